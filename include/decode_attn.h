@@ -1,0 +1,292 @@
+/*
+ * decode_attn.h - C ABI of the B200 (sm_100a) paged decode-attention library.
+ *
+ * The operation (Section 3.1 and Algorithm 1 step 2 of the vSkipper paper):
+ * in one decode step every sequence ("row") has one query token that attends
+ * over all of that sequence's cached keys and values, which live in a paged
+ * KV cache and are found through per-sequence page mappings (Invariant 2).
+ * The row's own K/V is written before attention, so the whole cached range
+ * [0, seq_len) is attended and no causal mask is applied.  Query heads are
+ * grouped: query head h reads KV head h / (num_q_heads / num_kv_heads).
+ *
+ *   s_t = sm_scale * <q[b,h,:], K[page(t), slot(t), g, :]>,  page(t) = block_table[b][t / page_size]
+ *   out[b,h,:] = sum_t softmax_t(s)_t * V[page(t), slot(t), g, :],   lse[b,h] = log sum_t exp(s_t)
+ *
+ * The library splits each sequence's token range into partitions ("splits"),
+ * computes one partial result per (sequence, KV head, split) with a running
+ * maximum and sum of exponentials in fp32, and merges the partials of a
+ * sequence by their log-sum-exp weights.  The paper does not describe the
+ * split or the merge; they are an exact re-association of the formula above.
+ *
+ * Conventions
+ *  - Every pointer marked "device" is caller-owned device memory of the
+ *    current CUDA device; "host" is ordinary host memory.  The library never
+ *    allocates or frees device memory in run/combine and never synchronises
+ *    the caller's stream there.  It owns only the plan object.
+ *  - Every function returns an int status (da_status_t); nothing throws or
+ *    aborts across this boundary and no kernel traps.  Conditions detected on
+ *    the device (stale lengths, page ids outside the pool, a wait that gave
+ *    up) are recorded in a status word read by decode_attn_last_device_status.
+ *  - Strides are in elements.  The innermost (head_dim) axis is contiguous.
+ *  - There is no CPU fallback: without a usable CUDA device the compute entry
+ *    points return DA_ERR_CUDA.
+ */
+#ifndef DECODE_ATTN_H_
+#define DECODE_ATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__CUDACC__) || defined(__CUDA_RUNTIME_API_H__) || defined(__DRIVER_TYPES_H__)
+#include <cuda_runtime_api.h>
+#else
+typedef struct CUstream_st *cudaStream_t;
+#endif
+
+typedef struct decode_attn_plan decode_attn_plan_t; /* opaque, library-owned */
+
+typedef enum {
+    DA_OK = 0,
+    DA_ERR_INVALID_ARG = -1,         /* null pointer, non-positive size, misaligned pointer or stride */
+    DA_ERR_UNSUPPORTED = -2,         /* a shape, dtype or policy this build has no kernel for          */
+    DA_ERR_WORKSPACE_TOO_SMALL = -3,
+    DA_ERR_STALE_PLAN = -4,          /* seq_lens differ from the ones the plan was made for            */
+    DA_ERR_CUDA = -5,                /* a CUDA runtime/driver call failed, or no device                */
+    DA_ERR_BAD_PAGE = -6,            /* a referenced block-table entry lies outside [0, num_pages)     */
+    DA_ERR_TIMEOUT = -7              /* a bounded device-side wait gave up                             */
+} da_status_t;
+
+enum { DA_DTYPE_BF16 = 1, DA_DTYPE_FP32 = 2 };
+
+typedef enum {
+    DA_SPLIT_AUTO = 0,          /* chunk length chosen from the length mix and the SM count          */
+    DA_SPLIT_FIXED_COUNT = 1,   /* every sequence gets exactly fixed_count splits (some may be empty) */
+    DA_SPLIT_DETERMINISTIC = 2  /* boundaries at multiples of chunk_tokens: a function of seq_len only */
+} da_split_mode_t;
+
+typedef enum {
+    DA_KERNEL_AUTO = 0,     /* tensor-core kernel when the GQA group has >= 2 heads, else SIMT       */
+    DA_KERNEL_SIMT = 1,     /* CUDA-core kernel, 16-byte vectorised global loads                      */
+    DA_KERNEL_MMA_TMA = 2   /* TMA-staged pages in shared memory, mma.sync bf16 for QK^T and PV       */
+} da_kernel_t;
+
+/* Split policy.  Zero-initialise for the defaults. */
+typedef struct {
+    int32_t split_mode;     /* da_split_mode_t                                                       */
+    int32_t fixed_count;    /* FIXED_COUNT: splits per sequence (>= 1)                               */
+    int32_t chunk_tokens;   /* DETERMINISTIC: chunk length, a multiple of page_size (0: 1024).
+                               AUTO: smallest chunk the planner may choose (0: 256)                  */
+    int32_t max_splits;     /* upper bound on the splits of one sequence (0: 512)                    */
+    int32_t sm_count;       /* 0: the current device's multiprocessor count                          */
+    int32_t kernel;         /* da_kernel_t                                                           */
+    int32_t fuse_combine;   /* 0: decode_attn_combine must follow decode_attn_run.
+                               1: the last partition of a sequence to finish merges inside run       */
+    int32_t capacity_batch; /* > 0: the plan can be refreshed in place for any batch <= this value
+                               (decode_attn_plan_update) and launches a fixed grid whose surplus
+                               blocks exit at once (Algorithm 1 step 6, "grid exit")                  */
+    int32_t capacity_tokens;/* with capacity_batch: upper bound on sum(seq_lens) of any refresh      */
+    int32_t ctas_per_sm;    /* 0: from the occupancy of the chosen kernel                            */
+    int32_t reserved[6];
+} decode_attn_policy_t;
+
+typedef struct {
+    int32_t batch;              /* live sequences B (rows of q, out, block_table)                    */
+    int32_t num_q_heads;
+    int32_t num_kv_heads;       /* divides num_q_heads; group size <= 8                              */
+    int32_t head_dim;           /* 64 or 128                                                         */
+    int32_t page_size;          /* tokens per page: 16                                               */
+    int32_t max_pages_per_seq;  /* row stride of block_table, in entries                             */
+    int64_t num_pages;          /* pages in each pool                                                */
+    int64_t k_stride_page, k_stride_token, k_stride_head;   /* elements; multiples of 8              */
+    int64_t v_stride_page, v_stride_token, v_stride_head;
+    int32_t kv_dtype;           /* DA_DTYPE_BF16                                                     */
+    int32_t q_dtype;            /* DA_DTYPE_BF16                                                     */
+    int32_t out_dtype;          /* DA_DTYPE_FP32 or DA_DTYPE_BF16                                    */
+    float sm_scale;             /* 0: 1/sqrtf(head_dim) evaluated in fp32                            */
+} decode_attn_shape_t;
+
+/* One unit of work: one KV head of one sequence over one token range. */
+typedef struct {
+    int32_t seq;          /* b                                                                       */
+    int32_t kv_head;      /* g                                                                       */
+    int32_t tok_begin;    /* first token, a multiple of page_size                                    */
+    int32_t tok_end;      /* one past the last token; tok_end == tok_begin marks an empty split      */
+    int32_t slot;         /* index of the partial in the workspace, -1: writes `out` directly        */
+    int32_t seq_len;      /* the length the plan was made for (checked against device seq_lens)      */
+    int32_t split_index;  /* position of this split within its sequence                              */
+    int32_t n_splits;     /* splits of this sequence                                                 */
+} decode_attn_unit_t;
+
+typedef struct {
+    int64_t n_units;          /* work units = thread blocks that do work                             */
+    int64_t grid;             /* thread blocks launched (>= n_units with a capacity plan)            */
+    int64_t n_slots;          /* partial results held in the workspace                               */
+    int64_t workspace_bytes;
+    int32_t chunk_tokens;     /* AUTO / DETERMINISTIC: the chunk length in use (0 for FIXED_COUNT)   */
+    int32_t kernel;           /* the da_kernel_t actually used                                       */
+    int32_t ctas_per_sm;      /* resident blocks per SM the planner assumed                          */
+    int32_t sm_count;
+    int32_t fuse_combine;
+    int32_t max_splits_used;  /* largest split count of any sequence                                 */
+    int32_t block_threads;
+    int32_t dynamic_smem_bytes;
+} decode_attn_plan_info_t;
+
+/* ---------------------------------------------------------------------------
+ * Planner.  The paper gives no split policy; it only requires that launch
+ * metadata is never stale (Invariant 2) and that launches are capture-safe
+ * (Algorithm 1 step 6).
+ *
+ * decode_attn_plan_layout is the pure host function behind decode_attn_plan:
+ * from the length mix it chooses the splits of every sequence and emits the
+ * work list.  It touches no device.  units_out may be NULL to query sizes;
+ * otherwise it must hold max_units entries (DA_ERR_INVALID_ARG if too few).
+ * splits_out and slot_base_out are [batch] or NULL.  The result is a
+ * deterministic function of (shape, policy, seq_lens, sm_count, ctas_per_sm);
+ * in DETERMINISTIC mode each sequence's boundaries depend on its own length
+ * and policy.chunk_tokens only.
+ * ------------------------------------------------------------------------- */
+int decode_attn_plan_layout(const decode_attn_shape_t *shape, const decode_attn_policy_t *policy,
+                            const int32_t *seq_lens_host, int32_t sm_count, int32_t ctas_per_sm,
+                            decode_attn_unit_t *units_out, int64_t max_units, int64_t *n_units_out,
+                            int32_t *splits_out, int32_t *slot_base_out, int64_t *n_slots_out,
+                            int32_t *chunk_tokens_out);
+
+/* Builds a plan for one decode step: validates shape and policy, runs the
+ * planner on seq_lens_host [batch] (host), uploads the work list to a small
+ * device buffer the plan owns (synchronously, on an internal stream) and
+ * reports the workspace size run/combine need.  *plan_out is set only on
+ * DA_OK.  A plan is tied to the CUDA device current at creation and must not
+ * be used by two launches that overlap on the GPU. */
+int decode_attn_plan(const decode_attn_shape_t *shape, const decode_attn_policy_t *policy,
+                     const int32_t *seq_lens_host, decode_attn_plan_t **plan_out,
+                     size_t *workspace_bytes_out);
+
+/* Re-plans in place for new lengths (and a new live batch <= capacity_batch)
+ * and enqueues the upload of the refreshed work list on `stream`; the device
+ * addresses, grid and kernel stay the same, so a CUDA graph captured around
+ * run/combine keeps working.  Only for plans made with capacity_batch > 0.
+ * seq_lens_host must stay valid until the call returns (it is copied). */
+int decode_attn_plan_update(decode_attn_plan_t *plan, int32_t batch, const int32_t *seq_lens_host,
+                            cudaStream_t stream);
+
+int decode_attn_plan_get_info(const decode_attn_plan_t *plan, decode_attn_plan_info_t *info_out);
+
+/* Copies the plan's work list (host copy) into units_out[max_units]. */
+int decode_attn_plan_get_units(const decode_attn_plan_t *plan, decode_attn_unit_t *units_out,
+                               int64_t max_units);
+
+/* DA_OK if seq_lens_host [batch] equals the lengths the plan was made for,
+ * DA_ERR_STALE_PLAN otherwise (Invariant 2: row metadata is never stale). */
+int decode_attn_plan_check(const decode_attn_plan_t *plan, int32_t batch, const int32_t *seq_lens_host);
+
+int decode_attn_plan_destroy(decode_attn_plan_t *plan);
+
+/* ---------------------------------------------------------------------------
+ * Split-KV partial kernel (Algorithm 1 step 2, the attention read).
+ *
+ *   q            device, bf16 [batch, num_q_heads, head_dim], contiguous, 16-byte aligned
+ *   k_cache      device, bf16 pool addressed by the k_stride_* of the shape, 16-byte aligned
+ *   v_cache      device, same with v_stride_*
+ *   block_table  device, int32 [batch, max_pages_per_seq]; entries at or beyond
+ *                ceil(seq_len / page_size) are never read; pages may be shared by rows
+ *   seq_lens     device, int32 [batch]; must equal the planned lengths (checked per block)
+ *   out          device, [batch, num_q_heads, head_dim] in shape.out_dtype
+ *   lse_or_null  device, fp32 [batch, num_q_heads] or NULL
+ *   workspace    device, >= workspace_bytes from the plan, 256-byte aligned (may be NULL if 0)
+ *
+ * One launch on `stream`.  Sequences with a single split write `out` (and
+ * lse) directly; the others write unnormalised fp32 partials with their
+ * running maximum and sum into the workspace, and - with fuse_combine - the
+ * last block of a (sequence, KV head) to finish merges them into `out`.
+ * Rows with seq_len 0 get zeros and lse = -inf.  Capture-safe.
+ * ------------------------------------------------------------------------- */
+int decode_attn_run(const decode_attn_plan_t *plan, const void *q, const void *k_cache,
+                    const void *v_cache, const int32_t *block_table, const int32_t *seq_lens, void *out,
+                    float *lse_or_null, void *workspace, size_t workspace_bytes, cudaStream_t stream);
+
+/* Extended arguments; set struct_size = sizeof(decode_attn_run_args_t). */
+typedef struct {
+    uint32_t struct_size;
+    uint32_t flags;             /* must be 0 */
+    const void *q;
+    const void *k_cache;
+    const void *v_cache;
+    const int32_t *block_table;
+    const int32_t *seq_lens;
+    const uint8_t *run_mask;    /* device, [batch] or NULL.  A row whose byte is 0 reads no KV and
+                                   emits zero (lse = -inf): the RUN mask of Algorithm 1 step 2. */
+    void *out;
+    float *lse;
+    void *workspace;
+    size_t workspace_bytes;
+} decode_attn_run_args_t;
+
+int decode_attn_run_ex(const decode_attn_plan_t *plan, const decode_attn_run_args_t *args,
+                       cudaStream_t stream);
+
+/* LSE combine: merges the partials `run` left in the workspace, per
+ * (sequence, query head), in ascending split order:
+ *   M = max_i m_i;  out = sum_i e^{m_i-M} o_i / sum_i e^{m_i-M} l_i;  lse = M + log(sum_i e^{m_i-M} l_i)
+ * Empty splits weigh exactly zero.  One launch on `stream` (none if no
+ * sequence was split).  With a fuse_combine plan the call is redundant but
+ * valid: it recomputes the same bits. */
+int decode_attn_combine(const decode_attn_plan_t *plan, const void *workspace, void *out,
+                        float *lse_or_null, cudaStream_t stream);
+
+/* Synchronises `stream`, returns the worst condition the kernels recorded
+ * since the last call (DA_OK, DA_ERR_STALE_PLAN, DA_ERR_BAD_PAGE,
+ * DA_ERR_TIMEOUT) and clears it.  For tests and debugging. */
+int decode_attn_last_device_status(const decode_attn_plan_t *plan, cudaStream_t stream);
+
+/* Host-only check of a block table against the shape: every entry below
+ * ceil(seq_len / page_size) must lie in [0, num_pages). */
+int decode_attn_validate_block_table(const decode_attn_shape_t *shape, const int32_t *seq_lens_host,
+                                     const int32_t *block_table_host);
+
+/* ---------------------------------------------------------------------------
+ * Debug / measurement helpers that reuse the kernels' page addressing.
+ * ------------------------------------------------------------------------- */
+
+/* Writes sequence `seq`'s K and V rows in logical token order,
+ * k_out / v_out: device bf16 [seq_len, num_kv_heads, head_dim], fetched
+ * through the same tensor maps and page lookups as the MMA/TMA kernel.
+ * Must be bit-exact with a host gather. */
+int decode_attn_debug_gather(const decode_attn_plan_t *plan, int32_t seq, const void *k_cache,
+                             const void *v_cache, const int32_t *block_table, void *k_out, void *v_out,
+                             cudaStream_t stream);
+
+/* Gather-only probe: streams exactly the K/V bytes `run` would read, through
+ * the same loads, and folds them into checksum_out (device, uint32 [grid]);
+ * no attention arithmetic.  Its time is the ceiling for this access pattern. */
+int decode_attn_gather_probe(const decode_attn_plan_t *plan, const void *k_cache, const void *v_cache,
+                             const int32_t *block_table, uint32_t *checksum_out, cudaStream_t stream);
+
+/* ---------------------------------------------------------------------------
+ * Whole step from host buffers: copies q, both pools, block table and
+ * lengths to the device (into a grow-only arena the library keeps), plans,
+ * runs, combines, copies `out` (and lse) back and synchronises.  pool_elems
+ * is the element count of each pool.  For end-to-end measurement and simple
+ * callers; serving engines keep the pools resident and use plan/run/combine.
+ * ------------------------------------------------------------------------- */
+int decode_attn_host_step(const decode_attn_shape_t *shape, const decode_attn_policy_t *policy,
+                          const void *q_host, const void *k_cache_host, const void *v_cache_host,
+                          int64_t pool_elems, const int32_t *block_table_host,
+                          const int32_t *seq_lens_host, void *out_host, float *lse_host_or_null);
+
+/* Frees the arena decode_attn_host_step keeps. */
+int decode_attn_host_release(void);
+
+const char *decode_attn_strerror(int status);
+
+/* "major.minor arch" of this build, e.g. "0.1 sm_100a". */
+const char *decode_attn_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DECODE_ATTN_H_ */

@@ -1,0 +1,547 @@
+// Host side of the C ABI: plan objects, argument checks, kernel selection and
+// launches.  No device memory is allocated in run/combine; the plan owns one
+// small device buffer (work list, per-sequence split table, tickets, status).
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <mutex>
+#include <new>
+#include <vector>
+
+#include "combine.cuh"
+#include "common.cuh"
+#include "decode_attn.h"
+#include "kernel_mma.cuh"
+#include "kernel_simt.cuh"
+#include "planner.h"
+
+using namespace da;
+
+#define DA_CUDA_TRY(expr)                         \
+    do {                                          \
+        cudaError_t err__ = (expr);               \
+        if (err__ != cudaSuccess) {               \
+            (void)cudaGetLastError();             \
+            return DA_ERR_CUDA;                   \
+        }                                         \
+    } while (0)
+
+struct decode_attn_plan {
+    decode_attn_shape_t shape;
+    decode_attn_policy_t policy;
+    Layout layout;
+    std::vector<int32_t> seq_lens;
+    int device = -1;
+    int sm_count = 0;
+    int ctas_per_sm = 0;
+    int kernel = DA_KERNEL_SIMT;
+    int group = 1;
+    int block_threads = 0;
+    int dyn_smem = 0;
+    float scale = 0.f;
+    int64_t max_units = 0;   // capacity of the device work list
+    int64_t max_batch = 0;
+    int64_t max_slots = 0;   // what the workspace is sized for
+    int64_t grid = 0;
+    size_t workspace_bytes = 0;
+    size_t ws_ml_offset = 0;
+    // device buffer
+    char* dev = nullptr;
+    char* pinned = nullptr;
+    size_t upload_bytes = 0;
+    size_t off_units = 0, off_seq_info = 0, off_status = 0, off_tickets = 0, total_bytes = 0;
+    cudaStream_t stream = nullptr;
+    cudaEvent_t upload_done = nullptr;  // last refresh of the device work list
+};
+
+namespace {
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+typedef void (*simt_kernel_t)(const KernelParams);
+
+template <int D>
+simt_kernel_t simt_for_group(int G)
+{
+    switch (G) {
+        case 1: return decode_attn_simt_kernel<D, 1>;
+        case 2: return decode_attn_simt_kernel<D, 2>;
+        case 3: return decode_attn_simt_kernel<D, 3>;
+        case 4: return decode_attn_simt_kernel<D, 4>;
+        case 5: return decode_attn_simt_kernel<D, 5>;
+        case 6: return decode_attn_simt_kernel<D, 6>;
+        case 7: return decode_attn_simt_kernel<D, 7>;
+        case 8: return decode_attn_simt_kernel<D, 8>;
+        default: return nullptr;
+    }
+}
+
+simt_kernel_t simt_kernel_for(int D, int G)
+{
+    return D == 64 ? simt_for_group<64>(G) : D == 128 ? simt_for_group<128>(G) : nullptr;
+}
+
+int pick_kernel(const decode_attn_shape_t& s, const decode_attn_policy_t& p)
+{
+    if (p.kernel != DA_KERNEL_AUTO) return p.kernel;
+    const int G = s.num_q_heads / s.num_kv_heads;
+    return (G >= 2 && mma_supports(s.head_dim, G)) ? DA_KERNEL_MMA_TMA : DA_KERNEL_SIMT;
+}
+
+// Resident blocks per SM of the kernel a plan will launch.
+int query_occupancy(int kernel, int D, int G, int* block_threads, int* dyn_smem)
+{
+    int n = 0;
+    if (kernel == DA_KERNEL_SIMT) {
+        simt_kernel_t fn = simt_kernel_for(D, G);
+        if (!fn) return -1;
+        *block_threads = kSimtThreads;
+        *dyn_smem = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, fn, kSimtThreads, 0) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return -1;
+        }
+        return n;
+    }
+    return mma_query_occupancy(D, G, block_threads, dyn_smem);
+}
+
+void fill_host_mirror(decode_attn_plan_t* pl)
+{
+    DevHeader* hdr = reinterpret_cast<DevHeader*>(pl->pinned);
+    hdr->n_units = (int32_t)pl->layout.units.size();
+    hdr->batch = pl->shape.batch;
+    hdr->pad[0] = hdr->pad[1] = 0;
+    std::memcpy(pl->pinned + pl->off_units, pl->layout.units.data(),
+                pl->layout.units.size() * sizeof(decode_attn_unit_t));
+    SeqInfo* si = reinterpret_cast<SeqInfo*>(pl->pinned + pl->off_seq_info);
+    for (int b = 0; b < pl->shape.batch; ++b) {
+        si[b].slot_base = pl->layout.slot_base[b];
+        si[b].n_splits = pl->layout.splits[b];
+    }
+}
+
+KernelParams make_params(const decode_attn_plan_t* pl, const decode_attn_run_args_t& a)
+{
+    KernelParams kp;
+    std::memset(&kp, 0, sizeof kp);
+    const decode_attn_shape_t& s = pl->shape;
+    kp.q = static_cast<const __nv_bfloat16*>(a.q);
+    kp.k = static_cast<const __nv_bfloat16*>(a.k_cache);
+    kp.v = static_cast<const __nv_bfloat16*>(a.v_cache);
+    kp.block_table = a.block_table;
+    kp.seq_lens = a.seq_lens;
+    kp.run_mask = a.run_mask;
+    kp.out = a.out;
+    kp.lse = a.lse;
+    kp.ws_o = static_cast<float*>(a.workspace);
+    kp.ws_ml = reinterpret_cast<float*>(static_cast<char*>(a.workspace) + pl->ws_ml_offset);
+    kp.header = reinterpret_cast<const DevHeader*>(pl->dev);
+    kp.units = reinterpret_cast<const decode_attn_unit_t*>(pl->dev + pl->off_units);
+    kp.seq_info = reinterpret_cast<const SeqInfo*>(pl->dev + pl->off_seq_info);
+    kp.tickets = reinterpret_cast<int32_t*>(pl->dev + pl->off_tickets);
+    kp.status = reinterpret_cast<int32_t*>(pl->dev + pl->off_status);
+    kp.k_stride_page = s.k_stride_page; kp.k_stride_token = s.k_stride_token; kp.k_stride_head = s.k_stride_head;
+    kp.v_stride_page = s.v_stride_page; kp.v_stride_token = s.v_stride_token; kp.v_stride_head = s.v_stride_head;
+    kp.num_pages = s.num_pages;
+    kp.num_q_heads = s.num_q_heads;
+    kp.num_kv_heads = s.num_kv_heads;
+    kp.max_pages_per_seq = s.max_pages_per_seq;
+    kp.scale_log2 = pl->scale * kLog2e;
+    kp.out_bf16 = s.out_dtype == DA_DTYPE_BF16;
+    kp.fused = pl->policy.fuse_combine;
+    return kp;
+}
+
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+}  // namespace
+
+extern "C" {
+
+int decode_attn_plan(const decode_attn_shape_t* shape, const decode_attn_policy_t* policy,
+                     const int32_t* seq_lens_host, decode_attn_plan_t** plan_out, size_t* workspace_bytes_out)
+{
+    if (!shape || !policy || !plan_out) return DA_ERR_INVALID_ARG;
+    if (shape->batch > 0 && !seq_lens_host) return DA_ERR_INVALID_ARG;
+    int rc = validate_shape(*shape);
+    if (rc != DA_OK) return rc;
+    rc = validate_policy(*shape, *policy);
+    if (rc != DA_OK) return rc;
+
+    decode_attn_plan_t* pl = new (std::nothrow) decode_attn_plan_t();
+    if (!pl) return DA_ERR_INVALID_ARG;
+    struct Guard {
+        decode_attn_plan_t* p;
+        ~Guard() { if (p) decode_attn_plan_destroy(p); }
+    } guard{pl};
+
+    pl->shape = *shape;
+    pl->policy = *policy;
+    pl->group = shape->num_q_heads / shape->num_kv_heads;
+    pl->scale = shape->sm_scale > 0.f ? shape->sm_scale : 1.0f / sqrtf((float)shape->head_dim);
+    pl->kernel = pick_kernel(*shape, *policy);
+    if (pl->kernel == DA_KERNEL_MMA_TMA && !mma_supports(shape->head_dim, pl->group)) return DA_ERR_UNSUPPORTED;
+
+    DA_CUDA_TRY(cudaGetDevice(&pl->device));
+    if (policy->sm_count > 0) {
+        pl->sm_count = policy->sm_count;
+    } else {
+        DA_CUDA_TRY(cudaDeviceGetAttribute(&pl->sm_count, cudaDevAttrMultiProcessorCount, pl->device));
+    }
+    int occ = query_occupancy(pl->kernel, shape->head_dim, pl->group, &pl->block_threads, &pl->dyn_smem);
+    if (occ <= 0) return DA_ERR_CUDA;
+    pl->ctas_per_sm = policy->ctas_per_sm > 0 ? policy->ctas_per_sm : occ;
+
+    pl->seq_lens.assign(seq_lens_host, seq_lens_host + shape->batch);
+    rc = make_layout(*shape, *policy, pl->seq_lens.data(), pl->sm_count, pl->ctas_per_sm, pl->layout);
+    if (rc != DA_OK) return rc;
+
+    if (policy->capacity_batch > 0) {
+        pl->max_batch = policy->capacity_batch;
+        pl->max_slots = capacity_slots(*shape, *policy);
+        pl->max_units = (pl->max_slots + pl->max_batch) * shape->num_kv_heads;
+        if ((int64_t)pl->layout.units.size() > pl->max_units || pl->layout.n_slots > pl->max_slots)
+            return DA_ERR_INVALID_ARG;  // the lengths exceed the declared capacity
+        pl->grid = pl->max_units;
+    } else {
+        pl->max_batch = shape->batch;
+        pl->max_slots = pl->layout.n_slots;
+        pl->max_units = (int64_t)pl->layout.units.size();
+        pl->grid = pl->max_units;
+    }
+    if (pl->grid > 0x7fffffffLL) return DA_ERR_UNSUPPORTED;
+
+    const size_t o_bytes = (size_t)pl->max_slots * shape->num_q_heads * shape->head_dim * sizeof(float);
+    pl->ws_ml_offset = align_up(o_bytes, 256);
+    pl->workspace_bytes = pl->max_slots ? pl->ws_ml_offset + (size_t)pl->max_slots * shape->num_q_heads * 2 * sizeof(float) : 0;
+
+    pl->off_units = align_up(sizeof(DevHeader), 32);
+    pl->off_seq_info = pl->off_units + align_up((size_t)std::max<int64_t>(pl->max_units, 1) * sizeof(decode_attn_unit_t), 32);
+    pl->upload_bytes = pl->off_seq_info + align_up((size_t)std::max<int64_t>(pl->max_batch, 1) * sizeof(SeqInfo), 32);
+    pl->off_status = pl->upload_bytes;
+    pl->off_tickets = pl->off_status + 32;
+    pl->total_bytes = pl->off_tickets +
+                      align_up((size_t)std::max<int64_t>(pl->max_batch, 1) * shape->num_kv_heads * sizeof(int32_t), 32);
+
+    DA_CUDA_TRY(cudaStreamCreateWithFlags(&pl->stream, cudaStreamNonBlocking));
+    DA_CUDA_TRY(cudaEventCreateWithFlags(&pl->upload_done, cudaEventDisableTiming));
+    DA_CUDA_TRY(cudaMalloc(&pl->dev, pl->total_bytes));
+    DA_CUDA_TRY(cudaMallocHost(&pl->pinned, pl->upload_bytes));
+    std::memset(pl->pinned, 0, pl->upload_bytes);
+    fill_host_mirror(pl);
+    DA_CUDA_TRY(cudaMemsetAsync(pl->dev + pl->off_status, 0, pl->total_bytes - pl->off_status, pl->stream));
+    DA_CUDA_TRY(cudaMemcpyAsync(pl->dev, pl->pinned, pl->upload_bytes, cudaMemcpyHostToDevice, pl->stream));
+    DA_CUDA_TRY(cudaStreamSynchronize(pl->stream));
+
+    if (workspace_bytes_out) *workspace_bytes_out = pl->workspace_bytes;
+    *plan_out = pl;
+    guard.p = nullptr;
+    return DA_OK;
+}
+
+int decode_attn_plan_update(decode_attn_plan_t* pl, int32_t batch, const int32_t* seq_lens_host, cudaStream_t stream)
+{
+    if (!pl || batch < 0 || (batch > 0 && !seq_lens_host)) return DA_ERR_INVALID_ARG;
+    if (pl->policy.capacity_batch <= 0) return DA_ERR_UNSUPPORTED;
+    if (batch > pl->max_batch) return DA_ERR_INVALID_ARG;
+    int64_t total = 0;
+    for (int b = 0; b < batch; ++b) total += seq_lens_host[b];
+    if (total > pl->policy.capacity_tokens) return DA_ERR_INVALID_ARG;
+    decode_attn_shape_t s = pl->shape;
+    s.batch = batch;
+    Layout lay;
+    int rc = make_layout(s, pl->policy, seq_lens_host, pl->sm_count, pl->ctas_per_sm, lay);
+    if (rc != DA_OK) return rc;
+    if ((int64_t)lay.units.size() > pl->max_units || lay.n_slots > pl->max_slots) return DA_ERR_INVALID_ARG;
+    // the previous refresh may still be reading the pinned mirror
+    DA_CUDA_TRY(cudaEventSynchronize(pl->upload_done));
+    pl->shape.batch = batch;
+    pl->layout = std::move(lay);
+    pl->seq_lens.assign(seq_lens_host, seq_lens_host + batch);
+    fill_host_mirror(pl);
+    // the copy is ordered on the caller's stream, behind any launch that still reads the old list
+    DA_CUDA_TRY(cudaMemcpyAsync(pl->dev, pl->pinned, pl->upload_bytes, cudaMemcpyHostToDevice, stream));
+    DA_CUDA_TRY(cudaEventRecord(pl->upload_done, stream));
+    return DA_OK;
+}
+
+int decode_attn_plan_get_info(const decode_attn_plan_t* pl, decode_attn_plan_info_t* info)
+{
+    if (!pl || !info) return DA_ERR_INVALID_ARG;
+    std::memset(info, 0, sizeof *info);
+    info->n_units = (int64_t)pl->layout.units.size();
+    info->grid = pl->grid;
+    info->n_slots = pl->layout.n_slots;
+    info->workspace_bytes = (int64_t)pl->workspace_bytes;
+    info->chunk_tokens = pl->layout.chunk_tokens;
+    info->kernel = pl->kernel;
+    info->ctas_per_sm = pl->ctas_per_sm;
+    info->sm_count = pl->sm_count;
+    info->fuse_combine = pl->policy.fuse_combine;
+    info->max_splits_used = pl->layout.max_splits_used;
+    info->block_threads = pl->block_threads;
+    info->dynamic_smem_bytes = pl->dyn_smem;
+    return DA_OK;
+}
+
+int decode_attn_plan_get_units(const decode_attn_plan_t* pl, decode_attn_unit_t* units_out, int64_t max_units)
+{
+    if (!pl || !units_out) return DA_ERR_INVALID_ARG;
+    if (max_units < (int64_t)pl->layout.units.size()) return DA_ERR_INVALID_ARG;
+    std::copy(pl->layout.units.begin(), pl->layout.units.end(), units_out);
+    return DA_OK;
+}
+
+int decode_attn_plan_check(const decode_attn_plan_t* pl, int32_t batch, const int32_t* seq_lens_host)
+{
+    if (!pl || (batch > 0 && !seq_lens_host)) return DA_ERR_INVALID_ARG;
+    if (batch != pl->shape.batch) return DA_ERR_STALE_PLAN;
+    for (int b = 0; b < batch; ++b)
+        if (seq_lens_host[b] != pl->seq_lens[b]) return DA_ERR_STALE_PLAN;
+    return DA_OK;
+}
+
+int decode_attn_plan_destroy(decode_attn_plan_t* pl)
+{
+    if (!pl) return DA_OK;
+    if (pl->stream) {
+        cudaStreamSynchronize(pl->stream);
+        cudaStreamDestroy(pl->stream);
+    }
+    if (pl->upload_done) {
+        cudaEventSynchronize(pl->upload_done);
+        cudaEventDestroy(pl->upload_done);
+    }
+    if (pl->dev) cudaFree(pl->dev);
+    if (pl->pinned) cudaFreeHost(pl->pinned);
+    (void)cudaGetLastError();
+    delete pl;
+    return DA_OK;
+}
+
+int decode_attn_run_ex(const decode_attn_plan_t* pl, const decode_attn_run_args_t* a, cudaStream_t stream)
+{
+    if (!pl || !a) return DA_ERR_INVALID_ARG;
+    if (a->struct_size != sizeof(decode_attn_run_args_t) || a->flags != 0) return DA_ERR_INVALID_ARG;
+    if (pl->shape.batch == 0 && pl->policy.capacity_batch == 0) return DA_OK;
+    if (!a->q || !a->k_cache || !a->v_cache || !a->block_table || !a->seq_lens || !a->out) return DA_ERR_INVALID_ARG;
+    if (!aligned(a->q, 16) || !aligned(a->k_cache, 16) || !aligned(a->v_cache, 16) || !aligned(a->out, 16) ||
+        !aligned(a->block_table, 4) || !aligned(a->seq_lens, 4))
+        return DA_ERR_INVALID_ARG;
+    if (pl->workspace_bytes > 0) {
+        if (!a->workspace || !aligned(a->workspace, 256)) return DA_ERR_INVALID_ARG;
+        if (a->workspace_bytes < pl->workspace_bytes) return DA_ERR_WORKSPACE_TOO_SMALL;
+    }
+    if (pl->grid == 0) return DA_OK;
+    const KernelParams kp = make_params(pl, *a);
+    if (pl->kernel == DA_KERNEL_SIMT) {
+        simt_kernel_t fn = simt_kernel_for(pl->shape.head_dim, pl->group);
+        if (!fn) return DA_ERR_UNSUPPORTED;
+        fn<<<(unsigned)pl->grid, kSimtThreads, 0, stream>>>(kp);
+    } else {
+        int rc = mma_launch(pl->shape, pl->group, kp, (unsigned)pl->grid, stream);
+        if (rc != DA_OK) return rc;
+    }
+    DA_CUDA_TRY(cudaGetLastError());
+    return DA_OK;
+}
+
+int decode_attn_run(const decode_attn_plan_t* pl, const void* q, const void* k_cache, const void* v_cache,
+                    const int32_t* block_table, const int32_t* seq_lens, void* out, float* lse_or_null,
+                    void* workspace, size_t workspace_bytes, cudaStream_t stream)
+{
+    decode_attn_run_args_t a;
+    std::memset(&a, 0, sizeof a);
+    a.struct_size = sizeof a;
+    a.q = q; a.k_cache = k_cache; a.v_cache = v_cache;
+    a.block_table = block_table; a.seq_lens = seq_lens;
+    a.out = out; a.lse = lse_or_null;
+    a.workspace = workspace; a.workspace_bytes = workspace_bytes;
+    return decode_attn_run_ex(pl, &a, stream);
+}
+
+int decode_attn_combine(const decode_attn_plan_t* pl, const void* workspace, void* out, float* lse_or_null,
+                        cudaStream_t stream)
+{
+    if (!pl || !out) return DA_ERR_INVALID_ARG;
+    if (pl->max_slots == 0) return DA_OK;  // nothing was split: run wrote every row
+    if (!workspace || !aligned(workspace, 256) || !aligned(out, 16)) return DA_ERR_INVALID_ARG;
+    decode_attn_run_args_t a;
+    std::memset(&a, 0, sizeof a);
+    a.out = out;
+    a.lse = lse_or_null;
+    a.workspace = const_cast<void*>(workspace);
+    const KernelParams kp = make_params(pl, a);
+    const unsigned grid = (unsigned)(pl->max_batch * pl->shape.num_kv_heads);
+    if (grid == 0) return DA_OK;
+    int rc = combine_launch(pl->shape.head_dim, pl->group, kp, grid, stream);
+    if (rc != DA_OK) return rc;
+    DA_CUDA_TRY(cudaGetLastError());
+    return DA_OK;
+}
+
+int decode_attn_last_device_status(const decode_attn_plan_t* pl, cudaStream_t stream)
+{
+    if (!pl) return DA_ERR_INVALID_ARG;
+    int32_t st = 0;
+    DA_CUDA_TRY(cudaStreamSynchronize(stream));
+    DA_CUDA_TRY(cudaMemcpy(&st, pl->dev + pl->off_status, sizeof st, cudaMemcpyDeviceToHost));
+    if (st != 0) {
+        DA_CUDA_TRY(cudaMemset(pl->dev + pl->off_status, 0, sizeof(int32_t)));
+        // a failed launch may have left tickets half drawn
+        DA_CUDA_TRY(cudaMemset(pl->dev + pl->off_tickets, 0, pl->total_bytes - pl->off_tickets));
+    }
+    return st;
+}
+
+int decode_attn_validate_block_table(const decode_attn_shape_t* shape, const int32_t* seq_lens_host,
+                                     const int32_t* block_table_host)
+{
+    if (!shape || (shape->batch > 0 && (!seq_lens_host || !block_table_host))) return DA_ERR_INVALID_ARG;
+    int rc = validate_shape(*shape);
+    if (rc != DA_OK) return rc;
+    for (int b = 0; b < shape->batch; ++b) {
+        if (seq_lens_host[b] < 0) return DA_ERR_INVALID_ARG;
+        const int64_t pages = ((int64_t)seq_lens_host[b] + shape->page_size - 1) / shape->page_size;
+        if (pages > shape->max_pages_per_seq) return DA_ERR_INVALID_ARG;
+        for (int64_t i = 0; i < pages; ++i) {
+            const int32_t pg = block_table_host[(int64_t)b * shape->max_pages_per_seq + i];
+            if (pg < 0 || pg >= shape->num_pages) return DA_ERR_BAD_PAGE;
+        }
+    }
+    return DA_OK;
+}
+
+int decode_attn_debug_gather(const decode_attn_plan_t* pl, int32_t seq, const void* k_cache, const void* v_cache,
+                             const int32_t* block_table, void* k_out, void* v_out, cudaStream_t stream)
+{
+    if (!pl || !k_cache || !v_cache || !block_table || !k_out || !v_out) return DA_ERR_INVALID_ARG;
+    if (seq < 0 || seq >= pl->shape.batch) return DA_ERR_INVALID_ARG;
+    return mma_debug_gather(pl->shape, pl->seq_lens[seq], seq, k_cache, v_cache, block_table, k_out, v_out,
+                            reinterpret_cast<int32_t*>(pl->dev + pl->off_status), stream);
+}
+
+int decode_attn_gather_probe(const decode_attn_plan_t* pl, const void* k_cache, const void* v_cache,
+                             const int32_t* block_table, uint32_t* checksum_out, cudaStream_t stream)
+{
+    if (!pl || !k_cache || !v_cache || !block_table || !checksum_out) return DA_ERR_INVALID_ARG;
+    if (pl->grid == 0) return DA_OK;
+    decode_attn_run_args_t a;
+    std::memset(&a, 0, sizeof a);
+    a.k_cache = k_cache; a.v_cache = v_cache; a.block_table = block_table;
+    const KernelParams kp = make_params(pl, a);
+    return mma_gather_probe(pl->shape, pl->group, kp, checksum_out, (unsigned)pl->grid, stream);
+}
+
+// ------------------------------------------------------------------ host-buffer step
+
+namespace {
+struct HostArena {
+    std::mutex mu;
+    int device = -1;
+    char* base = nullptr;
+    size_t bytes = 0;
+} g_arena;
+}  // namespace
+
+int decode_attn_host_release(void)
+{
+    std::lock_guard<std::mutex> lock(g_arena.mu);
+    if (g_arena.base) {
+        cudaFree(g_arena.base);
+        (void)cudaGetLastError();
+    }
+    g_arena.base = nullptr;
+    g_arena.bytes = 0;
+    g_arena.device = -1;
+    return DA_OK;
+}
+
+int decode_attn_host_step(const decode_attn_shape_t* shape, const decode_attn_policy_t* policy, const void* q_host,
+                          const void* k_cache_host, const void* v_cache_host, int64_t pool_elems,
+                          const int32_t* block_table_host, const int32_t* seq_lens_host, void* out_host,
+                          float* lse_host_or_null)
+{
+    if (!shape || !policy || !q_host || !k_cache_host || !v_cache_host || !block_table_host || !seq_lens_host ||
+        !out_host || pool_elems <= 0)
+        return DA_ERR_INVALID_ARG;
+    if (policy->capacity_batch != 0) return DA_ERR_INVALID_ARG;
+    int rc = decode_attn_validate_block_table(shape, seq_lens_host, block_table_host);
+    if (rc != DA_OK) return rc;
+    if (shape->batch == 0) return DA_OK;
+
+    decode_attn_plan_t* plan = nullptr;
+    size_t ws_bytes = 0;
+    rc = decode_attn_plan(shape, policy, seq_lens_host, &plan, &ws_bytes);
+    if (rc != DA_OK) return rc;
+    struct PlanGuard {
+        decode_attn_plan_t* p;
+        ~PlanGuard() { decode_attn_plan_destroy(p); }
+    } pg{plan};
+
+    const size_t out_elem = shape->out_dtype == DA_DTYPE_BF16 ? 2 : 4;
+    const size_t q_bytes = (size_t)shape->batch * shape->num_q_heads * shape->head_dim * 2;
+    const size_t pool_bytes = (size_t)pool_elems * 2;
+    const size_t bt_bytes = (size_t)shape->batch * shape->max_pages_per_seq * 4;
+    const size_t sl_bytes = (size_t)shape->batch * 4;
+    const size_t out_bytes = (size_t)shape->batch * shape->num_q_heads * shape->head_dim * out_elem;
+    const size_t lse_bytes = (size_t)shape->batch * shape->num_q_heads * 4;
+    size_t off = 0;
+    auto take = [&off](size_t n) { size_t o = off; off = align_up(off + n, 256); return o; };
+    const size_t o_q = take(q_bytes), o_k = take(pool_bytes), o_v = take(pool_bytes), o_bt = take(bt_bytes),
+                 o_sl = take(sl_bytes), o_out = take(out_bytes), o_lse = take(lse_bytes), o_ws = take(ws_bytes);
+
+    std::lock_guard<std::mutex> lock(g_arena.mu);
+    int dev = -1;
+    DA_CUDA_TRY(cudaGetDevice(&dev));
+    if (g_arena.device != dev || g_arena.bytes < off) {
+        if (g_arena.base) cudaFree(g_arena.base);
+        g_arena.base = nullptr;
+        g_arena.bytes = 0;
+        DA_CUDA_TRY(cudaMalloc(&g_arena.base, off));
+        g_arena.bytes = off;
+        g_arena.device = dev;
+    }
+    char* A = g_arena.base;
+    cudaStream_t st = plan->stream;
+    DA_CUDA_TRY(cudaMemcpyAsync(A + o_q, q_host, q_bytes, cudaMemcpyHostToDevice, st));
+    DA_CUDA_TRY(cudaMemcpyAsync(A + o_k, k_cache_host, pool_bytes, cudaMemcpyHostToDevice, st));
+    DA_CUDA_TRY(cudaMemcpyAsync(A + o_v, v_cache_host, pool_bytes, cudaMemcpyHostToDevice, st));
+    DA_CUDA_TRY(cudaMemcpyAsync(A + o_bt, block_table_host, bt_bytes, cudaMemcpyHostToDevice, st));
+    DA_CUDA_TRY(cudaMemcpyAsync(A + o_sl, seq_lens_host, sl_bytes, cudaMemcpyHostToDevice, st));
+    float* lse_dev = lse_host_or_null ? reinterpret_cast<float*>(A + o_lse) : nullptr;
+    rc = decode_attn_run(plan, A + o_q, A + o_k, A + o_v, reinterpret_cast<const int32_t*>(A + o_bt),
+                         reinterpret_cast<const int32_t*>(A + o_sl), A + o_out, lse_dev, ws_bytes ? A + o_ws : nullptr,
+                         ws_bytes, st);
+    if (rc != DA_OK) return rc;
+    if (!policy->fuse_combine) {
+        rc = decode_attn_combine(plan, ws_bytes ? A + o_ws : nullptr, A + o_out, lse_dev, st);
+        if (rc != DA_OK) return rc;
+    }
+    DA_CUDA_TRY(cudaMemcpyAsync(out_host, A + o_out, out_bytes, cudaMemcpyDeviceToHost, st));
+    if (lse_host_or_null)
+        DA_CUDA_TRY(cudaMemcpyAsync(lse_host_or_null, A + o_lse, lse_bytes, cudaMemcpyDeviceToHost, st));
+    return decode_attn_last_device_status(plan, st);
+}
+
+const char* decode_attn_strerror(int status)
+{
+    switch (status) {
+        case DA_OK: return "ok";
+        case DA_ERR_INVALID_ARG: return "invalid argument";
+        case DA_ERR_UNSUPPORTED: return "unsupported shape, dtype or policy";
+        case DA_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+        case DA_ERR_STALE_PLAN: return "plan is stale: seq_lens differ from the planned lengths";
+        case DA_ERR_CUDA: return "CUDA call failed or no CUDA device";
+        case DA_ERR_BAD_PAGE: return "block table refers to a page outside the pool";
+        case DA_ERR_TIMEOUT: return "a bounded device-side wait gave up";
+        default: return "unknown status";
+    }
+}
+
+const char* decode_attn_version(void) { return "0.1 sm_100a"; }
+
+}  // extern "C"

@@ -1,0 +1,249 @@
+// Split-KV planner.  The paper leaves partitioning to the engine; what it
+// demands is that launch metadata is rebuilt from the current rows whenever
+// they change (Invariant 2) and that a fixed launch shape can serve any live
+// size (Algorithm 1 step 6).  The policy implemented here:
+//
+//  * a work unit is (sequence, KV head, run of whole pages); all query heads
+//    of the group are handled by the unit so each K/V byte is read once;
+//  * AUTO picks one chunk length c (pages) for the whole batch: the smallest
+//    c >= the policy's minimum for which the unit count fits in
+//    waves * sm_count * ctas_per_sm resident blocks, waves being the smallest
+//    integer for which that is possible at all.  Each sequence then gets
+//    ceil(pages / c) splits of near-equal size;
+//  * DETERMINISTIC cuts every sequence at multiples of policy.chunk_tokens,
+//    so a sequence's boundaries are a function of its own length alone;
+//  * FIXED_COUNT gives every sequence exactly n splits of ceil(pages / n)
+//    pages; trailing splits may be empty;
+//  * units are issued most expensive first, and the KV heads of one token
+//    range next to each other so their blocks run at the same time and touch
+//    neighbouring addresses of the same pages.
+#include "planner.h"
+
+#include <algorithm>
+#include <cmath>
+
+namespace da {
+
+static inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+int validate_shape(const decode_attn_shape_t& s)
+{
+    if (s.batch < 0 || s.num_q_heads <= 0 || s.num_kv_heads <= 0 || s.head_dim <= 0 || s.page_size <= 0 ||
+        s.max_pages_per_seq < 0 || s.num_pages <= 0)
+        return DA_ERR_INVALID_ARG;
+    if (s.num_q_heads % s.num_kv_heads != 0) return DA_ERR_INVALID_ARG;
+    if (!(s.sm_scale >= 0.0f) || std::isinf(s.sm_scale)) return DA_ERR_INVALID_ARG;
+    const int64_t strides[6] = {s.k_stride_page, s.k_stride_token, s.k_stride_head,
+                                s.v_stride_page, s.v_stride_token, s.v_stride_head};
+    for (int64_t st : strides) {
+        if (st <= 0) return DA_ERR_INVALID_ARG;
+        if (st % 8 != 0) return DA_ERR_INVALID_ARG;  // 16-byte rows for vector loads and TMA
+    }
+    if (s.k_stride_token < s.head_dim || s.k_stride_head < s.head_dim || s.v_stride_token < s.head_dim ||
+        s.v_stride_head < s.head_dim)
+        return DA_ERR_INVALID_ARG;  // rows of head_dim contiguous elements must not overlap
+    if (s.num_q_heads / s.num_kv_heads > kMaxGroup) return DA_ERR_UNSUPPORTED;
+    if (s.head_dim != 64 && s.head_dim != 128) return DA_ERR_UNSUPPORTED;
+    if (s.page_size != 16) return DA_ERR_UNSUPPORTED;
+    if (s.kv_dtype != DA_DTYPE_BF16 || s.q_dtype != DA_DTYPE_BF16) return DA_ERR_UNSUPPORTED;
+    if (s.out_dtype != DA_DTYPE_FP32 && s.out_dtype != DA_DTYPE_BF16) return DA_ERR_UNSUPPORTED;
+    if (s.num_pages > (int64_t)INT32_MAX) return DA_ERR_UNSUPPORTED;
+    return DA_OK;
+}
+
+int validate_policy(const decode_attn_shape_t& s, const decode_attn_policy_t& p)
+{
+    if (p.split_mode < DA_SPLIT_AUTO || p.split_mode > DA_SPLIT_DETERMINISTIC) return DA_ERR_INVALID_ARG;
+    if (p.kernel < DA_KERNEL_AUTO || p.kernel > DA_KERNEL_MMA_TMA) return DA_ERR_INVALID_ARG;
+    if (p.split_mode == DA_SPLIT_FIXED_COUNT && p.fixed_count < 1) return DA_ERR_INVALID_ARG;
+    if (p.chunk_tokens < 0 || p.max_splits < 0 || p.sm_count < 0 || p.ctas_per_sm < 0 ||
+        p.capacity_batch < 0 || p.capacity_tokens < 0)
+        return DA_ERR_INVALID_ARG;
+    if (p.chunk_tokens % s.page_size != 0) return DA_ERR_INVALID_ARG;
+    if (p.fuse_combine != 0 && p.fuse_combine != 1) return DA_ERR_INVALID_ARG;
+    if (p.capacity_batch > 0 && (p.capacity_tokens <= 0 || s.batch > p.capacity_batch))
+        return DA_ERR_INVALID_ARG;
+    for (int32_t r : p.reserved)
+        if (r != 0) return DA_ERR_INVALID_ARG;
+    return DA_OK;
+}
+
+static int max_splits_of(const decode_attn_policy_t& p) { return p.max_splits > 0 ? p.max_splits : kDefaultMaxSplits; }
+
+static int min_chunk_pages(const decode_attn_shape_t& s, const decode_attn_policy_t& p)
+{
+    int tokens;
+    if (p.split_mode == DA_SPLIT_DETERMINISTIC)
+        tokens = p.chunk_tokens > 0 ? p.chunk_tokens : kDefaultDeterministicChunk;
+    else
+        tokens = p.chunk_tokens > 0 ? p.chunk_tokens : kDefaultAutoMinChunk;
+    return (int)std::max<int64_t>(1, ceil_div(tokens, s.page_size));
+}
+
+int64_t capacity_slots(const decode_attn_shape_t& s, const decode_attn_policy_t& p)
+{
+    if (p.capacity_batch <= 0) return 0;
+    if (p.split_mode == DA_SPLIT_FIXED_COUNT) return (int64_t)p.fixed_count * p.capacity_batch;
+    const int64_t chunk_tokens = (int64_t)min_chunk_pages(s, p) * s.page_size;
+    return ceil_div(p.capacity_tokens, chunk_tokens) + p.capacity_batch;
+}
+
+namespace {
+
+struct SeqCut {
+    int64_t pages;
+    int64_t chunk;   // pages per split (upper bound)
+    int32_t splits;
+    bool even;       // spread the pages evenly instead of cutting at multiples of chunk
+};
+
+int64_t units_for_chunk(const std::vector<int64_t>& pages, int64_t c, int max_splits)
+{
+    int64_t total = 0;
+    for (int64_t pg : pages) {
+        if (pg == 0) {
+            total += 1;
+            continue;
+        }
+        const int64_t cb = std::max(c, ceil_div(pg, max_splits));
+        total += ceil_div(pg, cb);
+    }
+    return total;
+}
+
+}  // namespace
+
+int make_layout(const decode_attn_shape_t& s, const decode_attn_policy_t& p, const int32_t* seq_lens,
+                int sm_count, int ctas_per_sm, Layout& out)
+{
+    if (sm_count <= 0 || ctas_per_sm <= 0) return DA_ERR_INVALID_ARG;
+    if (s.batch > 0 && seq_lens == nullptr) return DA_ERR_INVALID_ARG;
+    const int B = s.batch, P = s.page_size, H = s.num_kv_heads;
+    const int max_splits = max_splits_of(p);
+    std::vector<int64_t> pages(B);
+    for (int b = 0; b < B; ++b) {
+        if (seq_lens[b] < 0) return DA_ERR_INVALID_ARG;
+        pages[b] = ceil_div(seq_lens[b], P);
+        if (pages[b] > s.max_pages_per_seq) return DA_ERR_INVALID_ARG;
+    }
+
+    std::vector<SeqCut> cuts(B);
+    out.chunk_tokens = 0;
+    if (p.split_mode == DA_SPLIT_FIXED_COUNT) {
+        for (int b = 0; b < B; ++b) {
+            cuts[b].pages = pages[b];
+            cuts[b].chunk = std::max<int64_t>(1, ceil_div(pages[b], p.fixed_count));
+            cuts[b].splits = p.fixed_count;
+            cuts[b].even = false;
+        }
+    } else {
+        int64_t c = min_chunk_pages(s, p);
+        if (p.split_mode == DA_SPLIT_AUTO && B > 0) {
+            const int64_t slots = (int64_t)sm_count * ctas_per_sm;
+            const int64_t floor_units = (int64_t)H * B;  // one unit per (sequence, KV head) at least
+            const int64_t waves = std::max<int64_t>(1, ceil_div(floor_units, slots));
+            const int64_t target = waves * slots;
+            int64_t lo = c, hi = std::max<int64_t>(c, *std::max_element(pages.begin(), pages.end()));
+            if (H * units_for_chunk(pages, lo, max_splits) > target) {
+                while (lo < hi) {  // smallest chunk whose unit count fits
+                    const int64_t mid = lo + (hi - lo) / 2;
+                    if (H * units_for_chunk(pages, mid, max_splits) <= target)
+                        hi = mid;
+                    else
+                        lo = mid + 1;
+                }
+            }
+            c = lo;
+        }
+        out.chunk_tokens = (int32_t)std::min<int64_t>(c * P, INT32_MAX);
+        for (int b = 0; b < B; ++b) {
+            cuts[b].pages = pages[b];
+            cuts[b].chunk = std::max(c, ceil_div(pages[b], max_splits));
+            cuts[b].splits = (int32_t)std::max<int64_t>(1, ceil_div(pages[b], cuts[b].chunk));
+            cuts[b].even = (p.split_mode == DA_SPLIT_AUTO);
+        }
+    }
+
+    out.splits.assign(B, 1);
+    out.slot_base.assign(B, -1);
+    out.units.clear();
+    out.n_slots = 0;
+    out.max_splits_used = B > 0 ? 1 : 0;
+    struct Keyed {
+        decode_attn_unit_t u;
+        int64_t cost;
+    };
+    std::vector<Keyed> keyed;
+    for (int b = 0; b < B; ++b) {
+        const SeqCut& cut = cuts[b];
+        const int32_t S = cut.splits;
+        out.splits[b] = S;
+        out.max_splits_used = std::max(out.max_splits_used, S);
+        int64_t base_slot = -1;
+        if (S > 1) {
+            base_slot = out.n_slots;
+            out.slot_base[b] = (int32_t)base_slot;
+            out.n_slots += S;
+            if (out.n_slots > INT32_MAX) return DA_ERR_UNSUPPORTED;
+        }
+        for (int32_t i = 0; i < S; ++i) {
+            int64_t pb, pe;
+            if (cut.even) {
+                const int64_t q = cut.pages / S, r = cut.pages % S;
+                pb = i * q + std::min<int64_t>(i, r);
+                pe = pb + q + (i < r ? 1 : 0);
+            } else {
+                pb = std::min(cut.pages, (int64_t)i * cut.chunk);
+                pe = std::min(cut.pages, (int64_t)(i + 1) * cut.chunk);
+            }
+            for (int g = 0; g < H; ++g) {
+                Keyed k;
+                k.u.seq = b;
+                k.u.kv_head = g;
+                k.u.tok_begin = (int32_t)(pb * P);
+                k.u.tok_end = (int32_t)std::min<int64_t>(pe * P, seq_lens[b]);
+                if (k.u.tok_end < k.u.tok_begin) k.u.tok_end = k.u.tok_begin;
+                k.u.slot = S > 1 ? (int32_t)(base_slot + i) : -1;
+                k.u.seq_len = seq_lens[b];
+                k.u.split_index = i;
+                k.u.n_splits = S;
+                k.cost = pe - pb;
+                keyed.push_back(k);
+            }
+        }
+    }
+    std::stable_sort(keyed.begin(), keyed.end(), [](const Keyed& a, const Keyed& b) { return a.cost > b.cost; });
+    out.units.reserve(keyed.size());
+    for (const Keyed& k : keyed) out.units.push_back(k.u);
+    return DA_OK;
+}
+
+}  // namespace da
+
+extern "C" int decode_attn_plan_layout(const decode_attn_shape_t* shape, const decode_attn_policy_t* policy,
+                                       const int32_t* seq_lens_host, int32_t sm_count, int32_t ctas_per_sm,
+                                       decode_attn_unit_t* units_out, int64_t max_units, int64_t* n_units_out,
+                                       int32_t* splits_out, int32_t* slot_base_out, int64_t* n_slots_out,
+                                       int32_t* chunk_tokens_out)
+{
+    if (!shape || !policy) return DA_ERR_INVALID_ARG;
+    int rc = da::validate_shape(*shape);
+    if (rc != DA_OK) return rc;
+    rc = da::validate_policy(*shape, *policy);
+    if (rc != DA_OK) return rc;
+    da::Layout lay;
+    rc = da::make_layout(*shape, *policy, seq_lens_host, sm_count, ctas_per_sm, lay);
+    if (rc != DA_OK) return rc;
+    if (n_units_out) *n_units_out = (int64_t)lay.units.size();
+    if (n_slots_out) *n_slots_out = lay.n_slots;
+    if (chunk_tokens_out) *chunk_tokens_out = lay.chunk_tokens;
+    for (int b = 0; b < shape->batch; ++b) {
+        if (splits_out) splits_out[b] = lay.splits[b];
+        if (slot_base_out) slot_base_out[b] = lay.slot_base[b];
+    }
+    if (units_out) {
+        if (max_units < (int64_t)lay.units.size()) return DA_ERR_INVALID_ARG;
+        std::copy(lay.units.begin(), lay.units.end(), units_out);
+    }
+    return DA_OK;
+}

@@ -1,0 +1,38 @@
+// Host-side split-KV planner: length mix -> work list.  Pure integer work, no
+// CUDA calls, so it is also what the CPU tests exercise.
+#pragma once
+
+#include <cstdint>
+#include <vector>
+
+#include "decode_attn.h"
+
+namespace da {
+
+constexpr int kDefaultDeterministicChunk = 1024;  // tokens
+constexpr int kDefaultAutoMinChunk = 256;         // tokens
+constexpr int kDefaultMaxSplits = 512;
+constexpr int kMaxGroup = 8;
+
+struct Layout {
+    std::vector<decode_attn_unit_t> units;  // launch order: most expensive first
+    std::vector<int32_t> splits;            // [batch]
+    std::vector<int32_t> slot_base;         // [batch], -1 when the sequence has one split
+    int64_t n_slots = 0;
+    int32_t chunk_tokens = 0;
+    int32_t max_splits_used = 0;
+};
+
+// Validates the fields the planner and the kernels rely on.
+int validate_shape(const decode_attn_shape_t& s);
+int validate_policy(const decode_attn_shape_t& s, const decode_attn_policy_t& p);
+
+// Fills `out` for the given lengths.  sm_count and ctas_per_sm must be > 0.
+int make_layout(const decode_attn_shape_t& s, const decode_attn_policy_t& p, const int32_t* seq_lens,
+                int sm_count, int ctas_per_sm, Layout& out);
+
+// Upper bounds for a capacity plan (any batch <= capacity_batch and
+// sum(seq_lens) <= capacity_tokens).
+int64_t capacity_slots(const decode_attn_shape_t& s, const decode_attn_policy_t& p);
+
+}  // namespace da

@@ -1,0 +1,215 @@
+"""Host-side checks that need no GPU: the library loads and exports what the
+header declares, argument validation answers with status codes, and the
+split planner's work lists cover every token exactly once."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+from paper_2609_37062_b200 import build as da_build
+
+da_build.build()
+from paper_2609_37062_b200 import binding as da  # noqa: E402
+from paper_2609_37062_b200 import workloads as wl  # noqa: E402
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "decode_attn.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(decode_attn_[a-z_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    names = declared_functions()
+    assert len(names) >= 15
+    lib = ctypes.CDLL(da.LIB_PATH)
+    for n in names:
+        assert hasattr(lib, n), n
+    assert sorted(da.EXPORTED) == names
+
+
+def test_version_and_strerror():
+    assert "sm_100a" in da.decode_attn_version()
+    assert da.decode_attn_strerror(da.DA_OK) == "ok"
+    for code in range(-7, 0):
+        assert da.decode_attn_strerror(code) != "unknown status"
+    assert da.decode_attn_strerror(-99) == "unknown status"
+
+
+def test_struct_sizes_match_the_header():
+    assert ctypes.sizeof(da.Unit) == 32
+    assert ctypes.sizeof(da.Policy) == 64
+    assert ctypes.sizeof(da.Shape) == 96
+    assert ctypes.sizeof(da.RunArgs) == 88
+
+
+def shape(B=4, Hq=32, Hkv=8, D=128, mpp=8192, pages=1 << 20):
+    return da.make_shape(B, Hq, Hkv, D, 16, mpp, pages, (16 * Hkv * D, Hkv * D, D))
+
+
+def layout(lens, policy, sm=148, ctas=2, **kw):
+    return da.decode_attn_plan_layout(shape(B=len(lens), **kw), policy, lens, sm, ctas)
+
+
+def covered_exactly_once(units, lens, Hkv):
+    """Every (sequence, KV head) token range is tiled by its units."""
+    per = {}
+    for u in units:
+        per.setdefault((u.seq, u.kv_head), []).append(u)
+    assert len(per) == len(lens) * Hkv
+    for (b, g), us in per.items():
+        us.sort(key=lambda u: u.split_index)
+        assert [u.split_index for u in us] == list(range(len(us)))
+        assert all(u.n_splits == len(us) and u.seq_len == lens[b] for u in us)
+        pos = 0
+        for u in us:
+            assert u.tok_begin % 16 == 0
+            if u.tok_end > u.tok_begin:
+                assert u.tok_begin == pos
+                pos = u.tok_end
+            else:
+                assert u.tok_end == u.tok_begin        # an empty split
+        assert pos == lens[b]
+        if len(us) == 1:
+            assert us[0].slot == -1
+        else:
+            slots = [u.slot for u in us]
+            assert slots == list(range(slots[0], slots[0] + len(us))) and slots[0] >= 0
+
+
+@pytest.mark.parametrize("lens", [[17, 64, 129, 300], [32768], [0, 1, 15, 16, 17], [5000] * 64,
+                                  wl.lengths_short_chat(64, 2), wl.lengths_shared_prefix(256, 3)])
+@pytest.mark.parametrize("mode", [da.DA_SPLIT_AUTO, da.DA_SPLIT_DETERMINISTIC, da.DA_SPLIT_FIXED_COUNT])
+def test_units_tile_every_sequence(lens, mode):
+    pol = da.make_policy(split_mode=mode, fixed_count=3)
+    units, splits, slot_base, n_slots, chunk = layout(lens, pol)
+    covered_exactly_once(units, lens, 8)
+    assert n_slots == sum(int(s) for s in splits if s > 1)
+    costs = [u.tok_end - u.tok_begin for u in units]
+    pages = [(c + 15) // 16 for c in costs]
+    assert pages == sorted(pages, reverse=True)         # most expensive first
+    for b, s in enumerate(splits):
+        assert (slot_base[b] == -1) == (s == 1)
+
+
+def test_auto_fills_the_machine_for_one_long_sequence():
+    units, splits, _, n_slots, chunk = layout([32768], da.make_policy(), sm=148, ctas=2)
+    assert 8 <= splits[0] <= 64
+    assert len(units) <= 296 and len(units) > 296 - 8
+    sizes = {u.tok_end - u.tok_begin for u in units}
+    assert max(sizes) - min(sizes) <= 16                # near-equal cost
+    assert chunk % 16 == 0 and chunk >= 256
+
+
+def test_auto_never_goes_below_the_minimum_chunk():
+    units, splits, _, _, chunk = layout([300, 200], da.make_policy())
+    assert chunk == 256 and list(splits) == [2, 1]
+    units, splits, _, _, chunk = layout([300, 200], da.make_policy(chunk_tokens=512))
+    assert list(splits) == [1, 1]
+
+
+def test_auto_uses_whole_waves_for_large_batches():
+    lens = [512] * 256
+    units, splits, _, n_slots, _ = layout(lens, da.make_policy())
+    assert set(splits) == {1} and n_slots == 0 and len(units) == 2048
+
+
+def test_auto_is_a_pure_function_of_its_inputs():
+    lens = wl.lengths_short_chat(64, 2)
+    a = layout(lens, da.make_policy())
+    b = layout(lens, da.make_policy())
+    assert [(u.seq, u.kv_head, u.tok_begin, u.tok_end, u.slot) for u in a[0]] == \
+           [(u.seq, u.kv_head, u.tok_begin, u.tok_end, u.slot) for u in b[0]]
+    c = layout(lens, da.make_policy(), sm=64)
+    assert c[4] >= a[4]                                 # fewer SMs, never shorter chunks
+
+
+def test_deterministic_boundaries_depend_on_the_length_alone():
+    pol = da.make_policy(split_mode=da.DA_SPLIT_DETERMINISTIC, chunk_tokens=512)
+
+    def cuts(lens, b, **kw):
+        units = layout(lens, pol, **kw)[0]
+        return sorted({(u.split_index, u.tok_begin, u.tok_end) for u in units if u.seq == b})
+
+    alone = cuts([5000], 0)
+    assert alone == [(i, 512 * i, min(512 * (i + 1), 5000)) for i in range(10)]
+    assert cuts([77, 5000, 123456], 1) == alone
+    assert cuts([5000] * 256, 200) == alone
+    assert cuts([5000, 9], 0, sm=16, ctas=1) == alone
+    assert layout([5000], da.make_policy(split_mode=da.DA_SPLIT_DETERMINISTIC))[4] == 1024
+
+
+def test_fixed_count_gives_empty_trailing_splits():
+    pol = da.make_policy(split_mode=da.DA_SPLIT_FIXED_COUNT, fixed_count=8)
+    units, splits, _, n_slots, _ = layout([40], pol)
+    assert list(splits) == [8] and n_slots == 8
+    mine = sorted([u for u in units if u.kv_head == 0], key=lambda u: u.split_index)
+    assert [(u.tok_begin, u.tok_end) for u in mine][:4] == [(0, 16), (16, 32), (32, 40), (48, 48)]
+    assert all(u.tok_end == u.tok_begin for u in mine[3:])
+
+
+def test_max_splits_caps_the_split_count():
+    units, splits, _, _, _ = layout([131072], da.make_policy(max_splits=16, chunk_tokens=16))
+    assert splits[0] == 16
+
+
+def test_invalid_shapes_and_policies_are_rejected():
+    L = [100]
+    ok = da.make_policy()
+    bad = [
+        (dict(Hq=30), ok, da.DA_ERR_INVALID_ARG),           # heads do not divide
+        (dict(Hq=128, Hkv=8), ok, da.DA_ERR_UNSUPPORTED),   # group of 16
+        (dict(D=96), ok, da.DA_ERR_INVALID_ARG),            # stride rule holds but dim unsupported
+        (dict(mpp=3), ok, da.DA_ERR_INVALID_ARG),           # block table row too short
+        ({}, da.make_policy(split_mode=7), da.DA_ERR_INVALID_ARG),
+        ({}, da.make_policy(split_mode=da.DA_SPLIT_FIXED_COUNT, fixed_count=0), da.DA_ERR_INVALID_ARG),
+        ({}, da.make_policy(chunk_tokens=100), da.DA_ERR_INVALID_ARG),
+        ({}, da.make_policy(kernel=9), da.DA_ERR_INVALID_ARG),
+    ]
+    for kw, pol, code in bad:
+        with pytest.raises(da.DecodeAttnError) as e:
+            layout(L, pol, **kw)
+        if kw.get("D") == 96:
+            assert e.value.status in (da.DA_ERR_INVALID_ARG, da.DA_ERR_UNSUPPORTED)
+        else:
+            assert e.value.status == code, (kw, e.value.status)
+    s = shape(B=1)
+    s.page_size = 32
+    with pytest.raises(da.DecodeAttnError) as e:
+        da.decode_attn_plan_layout(s, ok, L, 148, 2)
+    assert e.value.status == da.DA_ERR_UNSUPPORTED
+    s = shape(B=1)
+    s.k_stride_token = 100                                   # not a multiple of 8 elements
+    with pytest.raises(da.DecodeAttnError) as e:
+        da.decode_attn_plan_layout(s, ok, L, 148, 2)
+    assert e.value.status == da.DA_ERR_INVALID_ARG
+    with pytest.raises(da.DecodeAttnError):
+        layout([-1], ok)
+
+
+def test_validate_block_table():
+    w = wl.config_tiny()
+    s = da.shape_of_workload(w)
+    assert da.decode_attn_validate_block_table(s, w.seq_lens, w.block_table) == da.DA_OK
+    bt = w.block_table.clone()
+    bt[2, 3] = 64
+    assert da.decode_attn_validate_block_table(s, w.seq_lens, bt) == da.DA_ERR_BAD_PAGE
+    bt[2, 3] = -1
+    assert da.decode_attn_validate_block_table(s, w.seq_lens, bt) == da.DA_ERR_BAD_PAGE
+    bt = w.block_table.clone()
+    bt[0, 2] = 1000                                          # beyond ceil(17/16) pages: never read
+    assert da.decode_attn_validate_block_table(s, w.seq_lens, bt) == da.DA_OK
+
+
+def test_compute_entry_points_fail_loudly_without_a_device():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a device is present")
+    w = wl.config_tiny()
+    with pytest.raises(da.DecodeAttnError) as e:
+        da.decode_attn_plan(da.shape_of_workload(w), da.make_policy(), w.seq_lens)
+    assert e.value.status == da.DA_ERR_CUDA
