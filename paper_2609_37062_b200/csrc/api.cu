@@ -420,14 +420,21 @@ int decode_attn_debug_gather(const decode_attn_plan_t* pl, int32_t seq, const vo
 {
     if (!pl || !k_cache || !v_cache || !block_table || !k_out || !v_out) return DA_ERR_INVALID_ARG;
     if (seq < 0 || seq >= pl->shape.batch) return DA_ERR_INVALID_ARG;
-    return mma_debug_gather(pl->shape, pl->seq_lens[seq], seq, k_cache, v_cache, block_table, k_out, v_out,
-                            reinterpret_cast<int32_t*>(pl->dev + pl->off_status), stream);
+    if (!aligned(k_cache, 16) || !aligned(v_cache, 16) || !aligned(k_out, 16) || !aligned(v_out, 16))
+        return DA_ERR_INVALID_ARG;
+    if (pl->grid == 0) return DA_OK;
+    decode_attn_run_args_t a;
+    std::memset(&a, 0, sizeof a);
+    a.k_cache = k_cache; a.v_cache = v_cache; a.block_table = block_table;
+    const KernelParams kp = make_params(pl, a);
+    return mma_debug_gather(pl->shape, pl->group, kp, seq, k_out, v_out, (unsigned)pl->grid, stream);
 }
 
 int decode_attn_gather_probe(const decode_attn_plan_t* pl, const void* k_cache, const void* v_cache,
                              const int32_t* block_table, uint32_t* checksum_out, cudaStream_t stream)
 {
     if (!pl || !k_cache || !v_cache || !block_table || !checksum_out) return DA_ERR_INVALID_ARG;
+    if (!aligned(k_cache, 16) || !aligned(v_cache, 16)) return DA_ERR_INVALID_ARG;
     if (pl->grid == 0) return DA_OK;
     decode_attn_run_args_t a;
     std::memset(&a, 0, sizeof a);

@@ -1,14 +1,587 @@
-// Placeholder until the tensor-core kernel lands: nothing is supported.
+// Tensor-core split-KV partial kernel with TMA-staged pages.
+//
+// One block per work unit (sequence, KV head, run of pages): four consumer
+// warps and one producer warp.  The producer turns block-table entries into
+// TMA tile loads (cp.async.bulk.tensor over a 4-D map [dim, slot, head, page]
+// of each pool): one 16-token page of one KV head lands in shared memory as
+// 16 rows x 128 bytes per half of the head dimension, 128-byte swizzled, with
+// an mbarrier counting the bytes.  A stage is four pages of K and of V; a
+// ring of stages keeps tens of KB in flight per block with no register cost.
+//
+// Consumer warp w owns page w of every stage.  With the query heads of the
+// group as the N dimension (padded to 8) and the 16 tokens of the page as M,
+//   S^T[16 x 8]  = K_page[16 x D] . Q^T[D x 8]          (mma.sync m16n8k16 bf16, fp32 accumulate)
+//   O^T[D x 8]  += V_page^T[D x 16] . P^T[16 x 8]
+// so K and V are the A operands straight out of shared memory (ldmatrix, the
+// V tile transposed on the way) and each K/V byte is used for all heads of
+// the group.  Softmax runs on the accumulator fragments in fp32: running max
+// and sum per head, column maxima over the 8 lanes that share a head by warp
+// shuffles, exponentials in the base-2 domain.
+//
+// P must keep more than bf16 precision.  For groups of up to 4 heads the
+// query is duplicated into columns 4..7, so those columns see the same logits
+// and carry the low part: columns 0..3 hold bf16(p), columns 4..7 hold
+// bf16(p - bf16(p)), and one PV mma accumulates both; the two halves are
+// added at the end.  For groups of 5..8 heads the low part takes a second
+// mma.  P^T reaches the B-operand layout with one movmatrix transpose per
+// 8x8 block.
+//
+// Every wait on an mbarrier is bounded; a wait that gives up records
+// DA_ERR_TIMEOUT and the block drains without touching the tiles.
 #pragma once
+
+#include <cuda.h>
 
 #include "common.cuh"
 
 namespace da {
 
-inline bool mma_supports(int, int) { return false; }
-inline int mma_query_occupancy(int, int, int*, int*) { return -1; }
-inline int mma_launch(const decode_attn_shape_t&, int, const KernelParams&, unsigned, cudaStream_t) { return DA_ERR_UNSUPPORTED; }
-inline int mma_debug_gather(const decode_attn_shape_t&, int, int, const void*, const void*, const int32_t*, void*, void*, int32_t*, cudaStream_t) { return DA_ERR_UNSUPPORTED; }
-inline int mma_gather_probe(const decode_attn_shape_t&, int, const KernelParams&, uint32_t*, unsigned, cudaStream_t) { return DA_ERR_UNSUPPORTED; }
+constexpr int kMmaConsumerWarps = 4;
+constexpr int kMmaThreads = (kMmaConsumerWarps + 1) * 32;
+constexpr int kPagesPerStage = kMmaConsumerWarps;
+constexpr long long kWaitLimitCycles = 2000000000LL;  // about one second
+
+enum MmaMode { kModeAttend = 0, kModeProbe = 1, kModeGather = 2 };
+
+template <int D>
+struct MmaCfg {
+    static constexpr int kHalves = D / 64;                      // 128-byte column blocks per row
+    static constexpr int kBoxBytes = 16 * 128;                  // one TMA box: 16 rows x 128 B
+    static constexpr int kPageBytes = kHalves * kBoxBytes;      // one page of one tensor
+    static constexpr int kTensorBytes = kPagesPerStage * kPageBytes;
+    static constexpr int kStageBytes = 2 * kTensorBytes;        // K then V
+    static constexpr int kStages = (D == 128) ? 3 : 6;
+    static constexpr int kBarrierBytes = 1024;                  // barriers + small state, keeps tiles 1 KB aligned
+    static constexpr int kSmemBytes = kStages * kStageBytes + kBarrierBytes + 1024;  // + alignment slack
+};
+
+// ---------------------------------------------------------------- PTX wrappers
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+// Bounded wait: false if the phase did not complete within the limit.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if (clock64() - t0 > kWaitLimitCycles) return false;
+    }
+    return true;
+}
+
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
+                                            int c2, int c3)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+}
+
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4])
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr));
+}
+
+__device__ __forceinline__ void ldsm_x4_trans(uint32_t addr, uint32_t (&r)[4])
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr));
+}
+
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a)
+{
+    uint32_t d;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+    return d;
+}
+
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
+{
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
+{
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// Byte offset, inside one 16 x 128 B box written by TMA with the 128-byte
+// swizzle, of 16-byte chunk `chunk` (0..7) of row `row` (0..15).
+__device__ __forceinline__ uint32_t swz(int row, int chunk) { return row * 128 + ((chunk ^ (row & 7)) << 4); }
+
+// ---------------------------------------------------------------- the kernel
+
+struct MmaExtra {
+    // kModeProbe:  checksum [grid] (uint32).  kModeGather: dense K / V rows of one sequence.
+    uint32_t* checksum;
+    __nv_bfloat16* k_out;
+    __nv_bfloat16* v_out;
+    int32_t gather_seq;
+};
+
+template <int D, bool DUP, int MODE>
+__global__ void __launch_bounds__(kMmaThreads) decode_attn_mma_kernel(const KernelParams p,
+                                                                      const __grid_constant__ CUtensorMap k_map,
+                                                                      const __grid_constant__ CUtensorMap v_map,
+                                                                      const int G, const MmaExtra ex)
+{
+    using Cfg = MmaCfg<D>;
+    constexpr int NS = Cfg::kStages;
+    constexpr int KSTEPS = D / 16;
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;             // 1 KB aligned: the swizzle atom
+    uint8_t* const gbase = smem_raw + (base - raw);
+    const uint32_t bar_base = base + NS * Cfg::kStageBytes;   // full[NS], empty[NS]
+    volatile int* const sm_flags = reinterpret_cast<volatile int*>(gbase + NS * Cfg::kStageBytes + 256);
+    int* const sm_ticket = reinterpret_cast<int*>(gbase + NS * Cfg::kStageBytes + 256 + 16);
+
+    const int uid = blockIdx.x;
+    if (uid >= p.header->n_units) return;                     // grid exit: surplus blocks of a capacity launch
+    const decode_attn_unit_t u = load_unit(p.units, uid);
+    if (MODE == kModeGather && u.seq != ex.gather_seq) return;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int b = u.seq, g = u.kv_head;
+
+    int t0 = u.tok_begin, t1 = u.tok_end;
+    if (MODE == kModeAttend) {
+        if (__ldg(p.seq_lens + b) != u.seq_len) {             // Invariant 2: never run on stale lengths
+            if (tid == 0) record_status(p.status, DA_ERR_STALE_PLAN);
+            t1 = t0;
+        }
+        if (p.run_mask != nullptr && __ldg(p.run_mask + b) == 0) t1 = t0;   // masked row reads no KV
+    }
+    const int n_pages = (t1 - t0 + 15) >> 4;
+    const int n_iters = (n_pages + kPagesPerStage - 1) / kPagesPerStage;
+
+    if (tid == 0) {
+        for (int s = 0; s < NS; ++s) {
+            mbar_init(bar_base + 8 * s, 1);                             // full: the producer's expect_tx arrival
+            mbar_init(bar_base + 8 * (NS + s), kMmaConsumerWarps);      // empty: one arrival per consumer warp
+        }
+        sm_flags[0] = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+
+    // per-warp results (consumers only)
+    float oacc[D / 16][4];
+    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+#pragma unroll
+    for (int i = 0; i < D / 16; ++i) oacc[i][0] = oacc[i][1] = oacc[i][2] = oacc[i][3] = 0.f;
+    uint32_t probe_sum = 0;
+
+    if (warp == kMmaConsumerWarps) {
+        // ------------------------------------------------------------ producer
+        const int32_t* bt = p.block_table + (int64_t)b * p.max_pages_per_seq + (t0 >> 4);
+        int ids_next = (lane < n_pages) ? __ldg(bt + lane) : 0;
+        int ids_cur = 0;
+        bool alive = true;
+        for (int it = 0; it < n_iters && alive; ++it) {
+            if ((it & 7) == 0) {                                          // 32 page ids per 8 stages, one batch ahead
+                ids_cur = ids_next;
+                const int nxt = (it + 8) * kPagesPerStage + lane;
+                ids_next = (nxt < n_pages) ? __ldg(bt + nxt) : 0;
+            }
+            const int s = it % NS;
+            const uint32_t parity = ((it / NS) & 1) ^ 1;
+            if (it >= NS) {
+                bool ok = true;
+                if (lane == 0) ok = mbar_wait(bar_base + 8 * (NS + s), parity);
+                ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+                if (!ok) {
+                    if (lane == 0) {
+                        record_status(p.status, DA_ERR_TIMEOUT);
+                        sm_flags[0] = 1;
+                    }
+                    alive = false;
+                    break;
+                }
+            }
+            const int pages_here = min(kPagesPerStage, n_pages - it * kPagesPerStage);
+            const uint32_t full = bar_base + 8 * s;
+            if (lane == 0) mbar_arrive_expect_tx(full, (uint32_t)pages_here * 2u * Cfg::kPageBytes);
+            __syncwarp();
+            // lane j issues one box: page j / (2*halves), tensor (K, V), half of the head dimension
+            constexpr int OPS_PER_PAGE = 2 * Cfg::kHalves;
+            const int pg = lane / OPS_PER_PAGE;
+            const int which = (lane % OPS_PER_PAGE) / Cfg::kHalves;       // 0: K, 1: V
+            const int hf = lane % Cfg::kHalves;
+            int page_id = __shfl_sync(0xffffffffu, ids_cur, ((it & 7) * kPagesPerStage + pg) & 31);
+            if (lane < pages_here * OPS_PER_PAGE) {
+                if ((unsigned)page_id >= (unsigned)p.num_pages) {         // never hand TMA a page outside the pool
+                    record_status(p.status, DA_ERR_BAD_PAGE);
+                    page_id = 0;
+                }
+                const uint32_t dst = base + s * Cfg::kStageBytes + which * Cfg::kTensorBytes + pg * Cfg::kPageBytes +
+                                     hf * Cfg::kBoxBytes;
+                tma_load_4d(dst, which ? &v_map : &k_map, full, hf * 64, 0, g, page_id);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ consumers
+        const int r = lane >> 2, c = lane & 3;
+        // Q^T as B fragments: column n = r is query head (r mod 4 when duplicated)
+        uint32_t qb[KSTEPS][2];
+        if (MODE == kModeAttend) {
+            const int head = DUP ? (r & 3) : r;
+            const bool live = head < G;
+            const uint32_t* qrow = reinterpret_cast<const uint32_t*>(p.q + ((int64_t)b * p.num_q_heads + g * G + (live ? head : 0)) * D);
+#pragma unroll
+            for (int ks = 0; ks < KSTEPS; ++ks) {
+                qb[ks][0] = live ? __ldg(qrow + ks * 8 + c) : 0u;         // dims ks*16 + 2c, +1
+                qb[ks][1] = live ? __ldg(qrow + ks * 8 + 4 + c) : 0u;     // dims ks*16 + 8 + 2c, +1
+            }
+        }
+        const bool lo_role = DUP && (c >= 2);
+        bool alive = true;
+        for (int it = 0; it < n_iters && alive; ++it) {
+            const int s = it % NS;
+            const uint32_t parity = (it / NS) & 1;
+            if (!mbar_wait(bar_base + 8 * s, parity) || sm_flags[0] != 0) {
+                if (lane == 0) {
+                    record_status(p.status, DA_ERR_TIMEOUT);
+                    sm_flags[0] = 1;
+                }
+                alive = false;
+                break;
+            }
+            const int page_idx = it * kPagesPerStage + warp;
+            if (page_idx < n_pages) {
+                const int tok0 = t0 + page_idx * 16;
+                const int n_valid = min(16, t1 - tok0);
+                const uint32_t kpage = base + s * Cfg::kStageBytes + warp * Cfg::kPageBytes;
+                const uint32_t vpage = kpage + Cfg::kTensorBytes;
+                if (MODE == kModeProbe) {
+                    // fold every 16-byte chunk of the page's K and V tiles
+                    for (int i = lane; i < 2 * Cfg::kPageBytes / 16; i += 32) {
+                        const uint32_t a = (i < Cfg::kPageBytes / 16 ? kpage : vpage - Cfg::kPageBytes) + i * 16;
+                        uint32_t x, y, z, w;
+                        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(x), "=r"(y), "=r"(z), "=r"(w) : "r"(a));
+                        probe_sum ^= x ^ y ^ z ^ w;
+                    }
+                } else if (MODE == kModeGather) {
+                    // un-swizzle: token row, 16-byte chunk -> dense [token][head][dim]
+                    for (int i = lane; i < n_valid * (D / 8); i += 32) {
+                        const int row = i / (D / 8), ch = i % (D / 8);
+                        const uint32_t off = (ch >> 3) * Cfg::kBoxBytes + swz(row, ch & 7);
+                        uint4 kv, vv;
+                        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(kv.x), "=r"(kv.y), "=r"(kv.z), "=r"(kv.w) : "r"(kpage + off));
+                        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(vv.x), "=r"(vv.y), "=r"(vv.z), "=r"(vv.w) : "r"(vpage + off));
+                        const int64_t o = ((int64_t)(tok0 + row) * p.num_kv_heads + g) * D + ch * 8;
+                        *reinterpret_cast<uint4*>(ex.k_out + o) = kv;
+                        *reinterpret_cast<uint4*>(ex.v_out + o) = vv;
+                    }
+                } else {
+                    if (n_valid < 16) {
+                        // rows past the sequence end may hold anything (NaN patterns included) and a
+                        // zero weight does not silence them in an mma: clear those V rows
+                        for (int i = lane; i < (16 - n_valid) * (D / 8); i += 32) {
+                            const int row = n_valid + i / (D / 8), ch = i % (D / 8);
+                            const uint32_t a = vpage + (ch >> 3) * Cfg::kBoxBytes + swz(row, ch & 7);
+                            asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0u) : "memory");
+                        }
+                        __syncwarp();
+                    }
+                    // ---- S^T = K . Q^T
+                    float sacc[4] = {0.f, 0.f, 0.f, 0.f};
+                    const int arow = (lane & 7) + ((lane >> 3) & 1) * 8;
+                    const int achk = lane >> 4;
+#pragma unroll
+                    for (int ks = 0; ks < KSTEPS; ++ks) {
+                        uint32_t a[4];
+                        ldsm_x4(kpage + (ks >> 2) * Cfg::kBoxBytes + swz(arow, (ks & 3) * 2 + achk), a);
+                        mma_bf16_16816(sacc, a, qb[ks][0], qb[ks][1]);
+                    }
+                    // ---- online softmax on the fragment: rows r, r+8 (tokens), columns 2c, 2c+1 (heads)
+                    const bool v_lo = r < n_valid, v_hi = (r + 8) < n_valid;
+                    float s00 = v_lo ? sacc[0] * p.scale_log2 : -INFINITY;
+                    float s01 = v_lo ? sacc[1] * p.scale_log2 : -INFINITY;
+                    float s10 = v_hi ? sacc[2] * p.scale_log2 : -INFINITY;
+                    float s11 = v_hi ? sacc[3] * p.scale_log2 : -INFINITY;
+                    float mx0 = fmaxf(s00, s10), mx1 = fmaxf(s01, s11);
+#pragma unroll
+                    for (int off = 4; off <= 16; off <<= 1) {
+                        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, off));
+                        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, off));
+                    }
+                    const float mn0 = fmaxf(m_run[0], mx0), mn1 = fmaxf(m_run[1], mx1);   // finite: token 0 of the page is valid
+                    const float al0 = ex2f(m_run[0] - mn0), al1 = ex2f(m_run[1] - mn1);
+                    m_run[0] = mn0;
+                    m_run[1] = mn1;
+                    const float p00 = ex2f(s00 - mn0), p01 = ex2f(s01 - mn1);
+                    const float p10 = ex2f(s10 - mn0), p11 = ex2f(s11 - mn1);
+                    l_run[0] = fmaf(l_run[0], al0, p00 + p10);
+                    l_run[1] = fmaf(l_run[1], al1, p01 + p11);
+                    if (__any_sync(0xffffffffu, al0 != 1.f || al1 != 1.f)) {
+#pragma unroll
+                        for (int mt = 0; mt < D / 16; ++mt) {
+                            oacc[mt][0] *= al0; oacc[mt][1] *= al1;
+                            oacc[mt][2] *= al0; oacc[mt][3] *= al1;
+                        }
+                    }
+                    // ---- P^T as B fragments (high parts; low parts in the duplicated columns or a second set)
+                    uint32_t hi0 = pack_bf16(p00, p01), hi1 = pack_bf16(p10, p11);
+                    const float r00 = p00 - __uint_as_float(hi0 << 16), r01 = p01 - __uint_as_float(hi0 & 0xffff0000u);
+                    const float r10 = p10 - __uint_as_float(hi1 << 16), r11 = p11 - __uint_as_float(hi1 & 0xffff0000u);
+                    const uint32_t lo0 = pack_bf16(r00, r01), lo1 = pack_bf16(r10, r11);
+                    uint32_t b0, b1, b0l = 0, b1l = 0;
+                    if (DUP) {
+                        b0 = movmatrix_trans(lo_role ? lo0 : hi0);
+                        b1 = movmatrix_trans(lo_role ? lo1 : hi1);
+                    } else {
+                        b0 = movmatrix_trans(hi0);
+                        b1 = movmatrix_trans(hi1);
+                        b0l = movmatrix_trans(lo0);
+                        b1l = movmatrix_trans(lo1);
+                    }
+                    // ---- O^T += V^T . P^T
+                    const int vrow = (lane & 7) + (lane >> 4) * 8;
+                    const int vchk = (lane >> 3) & 1;
+#pragma unroll
+                    for (int mt = 0; mt < D / 16; ++mt) {
+                        uint32_t a[4];
+                        ldsm_x4_trans(vpage + (mt >> 2) * Cfg::kBoxBytes + swz(vrow, (mt & 3) * 2 + vchk), a);
+                        mma_bf16_16816(oacc[mt], a, b0, b1);
+                        if (!DUP) mma_bf16_16816(oacc[mt], a, b0l, b1l);
+                    }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_base + 8 * (NS + s));          // this warp is done with the stage
+        }
+    }
+
+    __syncthreads();   // every issued tile has landed and been consumed: the stage memory is free
+    if (MODE == kModeProbe) {
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) probe_sum ^= __shfl_xor_sync(0xffffffffu, probe_sum, off);
+        if (lane == 0 && warp < kMmaConsumerWarps) atomicXor(ex.checksum + uid, probe_sum);
+        return;
+    }
+    if (MODE == kModeGather) return;
+
+    // ---------------------------------------------------------------- block epilogue
+    // scratch aliases stage memory: per-warp accumulators [4][8][D], then the merged [G][D]
+    float* const sm_wo = reinterpret_cast<float*>(gbase);
+    float* const sm_o = sm_wo + kMmaConsumerWarps * 8 * D;
+    float* const sm_wm = sm_o + 8 * D;                       // [4][8]
+    float* const sm_wl = sm_wm + kMmaConsumerWarps * 8;      // [4][8]
+    float* const sm_m = sm_wl + kMmaConsumerWarps * 8;       // [8]
+    float* const sm_l = sm_m + 8;                            // [8]
+    const bool failed = sm_flags[0] != 0;
+    if (warp < kMmaConsumerWarps) {
+        const int r = lane >> 2, c = lane & 3;
+#pragma unroll
+        for (int off = 4; off <= 16; off <<= 1) {
+            l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], off);
+            l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], off);
+        }
+        if (failed) {
+            m_run[0] = m_run[1] = -INFINITY;
+            l_run[0] = l_run[1] = 0.f;
+        }
+        if (r == 0) {
+            sm_wm[warp * 8 + 2 * c] = m_run[0];
+            sm_wm[warp * 8 + 2 * c + 1] = m_run[1];
+            sm_wl[warp * 8 + 2 * c] = l_run[0];
+            sm_wl[warp * 8 + 2 * c + 1] = l_run[1];
+        }
+        float* wo = sm_wo + warp * 8 * D;
+#pragma unroll
+        for (int mt = 0; mt < D / 16; ++mt) {
+            wo[(2 * c) * D + mt * 16 + r] = oacc[mt][0];
+            wo[(2 * c + 1) * D + mt * 16 + r] = oacc[mt][1];
+            wo[(2 * c) * D + mt * 16 + r + 8] = oacc[mt][2];
+            wo[(2 * c + 1) * D + mt * 16 + r + 8] = oacc[mt][3];
+        }
+    }
+    __syncthreads();
+    for (int e = tid; e < G * D; e += kMmaThreads) {
+        const int h = e / D, d = e % D;
+        float M = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < kMmaConsumerWarps; ++w) M = fmaxf(M, sm_wm[w * 8 + h]);
+        float o = 0.f, ls = 0.f;
+        if (M != -INFINITY) {
+#pragma unroll
+            for (int w = 0; w < kMmaConsumerWarps; ++w) {
+                const float wgt = ex2f(sm_wm[w * 8 + h] - M);             // a warp that saw no page has m = -inf: 0
+                float v = sm_wo[(w * 8 + h) * D + d];
+                if (DUP) v += sm_wo[(w * 8 + h + 4) * D + d];             // low parts of P live in columns 4..7
+                o = fmaf(wgt, v, o);
+                ls = fmaf(wgt, sm_wl[w * 8 + h], ls);
+            }
+        }
+        sm_o[h * D + d] = o;
+        if (d == 0) {
+            sm_m[h] = M;
+            sm_l[h] = ls;
+        }
+    }
+    __syncthreads();
+    finish_unit<D>(p, u, G, sm_o, sm_m, sm_l, sm_ticket, tid, kMmaThreads);
+}
+
+// ---------------------------------------------------------------- host side
+
+inline bool mma_supports(int D, int G) { return (D == 64 || D == 128) && G >= 1 && G <= 8; }
+
+typedef CUresult (*encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+inline encode_tiled_fn get_encode_tiled()
+{
+    static encode_tiled_fn fn = [] {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess) {
+            (void)cudaGetLastError();
+            ptr = nullptr;
+        }
+        return reinterpret_cast<encode_tiled_fn>(ptr);
+    }();
+    return fn;
+}
+
+// 4-D map of one pool: [head_dim, slot, kv head, page]; a box is 64 dims x 16 slots of one head of one page.
+inline int make_pool_map(CUtensorMap* map, const void* pool, const decode_attn_shape_t& s, int64_t stride_page,
+                         int64_t stride_token, int64_t stride_head)
+{
+    encode_tiled_fn enc = get_encode_tiled();
+    if (!enc) return DA_ERR_CUDA;
+    const cuuint64_t dims[4] = {(cuuint64_t)s.head_dim, (cuuint64_t)s.page_size, (cuuint64_t)s.num_kv_heads,
+                                (cuuint64_t)s.num_pages};
+    const cuuint64_t strides[3] = {(cuuint64_t)stride_token * 2, (cuuint64_t)stride_head * 2,
+                                   (cuuint64_t)stride_page * 2};
+    const cuuint32_t box[4] = {64, 16, 1, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(pool), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? DA_OK : DA_ERR_CUDA;
+}
+
+typedef void (*mma_kernel_t)(const KernelParams, const CUtensorMap, const CUtensorMap, const int, const MmaExtra);
+
+template <int MODE>
+inline mma_kernel_t mma_kernel_for(int D, int G)
+{
+    const bool dup = G <= 4;
+    if (D == 128) return dup ? decode_attn_mma_kernel<128, true, MODE> : decode_attn_mma_kernel<128, false, MODE>;
+    if (D == 64) return dup ? decode_attn_mma_kernel<64, true, MODE> : decode_attn_mma_kernel<64, false, MODE>;
+    return nullptr;
+}
+
+inline int mma_smem_bytes(int D) { return D == 128 ? MmaCfg<128>::kSmemBytes : MmaCfg<64>::kSmemBytes; }
+
+template <int MODE>
+inline int mma_prepare(int D, int G, mma_kernel_t* fn_out)
+{
+    mma_kernel_t fn = mma_kernel_for<MODE>(D, G);
+    if (!fn) return DA_ERR_UNSUPPORTED;
+    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, mma_smem_bytes(D)) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return DA_ERR_CUDA;
+    }
+    *fn_out = fn;
+    return DA_OK;
+}
+
+inline int mma_query_occupancy(int D, int G, int* block_threads, int* dyn_smem)
+{
+    mma_kernel_t fn;
+    if (mma_prepare<kModeAttend>(D, G, &fn) != DA_OK) return -1;
+    *block_threads = kMmaThreads;
+    *dyn_smem = mma_smem_bytes(D);
+    int n = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, fn, kMmaThreads, mma_smem_bytes(D)) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return -1;
+    }
+    return n;
+}
+
+template <int MODE>
+inline int mma_launch_mode(const decode_attn_shape_t& s, int G, const KernelParams& kp, const MmaExtra& ex,
+                           unsigned grid, cudaStream_t stream)
+{
+    mma_kernel_t fn;
+    int rc = mma_prepare<MODE>(s.head_dim, G, &fn);
+    if (rc != DA_OK) return rc;
+    CUtensorMap kmap, vmap;
+    rc = make_pool_map(&kmap, kp.k, s, s.k_stride_page, s.k_stride_token, s.k_stride_head);
+    if (rc != DA_OK) return rc;
+    rc = make_pool_map(&vmap, kp.v, s, s.v_stride_page, s.v_stride_token, s.v_stride_head);
+    if (rc != DA_OK) return rc;
+    fn<<<grid, kMmaThreads, mma_smem_bytes(s.head_dim), stream>>>(kp, kmap, vmap, G, ex);
+    if (cudaGetLastError() != cudaSuccess) return DA_ERR_CUDA;
+    return DA_OK;
+}
+
+inline int mma_launch(const decode_attn_shape_t& s, int G, const KernelParams& kp, unsigned grid, cudaStream_t stream)
+{
+    MmaExtra ex = {nullptr, nullptr, nullptr, 0};
+    return mma_launch_mode<kModeAttend>(s, G, kp, ex, grid, stream);
+}
+
+inline int mma_gather_probe(const decode_attn_shape_t& s, int G, const KernelParams& kp, uint32_t* checksum,
+                            unsigned grid, cudaStream_t stream)
+{
+    if (cudaMemsetAsync(checksum, 0, sizeof(uint32_t) * grid, stream) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return DA_ERR_CUDA;
+    }
+    MmaExtra ex = {checksum, nullptr, nullptr, 0};
+    return mma_launch_mode<kModeProbe>(s, G, kp, ex, grid, stream);
+}
+
+inline int mma_debug_gather(const decode_attn_shape_t& s, int G, const KernelParams& kp, int seq, void* k_out,
+                            void* v_out, unsigned grid, cudaStream_t stream)
+{
+    MmaExtra ex = {nullptr, static_cast<__nv_bfloat16*>(k_out), static_cast<__nv_bfloat16*>(v_out), seq};
+    return mma_launch_mode<kModeGather>(s, G, kp, ex, grid, stream);
+}
 
 }  // namespace da
