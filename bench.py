@@ -56,6 +56,8 @@ def parse_args():
     ap.add_argument("--kernel", default="auto", choices=["auto", "simt", "mma"])
     ap.add_argument("--no-fuse", action="store_true", help="separate combine launch")
     ap.add_argument("--no-graph", action="store_true", help="launch every step from the host")
+    ap.add_argument("--partial-only", action="store_true",
+                    help="diagnostic: with --no-fuse, time the partial kernel alone (results are not merged)")
     ap.add_argument("--ctas-per-sm", type=int, default=0)
     ap.add_argument("--skip-cpu", action="store_true", help="leave out the cpu_baseline leg")
     ap.add_argument("--skip-e2e", action="store_true")
@@ -255,7 +257,7 @@ def main():
         w = pools[i % copies]
         da.decode_attn_run(plan, w.q_bits, w.k_pool, w.v_pool, w.block_table, w.seq_lens, out, lse, ws,
                            plan.workspace_bytes)
-        if not policy.fuse_combine:
+        if not policy.fuse_combine and not args.partial_only:
             da.decode_attn_combine(plan, ws, out, lse)
 
     def make_runner(n_steps, first_index):

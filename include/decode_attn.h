@@ -80,7 +80,7 @@ typedef struct {
     int32_t fixed_count;    /* FIXED_COUNT: splits per sequence (>= 1)                               */
     int32_t chunk_tokens;   /* DETERMINISTIC: chunk length, a multiple of page_size (0: 1024).
                                AUTO: smallest chunk the planner may choose (0: 256)                  */
-    int32_t max_splits;     /* upper bound on the splits of one sequence (0: 512)                    */
+    int32_t max_splits;     /* upper bound on the splits of one sequence (0: 512; at most 1024)      */
     int32_t sm_count;       /* 0: the current device's multiprocessor count                          */
     int32_t kernel;         /* da_kernel_t                                                           */
     int32_t fuse_combine;   /* 0: decode_attn_combine must follow decode_attn_run.
@@ -160,7 +160,9 @@ int decode_attn_plan_layout(const decode_attn_shape_t *shape, const decode_attn_
  * planner on seq_lens_host [batch] (host), uploads the work list to a small
  * device buffer the plan owns (synchronously, on an internal stream) and
  * reports the workspace size run/combine need.  *plan_out is set only on
- * DA_OK.  A plan is tied to the CUDA device current at creation and must not
+ * DA_OK.  The device buffer, its pinned mirror and the stream come from a
+ * small cache fed by destroyed plans, so re-planning every step does not
+ * allocate.  A plan is tied to the CUDA device current at creation and must not
  * be used by two launches that overlap on the GPU. */
 int decode_attn_plan(const decode_attn_shape_t *shape, const decode_attn_policy_t *policy,
                      const int32_t *seq_lens_host, decode_attn_plan_t **plan_out,
@@ -278,7 +280,8 @@ int decode_attn_host_step(const decode_attn_shape_t *shape, const decode_attn_po
                           int64_t pool_elems, const int32_t *block_table_host,
                           const int32_t *seq_lens_host, void *out_host, float *lse_host_or_null);
 
-/* Frees the arena decode_attn_host_step keeps. */
+/* Frees what the library caches between calls: the arena of
+ * decode_attn_host_step and the buffers parked by destroyed plans. */
 int decode_attn_host_release(void);
 
 const char *decode_attn_strerror(int status);

@@ -46,19 +46,105 @@ struct decode_attn_plan {
     int64_t max_slots = 0;   // what the workspace is sized for
     int64_t grid = 0;
     size_t workspace_bytes = 0;
-    size_t ws_ml_offset = 0;
-    // device buffer
+    // device buffer (views into the cached allocation the plan holds)
     char* dev = nullptr;
     char* pinned = nullptr;
     size_t upload_bytes = 0;
     size_t off_units = 0, off_seq_info = 0, off_status = 0, off_tickets = 0, total_bytes = 0;
     cudaStream_t stream = nullptr;
     cudaEvent_t upload_done = nullptr;  // last refresh of the device work list
+    void* buffers = nullptr;            // PlanBuffers*, returned to the cache on destroy
 };
 
+#ifdef DA_TRACE
+static unsigned long long* g_trace_buffer = nullptr;
+#endif
 namespace {
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Device buffer, pinned mirror, stream and event of a plan.  Creating these
+// costs far more than planning a step, so destroyed plans park theirs here
+// and the next plan of a similar size picks them up.
+struct PlanBuffers {
+    int device = -1;
+    char* dev = nullptr;
+    char* pinned = nullptr;
+    size_t dev_bytes = 0, pinned_bytes = 0;
+    cudaStream_t stream = nullptr;
+    cudaEvent_t event = nullptr;
+};
+
+void free_buffers(PlanBuffers& b)
+{
+    if (b.stream) {
+        cudaStreamSynchronize(b.stream);
+        cudaStreamDestroy(b.stream);
+    }
+    if (b.event) cudaEventDestroy(b.event);
+    if (b.dev) cudaFree(b.dev);
+    if (b.pinned) cudaFreeHost(b.pinned);
+    (void)cudaGetLastError();
+    b = PlanBuffers();
+}
+
+struct BufferCache {
+    std::mutex mu;
+    std::vector<PlanBuffers> free_list;
+    static constexpr size_t kMaxParked = 8;
+} g_buffers;
+
+size_t round_pow2(size_t x)
+{
+    size_t r = 4096;
+    while (r < x) r <<= 1;
+    return r;
+}
+
+int acquire_buffers(int device, size_t dev_bytes, size_t pinned_bytes, PlanBuffers* out)
+{
+    {
+        std::lock_guard<std::mutex> lock(g_buffers.mu);
+        for (size_t i = 0; i < g_buffers.free_list.size(); ++i) {
+            PlanBuffers& b = g_buffers.free_list[i];
+            if (b.device == device && b.dev_bytes >= dev_bytes && b.pinned_bytes >= pinned_bytes) {
+                *out = b;
+                g_buffers.free_list.erase(g_buffers.free_list.begin() + i);
+                return DA_OK;
+            }
+        }
+    }
+    PlanBuffers b;
+    b.device = device;
+    b.dev_bytes = round_pow2(dev_bytes);
+    b.pinned_bytes = round_pow2(pinned_bytes);
+    if (cudaStreamCreateWithFlags(&b.stream, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&b.event, cudaEventDisableTiming) != cudaSuccess ||
+        cudaMalloc(&b.dev, b.dev_bytes) != cudaSuccess || cudaMallocHost(&b.pinned, b.pinned_bytes) != cudaSuccess) {
+        (void)cudaGetLastError();
+        free_buffers(b);
+        return DA_ERR_CUDA;
+    }
+    *out = b;
+    return DA_OK;
+}
+
+void release_buffers(PlanBuffers& b)
+{
+    if (!b.dev) return;
+    if (b.stream) cudaStreamSynchronize(b.stream);
+    if (b.event) cudaEventSynchronize(b.event);
+    (void)cudaGetLastError();
+    {
+        std::lock_guard<std::mutex> lock(g_buffers.mu);
+        if (g_buffers.free_list.size() < BufferCache::kMaxParked) {
+            g_buffers.free_list.push_back(b);
+            b = PlanBuffers();
+            return;
+        }
+    }
+    free_buffers(b);
+}
 
 typedef void (*simt_kernel_t)(const KernelParams);
 
@@ -136,8 +222,7 @@ KernelParams make_params(const decode_attn_plan_t* pl, const decode_attn_run_arg
     kp.run_mask = a.run_mask;
     kp.out = a.out;
     kp.lse = a.lse;
-    kp.ws_o = static_cast<float*>(a.workspace);
-    kp.ws_ml = reinterpret_cast<float*>(static_cast<char*>(a.workspace) + pl->ws_ml_offset);
+    kp.ws = static_cast<float*>(a.workspace);
     kp.header = reinterpret_cast<const DevHeader*>(pl->dev);
     kp.units = reinterpret_cast<const decode_attn_unit_t*>(pl->dev + pl->off_units);
     kp.seq_info = reinterpret_cast<const SeqInfo*>(pl->dev + pl->off_seq_info);
@@ -152,6 +237,10 @@ KernelParams make_params(const decode_attn_plan_t* pl, const decode_attn_run_arg
     kp.scale_log2 = pl->scale * kLog2e;
     kp.out_bf16 = s.out_dtype == DA_DTYPE_BF16;
     kp.fused = pl->policy.fuse_combine;
+    kp.grid_exit = pl->policy.capacity_batch > 0;
+#ifdef DA_TRACE
+    kp.trace = g_trace_buffer;
+#endif
     return kp;
 }
 
@@ -214,9 +303,7 @@ int decode_attn_plan(const decode_attn_shape_t* shape, const decode_attn_policy_
     }
     if (pl->grid > 0x7fffffffLL) return DA_ERR_UNSUPPORTED;
 
-    const size_t o_bytes = (size_t)pl->max_slots * shape->num_q_heads * shape->head_dim * sizeof(float);
-    pl->ws_ml_offset = align_up(o_bytes, 256);
-    pl->workspace_bytes = pl->max_slots ? pl->ws_ml_offset + (size_t)pl->max_slots * shape->num_q_heads * 2 * sizeof(float) : 0;
+    pl->workspace_bytes = (size_t)pl->max_slots * shape->num_kv_heads * rec_floats(pl->group, shape->head_dim) * sizeof(float);
 
     pl->off_units = align_up(sizeof(DevHeader), 32);
     pl->off_seq_info = pl->off_units + align_up((size_t)std::max<int64_t>(pl->max_units, 1) * sizeof(decode_attn_unit_t), 32);
@@ -226,10 +313,15 @@ int decode_attn_plan(const decode_attn_shape_t* shape, const decode_attn_policy_
     pl->total_bytes = pl->off_tickets +
                       align_up((size_t)std::max<int64_t>(pl->max_batch, 1) * shape->num_kv_heads * sizeof(int32_t), 32);
 
-    DA_CUDA_TRY(cudaStreamCreateWithFlags(&pl->stream, cudaStreamNonBlocking));
-    DA_CUDA_TRY(cudaEventCreateWithFlags(&pl->upload_done, cudaEventDisableTiming));
-    DA_CUDA_TRY(cudaMalloc(&pl->dev, pl->total_bytes));
-    DA_CUDA_TRY(cudaMallocHost(&pl->pinned, pl->upload_bytes));
+    PlanBuffers* pb = new (std::nothrow) PlanBuffers();
+    if (!pb) return DA_ERR_INVALID_ARG;
+    pl->buffers = pb;
+    rc = acquire_buffers(pl->device, pl->total_bytes, pl->upload_bytes, pb);
+    if (rc != DA_OK) return rc;
+    pl->dev = pb->dev;
+    pl->pinned = pb->pinned;
+    pl->stream = pb->stream;
+    pl->upload_done = pb->event;
     std::memset(pl->pinned, 0, pl->upload_bytes);
     fill_host_mirror(pl);
     DA_CUDA_TRY(cudaMemsetAsync(pl->dev + pl->off_status, 0, pl->total_bytes - pl->off_status, pl->stream));
@@ -307,17 +399,11 @@ int decode_attn_plan_check(const decode_attn_plan_t* pl, int32_t batch, const in
 int decode_attn_plan_destroy(decode_attn_plan_t* pl)
 {
     if (!pl) return DA_OK;
-    if (pl->stream) {
-        cudaStreamSynchronize(pl->stream);
-        cudaStreamDestroy(pl->stream);
+    if (pl->buffers) {
+        PlanBuffers* pb = static_cast<PlanBuffers*>(pl->buffers);
+        release_buffers(*pb);
+        delete pb;
     }
-    if (pl->upload_done) {
-        cudaEventSynchronize(pl->upload_done);
-        cudaEventDestroy(pl->upload_done);
-    }
-    if (pl->dev) cudaFree(pl->dev);
-    if (pl->pinned) cudaFreeHost(pl->pinned);
-    (void)cudaGetLastError();
     delete pl;
     return DA_OK;
 }
@@ -464,6 +550,9 @@ int decode_attn_host_release(void)
     g_arena.base = nullptr;
     g_arena.bytes = 0;
     g_arena.device = -1;
+    std::lock_guard<std::mutex> lock2(g_buffers.mu);
+    for (PlanBuffers& b : g_buffers.free_list) free_buffers(b);
+    g_buffers.free_list.clear();
     return DA_OK;
 }
 
@@ -550,5 +639,14 @@ const char* decode_attn_strerror(int status)
 }
 
 const char* decode_attn_version(void) { return "0.1 sm_100a"; }
+
+#ifdef DA_TRACE
+// Debug builds only: device buffer of 32 uint64 stamps per block (NULL switches tracing off).
+int decode_attn_trace_set_buffer(unsigned long long* device_buffer)
+{
+    g_trace_buffer = device_buffer;
+    return DA_OK;
+}
+#endif
 
 }  // extern "C"

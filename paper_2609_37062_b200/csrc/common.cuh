@@ -33,8 +33,7 @@ struct KernelParams {
     const uint8_t* run_mask;
     void* out;
     float* lse;
-    float* ws_o;   // [n_slots][Hq][D]   unnormalised partial outputs
-    float* ws_ml;  // [n_slots][Hq][2]   running max (log2 domain) and sum of exponentials
+    float* ws;     // [n_slots][Hkv] partial records, see rec_floats()
     const DevHeader* header;
     const decode_attn_unit_t* units;
     const SeqInfo* seq_info;
@@ -47,7 +46,32 @@ struct KernelParams {
     float scale_log2;  // sm_scale * log2(e): logits are kept in the base-2 domain
     int32_t out_bf16;
     int32_t fused;
+    int32_t grid_exit;  // capacity plans: blocks at or beyond header->n_units leave at once
+#ifdef DA_TRACE
+    unsigned long long* trace;  // debug builds: 32 stamps per block, or NULL
+#endif
 };
+
+// Optional per-block timeline (builds with -DDA_TRACE only): stamps at a few
+// points of each block.  Compiled out of the product library.
+#ifdef DA_TRACE
+#define DA_TRACE_STAMP(uid, slot)                                                \
+    do {                                                                         \
+        if (p.trace != nullptr) {                                                \
+            unsigned long long t__;                                              \
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t__));              \
+            p.trace[(long long)(uid) * 32 + (slot)] = t__;                       \
+        }                                                                        \
+    } while (0)
+#define DA_TRACE_CLOCK(uid, slot)                                                                         \
+    do {                                                                                                  \
+        if (p.trace != nullptr) p.trace[(long long)(uid) * 32 + (slot)] = (unsigned long long)clock64();  \
+    } while (0)
+#else
+#define DA_TRACE_STAMP(uid, slot) ((void)0)
+#define DA_TRACE_CLOCK(uid, slot) ((void)0)
+#endif
+
 
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kLog2e = 1.4426950408889634f;
@@ -75,7 +99,6 @@ __device__ __forceinline__ decode_attn_unit_t load_unit(const decode_attn_unit_t
     return u;
 }
 
-template <typename T>
 __device__ __forceinline__ void store_out4(void* out, int64_t idx, float4 v, int out_bf16)
 {
     if (out_bf16) {
@@ -90,97 +113,306 @@ __device__ __forceinline__ void store_out4(void* out, int64_t idx, float4 v, int
     }
 }
 
-// LSE merge of the splits of one (sequence, KV head): all G query heads of
-// the group, ascending split order, by `nthreads` threads of one block.  Used
+// ---------------------------------------------------------------- partial records
+//
+// The partial result of one (split, KV head) is one contiguous record:
+// G x D floats of unnormalised output followed by (running max in the log2
+// domain, sum of exponentials) for each of the G heads, padded to 16 bytes so
+// a record can be moved with one bulk copy.  Record r = slot * Hkv + kv_head.
+__host__ __device__ constexpr int rec_floats(int G, int D) { return (G * D + 2 * G + 3) / 4 * 4; }
+
+// Shared memory merge_group needs to stage `cap` records at a time.
+__host__ __device__ constexpr int merge_stage_bytes(int G, int D, int cap)
+{
+    return cap * rec_floats(G, D) * 4 + cap * G * 4 + 64;
+}
+
+// ---------------------------------------------------------------- mbarrier / bulk copy
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+
+__device__ __forceinline__ void mbar_init_fence()
+{
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+constexpr long long kWaitLimitCycles = 2000000000LL;  // about one second
+
+// Bounded wait: false if the phase did not complete within the limit.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if (clock64() - t0 > kWaitLimitCycles) return false;
+    }
+    return true;
+}
+
+// 1-D bulk copy global -> shared, completion counted in bytes on `bar`.
+// Addresses 16-byte aligned, size a multiple of 16.
+__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+
+// ---------------------------------------------------------------- LSE merge
+//
+// Merge of the splits of one (sequence, KV head): all G query heads of the
+// group, ascending split order, by the `nthreads` threads of one block.  Used
 // by the combine kernel and by the last block to finish in a fused launch, so
-// both give the same bits.  Partials are read around L1 (they were written by
-// other SMs in the same launch when fused).
+// both give the same bits.  The records (written by other SMs) are pulled
+// into shared memory `cap` at a time by bulk copies, one per record, issued
+// by as many threads in parallel as there are records (a bulk copy costs its
+// issuer about one round trip to L2); warp w reduces the running maxima of
+// heads w, w + nwarps, ... by shuffles and leaves the weights e^{m_i - M} in
+// shared memory; the accumulation runs split by split in ascending order
+// whatever `cap` is.  `stage`: merge_stage_bytes(G, D, cap) bytes of shared
+// memory, 16-byte aligned, that no thread still reads.  `bar`: an initialised
+// mbarrier (count 1) whose current phase parity is `parity` (updated).
 template <int D>
 __device__ __forceinline__ void merge_group(const KernelParams& p, int b, int g, int G, int slot_base, int S,
-                                            int tid, int nthreads)
+                                            int tid, int nthreads, uint8_t* stage, int cap, uint32_t bar,
+                                            uint32_t& parity)
 {
     constexpr int D4 = D / 4;
-    const int Hq = p.num_q_heads;
-    for (int task = tid; task < G * D4; task += nthreads) {
-        const int h = g * G + task / D4;
-        const int d4 = task % D4;
-        const float2* ml = reinterpret_cast<const float2*>(p.ws_ml) + ((int64_t)slot_base * Hq + h);
-        const float4* po = reinterpret_cast<const float4*>(p.ws_o) + ((int64_t)slot_base * Hq + h) * D4 + d4;
-        float M = -INFINITY;
-        for (int i = 0; i < S; ++i) M = fmaxf(M, __ldcg(ml + (int64_t)i * Hq).x);
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        float lsum = 0.f;
-        if (M != -INFINITY) {
-#pragma unroll 8
-            for (int i = 0; i < S; ++i) {
-                const float2 mli = __ldcg(ml + (int64_t)i * Hq);
-                const float4 o = __ldcg(po + (int64_t)i * Hq * D4);
-                const float w = ex2f(mli.x - M);  // an empty split has m = -inf: w = 0 exactly
-                lsum = fmaf(w, mli.y, lsum);
-                acc.x = fmaf(w, o.x, acc.x);
-                acc.y = fmaf(w, o.y, acc.y);
-                acc.z = fmaf(w, o.z, acc.z);
-                acc.w = fmaf(w, o.w, acc.w);
+    constexpr int kMaxTasks = 2;                        // G * D4 <= 256 tasks over >= 128 threads
+    const int Hq = p.num_q_heads, Hkv = p.num_kv_heads;
+    const int RF = rec_floats(G, D), RF4 = RF / 4;
+    const int GD4 = G * D4;
+    const int lane = tid & 31, warp = tid >> 5, nwarps = nthreads >> 5;
+    float* const st_rec = reinterpret_cast<float*>(stage);          // [cap][RF]
+    float* const st_w = st_rec + (size_t)cap * RF;                  // [cap][G] weights
+    float* const st_M = st_w + cap * G;                             // [8] maxima
+    float* const st_l = st_M + 8;                                   // [8] sums
+    const float* const recs = p.ws + ((int64_t)slot_base * Hkv + g) * RF;
+    const int64_t rec_stride = (int64_t)Hkv * RF;                   // next split of the same KV head
+
+    float4 acc[kMaxTasks];
+#pragma unroll
+    for (int k = 0; k < kMaxTasks; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+    // warp w owns heads w, w + nwarps, ...: lane l keeps the running sum of splits i = l (mod 32)
+    float lpart[2] = {0.f, 0.f};
+
+    for (int i0 = 0; i0 < S; i0 += cap) {
+        const int n = min(cap, S - i0);
+        // The proxy fence orders the generic-proxy accesses made so far (this block's use of the
+        // stage memory, other blocks' record stores seen through the ticket) before the copies.
+        if (tid < n) asm volatile("fence.proxy.async;" ::: "memory");
+        if (tid == 0) mbar_arrive_expect_tx(bar, (uint32_t)(n * RF * 4));
+        for (int j = tid; j < n; j += nthreads)
+            bulk_copy_g2s(smem_u32(st_rec + (size_t)j * RF), recs + (i0 + j) * rec_stride, (uint32_t)(RF * 4), bar);
+        if (i0 == 0 && S > cap) {
+            // several batches: the maximum of every head over ALL splits must be known before the
+            // first weight, so read the maxima from global memory while the first batch flies
+            for (int h = warp; h < G; h += nwarps) {
+                float m = -INFINITY;
+                for (int i = lane; i < S; i += 32) m = fmaxf(m, __ldcg(recs + i * rec_stride + G * D + 2 * h));
+#pragma unroll
+                for (int off = 16; off >= 1; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+                if (lane == 0) st_M[h] = m;
             }
-            const float inv = 1.0f / lsum;
-            acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
         }
-        store_out4<void>(p.out, ((int64_t)b * Hq + h) * D + d4 * 4, acc, p.out_bf16);
-        if (p.lse != nullptr && d4 == 0)
-            p.lse[(int64_t)b * Hq + h] = (M != -INFINITY) ? (M + log2f(lsum)) * kLn2 : -INFINITY;
+        if (!mbar_wait(bar, parity) && tid == 0) record_status(p.status, DA_ERR_TIMEOUT);
+        parity ^= 1u;
+        if (S <= cap) {
+            // one batch: every record is here, take the maxima from shared memory
+            for (int h = warp; h < G; h += nwarps) {
+                float m = -INFINITY;
+                for (int j = lane; j < n; j += 32) m = fmaxf(m, st_rec[(size_t)j * RF + G * D + 2 * h]);
+#pragma unroll
+                for (int off = 16; off >= 1; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+                if (lane == 0) st_M[h] = m;
+            }
+        }
+        __syncthreads();
+        // weights e^{m_i - M} once per (split, head); the head's sum of w_i * l_i alongside
+        {
+            int k = 0;
+            for (int h = warp; h < G; h += nwarps, ++k) {
+                const float M = st_M[h];
+                // lane l takes the splits with global index i = l (mod 32), whatever the batching
+                for (int j = (lane - i0) & 31; j < n; j += 32) {
+                    const float2 ml = *reinterpret_cast<const float2*>(st_rec + (size_t)j * RF + G * D + 2 * h);
+                    const float w = (M == -INFINITY) ? 0.f : ex2f(ml.x - M);   // empty split: m = -inf, w = 0
+                    st_w[j * G + h] = w;
+                    lpart[k] = fmaf(w, ml.y, lpart[k]);
+                }
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int k = 0; k < kMaxTasks; ++k) {
+            const int task = tid + k * nthreads;
+            if (task < GD4) {
+                const int h = task / D4;
+                const float4* o = reinterpret_cast<const float4*>(st_rec) + task;
+                const float* wp = st_w + h;
+                float4 a4 = acc[k];
+                int j = 0;
+                for (; j + 4 <= n; j += 4) {       // four records in flight; the sums stay in split order
+                    const float w0 = wp[j * G], w1 = wp[(j + 1) * G], w2 = wp[(j + 2) * G], w3 = wp[(j + 3) * G];
+                    const float4 v0 = o[j * RF4], v1 = o[(j + 1) * RF4], v2 = o[(j + 2) * RF4], v3 = o[(j + 3) * RF4];
+                    a4.x = fmaf(w3, v3.x, fmaf(w2, v2.x, fmaf(w1, v1.x, fmaf(w0, v0.x, a4.x))));
+                    a4.y = fmaf(w3, v3.y, fmaf(w2, v2.y, fmaf(w1, v1.y, fmaf(w0, v0.y, a4.y))));
+                    a4.z = fmaf(w3, v3.z, fmaf(w2, v2.z, fmaf(w1, v1.z, fmaf(w0, v0.z, a4.z))));
+                    a4.w = fmaf(w3, v3.w, fmaf(w2, v2.w, fmaf(w1, v1.w, fmaf(w0, v0.w, a4.w))));
+                }
+                for (; j < n; ++j) {
+                    const float w = wp[j * G];
+                    const float4 v = o[j * RF4];
+                    a4.x = fmaf(w, v.x, a4.x);
+                    a4.y = fmaf(w, v.y, a4.y);
+                    a4.z = fmaf(w, v.z, a4.z);
+                    a4.w = fmaf(w, v.w, a4.w);
+                }
+                acc[k] = a4;
+            }
+        }
+        __syncthreads();
+    }
+    // the heads' sums: a fixed butterfly over the 32 lane partials
+    {
+        int k = 0;
+        for (int h = warp; h < G; h += nwarps, ++k) {
+            float l = lpart[k];
+#pragma unroll
+            for (int off = 16; off >= 1; off >>= 1) l += __shfl_xor_sync(0xffffffffu, l, off);
+            if (lane == 0) st_l[h] = l;
+        }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < kMaxTasks; ++k) {
+        const int task = tid + k * nthreads;
+        if (task < GD4) {
+            const int h = task / D4, d4 = task % D4;
+            const float M = st_M[h], ls = st_l[h];
+            float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (M != -INFINITY && ls > 0.f) {
+                const float inv = 1.0f / ls;
+                o = make_float4(acc[k].x * inv, acc[k].y * inv, acc[k].z * inv, acc[k].w * inv);
+            }
+            store_out4(p.out, ((int64_t)b * Hq + g * G + h) * D + d4 * 4, o, p.out_bf16);
+            if (p.lse != nullptr && d4 == 0)
+                p.lse[(int64_t)b * Hq + g * G + h] = (M != -INFINITY && ls > 0.f) ? (M + log2f(ls)) * kLn2 : -INFINITY;
+        }
     }
 }
 
-// End of a unit.  sm_o [G][D] holds the block's unnormalised accumulator,
-// sm_m [G] its running max (log2 domain, -inf if nothing was attended) and
-// sm_l [G] its sum of exponentials; all threads of the block call this after
-// a __syncthreads() that made those visible.
-template <int D>
-__device__ __forceinline__ void finish_unit(const KernelParams& p, const decode_attn_unit_t& u, int G,
-                                            const float* sm_o, const float* sm_m, const float* sm_l,
-                                            int* sm_ticket, int tid, int nthreads)
+// ---------------------------------------------------------------- end of a unit
+//
+// The block's R partial states (one per warp or row group) sit in shared
+// memory: src_o [R][COLS][D] unnormalised accumulators, src_m / src_l
+// [R][COLS] running maxima (log2 domain, -inf if nothing was attended) and
+// sums.  With DUP, columns h and h + 4 hold the high and low parts of the
+// same head and are added.  All threads call this after a __syncthreads()
+// that made the sources visible.  The states are merged in the fixed order
+// r = 0..R-1 and the result goes straight to `out` (single split) or to the
+// unit's record; with a fused plan the block then draws a ticket and, if it
+// is the last of its (sequence, KV head), merges all records.  `stage` /
+// `cap`: shared memory the merge may overwrite (it may alias the sources).
+template <int D, int R, int COLS, bool DUP>
+__device__ __forceinline__ void block_finish(const KernelParams& p, const decode_attn_unit_t& u, int G,
+                                             const float* src_o, const float* src_m, const float* src_l,
+                                             int* sm_ticket, uint32_t merge_bar, int tid, int nthreads,
+                                             uint8_t* stage, int cap)
 {
     constexpr int D4 = D / 4;
+    constexpr int kUnroll = R <= 4 ? R : 1;     // many row groups: keep the loop rolled, registers matter more
     const int Hq = p.num_q_heads;
     const int h0 = u.kv_head * G;
-    if (u.slot < 0) {
-        for (int task = tid; task < G * D4; task += nthreads) {
-            const int h = task / D4, d4 = task % D4;
-            const float l = sm_l[h];
-            float4 o = reinterpret_cast<const float4*>(sm_o)[h * D4 + d4];
-            if (l > 0.f) {
-                const float inv = 1.0f / l;
+    const int RF = rec_floats(G, D);
+    float* const rec = (u.slot >= 0) ? p.ws + ((int64_t)u.slot * p.num_kv_heads + u.kv_head) * RF : nullptr;
+    for (int task = tid; task < G * D4; task += nthreads) {
+        const int h = task / D4, d4 = task % D4;
+        float M = -INFINITY;
+#pragma unroll kUnroll
+        for (int r = 0; r < R; ++r) M = fmaxf(M, src_m[r * COLS + h]);
+        float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+        float ls = 0.f;
+        if (M != -INFINITY) {
+#pragma unroll kUnroll
+            for (int r = 0; r < R; ++r) {
+                const float w = ex2f(src_m[r * COLS + h] - M);          // a source that saw nothing: w = 0
+                float4 v = reinterpret_cast<const float4*>(src_o)[(r * COLS + h) * D4 + d4];
+                if (DUP) {
+                    const float4 v2 = reinterpret_cast<const float4*>(src_o)[(r * COLS + h + 4) * D4 + d4];
+                    v.x += v2.x; v.y += v2.y; v.z += v2.z; v.w += v2.w;
+                }
+                o.x = fmaf(w, v.x, o.x);
+                o.y = fmaf(w, v.y, o.y);
+                o.z = fmaf(w, v.z, o.z);
+                o.w = fmaf(w, v.w, o.w);
+                ls = fmaf(w, src_l[r * COLS + h], ls);
+            }
+        }
+        if (rec == nullptr) {
+            if (ls > 0.f) {
+                const float inv = 1.0f / ls;
                 o.x *= inv; o.y *= inv; o.z *= inv; o.w *= inv;
             } else {
                 o = make_float4(0.f, 0.f, 0.f, 0.f);
             }
-            store_out4<void>(p.out, ((int64_t)u.seq * Hq + h0 + h) * D + d4 * 4, o, p.out_bf16);
+            store_out4(p.out, ((int64_t)u.seq * Hq + h0 + h) * D + d4 * 4, o, p.out_bf16);
+            if (p.lse != nullptr && d4 == 0)
+                p.lse[(int64_t)u.seq * Hq + h0 + h] = (ls > 0.f) ? (M + log2f(ls)) * kLn2 : -INFINITY;
+        } else {
+            __stcg(reinterpret_cast<float4*>(rec) + task, o);
+            if (d4 == 0) __stcg(reinterpret_cast<float2*>(rec + G * D) + h, make_float2(M, ls));
         }
-        if (p.lse != nullptr && tid < G) {
-            const float l = sm_l[tid];
-            p.lse[(int64_t)u.seq * Hq + h0 + tid] = (l > 0.f) ? (sm_m[tid] + log2f(l)) * kLn2 : -INFINITY;
-        }
-        return;
     }
-    for (int task = tid; task < G * D4; task += nthreads) {
-        const int h = task / D4, d4 = task % D4;
-        reinterpret_cast<float4*>(p.ws_o)[((int64_t)u.slot * Hq + h0 + h) * D4 + d4] =
-            reinterpret_cast<const float4*>(sm_o)[h * D4 + d4];
-    }
-    if (tid < G)
-        reinterpret_cast<float2*>(p.ws_ml)[(int64_t)u.slot * Hq + h0 + tid] = make_float2(sm_m[tid], sm_l[tid]);
-    if (!p.fused) return;
-    // Ticket: nobody waits.  The block that draws the last ticket of its
-    // (sequence, KV head) sees every other block's partials (fence before
-    // the ticket, fence after) and merges them in ascending split order.
-    __threadfence();
+    if (rec == nullptr || !p.fused) return;
+    // Ticket: nobody waits.  The block barrier orders every thread's record
+    // stores before thread 0's fence, which publishes them device-wide ahead
+    // of the ticket; the block that draws the last ticket of its (sequence,
+    // KV head) therefore sees all the other records.
     __syncthreads();
+    if (tid == 0) DA_TRACE_CLOCK(blockIdx.x, 13);
     int32_t* ticket = p.tickets + (int64_t)u.seq * p.num_kv_heads + u.kv_head;
-    if (tid == 0) *sm_ticket = atomicAdd(ticket, 1);
+    if (tid == 0) {
+        __threadfence();
+        *sm_ticket = atomicAdd(ticket, 1);
+        __threadfence();
+    }
     __syncthreads();
+    if (tid == 0) DA_TRACE_CLOCK(blockIdx.x, 14);
     if (*sm_ticket != u.n_splits - 1) return;
-    __threadfence();
-    merge_group<D>(p, u.seq, u.kv_head, G, u.slot - u.split_index, u.n_splits, tid, nthreads);
+    uint32_t parity = 0;
+    merge_group<D>(p, u.seq, u.kv_head, G, u.slot - u.split_index, u.n_splits, tid, nthreads, stage, cap, merge_bar,
+                   parity);
+    if (tid == 0) DA_TRACE_CLOCK(blockIdx.x, 19);
     if (tid == 0) *ticket = 0;  // ready for the next launch
 }
 

@@ -39,7 +39,6 @@ namespace da {
 constexpr int kMmaConsumerWarps = 4;
 constexpr int kMmaThreads = (kMmaConsumerWarps + 1) * 32;
 constexpr int kPagesPerStage = kMmaConsumerWarps;
-constexpr long long kWaitLimitCycles = 2000000000LL;  // about one second
 
 enum MmaMode { kModeAttend = 0, kModeProbe = 1, kModeGather = 2 };
 
@@ -57,54 +56,29 @@ struct MmaCfg {
 
 // ---------------------------------------------------------------- PTX wrappers
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-
-// Bounded wait: false if the phase did not complete within the limit.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
-{
-    if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    while (!mbar_try_wait(bar, parity)) {
-        if (clock64() - t0 > kWaitLimitCycles) return false;
-    }
-    return true;
-}
-
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
-                                            int c2, int c3)
+                                            int c2, int c3, uint64_t l2_policy)
 {
     asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1, {%3, %4, %5, %6}], [%2], %7;"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "l"(l2_policy)
         : "memory");
+}
+
+__device__ __forceinline__ void tma_prefetch_descriptor(const CUtensorMap* map)
+{
+    asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+
+// K/V bytes are read once per step: mark their L2 lines first in line for
+// eviction so the stream does not push out the work list, block tables,
+// partial records and instructions that are reused.
+__device__ __forceinline__ uint64_t l2_policy_evict_first()
+{
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
 }
 
 __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4])
@@ -170,38 +144,44 @@ __global__ void __launch_bounds__(kMmaThreads) decode_attn_mma_kernel(const Kern
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;             // 1 KB aligned: the swizzle atom
     uint8_t* const gbase = smem_raw + (base - raw);
-    const uint32_t bar_base = base + NS * Cfg::kStageBytes;   // full[NS], empty[NS]
+    const uint32_t bar_base = base + NS * Cfg::kStageBytes;   // full[NS], empty[NS], merge
     volatile int* const sm_flags = reinterpret_cast<volatile int*>(gbase + NS * Cfg::kStageBytes + 256);
     int* const sm_ticket = reinterpret_cast<int*>(gbase + NS * Cfg::kStageBytes + 256 + 16);
 
     const int uid = blockIdx.x;
-    if (uid >= p.header->n_units) return;                     // grid exit: surplus blocks of a capacity launch
+    if (p.grid_exit && uid >= p.header->n_units) return;      // surplus blocks of a capacity launch
     const decode_attn_unit_t u = load_unit(p.units, uid);
     if (MODE == kModeGather && u.seq != ex.gather_seq) return;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = u.seq, g = u.kv_head;
+    if (tid == 0) DA_TRACE_STAMP(uid, 0);
 
-    int t0 = u.tok_begin, t1 = u.tok_end;
+    const int t0 = u.tok_begin;
+    int t1 = u.tok_end;
+    // Invariant 2 (never run on stale lengths): the device length is fetched now and compared
+    // in the epilogue, off the critical path; a mismatch voids the block's result.  Reads stay
+    // inside the planned range and page ids are range-checked, so nothing can fault meanwhile.
+    int dev_len = u.seq_len;
     if (MODE == kModeAttend) {
-        if (__ldg(p.seq_lens + b) != u.seq_len) {             // Invariant 2: never run on stale lengths
-            if (tid == 0) record_status(p.status, DA_ERR_STALE_PLAN);
-            t1 = t0;
-        }
+        dev_len = __ldg(p.seq_lens + b);
         if (p.run_mask != nullptr && __ldg(p.run_mask + b) == 0) t1 = t0;   // masked row reads no KV
     }
     const int n_pages = (t1 - t0 + 15) >> 4;
     const int n_iters = (n_pages + kPagesPerStage - 1) / kPagesPerStage;
 
     if (tid == 0) {
+        tma_prefetch_descriptor(&k_map);
+        tma_prefetch_descriptor(&v_map);
         for (int s = 0; s < NS; ++s) {
             mbar_init(bar_base + 8 * s, 1);                             // full: the producer's expect_tx arrival
             mbar_init(bar_base + 8 * (NS + s), kMmaConsumerWarps);      // empty: one arrival per consumer warp
         }
+        mbar_init(bar_base + 8 * 2 * NS, 1);                            // the in-kernel merge's copies
         sm_flags[0] = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        mbar_init_fence();
     }
     __syncthreads();
+    if (tid == 0) DA_TRACE_STAMP(uid, 1);
 
     // per-warp results (consumers only)
     float oacc[D / 16][4];
@@ -216,6 +196,7 @@ __global__ void __launch_bounds__(kMmaThreads) decode_attn_mma_kernel(const Kern
         int ids_next = (lane < n_pages) ? __ldg(bt + lane) : 0;
         int ids_cur = 0;
         bool alive = true;
+        const uint64_t l2_policy = l2_policy_evict_first();
         for (int it = 0; it < n_iters && alive; ++it) {
             if ((it & 7) == 0) {                                          // 32 page ids per 8 stages, one batch ahead
                 ids_cur = ids_next;
@@ -254,7 +235,8 @@ __global__ void __launch_bounds__(kMmaThreads) decode_attn_mma_kernel(const Kern
                 }
                 const uint32_t dst = base + s * Cfg::kStageBytes + which * Cfg::kTensorBytes + pg * Cfg::kPageBytes +
                                      hf * Cfg::kBoxBytes;
-                tma_load_4d(dst, which ? &v_map : &k_map, full, hf * 64, 0, g, page_id);
+                tma_load_4d(dst, which ? &v_map : &k_map, full, hf * 64, 0, g, page_id, l2_policy);
+                if (it == 0 && lane == 0) DA_TRACE_STAMP(uid, 2);
             }
         }
     } else {
@@ -285,6 +267,7 @@ __global__ void __launch_bounds__(kMmaThreads) decode_attn_mma_kernel(const Kern
                 alive = false;
                 break;
             }
+            if (it == 0 && tid == 0) DA_TRACE_STAMP(uid, 3);
             const int page_idx = it * kPagesPerStage + warp;
             if (page_idx < n_pages) {
                 const int tok0 = t0 + page_idx * 16;
@@ -391,6 +374,7 @@ __global__ void __launch_bounds__(kMmaThreads) decode_attn_mma_kernel(const Kern
         }
     }
 
+    if (tid == 0) DA_TRACE_STAMP(uid, 4);
     __syncthreads();   // every issued tile has landed and been consumed: the stage memory is free
     if (MODE == kModeProbe) {
 #pragma unroll
@@ -401,14 +385,15 @@ __global__ void __launch_bounds__(kMmaThreads) decode_attn_mma_kernel(const Kern
     if (MODE == kModeGather) return;
 
     // ---------------------------------------------------------------- block epilogue
-    // scratch aliases stage memory: per-warp accumulators [4][8][D], then the merged [G][D]
+    // scratch aliases stage memory: the four warps' accumulators [4][8][D], maxima and sums [4][8]
     float* const sm_wo = reinterpret_cast<float*>(gbase);
-    float* const sm_o = sm_wo + kMmaConsumerWarps * 8 * D;
-    float* const sm_wm = sm_o + 8 * D;                       // [4][8]
-    float* const sm_wl = sm_wm + kMmaConsumerWarps * 8;      // [4][8]
-    float* const sm_m = sm_wl + kMmaConsumerWarps * 8;       // [8]
-    float* const sm_l = sm_m + 8;                            // [8]
-    const bool failed = sm_flags[0] != 0;
+    float* const sm_wm = sm_wo + kMmaConsumerWarps * 8 * D;
+    float* const sm_wl = sm_wm + kMmaConsumerWarps * 8;
+    bool failed = sm_flags[0] != 0;
+    if (dev_len != u.seq_len) {                               // stale plan: void the result, report it
+        if (tid == 0) record_status(p.status, DA_ERR_STALE_PLAN);
+        failed = true;
+    }
     if (warp < kMmaConsumerWarps) {
         const int r = lane >> 2, c = lane & 3;
 #pragma unroll
@@ -436,30 +421,10 @@ __global__ void __launch_bounds__(kMmaThreads) decode_attn_mma_kernel(const Kern
         }
     }
     __syncthreads();
-    for (int e = tid; e < G * D; e += kMmaThreads) {
-        const int h = e / D, d = e % D;
-        float M = -INFINITY;
-#pragma unroll
-        for (int w = 0; w < kMmaConsumerWarps; ++w) M = fmaxf(M, sm_wm[w * 8 + h]);
-        float o = 0.f, ls = 0.f;
-        if (M != -INFINITY) {
-#pragma unroll
-            for (int w = 0; w < kMmaConsumerWarps; ++w) {
-                const float wgt = ex2f(sm_wm[w * 8 + h] - M);             // a warp that saw no page has m = -inf: 0
-                float v = sm_wo[(w * 8 + h) * D + d];
-                if (DUP) v += sm_wo[(w * 8 + h + 4) * D + d];             // low parts of P live in columns 4..7
-                o = fmaf(wgt, v, o);
-                ls = fmaf(wgt, sm_wl[w * 8 + h], ls);
-            }
-        }
-        sm_o[h * D + d] = o;
-        if (d == 0) {
-            sm_m[h] = M;
-            sm_l[h] = ls;
-        }
-    }
-    __syncthreads();
-    finish_unit<D>(p, u, G, sm_o, sm_m, sm_l, sm_ticket, tid, kMmaThreads);
+    const int cap = (NS * Cfg::kStageBytes - 64 - 4 * G) / (rec_floats(G, D) * 4 + 4 * G);
+    block_finish<D, kMmaConsumerWarps, 8, DUP>(p, u, G, sm_wo, sm_wm, sm_wl, sm_ticket, bar_base + 8 * 2 * NS, tid,
+                                               kMmaThreads, gbase, cap);
+    if (tid == 0) DA_TRACE_STAMP(uid, 6);
 }
 
 // ---------------------------------------------------------------- host side

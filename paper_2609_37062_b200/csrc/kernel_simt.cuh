@@ -46,28 +46,34 @@ __global__ void __launch_bounds__(kSimtThreads) decode_attn_simt_kernel(const Ke
     constexpr int ROWS = kSimtWarps * RPW;      // row groups per block
     constexpr int U = 4;                        // rows in flight per thread
 
-    __shared__ __align__(16) float sm_acc[ROWS][G][D];
-    __shared__ float sm_rm[ROWS][G];
-    __shared__ float sm_rl[ROWS][G];
-    __shared__ __align__(16) float sm_o[G][D];
-    __shared__ float sm_m[G];
-    __shared__ float sm_l[G];
+    // one raw block so the in-kernel merge can reuse it as its staging area
+    constexpr int kOwnBytes = ROWS * G * D * 4 + 2 * ROWS * G * 4;
+    constexpr int kRawBytes = kOwnBytes > merge_stage_bytes(G, D, ROWS) ? kOwnBytes : merge_stage_bytes(G, D, ROWS);
+    __shared__ __align__(16) uint8_t sm_raw[kRawBytes];
+    float (*sm_acc)[G][D] = reinterpret_cast<float (*)[G][D]>(sm_raw);
+    float (*sm_rm)[G] = reinterpret_cast<float (*)[G]>(sm_raw + ROWS * G * D * 4);
+    float (*sm_rl)[G] = reinterpret_cast<float (*)[G]>(sm_raw + ROWS * G * D * 4 + ROWS * G * 4);
+    __shared__ __align__(8) uint64_t sm_merge_bar;
     __shared__ int sm_ticket;
 
     const int uid = blockIdx.x;
-    if (uid >= p.header->n_units) return;       // grid exit: surplus blocks of a capacity launch
+    if (p.grid_exit && uid >= p.header->n_units) return;   // surplus blocks of a capacity launch
     const decode_attn_unit_t u = load_unit(p.units, uid);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int rg = warp * RPW + lane / LPR;     // row group of this thread
     const int li = lane % LPR;                  // 8-dim slice within the row
     const int b = u.seq, g = u.kv_head;
 
-    int t0 = u.tok_begin, t1 = u.tok_end;
-    if (__ldg(p.seq_lens + b) != u.seq_len) {   // Invariant 2: never run on stale lengths
-        if (tid == 0) record_status(p.status, DA_ERR_STALE_PLAN);
-        t1 = t0;
-    }
+    const int t0 = u.tok_begin;
+    int t1 = u.tok_end;
+    // Invariant 2 (never run on stale lengths): fetched now, compared in the epilogue so the
+    // load stays off the critical path; page ids are range-checked, so nothing can fault.
+    const int dev_len = __ldg(p.seq_lens + b);
     if (p.run_mask != nullptr && __ldg(p.run_mask + b) == 0) t1 = t0;   // masked row reads no KV
+    if (tid == 0) {
+        mbar_init(smem_u32(&sm_merge_bar), 1);
+        mbar_init_fence();
+    }
 
     float qf[G][8];
 #pragma unroll
@@ -164,7 +170,15 @@ __global__ void __launch_bounds__(kSimtThreads) decode_attn_simt_kernel(const Ke
         }
     }
 
-    // merge the row groups of the block in a fixed order
+    // the row groups' states go to shared memory; block_finish merges them in a fixed order
+    if (dev_len != u.seq_len) {                 // stale plan: void the result, report it
+        if (tid == 0) record_status(p.status, DA_ERR_STALE_PLAN);
+#pragma unroll
+        for (int h = 0; h < G; ++h) {
+            m[h] = -INFINITY;
+            l[h] = 0.f;
+        }
+    }
 #pragma unroll
     for (int h = 0; h < G; ++h) {
         if (li == 0) {
@@ -176,28 +190,8 @@ __global__ void __launch_bounds__(kSimtThreads) decode_attn_simt_kernel(const Ke
         dst[1] = make_float4(acc[h][4], acc[h][5], acc[h][6], acc[h][7]);
     }
     __syncthreads();
-    for (int e = tid; e < G * D; e += kSimtThreads) {
-        const int h = e / D, d = e % D;
-        float M = -INFINITY;
-#pragma unroll
-        for (int r = 0; r < ROWS; ++r) M = fmaxf(M, sm_rm[r][h]);
-        float o = 0.f, ls = 0.f;
-        if (M != -INFINITY) {
-#pragma unroll
-            for (int r = 0; r < ROWS; ++r) {
-                const float w = ex2f(sm_rm[r][h] - M);
-                o = fmaf(w, sm_acc[r][h][d], o);
-                ls = fmaf(w, sm_rl[r][h], ls);
-            }
-        }
-        sm_o[h][d] = o;
-        if (d == 0) {
-            sm_m[h] = M;
-            sm_l[h] = ls;
-        }
-    }
-    __syncthreads();
-    finish_unit<D>(p, u, G, &sm_o[0][0], sm_m, sm_l, &sm_ticket, tid, kSimtThreads);
+    block_finish<D, ROWS, G, false>(p, u, G, &sm_acc[0][0][0], &sm_rm[0][0], &sm_rl[0][0], &sm_ticket,
+                                    smem_u32(&sm_merge_bar), tid, kSimtThreads, sm_raw, ROWS);
 }
 
 }  // namespace da

@@ -60,6 +60,8 @@ int validate_policy(const decode_attn_shape_t& s, const decode_attn_policy_t& p)
         p.capacity_batch < 0 || p.capacity_tokens < 0)
         return DA_ERR_INVALID_ARG;
     if (p.chunk_tokens % s.page_size != 0) return DA_ERR_INVALID_ARG;
+    if (p.max_splits > kMaxSplits || (p.split_mode == DA_SPLIT_FIXED_COUNT && p.fixed_count > kMaxSplits))
+        return DA_ERR_INVALID_ARG;
     if (p.fuse_combine != 0 && p.fuse_combine != 1) return DA_ERR_INVALID_ARG;
     if (p.capacity_batch > 0 && (p.capacity_tokens <= 0 || s.batch > p.capacity_batch))
         return DA_ERR_INVALID_ARG;

@@ -12,6 +12,7 @@ namespace da {
 constexpr int kDefaultDeterministicChunk = 1024;  // tokens
 constexpr int kDefaultAutoMinChunk = 256;         // tokens
 constexpr int kDefaultMaxSplits = 512;
+constexpr int kMaxSplits = 1024;  // hard bound on the splits of one sequence
 constexpr int kMaxGroup = 8;
 
 struct Layout {
