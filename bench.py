@@ -4,8 +4,9 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
 
 A step is one pass of the whole path over one batch: the split-KV partial
-kernel and the LSE merge (fused into the same launch by default) over every
-sequence of the workload.  The default workload is the single long sequence
+kernel and the LSE combine kernel (launched with a programmatic dependency on
+it; --fuse merges inside the partial kernel instead) over every sequence of
+the workload.  The default workload is the single long sequence
 (batch 1, 32 query / 8 KV heads, head_dim 128, page 16, 32,768 tokens); the
 metric is KV-read GB/s = logical K+V bytes of the batch / time per step.
 
@@ -54,10 +55,11 @@ def parse_args():
     ap.add_argument("--split", default="auto", choices=["auto", "deterministic"])
     ap.add_argument("--chunk-tokens", type=int, default=0)
     ap.add_argument("--kernel", default="auto", choices=["auto", "simt", "mma"])
-    ap.add_argument("--no-fuse", action="store_true", help="separate combine launch")
+    ap.add_argument("--fuse", action="store_true",
+                    help="merge inside the partial kernel (one launch per step) instead of the combine kernel")
     ap.add_argument("--no-graph", action="store_true", help="launch every step from the host")
     ap.add_argument("--partial-only", action="store_true",
-                    help="diagnostic: with --no-fuse, time the partial kernel alone (results are not merged)")
+                    help="diagnostic: time the partial kernel alone (results are not merged)")
     ap.add_argument("--ctas-per-sm", type=int, default=0)
     ap.add_argument("--skip-cpu", action="store_true", help="leave out the cpu_baseline leg")
     ap.add_argument("--skip-e2e", action="store_true")
@@ -241,7 +243,7 @@ def main():
     kernel = {"auto": da.DA_KERNEL_AUTO, "simt": da.DA_KERNEL_SIMT, "mma": da.DA_KERNEL_MMA_TMA}[args.kernel]
     policy = da.make_policy(
         split_mode=da.DA_SPLIT_DETERMINISTIC if args.split == "deterministic" else da.DA_SPLIT_AUTO,
-        chunk_tokens=args.chunk_tokens, kernel=kernel, fuse_combine=0 if args.no_fuse else 1,
+        chunk_tokens=args.chunk_tokens, kernel=kernel, fuse_combine=1 if args.fuse else 0,
         ctas_per_sm=args.ctas_per_sm)
     shape = da.shape_of_workload(first)
     t0 = time.perf_counter()
@@ -394,7 +396,7 @@ def main():
 
     if rank == 0:
         peak, peak_kind = peak_hbm()
-        achieved = kv_bytes / sec_per_step / 1e9 if launches_per_step == 1 else None
+        achieved = kv_bytes / sec_per_step / 1e9
         kname = {da.DA_KERNEL_SIMT: "decode_attn_simt_kernel", da.DA_KERNEL_MMA_TMA: "decode_attn_mma_kernel"}[info.kernel]
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -415,7 +417,8 @@ def main():
                          "frac": (achieved / peak) if achieved else None, "peak_kind": f"of {peak_kind}",
                          "kernel": kname, "traffic": NCU_TRAFFIC_BYTES.get(args.workload),
                          "algorithmic_bytes_per_launch": kv_bytes,
-                         "how": "logical K+V bytes of the batch / (event time of the timed region / launches)"},
+                         "how": "logical K+V bytes of the batch / (event time of the timed region / steps): the "
+                                "step's combine launch and launch gaps are charged to the partial kernel"},
             "gpu_launches": args.steps * launches_per_step,
             "clocks": clocks,
             "e2e": e2e,

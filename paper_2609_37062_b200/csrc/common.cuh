@@ -113,6 +113,15 @@ __device__ __forceinline__ void store_out4(void* out, int64_t idx, float4 v, int
     }
 }
 
+// ---------------------------------------------------------------- programmatic dependent launch
+//
+// The partial kernel lets the grid launched after it (the combine kernel)
+// start being scheduled once every block is past its main loop; that grid
+// still waits, at its top, for this one to finish and flush.  Both are no-ops
+// when the launches carry no programmatic dependency.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait_primary() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // ---------------------------------------------------------------- partial records
 //
 // The partial result of one (split, KV head) is one contiguous record:
@@ -192,13 +201,16 @@ __device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uin
 // Merge of the splits of one (sequence, KV head): all G query heads of the
 // group, ascending split order, by the `nthreads` threads of one block.  Used
 // by the combine kernel and by the last block to finish in a fused launch, so
-// both give the same bits.  The records (written by other SMs) are pulled
+// both give the same bits: every output column is the sum of four chains,
+// chain k taking the splits with index k (mod 4) in ascending order, added as
+// ((c0 + c1) + c2) + c3; the sums of exponentials follow the same scheme.
+// The records (written by other SMs) are pulled
 // into shared memory `cap` at a time by bulk copies, one per record, issued
 // by as many threads in parallel as there are records (a bulk copy costs its
 // issuer about one round trip to L2); warp w reduces the running maxima of
 // heads w, w + nwarps, ... by shuffles and leaves the weights e^{m_i - M} in
-// shared memory; the accumulation runs split by split in ascending order
-// whatever `cap` is.  `stage`: merge_stage_bytes(G, D, cap) bytes of shared
+// shared memory.  The result does not depend on `cap` (a multiple of 4).
+// `stage`: merge_stage_bytes(G, D, cap) bytes of shared
 // memory, 16-byte aligned, that no thread still reads.  `bar`: an initialised
 // mbarrier (count 1) whose current phase parity is `parity` (updated).
 template <int D>
@@ -215,15 +227,18 @@ __device__ __forceinline__ void merge_group(const KernelParams& p, int b, int g,
     float* const st_rec = reinterpret_cast<float*>(stage);          // [cap][RF]
     float* const st_w = st_rec + (size_t)cap * RF;                  // [cap][G] weights
     float* const st_M = st_w + cap * G;                             // [8] maxima
-    float* const st_l = st_M + 8;                                   // [8] sums
     const float* const recs = p.ws + ((int64_t)slot_base * Hkv + g) * RF;
     const int64_t rec_stride = (int64_t)Hkv * RF;                   // next split of the same KV head
 
-    float4 acc[kMaxTasks];
+    float4 acc[kMaxTasks][4];                                       // four chains per column
+    float lch[kMaxTasks][4];                                        // and per head (kept by every column thread)
 #pragma unroll
-    for (int k = 0; k < kMaxTasks; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-    // warp w owns heads w, w + nwarps, ...: lane l keeps the running sum of splits i = l (mod 32)
-    float lpart[2] = {0.f, 0.f};
+    for (int k = 0; k < kMaxTasks; ++k)
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            acc[k][q] = make_float4(0.f, 0.f, 0.f, 0.f);
+            lch[k][q] = 0.f;
+        }
 
     for (int i0 = 0; i0 < S; i0 += cap) {
         const int n = min(cap, S - i0);
@@ -257,19 +272,11 @@ __device__ __forceinline__ void merge_group(const KernelParams& p, int b, int g,
             }
         }
         __syncthreads();
-        // weights e^{m_i - M} once per (split, head); the head's sum of w_i * l_i alongside
-        {
-            int k = 0;
-            for (int h = warp; h < G; h += nwarps, ++k) {
-                const float M = st_M[h];
-                // lane l takes the splits with global index i = l (mod 32), whatever the batching
-                for (int j = (lane - i0) & 31; j < n; j += 32) {
-                    const float2 ml = *reinterpret_cast<const float2*>(st_rec + (size_t)j * RF + G * D + 2 * h);
-                    const float w = (M == -INFINITY) ? 0.f : ex2f(ml.x - M);   // empty split: m = -inf, w = 0
-                    st_w[j * G + h] = w;
-                    lpart[k] = fmaf(w, ml.y, lpart[k]);
-                }
-            }
+        // weights e^{m_i - M}, once per (split, head)
+        for (int c = tid; c < n * G; c += nthreads) {
+            const int j = c / G, h = c % G;
+            const float M = st_M[h];
+            st_w[c] = (M == -INFINITY) ? 0.f : ex2f(st_rec[(size_t)j * RF + G * D + 2 * h] - M);   // empty split: 0
         }
         __syncthreads();
 #pragma unroll
@@ -279,50 +286,50 @@ __device__ __forceinline__ void merge_group(const KernelParams& p, int b, int g,
                 const int h = task / D4;
                 const float4* o = reinterpret_cast<const float4*>(st_rec) + task;
                 const float* wp = st_w + h;
-                float4 a4 = acc[k];
+                const float* lp = st_rec + G * D + 2 * h + 1;
                 int j = 0;
-                for (; j + 4 <= n; j += 4) {       // four records in flight; the sums stay in split order
-                    const float w0 = wp[j * G], w1 = wp[(j + 1) * G], w2 = wp[(j + 2) * G], w3 = wp[(j + 3) * G];
-                    const float4 v0 = o[j * RF4], v1 = o[(j + 1) * RF4], v2 = o[(j + 2) * RF4], v3 = o[(j + 3) * RF4];
-                    a4.x = fmaf(w3, v3.x, fmaf(w2, v2.x, fmaf(w1, v1.x, fmaf(w0, v0.x, a4.x))));
-                    a4.y = fmaf(w3, v3.y, fmaf(w2, v2.y, fmaf(w1, v1.y, fmaf(w0, v0.y, a4.y))));
-                    a4.z = fmaf(w3, v3.z, fmaf(w2, v2.z, fmaf(w1, v1.z, fmaf(w0, v0.z, a4.z))));
-                    a4.w = fmaf(w3, v3.w, fmaf(w2, v2.w, fmaf(w1, v1.w, fmaf(w0, v0.w, a4.w))));
+                for (; j + 4 <= n; j += 4) {       // i0 and cap are multiples of 4: chain q takes j + q
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const float w = wp[(j + q) * G];
+                        const float4 v = o[(j + q) * RF4];
+                        acc[k][q].x = fmaf(w, v.x, acc[k][q].x);
+                        acc[k][q].y = fmaf(w, v.y, acc[k][q].y);
+                        acc[k][q].z = fmaf(w, v.z, acc[k][q].z);
+                        acc[k][q].w = fmaf(w, v.w, acc[k][q].w);
+                        lch[k][q] = fmaf(w, lp[(size_t)(j + q) * RF], lch[k][q]);
+                    }
                 }
-                for (; j < n; ++j) {
-                    const float w = wp[j * G];
-                    const float4 v = o[j * RF4];
-                    a4.x = fmaf(w, v.x, a4.x);
-                    a4.y = fmaf(w, v.y, a4.y);
-                    a4.z = fmaf(w, v.z, a4.z);
-                    a4.w = fmaf(w, v.w, a4.w);
+#pragma unroll
+                for (int q = 0; q < 3; ++q) {
+                    if (j + q < n) {
+                        const float w = wp[(j + q) * G];
+                        const float4 v = o[(j + q) * RF4];
+                        acc[k][q].x = fmaf(w, v.x, acc[k][q].x);
+                        acc[k][q].y = fmaf(w, v.y, acc[k][q].y);
+                        acc[k][q].z = fmaf(w, v.z, acc[k][q].z);
+                        acc[k][q].w = fmaf(w, v.w, acc[k][q].w);
+                        lch[k][q] = fmaf(w, lp[(size_t)(j + q) * RF], lch[k][q]);
+                    }
                 }
-                acc[k] = a4;
             }
         }
         __syncthreads();
     }
-    // the heads' sums: a fixed butterfly over the 32 lane partials
-    {
-        int k = 0;
-        for (int h = warp; h < G; h += nwarps, ++k) {
-            float l = lpart[k];
-#pragma unroll
-            for (int off = 16; off >= 1; off >>= 1) l += __shfl_xor_sync(0xffffffffu, l, off);
-            if (lane == 0) st_l[h] = l;
-        }
-    }
-    __syncthreads();
 #pragma unroll
     for (int k = 0; k < kMaxTasks; ++k) {
         const int task = tid + k * nthreads;
         if (task < GD4) {
             const int h = task / D4, d4 = task % D4;
-            const float M = st_M[h], ls = st_l[h];
+            const float M = st_M[h];
+            const float ls = ((lch[k][0] + lch[k][1]) + lch[k][2]) + lch[k][3];
             float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
             if (M != -INFINITY && ls > 0.f) {
                 const float inv = 1.0f / ls;
-                o = make_float4(acc[k].x * inv, acc[k].y * inv, acc[k].z * inv, acc[k].w * inv);
+                o.x = (((acc[k][0].x + acc[k][1].x) + acc[k][2].x) + acc[k][3].x) * inv;
+                o.y = (((acc[k][0].y + acc[k][1].y) + acc[k][2].y) + acc[k][3].y) * inv;
+                o.z = (((acc[k][0].z + acc[k][1].z) + acc[k][2].z) + acc[k][3].z) * inv;
+                o.w = (((acc[k][0].w + acc[k][1].w) + acc[k][2].w) + acc[k][3].w) * inv;
             }
             store_out4(p.out, ((int64_t)b * Hq + g * G + h) * D + d4 * 4, o, p.out_bf16);
             if (p.lse != nullptr && d4 == 0)

@@ -375,6 +375,7 @@ __global__ void __launch_bounds__(kMmaThreads) decode_attn_mma_kernel(const Kern
     }
 
     if (tid == 0) DA_TRACE_STAMP(uid, 4);
+    if (MODE == kModeAttend) pdl_launch_dependents();   // the combine kernel may start getting scheduled
     __syncthreads();   // every issued tile has landed and been consumed: the stage memory is free
     if (MODE == kModeProbe) {
 #pragma unroll
@@ -421,7 +422,7 @@ __global__ void __launch_bounds__(kMmaThreads) decode_attn_mma_kernel(const Kern
         }
     }
     __syncthreads();
-    const int cap = (NS * Cfg::kStageBytes - 64 - 4 * G) / (rec_floats(G, D) * 4 + 4 * G);
+    const int cap = ((NS * Cfg::kStageBytes - 64 - 4 * G) / (rec_floats(G, D) * 4 + 4 * G)) & ~3;
     block_finish<D, kMmaConsumerWarps, 8, DUP>(p, u, G, sm_wo, sm_wm, sm_wl, sm_ticket, bar_base + 8 * 2 * NS, tid,
                                                kMmaThreads, gbase, cap);
     if (tid == 0) DA_TRACE_STAMP(uid, 6);

@@ -170,6 +170,7 @@ __global__ void __launch_bounds__(kSimtThreads) decode_attn_simt_kernel(const Ke
         }
     }
 
+    pdl_launch_dependents();                    // the combine kernel may start getting scheduled
     // the row groups' states go to shared memory; block_finish merges them in a fixed order
     if (dev_len != u.seq_len) {                 // stale plan: void the result, report it
         if (tid == 0) record_status(p.status, DA_ERR_STALE_PLAN);
