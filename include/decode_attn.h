@@ -280,6 +280,42 @@ int decode_attn_host_step(const decode_attn_shape_t *shape, const decode_attn_po
                           int64_t pool_elems, const int32_t *block_table_host,
                           const int32_t *seq_lens_host, void *out_host, float *lse_host_or_null);
 
+/* ---------------------------------------------------------------------------
+ * Allocation-free step.  (The paper has no counterpart to this entry point;
+ * it exists for integration, not for the method.)
+ *
+ * One whole decode-attention step - the split-KV partial kernel followed by
+ * the combine kernel - that never asks the CUDA allocator for anything: no
+ * plan object, no cudaMalloc / cudaFree, no pinned allocation, no workspace
+ * argument.  It is meant for callers that cannot allocate device memory at
+ * the point of the call: a serving engine that handed every remaining byte of
+ * HBM to its KV pool at start-up (a later cudaMalloc simply fails), or a
+ * latency-critical path that cannot accept the device-wide synchronisation an
+ * allocation implies.
+ *
+ * The work list and the partial records live in a scratch array compiled
+ * into the library (8 MiB of device memory, held by every GPU that loads the
+ * library until the process exits).  The step is planned with the
+ * deterministic split policy at its default chunk length (1,024 tokens), so
+ * its result equals plan / run / combine with that policy.
+ *
+ * Limits: batch <= 1,024; at most 4,096 work units (batch x KV heads x
+ * splits); the partial records must fit in about 7.8 MiB (e.g. 470 split
+ * sequences' worth of slots at 8 KV heads x group 4 x head_dim 128).  A step
+ * beyond these returns DA_ERR_WORKSPACE_TOO_SMALL and launches nothing.
+ *
+ * All calls share the one array, which keeps whatever the previous call left
+ * there; the call itself clears what has to start at zero.  Two calls whose
+ * kernels overlap on the GPU (different streams, no ordering) race on it -
+ * order them.  The first call on a device looks up the array's device
+ * address and sets kernel attributes; make that first call outside any stream
+ * capture.  Arguments are those of decode_attn_plan + decode_attn_run:
+ * seq_lens_host [batch] on the host, everything else on the device.
+ * ------------------------------------------------------------------------- */
+int decode_attn_step_static(const decode_attn_shape_t *shape, const int32_t *seq_lens_host, const void *q,
+                            const void *k_cache, const void *v_cache, const int32_t *block_table,
+                            const int32_t *seq_lens, void *out, float *lse_or_null, cudaStream_t stream);
+
 /* Frees what the library caches between calls: the arena of
  * decode_attn_host_step and the buffers parked by destroyed plans. */
 int decode_attn_host_release(void);

@@ -50,6 +50,7 @@ EXPORTED = [
     "decode_attn_run_ex", "decode_attn_combine", "decode_attn_last_device_status",
     "decode_attn_validate_block_table", "decode_attn_debug_gather", "decode_attn_gather_probe",
     "decode_attn_host_step", "decode_attn_host_release", "decode_attn_strerror", "decode_attn_version",
+    "decode_attn_step_static",
 ]
 
 
@@ -118,6 +119,7 @@ _lib.decode_attn_gather_probe.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp]
 _lib.decode_attn_host_step.argtypes = [ctypes.POINTER(Shape), ctypes.POINTER(Policy), _vp, _vp, _vp,
                                        ctypes.c_int64, _vp, _vp, _vp, _vp]
 _lib.decode_attn_host_release.argtypes = []
+_lib.decode_attn_step_static.argtypes = [ctypes.POINTER(Shape), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.decode_attn_strerror.argtypes = [ctypes.c_int]
 _lib.decode_attn_strerror.restype = ctypes.c_char_p
 _lib.decode_attn_version.restype = ctypes.c_char_p
@@ -333,6 +335,18 @@ def decode_attn_host_step(shape: Shape, policy: Policy, q_host, k_cache_host, v_
     _check(_lib.decode_attn_host_step(ctypes.byref(shape), ctypes.byref(policy), _ptr(q_host), _ptr(k_cache_host),
                                       _ptr(v_cache_host), pool_elems, _ptr(block_table_host), _ptr(seq_lens_host),
                                       _ptr(out_host), _ptr(lse_host)), "decode_attn_host_step")
+
+
+def decode_attn_step_static(shape: Shape, seq_lens_host, q, k_cache, v_cache, block_table, seq_lens, out, lse=None,
+                            stream=None, check: bool = True) -> int:
+    """One whole step (partial + combine) that allocates nothing: for callers that cannot
+    call the CUDA allocator.  Scratch is an 8 MiB array built into the library."""
+    lens = _host_i32(seq_lens_host)
+    rc = _lib.decode_attn_step_static(ctypes.byref(shape), _ptr(lens), _ptr(q), _ptr(k_cache), _ptr(v_cache),
+                                      _ptr(block_table), _ptr(seq_lens), _ptr(out), _ptr(lse), _stream(stream))
+    if check:
+        _check(rc, "decode_attn_step_static")
+    return rc
 
 
 def decode_attn_host_release() -> None:

@@ -640,6 +640,145 @@ const char* decode_attn_strerror(int status)
 
 const char* decode_attn_version(void) { return "0.1 sm_100a"; }
 
+// ------------------------------------------------------------------ allocation-free step
+//
+// Scratch for decode_attn_step_static: work list, per-sequence split table,
+// status word and partial records, all inside one file-scope device array.
+// Every GPU that loads this library holds these bytes until the process ends.
+constexpr size_t kStaticScratchBytes = 8u << 20;       // 8 MiB
+constexpr int kStaticMaxUnits = 4096;
+constexpr int kStaticMaxBatch = 1024;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+namespace {
+
+constexpr size_t kStaticOffUnits = 256;                                                   // header first
+constexpr size_t kStaticOffSeqInfo = kStaticOffUnits + sizeof(decode_attn_unit_t) * kStaticMaxUnits;
+constexpr size_t kStaticOffStatus = kStaticOffSeqInfo + sizeof(SeqInfo) * kStaticMaxBatch;
+constexpr size_t kStaticOffTickets = kStaticOffStatus + 256;
+constexpr size_t kStaticOffRecords = (kStaticOffTickets + sizeof(int32_t) * kStaticMaxBatch * 8 + 255) / 256 * 256;
+static_assert(kStaticOffRecords < kStaticScratchBytes, "static scratch layout");
+
+struct StaticSetup {
+    std::mutex mu;
+    static constexpr int kMaxDevices = 64;
+    unsigned char* base[kMaxDevices] = {};      // device address of g_static_scratch, per device
+    int sm_count[kMaxDevices] = {};
+    // host copy of the upload region; calls are serialised by `mu` while it is filled and enqueued
+    alignas(16) unsigned char staging[kStaticOffStatus];
+} g_static;
+
+}  // namespace
+
+int decode_attn_step_static(const decode_attn_shape_t* shape, const int32_t* seq_lens_host, const void* q,
+                            const void* k_cache, const void* v_cache, const int32_t* block_table,
+                            const int32_t* seq_lens, void* out, float* lse_or_null, cudaStream_t stream)
+{
+    if (!shape || !q || !k_cache || !v_cache || !block_table || !seq_lens || !out) return DA_ERR_INVALID_ARG;
+    if (shape->batch > 0 && !seq_lens_host) return DA_ERR_INVALID_ARG;
+    int rc = validate_shape(*shape);
+    if (rc != DA_OK) return rc;
+    if (!aligned(q, 16) || !aligned(k_cache, 16) || !aligned(v_cache, 16) || !aligned(out, 16)) return DA_ERR_INVALID_ARG;
+    if (shape->batch == 0) return DA_OK;
+    if (shape->batch > kStaticMaxBatch || shape->num_kv_heads > 8) return DA_ERR_WORKSPACE_TOO_SMALL;
+
+    decode_attn_policy_t policy;
+    std::memset(&policy, 0, sizeof policy);
+    policy.split_mode = DA_SPLIT_DETERMINISTIC;     // boundaries from the lengths alone: no device query needed
+    const int G = shape->num_q_heads / shape->num_kv_heads;
+    const int kernel = pick_kernel(*shape, policy);
+
+    int dev = -1;
+    DA_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= StaticSetup::kMaxDevices) return DA_ERR_UNSUPPORTED;
+
+    std::lock_guard<std::mutex> lock(g_static.mu);
+    if (g_static.base[dev] == nullptr) {
+        // First call on this device (make it before any stream capture): in host code the
+        // array's name is only a stand-in, so ask the runtime for its address on the current
+        // device.  Also done once here: the kernels' shared-memory opt-in.
+        void* ptr = nullptr;
+        DA_CUDA_TRY(cudaGetSymbolAddress(&ptr, g_static_scratch));
+        int block_threads = 0, dyn_smem = 0;
+        if (query_occupancy(kernel, shape->head_dim, G, &block_threads, &dyn_smem) <= 0) return DA_ERR_CUDA;
+        DA_CUDA_TRY(cudaDeviceGetAttribute(&g_static.sm_count[dev], cudaDevAttrMultiProcessorCount, dev));
+        g_static.base[dev] = static_cast<unsigned char*>(ptr);
+    } else if (kernel == DA_KERNEL_MMA_TMA) {
+        int block_threads = 0, dyn_smem = 0;       // another head_dim / group may need its own opt-in
+        if (query_occupancy(kernel, shape->head_dim, G, &block_threads, &dyn_smem) <= 0) return DA_ERR_CUDA;
+    }
+    unsigned char* const base = g_static.base[dev];
+
+    Layout lay;
+    rc = make_layout(*shape, policy, seq_lens_host, g_static.sm_count[dev], 1, lay);
+    if (rc != DA_OK) return rc;
+    const size_t rec_bytes = (size_t)rec_floats(G, shape->head_dim) * sizeof(float);
+    if (lay.units.size() > (size_t)kStaticMaxUnits ||
+        (size_t)lay.n_slots * shape->num_kv_heads * rec_bytes > kStaticScratchBytes - kStaticOffRecords)
+        return DA_ERR_WORKSPACE_TOO_SMALL;          // the step does not fit the built-in scratch
+
+    // upload region: header, units, split table (host copy lives in g_static.staging)
+    DevHeader* hdr = reinterpret_cast<DevHeader*>(g_static.staging);
+    hdr->n_units = (int32_t)lay.units.size();
+    hdr->batch = shape->batch;
+    hdr->pad[0] = hdr->pad[1] = 0;
+    std::memcpy(g_static.staging + kStaticOffUnits, lay.units.data(), lay.units.size() * sizeof(decode_attn_unit_t));
+    SeqInfo* si = reinterpret_cast<SeqInfo*>(g_static.staging + kStaticOffSeqInfo);
+    for (int b = 0; b < shape->batch; ++b) {
+        si[b].slot_base = lay.slot_base[b];
+        si[b].n_splits = lay.splits[b];
+    }
+    const size_t upload = kStaticOffSeqInfo + sizeof(SeqInfo) * (size_t)shape->batch;
+    // The array keeps the previous call's contents: the status word and tickets must start at zero.
+    DA_CUDA_TRY(cudaMemsetAsync(base + kStaticOffStatus, 0, kStaticOffRecords - kStaticOffStatus, stream));
+    // Pageable source: the runtime stages the bytes before returning, so the staging area may be reused.
+    DA_CUDA_TRY(cudaMemcpyAsync(base, g_static.staging, upload, cudaMemcpyHostToDevice, stream));
+
+    KernelParams kp;
+    std::memset(&kp, 0, sizeof kp);
+    kp.q = static_cast<const __nv_bfloat16*>(q);
+    kp.k = static_cast<const __nv_bfloat16*>(k_cache);
+    kp.v = static_cast<const __nv_bfloat16*>(v_cache);
+    kp.block_table = block_table;
+    kp.seq_lens = seq_lens;
+    kp.out = out;
+    kp.lse = lse_or_null;
+    kp.ws = reinterpret_cast<float*>(base + kStaticOffRecords);
+    kp.header = reinterpret_cast<const DevHeader*>(base);
+    kp.units = reinterpret_cast<const decode_attn_unit_t*>(base + kStaticOffUnits);
+    kp.seq_info = reinterpret_cast<const SeqInfo*>(base + kStaticOffSeqInfo);
+    kp.tickets = reinterpret_cast<int32_t*>(base + kStaticOffTickets);
+    kp.status = reinterpret_cast<int32_t*>(base + kStaticOffStatus);
+    kp.k_stride_page = shape->k_stride_page; kp.k_stride_token = shape->k_stride_token; kp.k_stride_head = shape->k_stride_head;
+    kp.v_stride_page = shape->v_stride_page; kp.v_stride_token = shape->v_stride_token; kp.v_stride_head = shape->v_stride_head;
+    kp.num_pages = shape->num_pages;
+    kp.num_q_heads = shape->num_q_heads;
+    kp.num_kv_heads = shape->num_kv_heads;
+    kp.max_pages_per_seq = shape->max_pages_per_seq;
+    const float scale = shape->sm_scale > 0.f ? shape->sm_scale : 1.0f / sqrtf((float)shape->head_dim);
+    kp.scale_log2 = scale * kLog2e;
+    kp.out_bf16 = shape->out_dtype == DA_DTYPE_BF16;
+    kp.fused = 0;
+    kp.grid_exit = 0;
+
+    const unsigned grid = (unsigned)lay.units.size();
+    if (kernel == DA_KERNEL_SIMT) {
+        simt_kernel_t fn = simt_kernel_for(shape->head_dim, G);
+        if (!fn) return DA_ERR_UNSUPPORTED;
+        fn<<<grid, kSimtThreads, 0, stream>>>(kp);
+    } else {
+        rc = mma_launch(*shape, G, kp, grid, stream);
+        if (rc != DA_OK) return rc;
+    }
+    DA_CUDA_TRY(cudaGetLastError());
+    if (lay.n_slots > 0) {
+        rc = combine_launch(shape->head_dim, G, kp, (unsigned)(shape->batch * shape->num_kv_heads), stream);
+        if (rc != DA_OK) return rc;
+        DA_CUDA_TRY(cudaGetLastError());
+    }
+    return DA_OK;
+}
+
 #ifdef DA_TRACE
 // Debug builds only: device buffer of 32 uint64 stamps per block (NULL switches tracing off).
 int decode_attn_trace_set_buffer(unsigned long long* device_buffer)
