@@ -322,10 +322,8 @@ def main():
             stream.synchronize()
             probe_us = p0.elapsed_time(p1) * 1e3 / n_probe
 
-    if world > 1:
-        t = torch.tensor([ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    from paper_2609_37062_b200 import sharding
+    ms = sharding.max_over_ranks(ms, dev)
     sec_per_step = ms * 1e-3 / args.steps
     value = world * kv_bytes / sec_per_step / 1e9
 
@@ -348,10 +346,7 @@ def main():
             da.decode_attn_host_step(shape, policy, hq, hk, hv, hbt, hsl, hout)
         torch.cuda.synchronize()
         dt = time.perf_counter() - t0
-        if world > 1:
-            t = torch.tensor([dt], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            dt = float(t.item())
+        dt = sharding.max_over_ranks(dt, dev)
         e2e = {"value": world * kv_bytes * n_e2e / dt / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "steps": n_e2e, "ms_per_step": dt / n_e2e * 1e3,
                "what": "decode_attn_host_step: q, both pools, block table and lengths copied from pinned host "

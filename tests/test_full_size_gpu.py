@@ -1,0 +1,93 @@
+"""Parity at the benchmark's sizes, in the launch configuration bench.py
+times (AUTO split, tensor-core kernel, combine kernel): the whole batch
+against the oracle where the oracle finishes in seconds, sampled sequences
+where it does not, and bitwise determinism of a sequence across batch sizes
+at full contexts."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2609_37062_b200 import workloads as wl
+from gpu_util import assert_parity, da, oracle_of, to_device
+
+pytestmark = pytest.mark.gpu
+
+
+def extract_sequences(w, idxs):
+    """Host copy of the sequences `idxs` of a device workload: their pages are
+    gathered (bit for bit) into a small pool with an identity block table."""
+    P = w.page_size
+    lens = [int(w.seq_lens[i]) for i in idxs]
+    pages = [(l + P - 1) // P for l in lens]
+    total = max(sum(pages), 1)
+    k = torch.empty((total,) + tuple(w.k_pool.shape[1:]), dtype=torch.int16)
+    v = torch.empty_like(k)
+    bt = torch.full((len(idxs), max(max(pages), 1)), -1, dtype=torch.int32)
+    cur = 0
+    for r, (i, n) in enumerate(zip(idxs, pages)):
+        ids = w.block_table[i, :n].long()
+        k[cur:cur + n] = w.k_pool[ids].cpu()
+        v[cur:cur + n] = w.v_pool[ids].cpu()
+        bt[r, :n] = torch.arange(cur, cur + n, dtype=torch.int32)
+        cur += n
+    return dataclasses.replace(w, batch=len(idxs), num_pages=total, max_pages_per_seq=bt.shape[1],
+                               seq_lens=torch.tensor(lens, dtype=torch.int32), block_table=bt,
+                               q_bits=w.q_bits[idxs].cpu(), k_pool=k, v_pool=v)
+
+
+def bench_policy(**kw):
+    return da.make_policy(**kw)        # AUTO split, AUTO kernel (tensor cores at G = 4), combine kernel
+
+
+def test_long_sequence_full_size():
+    w = wl.config_long(device="cuda")
+    out, lse = da.run_workload(w, bench_policy())
+    ref_out, ref_lse = oracle_of(to_device(w, "cpu"))
+    assert_parity(out, lse, ref_out, ref_lse, "long_32k")
+    fused, fused_lse = da.run_workload(w, bench_policy(fuse_combine=1))
+    assert torch.equal(out, fused) and torch.equal(lse, fused_lse)
+
+
+def test_short_chat_full_size():
+    w = wl.config_short_chat(device="cuda")
+    out, lse = da.run_workload(w, bench_policy())
+    ref_out, ref_lse = oracle_of(to_device(w, "cpu"))
+    assert_parity(out, lse, ref_out, ref_lse, "short_chat")
+
+
+def test_shared_prefix_full_size():
+    w = wl.config_shared_prefix(device="cuda")
+    out, lse = da.run_workload(w, bench_policy())
+    ref_out, ref_lse = oracle_of(to_device(w, "cpu"))
+    assert_parity(out, lse, ref_out, ref_lse, "shared_prefix")
+
+
+@pytest.mark.parametrize("context,batch", [(512, 256), (2048, 64), (8192, 64), (32768, 8), (131072, 2)])
+def test_sweep_cells_on_sampled_sequences(context, batch):
+    """First, last and two seeded picks of the cell, one by one against the oracle."""
+    w = wl.config_sweep_cell(context, batch, device="cuda")
+    out, lse = da.run_workload(w, bench_policy())
+    g = torch.Generator().manual_seed(context + batch)
+    picks = sorted({0, batch - 1, *torch.randint(0, batch, (2,), generator=g).tolist()})
+    sub = extract_sequences(w, picks)
+    ref_out, ref_lse = oracle_of(sub)
+    assert_parity(out[picks], lse[picks], ref_out, ref_lse, f"{context}x{batch}")
+    assert torch.isfinite(out).all()
+
+
+@pytest.mark.parametrize("context,batches", [(8192, (1, 8, 64)), (32768, (1, 8)), (131072, (1, 2))])
+def test_deterministic_mode_across_batch_sizes_at_full_context(context, batches):
+    pol = da.make_policy(split_mode=da.DA_SPLIT_DETERMINISTIC)
+    first = None
+    for b in batches:
+        w = wl.config_sweep_cell(context, b, device="cuda", table_seed=b)
+        out, lse = da.run_workload(w, pol)
+        if first is None:
+            first = (out[0].clone(), lse[0].clone())
+            sub = extract_sequences(w, [0])
+            ref_out, ref_lse = oracle_of(sub)
+            assert_parity(out[:1], lse[:1], ref_out, ref_lse)
+        assert torch.equal(out[0], first[0]) and torch.equal(lse[0], first[1]), (context, b)
+        del w
