@@ -169,6 +169,26 @@ simt_kernel_t simt_kernel_for(int D, int G)
     return D == 64 ? simt_for_group<64>(G) : D == 128 ? simt_for_group<128>(G) : nullptr;
 }
 
+// Launch with a programmatic dependency on the kernel before (see pdl_wait_primary).
+int simt_launch(simt_kernel_t fn, const KernelParams& kp, unsigned grid, cudaStream_t stream)
+{
+    cudaLaunchConfig_t cfg;
+    cfg.gridDim = dim3(grid, 1, 1);
+    cfg.blockDim = dim3(kSimtThreads, 1, 1);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, fn, kp) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return DA_ERR_CUDA;
+    }
+    return DA_OK;
+}
+
 int pick_kernel(const decode_attn_shape_t& s, const decode_attn_policy_t& p)
 {
     if (p.kernel != DA_KERNEL_AUTO) return p.kernel;
@@ -426,7 +446,8 @@ int decode_attn_run_ex(const decode_attn_plan_t* pl, const decode_attn_run_args_
     if (pl->kernel == DA_KERNEL_SIMT) {
         simt_kernel_t fn = simt_kernel_for(pl->shape.head_dim, pl->group);
         if (!fn) return DA_ERR_UNSUPPORTED;
-        fn<<<(unsigned)pl->grid, kSimtThreads, 0, stream>>>(kp);
+        int rc = simt_launch(fn, kp, (unsigned)pl->grid, stream);
+        if (rc != DA_OK) return rc;
     } else {
         int rc = mma_launch(pl->shape, pl->group, kp, (unsigned)pl->grid, stream);
         if (rc != DA_OK) return rc;
@@ -765,7 +786,8 @@ int decode_attn_step_static(const decode_attn_shape_t* shape, const int32_t* seq
     if (kernel == DA_KERNEL_SIMT) {
         simt_kernel_t fn = simt_kernel_for(shape->head_dim, G);
         if (!fn) return DA_ERR_UNSUPPORTED;
-        fn<<<grid, kSimtThreads, 0, stream>>>(kp);
+        rc = simt_launch(fn, kp, grid, stream);
+        if (rc != DA_OK) return rc;
     } else {
         rc = mma_launch(*shape, G, kp, grid, stream);
         if (rc != DA_OK) return rc;

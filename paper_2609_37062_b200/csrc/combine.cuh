@@ -29,6 +29,7 @@ __global__ void __launch_bounds__(kCombineThreads) decode_attn_combine_kernel(co
     __shared__ float sm_l[4][32];
     __shared__ float4 sm_acc[4][32];
 
+    pdl_launch_dependents();                              // the next kernel may start its prologue
     pdl_wait_primary();                                   // the records of the launch before this one are complete
     const int slice = blockIdx.x % n_slices;
     const int bg = blockIdx.x / n_slices;

@@ -115,10 +115,12 @@ __device__ __forceinline__ void store_out4(void* out, int64_t idx, float4 v, int
 
 // ---------------------------------------------------------------- programmatic dependent launch
 //
-// The partial kernel lets the grid launched after it (the combine kernel)
-// start being scheduled once every block is past its main loop; that grid
-// still waits, at its top, for this one to finish and flush.  Both are no-ops
-// when the launches carry no programmatic dependency.
+// Kernels of this library are launched with a programmatic dependency on the
+// kernel before them in the stream: a kernel lets its successor start being
+// scheduled early (the partial kernel once every block is past its main loop,
+// the combine kernel at once), and the successor waits (pdl_wait_primary) for
+// its predecessor to finish and flush before it reads anything that
+// predecessor may have written.  Both are no-ops without such a dependency.
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait_primary() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 

@@ -158,17 +158,6 @@ __global__ void __launch_bounds__(kMmaThreads) decode_attn_mma_kernel(const Kern
 
     const int t0 = u.tok_begin;
     int t1 = u.tok_end;
-    // Invariant 2 (never run on stale lengths): the device length is fetched now and compared
-    // in the epilogue, off the critical path; a mismatch voids the block's result.  Reads stay
-    // inside the planned range and page ids are range-checked, so nothing can fault meanwhile.
-    int dev_len = u.seq_len;
-    if (MODE == kModeAttend) {
-        dev_len = __ldg(p.seq_lens + b);
-        if (p.run_mask != nullptr && __ldg(p.run_mask + b) == 0) t1 = t0;   // masked row reads no KV
-    }
-    const int n_pages = (t1 - t0 + 15) >> 4;
-    const int n_iters = (n_pages + kPagesPerStage - 1) / kPagesPerStage;
-
     if (tid == 0) {
         tma_prefetch_descriptor(&k_map);
         tma_prefetch_descriptor(&v_map);
@@ -182,6 +171,22 @@ __global__ void __launch_bounds__(kMmaThreads) decode_attn_mma_kernel(const Kern
     }
     __syncthreads();
     if (tid == 0) DA_TRACE_STAMP(uid, 1);
+    // Everything above touched only the plan's own work list and kernel parameters.  What the
+    // kernel launched before this one may have produced (q, new K/V rows, lengths, page
+    // mappings) is read only past this point; with a programmatic dependency the lines above
+    // overlap that kernel's tail.
+    pdl_wait_primary();
+
+    // Invariant 2 (never run on stale lengths): the device length is fetched now and compared
+    // in the epilogue, off the critical path; a mismatch voids the block's result.  Reads stay
+    // inside the planned range and page ids are range-checked, so nothing can fault meanwhile.
+    int dev_len = u.seq_len;
+    if (MODE == kModeAttend) {
+        dev_len = __ldg(p.seq_lens + b);
+        if (p.run_mask != nullptr && __ldg(p.run_mask + b) == 0) t1 = t0;   // masked row reads no KV
+    }
+    const int n_pages = (t1 - t0 + 15) >> 4;
+    const int n_iters = (n_pages + kPagesPerStage - 1) / kPagesPerStage;
 
     // per-warp results (consumers only)
     float oacc[D / 16][4];
@@ -521,8 +526,22 @@ inline int mma_launch_mode(const decode_attn_shape_t& s, int G, const KernelPara
     if (rc != DA_OK) return rc;
     rc = make_pool_map(&vmap, kp.v, s, s.v_stride_page, s.v_stride_token, s.v_stride_head);
     if (rc != DA_OK) return rc;
-    fn<<<grid, kMmaThreads, mma_smem_bytes(s.head_dim), stream>>>(kp, kmap, vmap, G, ex);
-    if (cudaGetLastError() != cudaSuccess) return DA_ERR_CUDA;
+    // programmatic dependency on the kernel launched before: this kernel's blocks may become
+    // resident and run their prologue while that kernel drains (see pdl_wait_primary above)
+    cudaLaunchConfig_t cfg;
+    cfg.gridDim = dim3(grid, 1, 1);
+    cfg.blockDim = dim3(kMmaThreads, 1, 1);
+    cfg.dynamicSmemBytes = (size_t)mma_smem_bytes(s.head_dim);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, fn, kp, kmap, vmap, G, ex) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return DA_ERR_CUDA;
+    }
     return DA_OK;
 }
 

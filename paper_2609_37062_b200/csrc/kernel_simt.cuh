@@ -66,14 +66,17 @@ __global__ void __launch_bounds__(kSimtThreads) decode_attn_simt_kernel(const Ke
 
     const int t0 = u.tok_begin;
     int t1 = u.tok_end;
-    // Invariant 2 (never run on stale lengths): fetched now, compared in the epilogue so the
-    // load stays off the critical path; page ids are range-checked, so nothing can fault.
-    const int dev_len = __ldg(p.seq_lens + b);
-    if (p.run_mask != nullptr && __ldg(p.run_mask + b) == 0) t1 = t0;   // masked row reads no KV
     if (tid == 0) {
         mbar_init(smem_u32(&sm_merge_bar), 1);
         mbar_init_fence();
     }
+    // Only the plan's work list was read so far; what the kernel launched before this one may
+    // have produced (q, new K/V rows, lengths, page mappings) is read past this point.
+    pdl_wait_primary();
+    // Invariant 2 (never run on stale lengths): fetched now, compared in the epilogue so the
+    // load stays off the critical path; page ids are range-checked, so nothing can fault.
+    const int dev_len = __ldg(p.seq_lens + b);
+    if (p.run_mask != nullptr && __ldg(p.run_mask + b) == 0) t1 = t0;   // masked row reads no KV
 
     float qf[G][8];
 #pragma unroll
