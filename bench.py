@@ -68,6 +68,8 @@ def parse_args():
     ap.add_argument("--skip-e2e", action="store_true")
     ap.add_argument("--probe", action="store_true", help="also time the gather-only probe")
     ap.add_argument("--copies", type=int, default=0, help="pool copies to rotate over (0: enough for 1 GiB)")
+    ap.add_argument("--mask-fraction", type=float, default=None,
+                    help="RUN mask (Alg. 1 step 2): this fraction of the rows, picked by a seeded hash, reads no KV")
     return ap.parse_args()
 
 
@@ -258,10 +260,20 @@ def main():
     ws = torch.empty(max(plan.workspace_bytes, 256), dtype=torch.uint8, device=dev)
     launches_per_step = 1 if (policy.fuse_combine or info.n_slots == 0) else 2
 
+    run_mask = None
+    masked_bytes = 0
+    if args.mask_fraction is not None:
+        g = torch.Generator().manual_seed(12345)
+        n_mask = int(round(args.mask_fraction * first.batch))
+        keep = torch.ones(first.batch, dtype=torch.uint8)
+        keep[torch.randperm(first.batch, generator=g)[:n_mask]] = 0
+        run_mask = keep.to(dev)
+        masked_bytes = int((first.seq_lens.cpu().long() * (1 - keep.long())).sum().item()) * first.kv_bytes_per_token
+
     def step(i):
         w = pools[i % copies]
         da.decode_attn_run(plan, w.q_bits, w.k_pool, w.v_pool, w.block_table, w.seq_lens, out, lse, ws,
-                           plan.workspace_bytes)
+                           plan.workspace_bytes, run_mask=run_mask)
         if not policy.fuse_combine and not args.partial_only:
             da.decode_attn_combine(plan, ws, out, lse)
 
@@ -423,6 +435,10 @@ def main():
             "e2e_resident_kv": e2e_resident,
             "cpu_baseline": cpu,
         }
+        if run_mask is not None:
+            line["run_mask"] = {"masked_fraction": args.mask_fraction, "masked_kv_bytes": masked_bytes,
+                                "read_kv_bytes": kv_bytes - masked_bytes,
+                                "read_GB/s": (kv_bytes - masked_bytes) / sec_per_step / 1e9}
         if probe_us is not None:
             line["gather_probe"] = {"us": probe_us, "GB/s": kv_bytes / probe_us / 1e3}
         print(json.dumps(line))

@@ -231,6 +231,20 @@ typedef struct {
 int decode_attn_run_ex(const decode_attn_plan_t *plan, const decode_attn_run_args_t *args,
                        cudaStream_t stream);
 
+/* Own-layer KV write (Invariant 1; Algorithm 1 step 2: every valid row's K/V
+ * is written through the cache-write path before attention, whether or not
+ * the row then attends).  Stores row b's new K and V rows at logical position
+ * seq_lens[b] - 1: page block_table[b][(L-1) / page_size], slot
+ * (L-1) % page_size.  Bit-exact copy; rows with seq_len 0 write nothing.
+ *   new_k, new_v  device, bf16 [batch, num_kv_heads, head_dim], 16-byte aligned
+ *   block_table, seq_lens  device (seq_lens are the lengths INCLUDING the new token)
+ *   k_cache, v_cache  device pools of the shape, modified in place
+ * One launch on `stream`; a decode_attn_run enqueued after it on the same
+ * stream sees the new rows.  The run mask plays no part here. */
+int decode_attn_append_kv(const decode_attn_shape_t *shape, const void *new_k, const void *new_v,
+                          const int32_t *block_table, const int32_t *seq_lens, void *k_cache, void *v_cache,
+                          cudaStream_t stream);
+
 /* LSE combine: merges the partials `run` left in the workspace, per
  * (sequence, query head), in ascending split order:
  *   M = max_i m_i;  out = sum_i e^{m_i-M} o_i / sum_i e^{m_i-M} l_i;  lse = M + log(sum_i e^{m_i-M} l_i)

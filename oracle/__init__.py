@@ -162,3 +162,14 @@ def gather_kv(inp: PagedInputs, b: int):
     lib.oracle_gather_kv(ctypes.byref(inp.shape), _p(inp.k), _p(inp.v), _p(inp.block_table),
                          _p(inp.seq_lens), b, _p(k), _p(v))
     return k, v
+
+
+def append_kv(inp: PagedInputs, new_k, new_v):
+    """Own-layer KV write: returns copies of the pools with every row's new K/V
+    stored at logical position seq_len - 1 (Invariant 1)."""
+    lib = _load()
+    nk, nv = _u16(new_k), _u16(new_v)
+    assert nk.shape == (inp.B, inp.Hkv, inp.D) and nv.shape == nk.shape
+    k, v = inp.k.copy(), inp.v.copy()
+    lib.oracle_append_kv(ctypes.byref(inp.shape), _p(nk), _p(nv), _p(inp.block_table), _p(inp.seq_lens), _p(k), _p(v))
+    return k, v

@@ -22,6 +22,9 @@
  * with seq_len 0, or a row whose RUN mask byte is 0 (a Project-Only row of
  * Algorithm 1 step 2), reads no KV and emits zeros, lse = -inf.
  *
+ * Also here: the own-layer KV write that precedes attention (Invariant 1),
+ * a byte copy pinned in tests/test_oracle_pins.py by reading the rows back.
+ *
  * Parity status: the paper prints no attention values, so the numerics are
  * "unpinned by the paper"; the functions below are pinned instead by
  * brute-force dense attention, closed forms, invariants and a library
@@ -209,5 +212,31 @@ int oracle_gather_kv(const oracle_shape_t *s, const uint16_t *k_pool, const uint
             memcpy(k_out + ((int64_t)t * H + g) * D, k_pool + ko, sizeof(uint16_t) * (size_t)D);
             memcpy(v_out + ((int64_t)t * H + g) * D, v_pool + vo, sizeof(uint16_t) * (size_t)D);
         }
+    return 0;
+}
+
+/* Own-layer KV write (Invariant 1; Algorithm 1 step 2, first sentence): every
+ * valid row - RUN or Project-Only alike - stores the K and V rows its layer
+ * projected for the current token at logical position seq_len - 1 of its
+ * sequence, i.e. page block_table[b][(L-1) / P], slot (L-1) % P, before
+ * attention runs.  new_k / new_v are [B][Hkv][D] bf16 bit patterns; rows with
+ * seq_len 0 write nothing.  Pools are modified in place; nothing else moves. */
+int oracle_append_kv(const oracle_shape_t *s, const uint16_t *new_k, const uint16_t *new_v,
+                     const int32_t *block_table, const int32_t *seq_lens, uint16_t *k_pool,
+                     uint16_t *v_pool)
+{
+    const int D = s->head_dim, H = s->num_kv_heads;
+    for (int b = 0; b < s->batch; ++b) {
+        if (seq_lens[b] <= 0) continue;
+        const int t = seq_lens[b] - 1;
+        for (int g = 0; g < H; ++g) {
+            int64_t ko = row_offset(s, block_table, b, t, g, s->k_stride_page, s->k_stride_token,
+                                    s->k_stride_head);
+            int64_t vo = row_offset(s, block_table, b, t, g, s->v_stride_page, s->v_stride_token,
+                                    s->v_stride_head);
+            memcpy(k_pool + ko, new_k + ((int64_t)b * H + g) * D, sizeof(uint16_t) * (size_t)D);
+            memcpy(v_pool + vo, new_v + ((int64_t)b * H + g) * D, sizeof(uint16_t) * (size_t)D);
+        }
+    }
     return 0;
 }

@@ -50,7 +50,7 @@ EXPORTED = [
     "decode_attn_run_ex", "decode_attn_combine", "decode_attn_last_device_status",
     "decode_attn_validate_block_table", "decode_attn_debug_gather", "decode_attn_gather_probe",
     "decode_attn_host_step", "decode_attn_host_release", "decode_attn_strerror", "decode_attn_version",
-    "decode_attn_step_static",
+    "decode_attn_step_static", "decode_attn_append_kv",
 ]
 
 
@@ -120,6 +120,7 @@ _lib.decode_attn_host_step.argtypes = [ctypes.POINTER(Shape), ctypes.POINTER(Pol
                                        ctypes.c_int64, _vp, _vp, _vp, _vp]
 _lib.decode_attn_host_release.argtypes = []
 _lib.decode_attn_step_static.argtypes = [ctypes.POINTER(Shape), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.decode_attn_append_kv.argtypes = [ctypes.POINTER(Shape), _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.decode_attn_strerror.argtypes = [ctypes.c_int]
 _lib.decode_attn_strerror.restype = ctypes.c_char_p
 _lib.decode_attn_version.restype = ctypes.c_char_p
@@ -346,6 +347,15 @@ def decode_attn_step_static(shape: Shape, seq_lens_host, q, k_cache, v_cache, bl
                                       _ptr(block_table), _ptr(seq_lens), _ptr(out), _ptr(lse), _stream(stream))
     if check:
         _check(rc, "decode_attn_step_static")
+    return rc
+
+
+def decode_attn_append_kv(shape: Shape, new_k, new_v, block_table, seq_lens, k_cache, v_cache, stream=None,
+                          check: bool = True) -> int:
+    rc = _lib.decode_attn_append_kv(ctypes.byref(shape), _ptr(new_k), _ptr(new_v), _ptr(block_table), _ptr(seq_lens),
+                                    _ptr(k_cache), _ptr(v_cache), _stream(stream))
+    if check:
+        _check(rc, "decode_attn_append_kv")
     return rc
 
 

@@ -10,6 +10,7 @@
 #include <new>
 #include <vector>
 
+#include "append.cuh"
 #include "combine.cuh"
 #include "common.cuh"
 #include "decode_attn.h"
@@ -548,6 +549,51 @@ int decode_attn_gather_probe(const decode_attn_plan_t* pl, const void* k_cache, 
     a.k_cache = k_cache; a.v_cache = v_cache; a.block_table = block_table;
     const KernelParams kp = make_params(pl, a);
     return mma_gather_probe(pl->shape, pl->group, kp, checksum_out, (unsigned)pl->grid, stream);
+}
+
+int decode_attn_append_kv(const decode_attn_shape_t* shape, const void* new_k, const void* new_v,
+                          const int32_t* block_table, const int32_t* seq_lens, void* k_cache, void* v_cache,
+                          cudaStream_t stream)
+{
+    if (!shape || !new_k || !new_v || !block_table || !seq_lens || !k_cache || !v_cache) return DA_ERR_INVALID_ARG;
+    int rc = validate_shape(*shape);
+    if (rc != DA_OK) return rc;
+    if (!aligned(new_k, 16) || !aligned(new_v, 16) || !aligned(k_cache, 16) || !aligned(v_cache, 16))
+        return DA_ERR_INVALID_ARG;
+    if (shape->batch == 0) return DA_OK;
+    AppendParams ap;
+    std::memset(&ap, 0, sizeof ap);
+    ap.new_k = static_cast<const __nv_bfloat16*>(new_k);
+    ap.new_v = static_cast<const __nv_bfloat16*>(new_v);
+    ap.k = static_cast<__nv_bfloat16*>(k_cache);
+    ap.v = static_cast<__nv_bfloat16*>(v_cache);
+    ap.block_table = block_table;
+    ap.seq_lens = seq_lens;
+    ap.status = nullptr;
+    ap.k_stride_page = shape->k_stride_page; ap.k_stride_token = shape->k_stride_token; ap.k_stride_head = shape->k_stride_head;
+    ap.v_stride_page = shape->v_stride_page; ap.v_stride_token = shape->v_stride_token; ap.v_stride_head = shape->v_stride_head;
+    ap.num_pages = shape->num_pages;
+    ap.batch = shape->batch;
+    ap.num_kv_heads = shape->num_kv_heads;
+    ap.head_dim = shape->head_dim;
+    ap.max_pages_per_seq = shape->max_pages_per_seq;
+    const int rows = shape->batch * shape->num_kv_heads;
+    const unsigned grid = (unsigned)((rows + kAppendThreads / 32 - 1) / (kAppendThreads / 32));
+    cudaLaunchConfig_t cfg;
+    cfg.gridDim = dim3(grid, 1, 1);
+    cfg.blockDim = dim3(kAppendThreads, 1, 1);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, decode_attn_append_kernel, ap) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return DA_ERR_CUDA;
+    }
+    return DA_OK;
 }
 
 // ------------------------------------------------------------------ host-buffer step

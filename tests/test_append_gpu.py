@@ -1,0 +1,61 @@
+"""Own-layer KV write on the GPU (Invariant 1; Alg. 1 step 2, first half):
+bit-exact against the oracle's byte copy, and seen by the attention launch
+that follows it on the same stream - for masked rows too."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2609_37062_b200 import workloads as wl
+from gpu_util import assert_parity, da, to_device
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("layout", ["token_major", "head_major"])
+@pytest.mark.parametrize("hq,hkv,d", [(8, 2, 64), (32, 8, 128)])
+def test_append_then_attend(layout, hq, hkv, d):
+    lens = [1, 16, 17, 300, 0, 1024, 1025, 77]
+    w = wl.make_workload("append", lens, hq, hkv, d, seed=17, layout=layout, pool_pages=300)
+    B = len(lens)
+    new_k = wl.normal_bf16_bits(wl.stream_key(17, wl.TENSOR_NEW_K, 0), 0, B * hkv * d).view(B, hkv, d)
+    new_v = wl.normal_bf16_bits(wl.stream_key(17, wl.TENSOR_NEW_V, 0), 0, B * hkv * d).view(B, hkv, d)
+    inp = oracle.PagedInputs.from_workload(w)
+    k_ref, v_ref = oracle.append_kv(inp, new_k, new_v)
+    wd = to_device(w)
+    shape = da.shape_of_workload(wd)
+    mask = torch.tensor([1, 0, 1, 0, 1, 1, 0, 1], dtype=torch.uint8, device="cuda")
+    plan = da.decode_attn_plan(shape, da.make_policy(chunk_tokens=256), w.seq_lens)
+    out = torch.empty((B, hq, d), dtype=torch.float32, device="cuda")
+    lse = torch.empty((B, hq), dtype=torch.float32, device="cuda")
+    ws = torch.empty(max(plan.workspace_bytes, 256), dtype=torch.uint8, device="cuda")
+    # write, then attend, back to back on one stream
+    da.decode_attn_append_kv(shape, new_k.cuda(), new_v.cuda(), wd.block_table, wd.seq_lens, wd.k_pool, wd.v_pool)
+    da.decode_attn_run(plan, wd.q_bits, wd.k_pool, wd.v_pool, wd.block_table, wd.seq_lens, out, lse, ws,
+                       plan.workspace_bytes, run_mask=mask)
+    da.decode_attn_combine(plan, ws, out, lse)
+    assert da.decode_attn_last_device_status(plan) == da.DA_OK
+    # the pools: bit for bit, masked rows included (every layer writes its own KV)
+    assert np.array_equal(wd.k_pool.cpu().numpy().view(np.uint16).ravel(), k_ref.ravel())
+    assert np.array_equal(wd.v_pool.cpu().numpy().view(np.uint16).ravel(), v_ref.ravel())
+    # attention over the appended cache
+    w.k_pool = torch.from_numpy(k_ref.view(np.int16).reshape(tuple(w.k_pool.shape)))
+    w.v_pool = torch.from_numpy(v_ref.view(np.int16).reshape(tuple(w.v_pool.shape)))
+    ref_out, ref_lse = oracle.paged_decode_attention(oracle.PagedInputs.from_workload(w), run_mask=mask.cpu().numpy())
+    assert_parity(out, lse, ref_out, ref_lse)
+
+
+def test_append_rejects_bad_arguments_and_skips_bad_pages():
+    w = to_device(wl.config_tiny())
+    shape = da.shape_of_workload(w)
+    nk = torch.zeros((4, 2, 64), dtype=torch.int16, device="cuda")
+    assert da.decode_attn_append_kv(shape, None, nk, w.block_table, w.seq_lens, w.k_pool, w.v_pool,
+                                    check=False) == da.DA_ERR_INVALID_ARG
+    assert da.decode_attn_append_kv(shape, nk.data_ptr() + 2, nk, w.block_table, w.seq_lens, w.k_pool, w.v_pool,
+                                    check=False) == da.DA_ERR_INVALID_ARG
+    before = w.k_pool.clone()
+    bt = w.block_table.clone()
+    bt[:, :] = 1 << 30                                   # every mapping points outside the pool
+    da.decode_attn_append_kv(shape, nk, nk, bt, w.seq_lens, w.k_pool, w.v_pool)
+    torch.cuda.synchronize()
+    assert torch.equal(before, w.k_pool)                 # nothing was written, nothing faulted

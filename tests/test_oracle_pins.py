@@ -326,3 +326,34 @@ def test_threads_do_not_change_results():
     a, _ = oracle.paged_decode_attention(inp, num_threads=1)
     b, _ = oracle.paged_decode_attention(inp, num_threads=4)
     assert np.array_equal(a, b)
+
+
+# --------------------------------------------------------------------------- own-layer KV write
+
+def test_append_writes_the_last_position_and_nothing_else():
+    """Invariant 1: position seq_len - 1 of the layer's cache holds the row's
+    own K/V after the write; every other byte of the pools is untouched."""
+    w = small_workload([1, 16, 17, 40, 0], Hq=4, Hkv=2, D=16, pool_pages=12)
+    inp = oracle.PagedInputs.from_workload(w)
+    new_k = wl.normal_bf16_bits(wl.stream_key(5, wl.TENSOR_NEW_K, 0), 0, 5 * 2 * 16).view(5, 2, 16)
+    new_v = wl.normal_bf16_bits(wl.stream_key(5, wl.TENSOR_NEW_V, 0), 0, 5 * 2 * 16).view(5, 2, 16)
+    k2, v2 = oracle.append_kv(inp, new_k, new_v)
+    expected_k, expected_v = w.k_pool.numpy().copy(), w.v_pool.numpy().copy()
+    for b, L in enumerate(w.seq_lens.tolist()):
+        if L == 0:
+            continue
+        page, slot = int(w.block_table[b, (L - 1) // 16]), (L - 1) % 16
+        expected_k[page, slot] = new_k[b].numpy()
+        expected_v[page, slot] = new_v[b].numpy()
+    assert np.array_equal(k2.view(np.int16).reshape(expected_k.shape), expected_k)
+    assert np.array_equal(v2.view(np.int16).reshape(expected_v.shape), expected_v)
+    # reading back through the gather gives the new rows at the last position
+    w2 = wl.make_workload("small", [1, 16, 17, 40, 0], 4, 2, 16, seed=11, pool_pages=12)
+    w2.k_pool = torch.from_numpy(k2.view(np.int16).reshape(expected_k.shape))
+    w2.v_pool = torch.from_numpy(v2.view(np.int16).reshape(expected_v.shape))
+    inp2 = oracle.PagedInputs.from_workload(w2)
+    for b, L in enumerate(w.seq_lens.tolist()):
+        if L:
+            gk, gv = oracle.gather_kv(inp2, b)
+            assert np.array_equal(gk[L - 1].view(np.int16), new_k[b].numpy())
+            assert np.array_equal(gv[L - 1].view(np.int16), new_v[b].numpy())
