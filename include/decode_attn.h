@@ -334,6 +334,27 @@ int decode_attn_step_static(const decode_attn_shape_t *shape, const int32_t *seq
  * decode_attn_host_step and the buffers parked by destroyed plans. */
 int decode_attn_host_release(void);
 
+/* ---------------------------------------------------------------------------
+ * Decode profitability rule (Section 3.3, Appendix D): what the RUN mask is
+ * worth.  A skipped row saves its KV read at each routed layer, so with a
+ * fraction s of decisions skipping over L_r routed layers a step holding V
+ * resident tokens saves s * L_r * b * V / BW seconds against a fixed per-step
+ * cost tau; routing pays above V* = tau * BW / (s * L_r * b).  Host only.
+ * ------------------------------------------------------------------------- */
+int decode_attn_breakeven_tokens(double tau_seconds, double bandwidth_bytes_per_s, double skip_fraction,
+                                 int32_t routed_layers, double kv_bytes_per_token_layer, double *v_star_out);
+
+/* Served thresholds of the rule: exit at V*, enter at 1.25 V*, each rounded
+ * half up to a multiple of round_to tokens (0: no rounding; the paper's
+ * printed thresholds use 10,000). */
+int decode_attn_switch_thresholds(double v_star, double round_to, double *exit_tokens_out,
+                                  double *enter_tokens_out);
+
+/* One step of the hysteresis: returns 1 (routed) once resident_tokens reaches
+ * enter_tokens, 0 (dense for newly starting requests) once it falls to
+ * exit_tokens, and routed_now in between. */
+int decode_attn_switch_next(int32_t routed_now, double resident_tokens, double exit_tokens, double enter_tokens);
+
 const char *decode_attn_strerror(int status);
 
 /* "major.minor arch" of this build, e.g. "0.1 sm_100a". */

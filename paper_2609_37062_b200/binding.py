@@ -50,7 +50,8 @@ EXPORTED = [
     "decode_attn_run_ex", "decode_attn_combine", "decode_attn_last_device_status",
     "decode_attn_validate_block_table", "decode_attn_debug_gather", "decode_attn_gather_probe",
     "decode_attn_host_step", "decode_attn_host_release", "decode_attn_strerror", "decode_attn_version",
-    "decode_attn_step_static", "decode_attn_append_kv",
+    "decode_attn_step_static", "decode_attn_append_kv", "decode_attn_breakeven_tokens",
+    "decode_attn_switch_thresholds", "decode_attn_switch_next",
 ]
 
 
@@ -121,6 +122,11 @@ _lib.decode_attn_host_step.argtypes = [ctypes.POINTER(Shape), ctypes.POINTER(Pol
 _lib.decode_attn_host_release.argtypes = []
 _lib.decode_attn_step_static.argtypes = [ctypes.POINTER(Shape), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.decode_attn_append_kv.argtypes = [ctypes.POINTER(Shape), _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.decode_attn_breakeven_tokens.argtypes = [ctypes.c_double, ctypes.c_double, ctypes.c_double, ctypes.c_int32,
+                                              ctypes.c_double, ctypes.POINTER(ctypes.c_double)]
+_lib.decode_attn_switch_thresholds.argtypes = [ctypes.c_double, ctypes.c_double, ctypes.POINTER(ctypes.c_double),
+                                               ctypes.POINTER(ctypes.c_double)]
+_lib.decode_attn_switch_next.argtypes = [ctypes.c_int32, ctypes.c_double, ctypes.c_double, ctypes.c_double]
 _lib.decode_attn_strerror.argtypes = [ctypes.c_int]
 _lib.decode_attn_strerror.restype = ctypes.c_char_p
 _lib.decode_attn_version.restype = ctypes.c_char_p
@@ -357,6 +363,25 @@ def decode_attn_append_kv(shape: Shape, new_k, new_v, block_table, seq_lens, k_c
     if check:
         _check(rc, "decode_attn_append_kv")
     return rc
+
+
+def decode_attn_breakeven_tokens(tau_seconds: float, bandwidth_bytes_per_s: float, skip_fraction: float,
+                                 routed_layers: int, kv_bytes_per_token_layer: float) -> float:
+    v = ctypes.c_double()
+    _check(_lib.decode_attn_breakeven_tokens(tau_seconds, bandwidth_bytes_per_s, skip_fraction, routed_layers,
+                                             kv_bytes_per_token_layer, ctypes.byref(v)), "decode_attn_breakeven_tokens")
+    return v.value
+
+
+def decode_attn_switch_thresholds(v_star: float, round_to: float = 10_000.0):
+    ex, en = ctypes.c_double(), ctypes.c_double()
+    _check(_lib.decode_attn_switch_thresholds(v_star, round_to, ctypes.byref(ex), ctypes.byref(en)),
+           "decode_attn_switch_thresholds")
+    return ex.value, en.value
+
+
+def decode_attn_switch_next(routed_now: bool, resident_tokens: float, exit_tokens: float, enter_tokens: float) -> bool:
+    return bool(_lib.decode_attn_switch_next(int(bool(routed_now)), resident_tokens, exit_tokens, enter_tokens))
 
 
 def decode_attn_host_release() -> None:

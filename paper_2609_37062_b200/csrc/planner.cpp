@@ -249,3 +249,39 @@ extern "C" int decode_attn_plan_layout(const decode_attn_shape_t* shape, const d
     }
     return DA_OK;
 }
+
+// ---------------------------------------------------------------------------
+// Decode profitability rule (Section 3.3, Appendix D).  Host arithmetic only.
+// ---------------------------------------------------------------------------
+extern "C" int decode_attn_breakeven_tokens(double tau_seconds, double bandwidth_bytes_per_s, double skip_fraction,
+                                            int32_t routed_layers, double kv_bytes_per_token_layer, double* v_star_out)
+{
+    if (!v_star_out) return DA_ERR_INVALID_ARG;
+    if (!(tau_seconds >= 0.0) || !(bandwidth_bytes_per_s > 0.0) || !(skip_fraction > 0.0) || skip_fraction > 1.0 ||
+        routed_layers <= 0 || !(kv_bytes_per_token_layer > 0.0))
+        return DA_ERR_INVALID_ARG;
+    *v_star_out = tau_seconds * bandwidth_bytes_per_s / (skip_fraction * (double)routed_layers * kv_bytes_per_token_layer);
+    return DA_OK;
+}
+
+extern "C" int decode_attn_switch_thresholds(double v_star, double round_to, double* exit_tokens_out,
+                                             double* enter_tokens_out)
+{
+    if (!exit_tokens_out || !enter_tokens_out || !(v_star >= 0.0) || !(round_to >= 0.0)) return DA_ERR_INVALID_ARG;
+    double ex = v_star, en = 1.25 * v_star;
+    if (round_to > 0.0) {
+        ex = std::floor(ex / round_to + 0.5) * round_to;
+        en = std::floor(en / round_to + 0.5) * round_to;
+    }
+    *exit_tokens_out = ex;
+    *enter_tokens_out = en;
+    return DA_OK;
+}
+
+extern "C" int decode_attn_switch_next(int32_t routed_now, double resident_tokens, double exit_tokens,
+                                       double enter_tokens)
+{
+    if (resident_tokens >= enter_tokens) return 1;
+    if (resident_tokens <= exit_tokens) return 0;
+    return routed_now ? 1 : 0;
+}
