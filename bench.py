@@ -322,7 +322,7 @@ def main():
 
         probe_us = None
         if args.probe and info.kernel == da.DA_KERNEL_MMA_TMA:
-            chk = torch.empty(int(info.grid), dtype=torch.int32, device=dev)
+            chk = torch.empty(int(info.n_units), dtype=torch.int32, device=dev)
             for i in range(3):
                 w = pools[i % copies]
                 da.decode_attn_gather_probe(plan, w.k_pool, w.v_pool, w.block_table, chk)

@@ -123,7 +123,8 @@ typedef struct {
 
 typedef struct {
     int64_t n_units;          /* work units = thread blocks that do work                             */
-    int64_t grid;             /* thread blocks launched (>= n_units with a capacity plan)            */
+    int64_t grid;             /* thread blocks launched: the tensor-core kernel walks the work list
+                                 with at most sm_count * ctas_per_sm blocks; fixed for a capacity plan */
     int64_t n_slots;          /* partial results held in the workspace                               */
     int64_t workspace_bytes;
     int32_t chunk_tokens;     /* AUTO / DETERMINISTIC: the chunk length in use (0 for FIXED_COUNT)   */
@@ -277,7 +278,7 @@ int decode_attn_debug_gather(const decode_attn_plan_t *plan, int32_t seq, const 
                              cudaStream_t stream);
 
 /* Gather-only probe: streams exactly the K/V bytes `run` would read, through
- * the same loads, and folds them into checksum_out (device, uint32 [grid]);
+ * the same loads, and folds them into checksum_out (device, uint32 [n_units]);
  * no attention arithmetic.  Its time is the ceiling for this access pattern. */
 int decode_attn_gather_probe(const decode_attn_plan_t *plan, const void *k_cache, const void *v_cache,
                              const int32_t *block_table, uint32_t *checksum_out, cudaStream_t stream);

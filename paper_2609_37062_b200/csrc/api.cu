@@ -259,6 +259,7 @@ KernelParams make_params(const decode_attn_plan_t* pl, const decode_attn_run_arg
     kp.out_bf16 = s.out_dtype == DA_DTYPE_BF16;
     kp.fused = pl->policy.fuse_combine;
     kp.grid_exit = pl->policy.capacity_batch > 0;
+    kp.n_units = (int32_t)pl->layout.units.size();
 #ifdef DA_TRACE
     kp.trace = g_trace_buffer;
 #endif
@@ -323,6 +324,10 @@ int decode_attn_plan(const decode_attn_shape_t* shape, const decode_attn_policy_
         pl->grid = pl->max_units;
     }
     if (pl->grid > 0x7fffffffLL) return DA_ERR_UNSUPPORTED;
+    // The tensor-core kernel walks the work list with a fixed number of blocks (what fits on the
+    // machine at once) unless the merge is fused, which needs one unit per block.
+    if (pl->kernel == DA_KERNEL_MMA_TMA && !policy->fuse_combine)
+        pl->grid = std::min<int64_t>(pl->grid, (int64_t)pl->sm_count * pl->ctas_per_sm);
 
     pl->workspace_bytes = (size_t)pl->max_slots * shape->num_kv_heads * rec_floats(pl->group, shape->head_dim) * sizeof(float);
 
@@ -548,7 +553,8 @@ int decode_attn_gather_probe(const decode_attn_plan_t* pl, const void* k_cache, 
     std::memset(&a, 0, sizeof a);
     a.k_cache = k_cache; a.v_cache = v_cache; a.block_table = block_table;
     const KernelParams kp = make_params(pl, a);
-    return mma_gather_probe(pl->shape, pl->group, kp, checksum_out, (unsigned)pl->grid, stream);
+    return mma_gather_probe(pl->shape, pl->group, kp, checksum_out, (unsigned)pl->layout.units.size(), (unsigned)pl->grid,
+                            stream);
 }
 
 int decode_attn_append_kv(const decode_attn_shape_t* shape, const void* new_k, const void* new_v,
@@ -827,6 +833,7 @@ int decode_attn_step_static(const decode_attn_shape_t* shape, const int32_t* seq
     kp.out_bf16 = shape->out_dtype == DA_DTYPE_BF16;
     kp.fused = 0;
     kp.grid_exit = 0;
+    kp.n_units = (int32_t)lay.units.size();
 
     const unsigned grid = (unsigned)lay.units.size();
     if (kernel == DA_KERNEL_SIMT) {

@@ -46,7 +46,8 @@ struct KernelParams {
     float scale_log2;  // sm_scale * log2(e): logits are kept in the base-2 domain
     int32_t out_bf16;
     int32_t fused;
-    int32_t grid_exit;  // capacity plans: blocks at or beyond header->n_units leave at once
+    int32_t grid_exit;  // capacity plans: the unit count is read from header->n_units, surplus blocks leave at once
+    int32_t n_units;    // otherwise: the unit count
 #ifdef DA_TRACE
     unsigned long long* trace;  // debug builds: 32 stamps per block, or NULL
 #endif
@@ -123,6 +124,13 @@ __device__ __forceinline__ void store_out4(void* out, int64_t idx, float4 v, int
 // predecessor may have written.  Both are no-ops without such a dependency.
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait_primary() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// Barrier over `nthreads` threads of the block (a multiple of 32) on hardware barrier `id`;
+// id 0 with the whole block is __syncthreads().
+__device__ __forceinline__ void block_sync(int id, int nthreads)
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
 
 // ---------------------------------------------------------------- partial records
 //
@@ -212,12 +220,13 @@ __device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uin
 // issuer about one round trip to L2); warp w reduces the running maxima of
 // heads w, w + nwarps, ... by shuffles and leaves the weights e^{m_i - M} in
 // shared memory.  The result does not depend on `cap` (a multiple of 4).
+// The `nthreads` threads synchronise on hardware barrier `bar_id`.
 // `stage`: merge_stage_bytes(G, D, cap) bytes of shared
 // memory, 16-byte aligned, that no thread still reads.  `bar`: an initialised
 // mbarrier (count 1) whose current phase parity is `parity` (updated).
 template <int D>
 __device__ __forceinline__ void merge_group(const KernelParams& p, int b, int g, int G, int slot_base, int S,
-                                            int tid, int nthreads, uint8_t* stage, int cap, uint32_t bar,
+                                            int tid, int nthreads, int bar_id, uint8_t* stage, int cap, uint32_t bar,
                                             uint32_t& parity)
 {
     constexpr int D4 = D / 4;
@@ -273,14 +282,14 @@ __device__ __forceinline__ void merge_group(const KernelParams& p, int b, int g,
                 if (lane == 0) st_M[h] = m;
             }
         }
-        __syncthreads();
+        block_sync(bar_id, nthreads);
         // weights e^{m_i - M}, once per (split, head)
         for (int c = tid; c < n * G; c += nthreads) {
             const int j = c / G, h = c % G;
             const float M = st_M[h];
             st_w[c] = (M == -INFINITY) ? 0.f : ex2f(st_rec[(size_t)j * RF + G * D + 2 * h] - M);   // empty split: 0
         }
-        __syncthreads();
+        block_sync(bar_id, nthreads);
 #pragma unroll
         for (int k = 0; k < kMaxTasks; ++k) {
             const int task = tid + k * nthreads;
@@ -316,7 +325,7 @@ __device__ __forceinline__ void merge_group(const KernelParams& p, int b, int g,
                 }
             }
         }
-        __syncthreads();
+        block_sync(bar_id, nthreads);
     }
 #pragma unroll
     for (int k = 0; k < kMaxTasks; ++k) {
@@ -350,13 +359,16 @@ __device__ __forceinline__ void merge_group(const KernelParams& p, int b, int g,
 // that made the sources visible.  The states are merged in the fixed order
 // r = 0..R-1 and the result goes straight to `out` (single split) or to the
 // unit's record; with a fused plan the block then draws a ticket and, if it
-// is the last of its (sequence, KV head), merges all records.  `stage` /
-// `cap`: shared memory the merge may overwrite (it may alias the sources).
+// is the last of its (sequence, KV head), merges all records.  The calling
+// threads (`nthreads`, ids 0..nthreads-1) synchronise on hardware barrier
+// `bar_id`.  `stage` / `cap`: shared memory the merge may overwrite (it may
+// alias the sources); cap == 0 means none is available (the block still has
+// units to stream) and a fused plan must not get here.
 template <int D, int R, int COLS, bool DUP>
 __device__ __forceinline__ void block_finish(const KernelParams& p, const decode_attn_unit_t& u, int G,
                                              const float* src_o, const float* src_m, const float* src_l,
-                                             int* sm_ticket, uint32_t merge_bar, int tid, int nthreads,
-                                             uint8_t* stage, int cap)
+                                             int* sm_ticket, uint32_t merge_bar, uint32_t* merge_parity, int tid,
+                                             int nthreads, int bar_id, uint8_t* stage, int cap)
 {
     constexpr int D4 = D / 4;
     constexpr int kUnroll = R <= 4 ? R : 1;     // many row groups: keep the loop rolled, registers matter more
@@ -407,7 +419,7 @@ __device__ __forceinline__ void block_finish(const KernelParams& p, const decode
     // stores before thread 0's fence, which publishes them device-wide ahead
     // of the ticket; the block that draws the last ticket of its (sequence,
     // KV head) therefore sees all the other records.
-    __syncthreads();
+    block_sync(bar_id, nthreads);
     if (tid == 0) DA_TRACE_CLOCK(blockIdx.x, 13);
     int32_t* ticket = p.tickets + (int64_t)u.seq * p.num_kv_heads + u.kv_head;
     if (tid == 0) {
@@ -415,12 +427,17 @@ __device__ __forceinline__ void block_finish(const KernelParams& p, const decode
         *sm_ticket = atomicAdd(ticket, 1);
         __threadfence();
     }
-    __syncthreads();
+    block_sync(bar_id, nthreads);
     if (tid == 0) DA_TRACE_CLOCK(blockIdx.x, 14);
     if (*sm_ticket != u.n_splits - 1) return;
-    uint32_t parity = 0;
-    merge_group<D>(p, u.seq, u.kv_head, G, u.slot - u.split_index, u.n_splits, tid, nthreads, stage, cap, merge_bar,
+    if (cap <= 0) {                              // host-side contract broken: fused plans run one unit per block
+        if (tid == 0) record_status(p.status, DA_ERR_UNSUPPORTED);
+        return;
+    }
+    uint32_t parity = *merge_parity;
+    merge_group<D>(p, u.seq, u.kv_head, G, u.slot - u.split_index, u.n_splits, tid, nthreads, bar_id, stage, cap, merge_bar,
                    parity);
+    *merge_parity = parity;
     if (tid == 0) DA_TRACE_CLOCK(blockIdx.x, 19);
     if (tid == 0) *ticket = 0;  // ready for the next launch
 }

@@ -1,7 +1,11 @@
 // Tensor-core split-KV partial kernel with TMA-staged pages.
 //
-// One block per work unit (sequence, KV head, run of pages): four consumer
-// warps and one producer warp.  The producer turns block-table entries into
+// A block is four consumer warps and one producer warp.  It works through
+// the units blockIdx.x, blockIdx.x + gridDim.x, ... of the work list (a unit
+// is one sequence, one KV head, a run of pages) without ever draining its
+// pipeline: the producer keeps filling the ring of stages with the next
+// unit's pages while the consumers finish the previous unit.  With a grid as
+// large as the work list every block has one unit.  The producer turns block-table entries into
 // TMA tile loads (cp.async.bulk.tensor over a 4-D map [dim, slot, head, page]
 // of each pool): one 16-token page of one KV head lands in shared memory as
 // 16 rows x 128 bytes per half of the head dimension, 128-byte swizzled, with
@@ -42,16 +46,18 @@ constexpr int kPagesPerStage = kMmaConsumerWarps;
 
 enum MmaMode { kModeAttend = 0, kModeProbe = 1, kModeGather = 2 };
 
-template <int D>
+template <int D, bool DUP>
 struct MmaCfg {
     static constexpr int kHalves = D / 64;                      // 128-byte column blocks per row
     static constexpr int kBoxBytes = 16 * 128;                  // one TMA box: 16 rows x 128 B
     static constexpr int kPageBytes = kHalves * kBoxBytes;      // one page of one tensor
     static constexpr int kTensorBytes = kPagesPerStage * kPageBytes;
     static constexpr int kStageBytes = 2 * kTensorBytes;        // K then V
-    static constexpr int kStages = (D == 128) ? 3 : 6;
+    static constexpr int kColsOut = DUP ? 4 : 8;                // output columns a warp hands to the block merge
+    static constexpr int kStages = (D == 128) ? (DUP ? 3 : 2) : 6;   // two blocks per SM must fit
     static constexpr int kBarrierBytes = 1024;                  // barriers + small state, keeps tiles 1 KB aligned
-    static constexpr int kSmemBytes = kStages * kStageBytes + kBarrierBytes + 1024;  // + alignment slack
+    static constexpr int kScratchBytes = kMmaConsumerWarps * kColsOut * D * 4 + 256;   // warps' results for the merge
+    static constexpr int kSmemBytes = kStages * kStageBytes + kBarrierBytes + kScratchBytes + 1024;  // + alignment slack
 };
 
 // ---------------------------------------------------------------- PTX wrappers
@@ -123,7 +129,7 @@ __device__ __forceinline__ uint32_t swz(int row, int chunk) { return row * 128 +
 // ---------------------------------------------------------------- the kernel
 
 struct MmaExtra {
-    // kModeProbe:  checksum [grid] (uint32).  kModeGather: dense K / V rows of one sequence.
+    // kModeProbe:  checksum [n_units] (uint32).  kModeGather: dense K / V rows of one sequence.
     uint32_t* checksum;
     __nv_bfloat16* k_out;
     __nv_bfloat16* v_out;
@@ -136,9 +142,11 @@ __global__ void __launch_bounds__(kMmaThreads) decode_attn_mma_kernel(const Kern
                                                                       const __grid_constant__ CUtensorMap v_map,
                                                                       const int G, const MmaExtra ex)
 {
-    using Cfg = MmaCfg<D>;
+    using Cfg = MmaCfg<D, DUP>;
     constexpr int NS = Cfg::kStages;
     constexpr int KSTEPS = D / 16;
+    constexpr int COLS = Cfg::kColsOut;
+    constexpr int kConsumerThreads = kMmaConsumerWarps * 32;
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -147,17 +155,15 @@ __global__ void __launch_bounds__(kMmaThreads) decode_attn_mma_kernel(const Kern
     const uint32_t bar_base = base + NS * Cfg::kStageBytes;   // full[NS], empty[NS], merge
     volatile int* const sm_flags = reinterpret_cast<volatile int*>(gbase + NS * Cfg::kStageBytes + 256);
     int* const sm_ticket = reinterpret_cast<int*>(gbase + NS * Cfg::kStageBytes + 256 + 16);
+    float* const sm_wo = reinterpret_cast<float*>(gbase + NS * Cfg::kStageBytes + Cfg::kBarrierBytes);   // [4][COLS][D]
+    float* const sm_wm = sm_wo + kMmaConsumerWarps * COLS * D;                                           // [4][COLS]
+    float* const sm_wl = sm_wm + kMmaConsumerWarps * COLS;                                               // [4][COLS]
 
-    const int uid = blockIdx.x;
-    if (p.grid_exit && uid >= p.header->n_units) return;      // surplus blocks of a capacity launch
-    const decode_attn_unit_t u = load_unit(p.units, uid);
-    if (MODE == kModeGather && u.seq != ex.gather_seq) return;
+    const int n_units = p.grid_exit ? p.header->n_units : p.n_units;
+    if ((int)blockIdx.x >= n_units) return;                   // surplus blocks of a capacity launch
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int b = u.seq, g = u.kv_head;
-    if (tid == 0) DA_TRACE_STAMP(uid, 0);
+    if (tid == 0) DA_TRACE_STAMP(blockIdx.x, 0);
 
-    const int t0 = u.tok_begin;
-    int t1 = u.tok_end;
     if (tid == 0) {
         tma_prefetch_descriptor(&k_map);
         tma_prefetch_descriptor(&v_map);
@@ -169,84 +175,102 @@ __global__ void __launch_bounds__(kMmaThreads) decode_attn_mma_kernel(const Kern
         sm_flags[0] = 0;
         mbar_init_fence();
     }
+    decode_attn_unit_t u = load_unit(p.units, blockIdx.x);
     __syncthreads();
-    if (tid == 0) DA_TRACE_STAMP(uid, 1);
+    if (tid == 0) DA_TRACE_STAMP(blockIdx.x, 1);
     // Everything above touched only the plan's own work list and kernel parameters.  What the
     // kernel launched before this one may have produced (q, new K/V rows, lengths, page
     // mappings) is read only past this point; with a programmatic dependency the lines above
     // overlap that kernel's tail.
     pdl_wait_primary();
 
-    // Invariant 2 (never run on stale lengths): the device length is fetched now and compared
-    // in the epilogue, off the critical path; a mismatch voids the block's result.  Reads stay
-    // inside the planned range and page ids are range-checked, so nothing can fault meanwhile.
-    int dev_len = u.seq_len;
-    if (MODE == kModeAttend) {
-        dev_len = __ldg(p.seq_lens + b);
-        if (p.run_mask != nullptr && __ldg(p.run_mask + b) == 0) t1 = t0;   // masked row reads no KV
-    }
-    const int n_pages = (t1 - t0 + 15) >> 4;
-    const int n_iters = (n_pages + kPagesPerStage - 1) / kPagesPerStage;
-
-    // per-warp results (consumers only)
-    float oacc[D / 16][4];
-    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
-#pragma unroll
-    for (int i = 0; i < D / 16; ++i) oacc[i][0] = oacc[i][1] = oacc[i][2] = oacc[i][3] = 0.f;
-    uint32_t probe_sum = 0;
-
     if (warp == kMmaConsumerWarps) {
         // ------------------------------------------------------------ producer
-        const int32_t* bt = p.block_table + (int64_t)b * p.max_pages_per_seq + (t0 >> 4);
-        int ids_next = (lane < n_pages) ? __ldg(bt + lane) : 0;
-        int ids_cur = 0;
-        bool alive = true;
         const uint64_t l2_policy = l2_policy_evict_first();
-        for (int it = 0; it < n_iters && alive; ++it) {
-            if ((it & 7) == 0) {                                          // 32 page ids per 8 stages, one batch ahead
-                ids_cur = ids_next;
-                const int nxt = (it + 8) * kPagesPerStage + lane;
-                ids_next = (nxt < n_pages) ? __ldg(bt + nxt) : 0;
-            }
-            const int s = it % NS;
-            const uint32_t parity = ((it / NS) & 1) ^ 1;
-            if (it >= NS) {
-                bool ok = true;
-                if (lane == 0) ok = mbar_wait(bar_base + 8 * (NS + s), parity);
-                ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
-                if (!ok) {
-                    if (lane == 0) {
-                        record_status(p.status, DA_ERR_TIMEOUT);
-                        sm_flags[0] = 1;
+        uint32_t git = 0;                                     // stages issued so far, over all units
+        bool alive = true;
+        for (int uid = blockIdx.x; uid < n_units && alive; uid += gridDim.x) {
+            decode_attn_unit_t nu = u;
+            if (uid + (int)gridDim.x < n_units) nu = load_unit(p.units, uid + gridDim.x);   // lands while this unit streams
+            const int b = u.seq, g = u.kv_head;
+            const int t0 = u.tok_begin;
+            int t1 = u.tok_end;
+            if (MODE == kModeAttend && p.run_mask != nullptr && __ldg(p.run_mask + b) == 0) t1 = t0;   // masked row reads no KV
+            if (MODE == kModeGather && b != ex.gather_seq) t1 = t0;
+            const int n_pages = (t1 - t0 + 15) >> 4;
+            const int n_iters = (n_pages + kPagesPerStage - 1) / kPagesPerStage;
+            const int32_t* bt = p.block_table + (int64_t)b * p.max_pages_per_seq + (t0 >> 4);
+            int ids_next = (lane < n_pages) ? __ldg(bt + lane) : 0;
+            int ids_cur = 0;
+            for (int it = 0; it < n_iters; ++it, ++git) {
+                if ((it & 7) == 0) {                                      // 32 page ids per 8 stages, one batch ahead
+                    ids_cur = ids_next;
+                    const int nxt = (it + 8) * kPagesPerStage + lane;
+                    ids_next = (nxt < n_pages) ? __ldg(bt + nxt) : 0;
+                }
+                const int s = git % NS;
+                if (git >= (uint32_t)NS) {
+                    bool ok = true;
+                    if (lane == 0) ok = mbar_wait(bar_base + 8 * (NS + s), ((git / NS) & 1) ^ 1);
+                    ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+                    if (!ok) {
+                        if (lane == 0) {
+                            record_status(p.status, DA_ERR_TIMEOUT);
+                            sm_flags[0] = 1;
+                        }
+                        alive = false;
+                        break;
                     }
-                    alive = false;
-                    break;
+                }
+                const int pages_here = min(kPagesPerStage, n_pages - it * kPagesPerStage);
+                const uint32_t full = bar_base + 8 * s;
+                if (lane == 0) mbar_arrive_expect_tx(full, (uint32_t)pages_here * 2u * Cfg::kPageBytes);
+                __syncwarp();
+                // lane j issues one box: page j / (2*halves), tensor (K, V), half of the head dimension
+                constexpr int OPS_PER_PAGE = 2 * Cfg::kHalves;
+                const int pg = lane / OPS_PER_PAGE;
+                const int which = (lane % OPS_PER_PAGE) / Cfg::kHalves;   // 0: K, 1: V
+                const int hf = lane % Cfg::kHalves;
+                int page_id = __shfl_sync(0xffffffffu, ids_cur, ((it & 7) * kPagesPerStage + pg) & 31);
+                if (lane < pages_here * OPS_PER_PAGE) {
+                    if ((unsigned)page_id >= (unsigned)p.num_pages) {     // never hand TMA a page outside the pool
+                        record_status(p.status, DA_ERR_BAD_PAGE);
+                        page_id = 0;
+                    }
+                    const uint32_t dst = base + s * Cfg::kStageBytes + which * Cfg::kTensorBytes +
+                                         pg * Cfg::kPageBytes + hf * Cfg::kBoxBytes;
+                    tma_load_4d(dst, which ? &v_map : &k_map, full, hf * 64, 0, g, page_id, l2_policy);
+                    if (git == 0 && lane == 0) DA_TRACE_STAMP(blockIdx.x, 2);
                 }
             }
-            const int pages_here = min(kPagesPerStage, n_pages - it * kPagesPerStage);
-            const uint32_t full = bar_base + 8 * s;
-            if (lane == 0) mbar_arrive_expect_tx(full, (uint32_t)pages_here * 2u * Cfg::kPageBytes);
-            __syncwarp();
-            // lane j issues one box: page j / (2*halves), tensor (K, V), half of the head dimension
-            constexpr int OPS_PER_PAGE = 2 * Cfg::kHalves;
-            const int pg = lane / OPS_PER_PAGE;
-            const int which = (lane % OPS_PER_PAGE) / Cfg::kHalves;       // 0: K, 1: V
-            const int hf = lane % Cfg::kHalves;
-            int page_id = __shfl_sync(0xffffffffu, ids_cur, ((it & 7) * kPagesPerStage + pg) & 31);
-            if (lane < pages_here * OPS_PER_PAGE) {
-                if ((unsigned)page_id >= (unsigned)p.num_pages) {         // never hand TMA a page outside the pool
-                    record_status(p.status, DA_ERR_BAD_PAGE);
-                    page_id = 0;
-                }
-                const uint32_t dst = base + s * Cfg::kStageBytes + which * Cfg::kTensorBytes + pg * Cfg::kPageBytes +
-                                     hf * Cfg::kBoxBytes;
-                tma_load_4d(dst, which ? &v_map : &k_map, full, hf * 64, 0, g, page_id, l2_policy);
-                if (it == 0 && lane == 0) DA_TRACE_STAMP(uid, 2);
-            }
+            u = nu;
         }
-    } else {
-        // ------------------------------------------------------------ consumers
-        const int r = lane >> 2, c = lane & 3;
+        return;
+    }
+
+    // ---------------------------------------------------------------- consumers
+    const int r = lane >> 2, c = lane & 3;
+    const bool lo_role = DUP && (c >= 2);
+    uint32_t git = 0;                                         // stages consumed so far, over all units
+    uint32_t merge_parity = 0;
+    for (int uid = blockIdx.x; uid < n_units; uid += gridDim.x) {
+        if (uid != (int)blockIdx.x) u = load_unit(p.units, uid);
+        const bool last_unit = uid + (int)gridDim.x >= n_units;
+        const int b = u.seq, g = u.kv_head;
+        const int t0 = u.tok_begin;
+        int t1 = u.tok_end;
+        // Invariant 2 (never run on stale lengths): the device length is fetched now and compared
+        // at the end of the unit, off the critical path; a mismatch voids the unit's result.  Reads
+        // stay inside the planned range and page ids are range-checked, so nothing can fault.
+        int dev_len = u.seq_len;
+        if (MODE == kModeAttend) {
+            dev_len = __ldg(p.seq_lens + b);
+            if (p.run_mask != nullptr && __ldg(p.run_mask + b) == 0) t1 = t0;
+        }
+        if (MODE == kModeGather && b != ex.gather_seq) t1 = t0;
+        const int n_pages = (t1 - t0 + 15) >> 4;
+        const int n_iters = (n_pages + kPagesPerStage - 1) / kPagesPerStage;
+
         // Q^T as B fragments: column n = r is query head (r mod 4 when duplicated)
         uint32_t qb[KSTEPS][2];
         if (MODE == kModeAttend) {
@@ -259,20 +283,24 @@ __global__ void __launch_bounds__(kMmaThreads) decode_attn_mma_kernel(const Kern
                 qb[ks][1] = live ? __ldg(qrow + ks * 8 + 4 + c) : 0u;     // dims ks*16 + 8 + 2c, +1
             }
         }
-        const bool lo_role = DUP && (c >= 2);
-        bool alive = true;
-        for (int it = 0; it < n_iters && alive; ++it) {
-            const int s = it % NS;
-            const uint32_t parity = (it / NS) & 1;
-            if (!mbar_wait(bar_base + 8 * s, parity) || sm_flags[0] != 0) {
+        float oacc[D / 16][4];
+        float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+#pragma unroll
+        for (int i = 0; i < D / 16; ++i) oacc[i][0] = oacc[i][1] = oacc[i][2] = oacc[i][3] = 0.f;
+        uint32_t probe_sum = 0;
+        bool failed = false;
+
+        for (int it = 0; it < n_iters; ++it, ++git) {
+            const int s = git % NS;
+            if (!mbar_wait(bar_base + 8 * s, (git / NS) & 1) || sm_flags[0] != 0) {
                 if (lane == 0) {
                     record_status(p.status, DA_ERR_TIMEOUT);
                     sm_flags[0] = 1;
                 }
-                alive = false;
+                failed = true;
                 break;
             }
-            if (it == 0 && tid == 0) DA_TRACE_STAMP(uid, 3);
+            if (git == 0 && tid == 0) DA_TRACE_STAMP(blockIdx.x, 3);
             const int page_idx = it * kPagesPerStage + warp;
             if (page_idx < n_pages) {
                 const int tok0 = t0 + page_idx * 16;
@@ -302,12 +330,15 @@ __global__ void __launch_bounds__(kMmaThreads) decode_attn_mma_kernel(const Kern
                 } else {
                     if (n_valid < 16) {
                         // rows past the sequence end may hold anything (NaN patterns included) and a
-                        // zero weight does not silence them in an mma: clear those V rows
+                        // zero weight does not silence them in an mma: clear those V rows.  This is the
+                        // sequence's last page; the async-proxy fence orders the stores before the TMA
+                        // load that will reuse the stage for the next unit.
                         for (int i = lane; i < (16 - n_valid) * (D / 8); i += 32) {
                             const int row = n_valid + i / (D / 8), ch = i % (D / 8);
                             const uint32_t a = vpage + (ch >> 3) * Cfg::kBoxBytes + swz(row, ch & 7);
                             asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0u) : "memory");
                         }
+                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                         __syncwarp();
                     }
                     // ---- S^T = K . Q^T
@@ -377,31 +408,24 @@ __global__ void __launch_bounds__(kMmaThreads) decode_attn_mma_kernel(const Kern
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_base + 8 * (NS + s));          // this warp is done with the stage
         }
-    }
+        if (uid == (int)blockIdx.x && tid == 0) DA_TRACE_STAMP(blockIdx.x, 4);
+        if (last_unit && MODE == kModeAttend) pdl_launch_dependents();    // the combine kernel may start getting scheduled
 
-    if (tid == 0) DA_TRACE_STAMP(uid, 4);
-    if (MODE == kModeAttend) pdl_launch_dependents();   // the combine kernel may start getting scheduled
-    __syncthreads();   // every issued tile has landed and been consumed: the stage memory is free
-    if (MODE == kModeProbe) {
+        if (MODE == kModeProbe) {
 #pragma unroll
-        for (int off = 16; off >= 1; off >>= 1) probe_sum ^= __shfl_xor_sync(0xffffffffu, probe_sum, off);
-        if (lane == 0 && warp < kMmaConsumerWarps) atomicXor(ex.checksum + uid, probe_sum);
-        return;
-    }
-    if (MODE == kModeGather) return;
+            for (int off = 16; off >= 1; off >>= 1) probe_sum ^= __shfl_xor_sync(0xffffffffu, probe_sum, off);
+            if (lane == 0) atomicXor(ex.checksum + uid, probe_sum);
+        }
+        if (MODE != kModeAttend) {
+            if (failed) return;
+            continue;
+        }
 
-    // ---------------------------------------------------------------- block epilogue
-    // scratch aliases stage memory: the four warps' accumulators [4][8][D], maxima and sums [4][8]
-    float* const sm_wo = reinterpret_cast<float*>(gbase);
-    float* const sm_wm = sm_wo + kMmaConsumerWarps * 8 * D;
-    float* const sm_wl = sm_wm + kMmaConsumerWarps * 8;
-    bool failed = sm_flags[0] != 0;
-    if (dev_len != u.seq_len) {                               // stale plan: void the result, report it
-        if (tid == 0) record_status(p.status, DA_ERR_STALE_PLAN);
-        failed = true;
-    }
-    if (warp < kMmaConsumerWarps) {
-        const int r = lane >> 2, c = lane & 3;
+        // ------------------------------------------------------------ end of the unit
+        if (dev_len != u.seq_len) {                               // stale plan: void the result, report it
+            if (tid == 0) record_status(p.status, DA_ERR_STALE_PLAN);
+            failed = true;
+        }
 #pragma unroll
         for (int off = 4; off <= 16; off <<= 1) {
             l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], off);
@@ -411,26 +435,38 @@ __global__ void __launch_bounds__(kMmaThreads) decode_attn_mma_kernel(const Kern
             m_run[0] = m_run[1] = -INFINITY;
             l_run[0] = l_run[1] = 0.f;
         }
-        if (r == 0) {
-            sm_wm[warp * 8 + 2 * c] = m_run[0];
-            sm_wm[warp * 8 + 2 * c + 1] = m_run[1];
-            sm_wl[warp * 8 + 2 * c] = l_run[0];
-            sm_wl[warp * 8 + 2 * c + 1] = l_run[1];
-        }
-        float* wo = sm_wo + warp * 8 * D;
+        block_sync(1, kConsumerThreads);          // every warp is done reading the previous unit's results
+        if (DUP) {
+            // columns 4..7 carried the low parts of P for heads 0..3: lanes c = 2, 3 hand theirs to c = 0, 1
 #pragma unroll
-        for (int mt = 0; mt < D / 16; ++mt) {
-            wo[(2 * c) * D + mt * 16 + r] = oacc[mt][0];
-            wo[(2 * c + 1) * D + mt * 16 + r] = oacc[mt][1];
-            wo[(2 * c) * D + mt * 16 + r + 8] = oacc[mt][2];
-            wo[(2 * c + 1) * D + mt * 16 + r + 8] = oacc[mt][3];
+            for (int mt = 0; mt < D / 16; ++mt)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) oacc[mt][i] += __shfl_down_sync(0xffffffffu, oacc[mt][i], 2);
         }
+        if (!DUP || c < 2) {
+            if (r == 0) {
+                sm_wm[warp * COLS + 2 * c] = m_run[0];
+                sm_wm[warp * COLS + 2 * c + 1] = m_run[1];
+                sm_wl[warp * COLS + 2 * c] = l_run[0];
+                sm_wl[warp * COLS + 2 * c + 1] = l_run[1];
+            }
+            float* wo = sm_wo + warp * COLS * D;
+#pragma unroll
+            for (int mt = 0; mt < D / 16; ++mt) {
+                wo[(2 * c) * D + mt * 16 + r] = oacc[mt][0];
+                wo[(2 * c + 1) * D + mt * 16 + r] = oacc[mt][1];
+                wo[(2 * c) * D + mt * 16 + r + 8] = oacc[mt][2];
+                wo[(2 * c + 1) * D + mt * 16 + r + 8] = oacc[mt][3];
+            }
+        }
+        block_sync(1, kConsumerThreads);
+        // the in-kernel merge may take the stage ring as scratch only when nothing more will land in it
+        const int cap = last_unit ? (((NS * Cfg::kStageBytes - 64 - 4 * G) / (rec_floats(G, D) * 4 + 4 * G)) & ~3) : 0;
+        block_finish<D, kMmaConsumerWarps, COLS, false>(p, u, G, sm_wo, sm_wm, sm_wl, sm_ticket, bar_base + 8 * 2 * NS,
+                                                        &merge_parity, tid, kConsumerThreads, 1, gbase, cap);
+        if (uid == (int)blockIdx.x && tid == 0) DA_TRACE_STAMP(blockIdx.x, 6);
+        if (failed && sm_flags[0] != 0) return;
     }
-    __syncthreads();
-    const int cap = ((NS * Cfg::kStageBytes - 64 - 4 * G) / (rec_floats(G, D) * 4 + 4 * G)) & ~3;
-    block_finish<D, kMmaConsumerWarps, 8, DUP>(p, u, G, sm_wo, sm_wm, sm_wl, sm_ticket, bar_base + 8 * 2 * NS, tid,
-                                               kMmaThreads, gbase, cap);
-    if (tid == 0) DA_TRACE_STAMP(uid, 6);
 }
 
 // ---------------------------------------------------------------- host side
@@ -485,14 +521,19 @@ inline mma_kernel_t mma_kernel_for(int D, int G)
     return nullptr;
 }
 
-inline int mma_smem_bytes(int D) { return D == 128 ? MmaCfg<128>::kSmemBytes : MmaCfg<64>::kSmemBytes; }
+inline int mma_smem_bytes(int D, int G)
+{
+    const bool dup = G <= 4;
+    if (D == 128) return dup ? MmaCfg<128, true>::kSmemBytes : MmaCfg<128, false>::kSmemBytes;
+    return dup ? MmaCfg<64, true>::kSmemBytes : MmaCfg<64, false>::kSmemBytes;
+}
 
 template <int MODE>
 inline int mma_prepare(int D, int G, mma_kernel_t* fn_out)
 {
     mma_kernel_t fn = mma_kernel_for<MODE>(D, G);
     if (!fn) return DA_ERR_UNSUPPORTED;
-    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, mma_smem_bytes(D)) != cudaSuccess) {
+    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, mma_smem_bytes(D, G)) != cudaSuccess) {
         (void)cudaGetLastError();
         return DA_ERR_CUDA;
     }
@@ -505,9 +546,9 @@ inline int mma_query_occupancy(int D, int G, int* block_threads, int* dyn_smem)
     mma_kernel_t fn;
     if (mma_prepare<kModeAttend>(D, G, &fn) != DA_OK) return -1;
     *block_threads = kMmaThreads;
-    *dyn_smem = mma_smem_bytes(D);
+    *dyn_smem = mma_smem_bytes(D, G);
     int n = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, fn, kMmaThreads, mma_smem_bytes(D)) != cudaSuccess) {
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, fn, kMmaThreads, mma_smem_bytes(D, G)) != cudaSuccess) {
         (void)cudaGetLastError();
         return -1;
     }
@@ -531,7 +572,7 @@ inline int mma_launch_mode(const decode_attn_shape_t& s, int G, const KernelPara
     cudaLaunchConfig_t cfg;
     cfg.gridDim = dim3(grid, 1, 1);
     cfg.blockDim = dim3(kMmaThreads, 1, 1);
-    cfg.dynamicSmemBytes = (size_t)mma_smem_bytes(s.head_dim);
+    cfg.dynamicSmemBytes = (size_t)mma_smem_bytes(s.head_dim, G);
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -552,9 +593,9 @@ inline int mma_launch(const decode_attn_shape_t& s, int G, const KernelParams& k
 }
 
 inline int mma_gather_probe(const decode_attn_shape_t& s, int G, const KernelParams& kp, uint32_t* checksum,
-                            unsigned grid, cudaStream_t stream)
+                            unsigned n_units, unsigned grid, cudaStream_t stream)
 {
-    if (cudaMemsetAsync(checksum, 0, sizeof(uint32_t) * grid, stream) != cudaSuccess) {
+    if (cudaMemsetAsync(checksum, 0, sizeof(uint32_t) * n_units, stream) != cudaSuccess) {
         (void)cudaGetLastError();
         return DA_ERR_CUDA;
     }

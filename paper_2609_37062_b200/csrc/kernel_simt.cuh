@@ -57,7 +57,7 @@ __global__ void __launch_bounds__(kSimtThreads) decode_attn_simt_kernel(const Ke
     __shared__ int sm_ticket;
 
     const int uid = blockIdx.x;
-    if (p.grid_exit && uid >= p.header->n_units) return;   // surplus blocks of a capacity launch
+    if (uid >= (p.grid_exit ? p.header->n_units : p.n_units)) return;   // surplus blocks of a capacity launch
     const decode_attn_unit_t u = load_unit(p.units, uid);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int rg = warp * RPW + lane / LPR;     // row group of this thread
@@ -194,8 +194,9 @@ __global__ void __launch_bounds__(kSimtThreads) decode_attn_simt_kernel(const Ke
         dst[1] = make_float4(acc[h][4], acc[h][5], acc[h][6], acc[h][7]);
     }
     __syncthreads();
+    uint32_t merge_parity = 0;
     block_finish<D, ROWS, G, false>(p, u, G, &sm_acc[0][0][0], &sm_rm[0][0], &sm_rl[0][0], &sm_ticket,
-                                    smem_u32(&sm_merge_bar), tid, kSimtThreads, sm_raw, ROWS);
+                                    smem_u32(&sm_merge_bar), &merge_parity, tid, kSimtThreads, 0, sm_raw, ROWS);
 }
 
 }  // namespace da
