@@ -189,18 +189,33 @@ __global__ void __launch_bounds__(kMmaThreads) decode_attn_mma_kernel(const Kern
         const uint64_t l2_policy = l2_policy_evict_first();
         uint32_t git = 0;                                     // stages issued so far, over all units
         bool alive = true;
+        // range of a unit as this launch sees it: a masked row (or, in the gather mode, another
+        // sequence) has nothing to read
+        auto unit_end = [&](const decode_attn_unit_t& x) {
+            int e = x.tok_end;
+            if (MODE == kModeAttend && p.run_mask != nullptr && __ldg(p.run_mask + x.seq) == 0) e = x.tok_begin;
+            if (MODE == kModeGather && x.seq != ex.gather_seq) e = x.tok_begin;
+            return e;
+        };
+        auto first_ids = [&](const decode_attn_unit_t& x, int end) {
+            const int np = (end - x.tok_begin + 15) >> 4;
+            const int32_t* t = p.block_table + (int64_t)x.seq * p.max_pages_per_seq + (x.tok_begin >> 4);
+            return (lane < np) ? __ldg(t + lane) : 0;
+        };
+        int t1 = unit_end(u);
+        int ids_first = first_ids(u, t1);
         for (int uid = blockIdx.x; uid < n_units && alive; uid += gridDim.x) {
+            const bool has_next = uid + (int)gridDim.x < n_units;
             decode_attn_unit_t nu = u;
-            if (uid + (int)gridDim.x < n_units) nu = load_unit(p.units, uid + gridDim.x);   // lands while this unit streams
+            if (has_next) nu = load_unit(p.units, uid + gridDim.x);       // lands while this unit streams
+            int nt1 = 0, nids_first = 0;
+            bool next_ready = false;
             const int b = u.seq, g = u.kv_head;
             const int t0 = u.tok_begin;
-            int t1 = u.tok_end;
-            if (MODE == kModeAttend && p.run_mask != nullptr && __ldg(p.run_mask + b) == 0) t1 = t0;   // masked row reads no KV
-            if (MODE == kModeGather && b != ex.gather_seq) t1 = t0;
             const int n_pages = (t1 - t0 + 15) >> 4;
             const int n_iters = (n_pages + kPagesPerStage - 1) / kPagesPerStage;
             const int32_t* bt = p.block_table + (int64_t)b * p.max_pages_per_seq + (t0 >> 4);
-            int ids_next = (lane < n_pages) ? __ldg(bt + lane) : 0;
+            int ids_next = ids_first;
             int ids_cur = 0;
             for (int it = 0; it < n_iters; ++it, ++git) {
                 if ((it & 7) == 0) {                                      // 32 page ids per 8 stages, one batch ahead
@@ -242,8 +257,19 @@ __global__ void __launch_bounds__(kMmaThreads) decode_attn_mma_kernel(const Kern
                     tma_load_4d(dst, which ? &v_map : &k_map, full, hf * 64, 0, g, page_id, l2_policy);
                     if (git == 0 && lane == 0) DA_TRACE_STAMP(blockIdx.x, 2);
                 }
+                if (has_next && !next_ready) {                            // this unit is under way: look ahead
+                    nt1 = unit_end(nu);
+                    nids_first = first_ids(nu, nt1);
+                    next_ready = true;
+                }
+            }
+            if (has_next && !next_ready) {
+                nt1 = unit_end(nu);
+                nids_first = first_ids(nu, nt1);
             }
             u = nu;
+            t1 = nt1;
+            ids_first = nids_first;
         }
         return;
     }
@@ -253,36 +279,50 @@ __global__ void __launch_bounds__(kMmaThreads) decode_attn_mma_kernel(const Kern
     const bool lo_role = DUP && (c >= 2);
     uint32_t git = 0;                                         // stages consumed so far, over all units
     uint32_t merge_parity = 0;
+    // what a unit needs before its first tile: lengths / mask of its sequence and Q^T as B
+    // fragments (column n = r is query head r, or r mod 4 when duplicated); fetched one unit ahead
+    struct Pre {
+        int dev_len;
+        int masked;
+        uint32_t qb[KSTEPS][2];
+    };
+    auto prefetch = [&](const decode_attn_unit_t& x, Pre& o) {
+        o.dev_len = x.seq_len;
+        o.masked = 0;
+        if (MODE == kModeAttend) {
+            o.dev_len = __ldg(p.seq_lens + x.seq);
+            if (p.run_mask != nullptr) o.masked = __ldg(p.run_mask + x.seq) == 0;
+            const int head = DUP ? (r & 3) : r;
+            const bool live = head < G;
+            const uint32_t* qrow = reinterpret_cast<const uint32_t*>(
+                p.q + ((int64_t)x.seq * p.num_q_heads + x.kv_head * G + (live ? head : 0)) * D);
+#pragma unroll
+            for (int ks = 0; ks < KSTEPS; ++ks) {
+                o.qb[ks][0] = live ? __ldg(qrow + ks * 8 + c) : 0u;         // dims ks*16 + 2c, +1
+                o.qb[ks][1] = live ? __ldg(qrow + ks * 8 + 4 + c) : 0u;     // dims ks*16 + 8 + 2c, +1
+            }
+        }
+    };
+    Pre cur;
+    prefetch(u, cur);
     for (int uid = blockIdx.x; uid < n_units; uid += gridDim.x) {
-        if (uid != (int)blockIdx.x) u = load_unit(p.units, uid);
         const bool last_unit = uid + (int)gridDim.x >= n_units;
+        decode_attn_unit_t nu = u;
+        if (!last_unit) nu = load_unit(p.units, uid + gridDim.x);         // lands while this unit is consumed
+        Pre nxt = cur;
         const int b = u.seq, g = u.kv_head;
         const int t0 = u.tok_begin;
         int t1 = u.tok_end;
-        // Invariant 2 (never run on stale lengths): the device length is fetched now and compared
-        // at the end of the unit, off the critical path; a mismatch voids the unit's result.  Reads
-        // stay inside the planned range and page ids are range-checked, so nothing can fault.
-        int dev_len = u.seq_len;
-        if (MODE == kModeAttend) {
-            dev_len = __ldg(p.seq_lens + b);
-            if (p.run_mask != nullptr && __ldg(p.run_mask + b) == 0) t1 = t0;
-        }
+        // Invariant 2 (never run on stale lengths): the device length was fetched ahead and is
+        // compared at the end of the unit, off the critical path; a mismatch voids the unit's
+        // result.  Reads stay inside the planned range and page ids are range-checked.
+        const int dev_len = cur.dev_len;
+        if (cur.masked) t1 = t0;                                           // masked row reads no KV
         if (MODE == kModeGather && b != ex.gather_seq) t1 = t0;
         const int n_pages = (t1 - t0 + 15) >> 4;
         const int n_iters = (n_pages + kPagesPerStage - 1) / kPagesPerStage;
+        uint32_t (&qb)[KSTEPS][2] = cur.qb;
 
-        // Q^T as B fragments: column n = r is query head (r mod 4 when duplicated)
-        uint32_t qb[KSTEPS][2];
-        if (MODE == kModeAttend) {
-            const int head = DUP ? (r & 3) : r;
-            const bool live = head < G;
-            const uint32_t* qrow = reinterpret_cast<const uint32_t*>(p.q + ((int64_t)b * p.num_q_heads + g * G + (live ? head : 0)) * D);
-#pragma unroll
-            for (int ks = 0; ks < KSTEPS; ++ks) {
-                qb[ks][0] = live ? __ldg(qrow + ks * 8 + c) : 0u;         // dims ks*16 + 2c, +1
-                qb[ks][1] = live ? __ldg(qrow + ks * 8 + 4 + c) : 0u;     // dims ks*16 + 8 + 2c, +1
-            }
-        }
         float oacc[D / 16][4];
         float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
 #pragma unroll
@@ -410,6 +450,7 @@ __global__ void __launch_bounds__(kMmaThreads) decode_attn_mma_kernel(const Kern
         }
         if (uid == (int)blockIdx.x && tid == 0) DA_TRACE_STAMP(blockIdx.x, 4);
         if (last_unit && MODE == kModeAttend) pdl_launch_dependents();    // the combine kernel may start getting scheduled
+        if (!last_unit) prefetch(nu, nxt);                                // in flight during this unit's epilogue
 
         if (MODE == kModeProbe) {
 #pragma unroll
@@ -418,6 +459,8 @@ __global__ void __launch_bounds__(kMmaThreads) decode_attn_mma_kernel(const Kern
         }
         if (MODE != kModeAttend) {
             if (failed) return;
+            u = nu;
+            cur = nxt;
             continue;
         }
 
@@ -466,6 +509,8 @@ __global__ void __launch_bounds__(kMmaThreads) decode_attn_mma_kernel(const Kern
                                                         &merge_parity, tid, kConsumerThreads, 1, gbase, cap);
         if (uid == (int)blockIdx.x && tid == 0) DA_TRACE_STAMP(blockIdx.x, 6);
         if (failed && sm_flags[0] != 0) return;
+        u = nu;
+        cur = nxt;
     }
 }
 
