@@ -68,6 +68,8 @@ def parse_args():
     ap.add_argument("--skip-e2e", action="store_true")
     ap.add_argument("--probe", action="store_true", help="also time the gather-only probe")
     ap.add_argument("--copies", type=int, default=0, help="pool copies to rotate over (0: enough for 1 GiB)")
+    ap.add_argument("--prefix-aware", action="store_true",
+                    help="shared_prefix workload: tell the planner about the common prefix (attended once per block of sequences)")
     ap.add_argument("--mask-fraction", type=float, default=None,
                     help="RUN mask (Alg. 1 step 2): this fraction of the rows, picked by a seeded hash, reads no KV")
     return ap.parse_args()
@@ -249,7 +251,8 @@ def main():
     policy = da.make_policy(
         split_mode=da.DA_SPLIT_DETERMINISTIC if args.split == "deterministic" else da.DA_SPLIT_AUTO,
         chunk_tokens=args.chunk_tokens, kernel=kernel, fuse_combine=1 if args.fuse else 0,
-        ctas_per_sm=args.ctas_per_sm)
+        ctas_per_sm=args.ctas_per_sm,
+        shared_prefix_tokens=first.shared_prefix_tokens if args.prefix_aware else 0)
     shape = da.shape_of_workload(first)
     t0 = time.perf_counter()
     plan = da.decode_attn_plan(shape, policy, first.seq_lens)
@@ -419,6 +422,7 @@ def main():
                        "split": args.split, "chunk_tokens": info.chunk_tokens, "units": info.n_units,
                        "max_splits": info.max_splits_used, "kernel": kname, "ctas_per_sm": info.ctas_per_sm,
                        "fused_combine": bool(policy.fuse_combine), "cuda_graph": not args.no_graph,
+                       "shared_prefix_tokens": int(policy.shared_prefix_tokens),
                        "l2": f"rotating over {copies} physical pool copies ({copies * unique_bytes / 2**30:.2f} GiB)",
                        "plan_us": plan_us, "parallelism": f"dp{world} (sequences sharded, no collective)"},
             "pct_of_8tbs": value / world / 8000.0 * 100.0,

@@ -90,7 +90,14 @@ typedef struct {
                                blocks exit at once (Algorithm 1 step 6, "grid exit")                  */
     int32_t capacity_tokens;/* with capacity_batch: upper bound on sum(seq_lens) of any refresh      */
     int32_t ctas_per_sm;    /* 0: from the occupancy of the chosen kernel                            */
-    int32_t reserved[6];
+    int32_t shared_prefix_tokens; /* > 0: the caller promises that the first this-many tokens of every
+                               sequence live in the same physical pages (the block-table rows agree on
+                               their first shared_prefix_tokens / page_size entries, as with few-shot
+                               prompts served from a prefix cache).  A multiple of page_size, at most
+                               every seq_len.  The prefix is then attended once per block of
+                               sequences instead of once per sequence.  Tensor-core kernel, groups of
+                               up to 4 heads, separate combine, no capacity plan.                    */
+    int32_t reserved[5];
 } decode_attn_policy_t;
 
 typedef struct {
@@ -264,6 +271,14 @@ int decode_attn_last_device_status(const decode_attn_plan_t *plan, cudaStream_t 
  * ceil(seq_len / page_size) must lie in [0, num_pages). */
 int decode_attn_validate_block_table(const decode_attn_shape_t *shape, const int32_t *seq_lens_host,
                                      const int32_t *block_table_host);
+
+/* Host-only check of the promise behind policy.shared_prefix_tokens: every
+ * sequence is at least that long and every block-table row starts with the
+ * same shared_prefix_tokens / page_size page ids as row 0 (DA_ERR_BAD_PAGE if
+ * a row differs).  The prefix cache of the paper's engine serves few-shot
+ * prompts this way (Appendix J). */
+int decode_attn_validate_shared_prefix(const decode_attn_shape_t *shape, int32_t shared_prefix_tokens,
+                                       const int32_t *seq_lens_host, const int32_t *block_table_host);
 
 /* ---------------------------------------------------------------------------
  * Debug / measurement helpers that reuse the kernels' page addressing.

@@ -51,7 +51,7 @@ EXPORTED = [
     "decode_attn_validate_block_table", "decode_attn_debug_gather", "decode_attn_gather_probe",
     "decode_attn_host_step", "decode_attn_host_release", "decode_attn_strerror", "decode_attn_version",
     "decode_attn_step_static", "decode_attn_append_kv", "decode_attn_breakeven_tokens",
-    "decode_attn_switch_thresholds", "decode_attn_switch_next",
+    "decode_attn_switch_thresholds", "decode_attn_switch_next", "decode_attn_validate_shared_prefix",
 ]
 
 
@@ -61,7 +61,7 @@ class Policy(ctypes.Structure):
                 ("sm_count", ctypes.c_int32), ("kernel", ctypes.c_int32),
                 ("fuse_combine", ctypes.c_int32), ("capacity_batch", ctypes.c_int32),
                 ("capacity_tokens", ctypes.c_int32), ("ctas_per_sm", ctypes.c_int32),
-                ("reserved", ctypes.c_int32 * 6)]
+                ("shared_prefix_tokens", ctypes.c_int32), ("reserved", ctypes.c_int32 * 5)]
 
 
 class Shape(ctypes.Structure):
@@ -115,6 +115,7 @@ _lib.decode_attn_run_ex.argtypes = [_vp, ctypes.POINTER(RunArgs), _vp]
 _lib.decode_attn_combine.argtypes = [_vp, _vp, _vp, _vp, _vp]
 _lib.decode_attn_last_device_status.argtypes = [_vp, _vp]
 _lib.decode_attn_validate_block_table.argtypes = [ctypes.POINTER(Shape), _vp, _vp]
+_lib.decode_attn_validate_shared_prefix.argtypes = [ctypes.POINTER(Shape), ctypes.c_int32, _vp, _vp]
 _lib.decode_attn_debug_gather.argtypes = [_vp, ctypes.c_int32, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.decode_attn_gather_probe.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp]
 _lib.decode_attn_host_step.argtypes = [ctypes.POINTER(Shape), ctypes.POINTER(Policy), _vp, _vp, _vp,
@@ -178,11 +179,13 @@ def _host_i32(x) -> np.ndarray:
 
 def make_policy(split_mode: int = DA_SPLIT_AUTO, fixed_count: int = 0, chunk_tokens: int = 0,
                 max_splits: int = 0, sm_count: int = 0, kernel: int = DA_KERNEL_AUTO, fuse_combine: int = 0,
-                capacity_batch: int = 0, capacity_tokens: int = 0, ctas_per_sm: int = 0) -> Policy:
+                capacity_batch: int = 0, capacity_tokens: int = 0, ctas_per_sm: int = 0,
+                shared_prefix_tokens: int = 0) -> Policy:
     p = Policy()
     p.split_mode, p.fixed_count, p.chunk_tokens, p.max_splits = split_mode, fixed_count, chunk_tokens, max_splits
     p.sm_count, p.kernel, p.fuse_combine = sm_count, kernel, fuse_combine
     p.capacity_batch, p.capacity_tokens, p.ctas_per_sm = capacity_batch, capacity_tokens, ctas_per_sm
+    p.shared_prefix_tokens = shared_prefix_tokens
     return p
 
 
@@ -323,6 +326,12 @@ def decode_attn_validate_block_table(shape: Shape, seq_lens_host, block_table_ho
     lens = _host_i32(seq_lens_host)
     bt = _host_i32(block_table_host)
     return _lib.decode_attn_validate_block_table(ctypes.byref(shape), _ptr(lens), _ptr(bt))
+
+
+def decode_attn_validate_shared_prefix(shape: Shape, shared_prefix_tokens: int, seq_lens_host, block_table_host) -> int:
+    lens = _host_i32(seq_lens_host)
+    bt = _host_i32(block_table_host)
+    return _lib.decode_attn_validate_shared_prefix(ctypes.byref(shape), shared_prefix_tokens, _ptr(lens), _ptr(bt))
 
 
 def decode_attn_debug_gather(plan: Plan, seq: int, k_cache, v_cache, block_table, k_out, v_out, stream=None) -> None:

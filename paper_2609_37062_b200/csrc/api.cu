@@ -51,7 +51,8 @@ struct decode_attn_plan {
     char* dev = nullptr;
     char* pinned = nullptr;
     size_t upload_bytes = 0;
-    size_t off_units = 0, off_seq_info = 0, off_status = 0, off_tickets = 0, total_bytes = 0;
+    size_t off_units = 0, off_seq_info = 0, off_block_begin = 0, off_status = 0, off_tickets = 0, total_bytes = 0;
+    int max_bins = 0;        // > 0: the units are packed into per-block ranges (persistent tensor-core kernel)
     cudaStream_t stream = nullptr;
     cudaEvent_t upload_done = nullptr;  // last refresh of the device work list
     void* buffers = nullptr;            // PlanBuffers*, returned to the cache on destroy
@@ -198,7 +199,7 @@ int pick_kernel(const decode_attn_shape_t& s, const decode_attn_policy_t& p)
 }
 
 // Resident blocks per SM of the kernel a plan will launch.
-int query_occupancy(int kernel, int D, int G, int* block_threads, int* dyn_smem)
+int query_occupancy(int kernel, int D, int G, int* block_threads, int* dyn_smem, bool prefix = false)
 {
     int n = 0;
     if (kernel == DA_KERNEL_SIMT) {
@@ -212,7 +213,7 @@ int query_occupancy(int kernel, int D, int G, int* block_threads, int* dyn_smem)
         }
         return n;
     }
-    return mma_query_occupancy(D, G, block_threads, dyn_smem);
+    return mma_query_occupancy(D, G, block_threads, dyn_smem, prefix);
 }
 
 void fill_host_mirror(decode_attn_plan_t* pl)
@@ -227,6 +228,15 @@ void fill_host_mirror(decode_attn_plan_t* pl)
     for (int b = 0; b < pl->shape.batch; ++b) {
         si[b].slot_base = pl->layout.slot_base[b];
         si[b].n_splits = pl->layout.splits[b];
+        si[b].seq_len = pl->seq_lens[b];
+        si[b].pad = 0;
+    }
+    if (pl->max_bins > 0) {
+        // one range per launched block; blocks beyond the bins in use get an empty range
+        int32_t* bb = reinterpret_cast<int32_t*>(pl->pinned + pl->off_block_begin);
+        const std::vector<int32_t>& src = pl->layout.block_begin;
+        const int32_t end = (int32_t)pl->layout.units.size();
+        for (int64_t i = 0; i <= pl->grid; ++i) bb[i] = i < (int64_t)src.size() ? src[i] : end;
     }
 }
 
@@ -247,6 +257,7 @@ KernelParams make_params(const decode_attn_plan_t* pl, const decode_attn_run_arg
     kp.header = reinterpret_cast<const DevHeader*>(pl->dev);
     kp.units = reinterpret_cast<const decode_attn_unit_t*>(pl->dev + pl->off_units);
     kp.seq_info = reinterpret_cast<const SeqInfo*>(pl->dev + pl->off_seq_info);
+    kp.block_begin = pl->max_bins > 0 ? reinterpret_cast<const int32_t*>(pl->dev + pl->off_block_begin) : nullptr;
     kp.tickets = reinterpret_cast<int32_t*>(pl->dev + pl->off_tickets);
     kp.status = reinterpret_cast<int32_t*>(pl->dev + pl->off_status);
     kp.k_stride_page = s.k_stride_page; kp.k_stride_token = s.k_stride_token; kp.k_stride_head = s.k_stride_head;
@@ -302,12 +313,17 @@ int decode_attn_plan(const decode_attn_shape_t* shape, const decode_attn_policy_
     } else {
         DA_CUDA_TRY(cudaDeviceGetAttribute(&pl->sm_count, cudaDevAttrMultiProcessorCount, pl->device));
     }
-    int occ = query_occupancy(pl->kernel, shape->head_dim, pl->group, &pl->block_threads, &pl->dyn_smem);
+    const bool prefix = policy->shared_prefix_tokens > 0;
+    if (prefix && pl->kernel != DA_KERNEL_MMA_TMA) return DA_ERR_UNSUPPORTED;
+    int occ = query_occupancy(pl->kernel, shape->head_dim, pl->group, &pl->block_threads, &pl->dyn_smem, prefix);
     if (occ <= 0) return DA_ERR_CUDA;
     pl->ctas_per_sm = policy->ctas_per_sm > 0 ? policy->ctas_per_sm : occ;
 
     pl->seq_lens.assign(seq_lens_host, seq_lens_host + shape->batch);
-    rc = make_layout(*shape, *policy, pl->seq_lens.data(), pl->sm_count, pl->ctas_per_sm, pl->layout);
+    // The tensor-core kernel walks the work list with a fixed set of resident blocks unless the
+    // merge is fused, which needs one unit per block (its scratch is the stage ring).
+    if (pl->kernel == DA_KERNEL_MMA_TMA && !policy->fuse_combine) pl->max_bins = pl->sm_count * pl->ctas_per_sm;
+    rc = make_layout(*shape, *policy, pl->seq_lens.data(), pl->sm_count, pl->ctas_per_sm, pl->layout, pl->max_bins);
     if (rc != DA_OK) return rc;
 
     if (policy->capacity_batch > 0) {
@@ -324,16 +340,14 @@ int decode_attn_plan(const decode_attn_shape_t* shape, const decode_attn_policy_
         pl->grid = pl->max_units;
     }
     if (pl->grid > 0x7fffffffLL) return DA_ERR_UNSUPPORTED;
-    // The tensor-core kernel walks the work list with a fixed number of blocks (what fits on the
-    // machine at once) unless the merge is fused, which needs one unit per block.
-    if (pl->kernel == DA_KERNEL_MMA_TMA && !policy->fuse_combine)
-        pl->grid = std::min<int64_t>(pl->grid, (int64_t)pl->sm_count * pl->ctas_per_sm);
+    if (pl->max_bins > 0) pl->grid = std::min<int64_t>(pl->grid, pl->max_bins);
 
     pl->workspace_bytes = (size_t)pl->max_slots * shape->num_kv_heads * rec_floats(pl->group, shape->head_dim) * sizeof(float);
 
     pl->off_units = align_up(sizeof(DevHeader), 32);
     pl->off_seq_info = pl->off_units + align_up((size_t)std::max<int64_t>(pl->max_units, 1) * sizeof(decode_attn_unit_t), 32);
-    pl->upload_bytes = pl->off_seq_info + align_up((size_t)std::max<int64_t>(pl->max_batch, 1) * sizeof(SeqInfo), 32);
+    pl->off_block_begin = pl->off_seq_info + align_up((size_t)std::max<int64_t>(pl->max_batch, 1) * sizeof(SeqInfo), 32);
+    pl->upload_bytes = pl->off_block_begin + align_up((size_t)(pl->grid + 1) * sizeof(int32_t), 32);
     pl->off_status = pl->upload_bytes;
     pl->off_tickets = pl->off_status + 32;
     pl->total_bytes = pl->off_tickets +
@@ -371,7 +385,7 @@ int decode_attn_plan_update(decode_attn_plan_t* pl, int32_t batch, const int32_t
     decode_attn_shape_t s = pl->shape;
     s.batch = batch;
     Layout lay;
-    int rc = make_layout(s, pl->policy, seq_lens_host, pl->sm_count, pl->ctas_per_sm, lay);
+    int rc = make_layout(s, pl->policy, seq_lens_host, pl->sm_count, pl->ctas_per_sm, lay, pl->max_bins);
     if (rc != DA_OK) return rc;
     if ((int64_t)lay.units.size() > pl->max_units || lay.n_slots > pl->max_slots) return DA_ERR_INVALID_ARG;
     // the previous refresh may still be reading the pinned mirror
@@ -455,7 +469,7 @@ int decode_attn_run_ex(const decode_attn_plan_t* pl, const decode_attn_run_args_
         int rc = simt_launch(fn, kp, (unsigned)pl->grid, stream);
         if (rc != DA_OK) return rc;
     } else {
-        int rc = mma_launch(pl->shape, pl->group, kp, (unsigned)pl->grid, stream);
+        int rc = mma_launch(pl->shape, pl->group, kp, (unsigned)pl->grid, stream, pl->policy.shared_prefix_tokens > 0);
         if (rc != DA_OK) return rc;
     }
     DA_CUDA_TRY(cudaGetLastError());
@@ -528,11 +542,30 @@ int decode_attn_validate_block_table(const decode_attn_shape_t* shape, const int
     return DA_OK;
 }
 
+int decode_attn_validate_shared_prefix(const decode_attn_shape_t* shape, int32_t shared_prefix_tokens,
+                                       const int32_t* seq_lens_host, const int32_t* block_table_host)
+{
+    if (!shape || shared_prefix_tokens < 0 || (shape->batch > 0 && (!seq_lens_host || !block_table_host)))
+        return DA_ERR_INVALID_ARG;
+    int rc = validate_shape(*shape);
+    if (rc != DA_OK) return rc;
+    if (shared_prefix_tokens % shape->page_size != 0) return DA_ERR_INVALID_ARG;
+    const int64_t pages = shared_prefix_tokens / shape->page_size;
+    if (pages > shape->max_pages_per_seq) return DA_ERR_INVALID_ARG;
+    for (int b = 0; b < shape->batch; ++b) {
+        if (seq_lens_host[b] < shared_prefix_tokens) return DA_ERR_INVALID_ARG;
+        for (int64_t i = 0; i < pages; ++i)
+            if (block_table_host[(int64_t)b * shape->max_pages_per_seq + i] != block_table_host[i]) return DA_ERR_BAD_PAGE;
+    }
+    return DA_OK;
+}
+
 int decode_attn_debug_gather(const decode_attn_plan_t* pl, int32_t seq, const void* k_cache, const void* v_cache,
                              const int32_t* block_table, void* k_out, void* v_out, cudaStream_t stream)
 {
     if (!pl || !k_cache || !v_cache || !block_table || !k_out || !v_out) return DA_ERR_INVALID_ARG;
     if (seq < 0 || seq >= pl->shape.batch) return DA_ERR_INVALID_ARG;
+    if (pl->policy.shared_prefix_tokens > 0) return DA_ERR_UNSUPPORTED;
     if (!aligned(k_cache, 16) || !aligned(v_cache, 16) || !aligned(k_out, 16) || !aligned(v_out, 16))
         return DA_ERR_INVALID_ARG;
     if (pl->grid == 0) return DA_OK;
@@ -548,6 +581,7 @@ int decode_attn_gather_probe(const decode_attn_plan_t* pl, const void* k_cache, 
 {
     if (!pl || !k_cache || !v_cache || !block_table || !checksum_out) return DA_ERR_INVALID_ARG;
     if (!aligned(k_cache, 16) || !aligned(v_cache, 16)) return DA_ERR_INVALID_ARG;
+    if (pl->policy.shared_prefix_tokens > 0) return DA_ERR_UNSUPPORTED;
     if (pl->grid == 0) return DA_OK;
     decode_attn_run_args_t a;
     std::memset(&a, 0, sizeof a);
@@ -800,6 +834,8 @@ int decode_attn_step_static(const decode_attn_shape_t* shape, const int32_t* seq
     for (int b = 0; b < shape->batch; ++b) {
         si[b].slot_base = lay.slot_base[b];
         si[b].n_splits = lay.splits[b];
+        si[b].seq_len = seq_lens_host[b];
+        si[b].pad = 0;
     }
     const size_t upload = kStaticOffSeqInfo + sizeof(SeqInfo) * (size_t)shape->batch;
     // The array keeps the previous call's contents: the status word and tickets must start at zero.

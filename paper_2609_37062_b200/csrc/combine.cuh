@@ -36,7 +36,7 @@ __global__ void __launch_bounds__(kCombineThreads) decode_attn_combine_kernel(co
     const int b = bg / p.num_kv_heads, g = bg % p.num_kv_heads;
     if (b >= p.header->batch) return;                     // rows past the live batch of a capacity plan
     const SeqInfo si = p.seq_info[b];
-    if (si.n_splits <= 1 || si.slot_base < 0) return;     // written directly by the partial kernel
+    if (si.slot_base < 0) return;                         // a single split, written directly by the partial kernel
     const int S = si.n_splits;
     const int q = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int col = slice * 32 + lane;

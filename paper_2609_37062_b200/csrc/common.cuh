@@ -20,8 +20,10 @@ struct DevHeader {
 };
 
 struct SeqInfo {
-    int32_t slot_base;  // -1: single split
+    int32_t slot_base;  // -1: single split, written directly
     int32_t n_splits;
+    int32_t seq_len;    // the length the plan was made for
+    int32_t pad;
 };
 
 struct KernelParams {
@@ -37,6 +39,7 @@ struct KernelParams {
     const DevHeader* header;
     const decode_attn_unit_t* units;
     const SeqInfo* seq_info;
+    const int32_t* block_begin;  // [grid + 1]: block b walks units block_begin[b] .. block_begin[b+1]; NULL: unit b
     int32_t* tickets;  // [batch][Hkv], zero between launches
     int32_t* status;   // worst da_status_t seen by any block (0 = ok)
     int64_t k_stride_page, k_stride_token, k_stride_head;

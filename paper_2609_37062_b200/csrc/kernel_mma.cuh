@@ -1,8 +1,9 @@
 // Tensor-core split-KV partial kernel with TMA-staged pages.
 //
 // A block is four consumer warps and one producer warp.  It works through
-// the units blockIdx.x, blockIdx.x + gridDim.x, ... of the work list (a unit
-// is one sequence, one KV head, a run of pages) without ever draining its
+// its share of the work list - units block_begin[b] .. block_begin[b+1], packed
+// by the planner so that every block gets about the same cost (a unit is one
+// sequence, one KV head, a run of pages) - without ever draining its
 // pipeline: the producer keeps filling the ring of stages with the next
 // unit's pages while the consumers finish the previous unit.  With a grid as
 // large as the work list every block has one unit.  The producer turns block-table entries into
@@ -136,8 +137,8 @@ struct MmaExtra {
     int32_t gather_seq;
 };
 
-template <int D, bool DUP, int MODE>
-__global__ void __launch_bounds__(kMmaThreads) decode_attn_mma_kernel(const KernelParams p,
+template <int D, bool DUP, int MODE, bool PREFIX>
+__global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const KernelParams p,
                                                                       const __grid_constant__ CUtensorMap k_map,
                                                                       const __grid_constant__ CUtensorMap v_map,
                                                                       const int G, const MmaExtra ex)
@@ -159,8 +160,17 @@ __global__ void __launch_bounds__(kMmaThreads) decode_attn_mma_kernel(const Kern
     float* const sm_wm = sm_wo + kMmaConsumerWarps * COLS * D;                                           // [4][COLS]
     float* const sm_wl = sm_wm + kMmaConsumerWarps * COLS;                                               // [4][COLS]
 
-    const int n_units = p.grid_exit ? p.header->n_units : p.n_units;
-    if ((int)blockIdx.x >= n_units) return;                   // surplus blocks of a capacity launch
+    // this block's units: a range of the work list (the planner's packing), or just unit blockIdx.x
+    int ubeg, uend;
+    if (p.block_begin != nullptr) {
+        ubeg = __ldg(p.block_begin + blockIdx.x);
+        uend = __ldg(p.block_begin + blockIdx.x + 1);
+    } else {
+        const int n_units = p.grid_exit ? p.header->n_units : p.n_units;
+        ubeg = blockIdx.x;
+        uend = min(n_units, (int)blockIdx.x + 1);
+    }
+    if (ubeg >= uend) return;                                 // surplus blocks of a capacity launch
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     if (tid == 0) DA_TRACE_STAMP(blockIdx.x, 0);
 
@@ -175,7 +185,7 @@ __global__ void __launch_bounds__(kMmaThreads) decode_attn_mma_kernel(const Kern
         sm_flags[0] = 0;
         mbar_init_fence();
     }
-    decode_attn_unit_t u = load_unit(p.units, blockIdx.x);
+    decode_attn_unit_t u = load_unit(p.units, ubeg);
     __syncthreads();
     if (tid == 0) DA_TRACE_STAMP(blockIdx.x, 1);
     // Everything above touched only the plan's own work list and kernel parameters.  What the
@@ -193,7 +203,8 @@ __global__ void __launch_bounds__(kMmaThreads) decode_attn_mma_kernel(const Kern
         // sequence) has nothing to read
         auto unit_end = [&](const decode_attn_unit_t& x) {
             int e = x.tok_end;
-            if (MODE == kModeAttend && p.run_mask != nullptr && __ldg(p.run_mask + x.seq) == 0) e = x.tok_begin;
+            if (MODE == kModeAttend && p.run_mask != nullptr && (x.kv_head >> 16) == 0 && __ldg(p.run_mask + x.seq) == 0)
+                e = x.tok_begin;
             if (MODE == kModeGather && x.seq != ex.gather_seq) e = x.tok_begin;
             return e;
         };
@@ -204,13 +215,13 @@ __global__ void __launch_bounds__(kMmaThreads) decode_attn_mma_kernel(const Kern
         };
         int t1 = unit_end(u);
         int ids_first = first_ids(u, t1);
-        for (int uid = blockIdx.x; uid < n_units && alive; uid += gridDim.x) {
-            const bool has_next = uid + (int)gridDim.x < n_units;
+        for (int uid = ubeg; uid < uend && alive; ++uid) {
+            const bool has_next = uid + 1 < uend;
             decode_attn_unit_t nu = u;
-            if (has_next) nu = load_unit(p.units, uid + gridDim.x);       // lands while this unit streams
+            if (has_next) nu = load_unit(p.units, uid + 1);               // lands while this unit streams
             int nt1 = 0, nids_first = 0;
             bool next_ready = false;
-            const int b = u.seq, g = u.kv_head;
+            const int b = u.seq, g = u.kv_head & 0xffff;   // (a shared-prefix unit keeps its block size in the high half)
             const int t0 = u.tok_begin;
             const int n_pages = (t1 - t0 + 15) >> 4;
             const int n_iters = (n_pages + kPagesPerStage - 1) / kPagesPerStage;
@@ -295,7 +306,7 @@ __global__ void __launch_bounds__(kMmaThreads) decode_attn_mma_kernel(const Kern
             const int head = DUP ? (r & 3) : r;
             const bool live = head < G;
             const uint32_t* qrow = reinterpret_cast<const uint32_t*>(
-                p.q + ((int64_t)x.seq * p.num_q_heads + x.kv_head * G + (live ? head : 0)) * D);
+                p.q + ((int64_t)x.seq * p.num_q_heads + (x.kv_head & 0xffff) * G + (live ? head : 0)) * D);
 #pragma unroll
             for (int ks = 0; ks < KSTEPS; ++ks) {
                 o.qb[ks][0] = live ? __ldg(qrow + ks * 8 + c) : 0u;         // dims ks*16 + 2c, +1
@@ -305,23 +316,211 @@ __global__ void __launch_bounds__(kMmaThreads) decode_attn_mma_kernel(const Kern
     };
     Pre cur;
     prefetch(u, cur);
-    for (int uid = blockIdx.x; uid < n_units; uid += gridDim.x) {
-        const bool last_unit = uid + (int)gridDim.x >= n_units;
+    for (int uid = ubeg; uid < uend; ++uid) {
+        const bool last_unit = uid + 1 >= uend;
         decode_attn_unit_t nu = u;
-        if (!last_unit) nu = load_unit(p.units, uid + gridDim.x);         // lands while this unit is consumed
+        if (!last_unit) nu = load_unit(p.units, uid + 1);                 // lands while this unit is consumed
         Pre nxt = cur;
-        const int b = u.seq, g = u.kv_head;
+        const int b = u.seq, g = u.kv_head & 0xffff;
+        const int nseq = u.kv_head >> 16;                                  // > 0: a shared-prefix unit
         const int t0 = u.tok_begin;
         int t1 = u.tok_end;
         // Invariant 2 (never run on stale lengths): the device length was fetched ahead and is
         // compared at the end of the unit, off the critical path; a mismatch voids the unit's
         // result.  Reads stay inside the planned range and page ids are range-checked.
         const int dev_len = cur.dev_len;
-        if (cur.masked) t1 = t0;                                           // masked row reads no KV
+        if (cur.masked && nseq == 0) t1 = t0;                              // masked row reads no KV
         if (MODE == kModeGather && b != ex.gather_seq) t1 = t0;
         const int n_pages = (t1 - t0 + 15) >> 4;
         const int n_iters = (n_pages + kPagesPerStage - 1) / kPagesPerStage;
         uint32_t (&qb)[KSTEPS][2] = cur.qb;
+
+        if (PREFIX && MODE == kModeAttend && nseq > 0) {
+            // -------------------------------------------------------- shared-prefix unit
+            // The pages of this chunk are the same physical pages for every sequence of the block,
+            // so the block's query rows (sequence j, head h -> column j*G + h, 16 columns in two
+            // tiles) are attended in one pass: each K/V tile is read once for all of them.  P keeps
+            // its low part through a second mma.
+            constexpr int NT = 2;
+            const int spb = 16 / G;                                         // sequences per block
+            uint32_t pq[KSTEPS][NT][2];
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                const int col = nt * 8 + r, j = col / G, h = col - j * G;
+                const bool live = j < nseq && j < spb;
+                const uint32_t* qrow = reinterpret_cast<const uint32_t*>(
+                    p.q + ((int64_t)(b + (live ? j : 0)) * p.num_q_heads + g * G + h) * D);
+#pragma unroll
+                for (int ks = 0; ks < KSTEPS; ++ks) {
+                    pq[ks][nt][0] = live ? __ldg(qrow + ks * 8 + c) : 0u;
+                    pq[ks][nt][1] = live ? __ldg(qrow + ks * 8 + 4 + c) : 0u;
+                }
+            }
+            float pacc[D / 16][NT][4];
+            float pm[NT][2], pl[NT][2];
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                pm[nt][0] = pm[nt][1] = -INFINITY;
+                pl[nt][0] = pl[nt][1] = 0.f;
+#pragma unroll
+                for (int mt = 0; mt < D / 16; ++mt) pacc[mt][nt][0] = pacc[mt][nt][1] = pacc[mt][nt][2] = pacc[mt][nt][3] = 0.f;
+            }
+            bool pfailed = false;
+            for (int it = 0; it < n_iters; ++it, ++git) {
+                const int s = git % NS;
+                if (!mbar_wait(bar_base + 8 * s, (git / NS) & 1) || sm_flags[0] != 0) {
+                    if (lane == 0) {
+                        record_status(p.status, DA_ERR_TIMEOUT);
+                        sm_flags[0] = 1;
+                    }
+                    pfailed = true;
+                    break;
+                }
+                const int page_idx = it * kPagesPerStage + warp;
+                if (page_idx < n_pages) {                                   // prefix pages are always full
+                    const uint32_t kpage = base + s * Cfg::kStageBytes + warp * Cfg::kPageBytes;
+                    const uint32_t vpage = kpage + Cfg::kTensorBytes;
+                    float sacc[NT][4];
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) sacc[nt][0] = sacc[nt][1] = sacc[nt][2] = sacc[nt][3] = 0.f;
+                    const int arow = (lane & 7) + ((lane >> 3) & 1) * 8;
+                    const int achk = lane >> 4;
+#pragma unroll
+                    for (int ks = 0; ks < KSTEPS; ++ks) {
+                        uint32_t a[4];
+                        ldsm_x4(kpage + (ks >> 2) * Cfg::kBoxBytes + swz(arow, (ks & 3) * 2 + achk), a);
+#pragma unroll
+                        for (int nt = 0; nt < NT; ++nt) mma_bf16_16816(sacc[nt], a, pq[ks][nt][0], pq[ks][nt][1]);
+                    }
+                    uint32_t bh[NT][2], bl[NT][2];
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) {
+                        const float s00 = sacc[nt][0] * p.scale_log2, s01 = sacc[nt][1] * p.scale_log2;
+                        const float s10 = sacc[nt][2] * p.scale_log2, s11 = sacc[nt][3] * p.scale_log2;
+                        float mx0 = fmaxf(s00, s10), mx1 = fmaxf(s01, s11);
+#pragma unroll
+                        for (int off = 4; off <= 16; off <<= 1) {
+                            mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, off));
+                            mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, off));
+                        }
+                        const float mn0 = fmaxf(pm[nt][0], mx0), mn1 = fmaxf(pm[nt][1], mx1);
+                        const float al0 = ex2f(pm[nt][0] - mn0), al1 = ex2f(pm[nt][1] - mn1);
+                        pm[nt][0] = mn0;
+                        pm[nt][1] = mn1;
+                        const float p00 = ex2f(s00 - mn0), p01 = ex2f(s01 - mn1);
+                        const float p10 = ex2f(s10 - mn0), p11 = ex2f(s11 - mn1);
+                        pl[nt][0] = fmaf(pl[nt][0], al0, p00 + p10);
+                        pl[nt][1] = fmaf(pl[nt][1], al1, p01 + p11);
+                        if (__any_sync(0xffffffffu, al0 != 1.f || al1 != 1.f)) {
+#pragma unroll
+                            for (int mt = 0; mt < D / 16; ++mt) {
+                                pacc[mt][nt][0] *= al0; pacc[mt][nt][1] *= al1;
+                                pacc[mt][nt][2] *= al0; pacc[mt][nt][3] *= al1;
+                            }
+                        }
+                        const uint32_t hi0 = pack_bf16(p00, p01), hi1 = pack_bf16(p10, p11);
+                        const uint32_t lo0 = pack_bf16(p00 - __uint_as_float(hi0 << 16), p01 - __uint_as_float(hi0 & 0xffff0000u));
+                        const uint32_t lo1 = pack_bf16(p10 - __uint_as_float(hi1 << 16), p11 - __uint_as_float(hi1 & 0xffff0000u));
+                        bh[nt][0] = movmatrix_trans(hi0);
+                        bh[nt][1] = movmatrix_trans(hi1);
+                        bl[nt][0] = movmatrix_trans(lo0);
+                        bl[nt][1] = movmatrix_trans(lo1);
+                    }
+                    const int vrow = (lane & 7) + (lane >> 4) * 8;
+                    const int vchk = (lane >> 3) & 1;
+#pragma unroll
+                    for (int mt = 0; mt < D / 16; ++mt) {
+                        uint32_t a[4];
+                        ldsm_x4_trans(vpage + (mt >> 2) * Cfg::kBoxBytes + swz(vrow, (mt & 3) * 2 + vchk), a);
+#pragma unroll
+                        for (int nt = 0; nt < NT; ++nt) {
+                            mma_bf16_16816(pacc[mt][nt], a, bh[nt][0], bh[nt][1]);
+                            mma_bf16_16816(pacc[mt][nt], a, bl[nt][0], bl[nt][1]);
+                        }
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_base + 8 * (NS + s));
+            }
+            if (last_unit) pdl_launch_dependents();
+            if (!last_unit) prefetch(nu, nxt);
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+#pragma unroll
+                for (int off = 4; off <= 16; off <<= 1) {
+                    pl[nt][0] += __shfl_xor_sync(0xffffffffu, pl[nt][0], off);
+                    pl[nt][1] += __shfl_xor_sync(0xffffffffu, pl[nt][1], off);
+                }
+                if (pfailed) {
+                    pm[nt][0] = pm[nt][1] = -INFINITY;
+                    pl[nt][0] = pl[nt][1] = 0.f;
+                }
+            }
+            // The warps' results go through the block's scratch four columns at a time (it holds
+            // [4 warps][4 columns][D]): columns 4q .. 4q+3 live in tile q / 2, lanes c = 2 (q % 2), +1.
+            const int RF = rec_floats(G, D);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int nt = q >> 1;
+                block_sync(1, kConsumerThreads);                            // the scratch is free again
+                if ((c >> 1) == (q & 1)) {
+                    const int lc = 2 * (c & 1);                             // local columns lc, lc + 1
+                    if (r == 0) {
+                        sm_wm[warp * COLS + lc] = pm[nt][0];
+                        sm_wm[warp * COLS + lc + 1] = pm[nt][1];
+                        sm_wl[warp * COLS + lc] = pl[nt][0];
+                        sm_wl[warp * COLS + lc + 1] = pl[nt][1];
+                    }
+                    float* wo = sm_wo + (warp * COLS + lc) * D;
+#pragma unroll
+                    for (int mt = 0; mt < D / 16; ++mt) {
+                        wo[mt * 16 + r] = pacc[mt][nt][0];
+                        wo[D + mt * 16 + r] = pacc[mt][nt][1];
+                        wo[mt * 16 + r + 8] = pacc[mt][nt][2];
+                        wo[D + mt * 16 + r + 8] = pacc[mt][nt][3];
+                    }
+                }
+                block_sync(1, kConsumerThreads);
+                for (int task = tid; task < 4 * (D / 4); task += kConsumerThreads) {
+                    const int lc = task / (D / 4), d4 = task % (D / 4);
+                    const int col = 4 * q + lc;
+                    const int j = col / G, h = col - j * G;
+                    if (j >= nseq || j >= spb) continue;
+                    const SeqInfo si = p.seq_info[b + j];
+                    bool dead = p.run_mask != nullptr && __ldg(p.run_mask + b + j) == 0;      // masked row: an empty record
+                    if (__ldg(p.seq_lens + b + j) != si.seq_len) {                            // stale plan: void, report
+                        if (d4 == 0 && h == 0) record_status(p.status, DA_ERR_STALE_PLAN);
+                        dead = true;
+                    }
+                    float M = -INFINITY;
+#pragma unroll
+                    for (int w = 0; w < kMmaConsumerWarps; ++w) M = fmaxf(M, sm_wm[w * COLS + lc]);
+                    float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+                    float ls = 0.f;
+                    if (M != -INFINITY && !dead) {
+#pragma unroll
+                        for (int w = 0; w < kMmaConsumerWarps; ++w) {
+                            const float wgt = ex2f(sm_wm[w * COLS + lc] - M);
+                            const float4 v = reinterpret_cast<const float4*>(sm_wo)[(w * COLS + lc) * (D / 4) + d4];
+                            o.x = fmaf(wgt, v.x, o.x);
+                            o.y = fmaf(wgt, v.y, o.y);
+                            o.z = fmaf(wgt, v.z, o.z);
+                            o.w = fmaf(wgt, v.w, o.w);
+                            ls = fmaf(wgt, sm_wl[w * COLS + lc], ls);
+                        }
+                    } else {
+                        M = -INFINITY;
+                    }
+                    float* rec = p.ws + ((int64_t)(si.slot_base + u.split_index) * p.num_kv_heads + g) * RF;
+                    __stcg(reinterpret_cast<float4*>(rec + h * D) + d4, o);
+                    if (d4 == 0) __stcg(reinterpret_cast<float2*>(rec + G * D) + h, make_float2(M, ls));
+                }
+            }
+            if (pfailed) return;
+            u = nu;
+            cur = nxt;
+            continue;
+        }
 
         float oacc[D / 16][4];
         float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
@@ -448,7 +647,7 @@ __global__ void __launch_bounds__(kMmaThreads) decode_attn_mma_kernel(const Kern
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_base + 8 * (NS + s));          // this warp is done with the stage
         }
-        if (uid == (int)blockIdx.x && tid == 0) DA_TRACE_STAMP(blockIdx.x, 4);
+        if (uid == ubeg && tid == 0) DA_TRACE_STAMP(blockIdx.x, 4);
         if (last_unit && MODE == kModeAttend) pdl_launch_dependents();    // the combine kernel may start getting scheduled
         if (!last_unit) prefetch(nu, nxt);                                // in flight during this unit's epilogue
 
@@ -507,7 +706,7 @@ __global__ void __launch_bounds__(kMmaThreads) decode_attn_mma_kernel(const Kern
         const int cap = last_unit ? (((NS * Cfg::kStageBytes - 64 - 4 * G) / (rec_floats(G, D) * 4 + 4 * G)) & ~3) : 0;
         block_finish<D, kMmaConsumerWarps, COLS, false>(p, u, G, sm_wo, sm_wm, sm_wl, sm_ticket, bar_base + 8 * 2 * NS,
                                                         &merge_parity, tid, kConsumerThreads, 1, gbase, cap);
-        if (uid == (int)blockIdx.x && tid == 0) DA_TRACE_STAMP(blockIdx.x, 6);
+        if (uid == ubeg && tid == 0) DA_TRACE_STAMP(blockIdx.x, 6);
         if (failed && sm_flags[0] != 0) return;
         u = nu;
         cur = nxt;
@@ -558,11 +757,17 @@ inline int make_pool_map(CUtensorMap* map, const void* pool, const decode_attn_s
 typedef void (*mma_kernel_t)(const KernelParams, const CUtensorMap, const CUtensorMap, const int, const MmaExtra);
 
 template <int MODE>
-inline mma_kernel_t mma_kernel_for(int D, int G)
+inline mma_kernel_t mma_kernel_for(int D, int G, bool prefix = false)
 {
     const bool dup = G <= 4;
-    if (D == 128) return dup ? decode_attn_mma_kernel<128, true, MODE> : decode_attn_mma_kernel<128, false, MODE>;
-    if (D == 64) return dup ? decode_attn_mma_kernel<64, true, MODE> : decode_attn_mma_kernel<64, false, MODE>;
+    if (prefix) {   // shared-prefix plans: attention mode, groups of up to 4 heads
+        if (MODE != kModeAttend || !dup) return nullptr;
+        if (D == 128) return decode_attn_mma_kernel<128, true, kModeAttend, true>;
+        if (D == 64) return decode_attn_mma_kernel<64, true, kModeAttend, true>;
+        return nullptr;
+    }
+    if (D == 128) return dup ? decode_attn_mma_kernel<128, true, MODE, false> : decode_attn_mma_kernel<128, false, MODE, false>;
+    if (D == 64) return dup ? decode_attn_mma_kernel<64, true, MODE, false> : decode_attn_mma_kernel<64, false, MODE, false>;
     return nullptr;
 }
 
@@ -574,9 +779,9 @@ inline int mma_smem_bytes(int D, int G)
 }
 
 template <int MODE>
-inline int mma_prepare(int D, int G, mma_kernel_t* fn_out)
+inline int mma_prepare(int D, int G, mma_kernel_t* fn_out, bool prefix = false)
 {
-    mma_kernel_t fn = mma_kernel_for<MODE>(D, G);
+    mma_kernel_t fn = mma_kernel_for<MODE>(D, G, prefix);
     if (!fn) return DA_ERR_UNSUPPORTED;
     if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, mma_smem_bytes(D, G)) != cudaSuccess) {
         (void)cudaGetLastError();
@@ -586,10 +791,10 @@ inline int mma_prepare(int D, int G, mma_kernel_t* fn_out)
     return DA_OK;
 }
 
-inline int mma_query_occupancy(int D, int G, int* block_threads, int* dyn_smem)
+inline int mma_query_occupancy(int D, int G, int* block_threads, int* dyn_smem, bool prefix = false)
 {
     mma_kernel_t fn;
-    if (mma_prepare<kModeAttend>(D, G, &fn) != DA_OK) return -1;
+    if (mma_prepare<kModeAttend>(D, G, &fn, prefix) != DA_OK) return -1;
     *block_threads = kMmaThreads;
     *dyn_smem = mma_smem_bytes(D, G);
     int n = 0;
@@ -602,10 +807,10 @@ inline int mma_query_occupancy(int D, int G, int* block_threads, int* dyn_smem)
 
 template <int MODE>
 inline int mma_launch_mode(const decode_attn_shape_t& s, int G, const KernelParams& kp, const MmaExtra& ex,
-                           unsigned grid, cudaStream_t stream)
+                           unsigned grid, cudaStream_t stream, bool prefix = false)
 {
     mma_kernel_t fn;
-    int rc = mma_prepare<MODE>(s.head_dim, G, &fn);
+    int rc = mma_prepare<MODE>(s.head_dim, G, &fn, prefix);
     if (rc != DA_OK) return rc;
     CUtensorMap kmap, vmap;
     rc = make_pool_map(&kmap, kp.k, s, s.k_stride_page, s.k_stride_token, s.k_stride_head);
@@ -631,10 +836,11 @@ inline int mma_launch_mode(const decode_attn_shape_t& s, int G, const KernelPara
     return DA_OK;
 }
 
-inline int mma_launch(const decode_attn_shape_t& s, int G, const KernelParams& kp, unsigned grid, cudaStream_t stream)
+inline int mma_launch(const decode_attn_shape_t& s, int G, const KernelParams& kp, unsigned grid, cudaStream_t stream,
+                      bool prefix = false)
 {
     MmaExtra ex = {nullptr, nullptr, nullptr, 0};
-    return mma_launch_mode<kModeAttend>(s, G, kp, ex, grid, stream);
+    return mma_launch_mode<kModeAttend>(s, G, kp, ex, grid, stream, prefix);
 }
 
 inline int mma_gather_probe(const decode_attn_shape_t& s, int G, const KernelParams& kp, uint32_t* checksum,

@@ -21,6 +21,9 @@
 
 #include <algorithm>
 #include <cmath>
+#include <functional>
+#include <queue>
+#include <utility>
 
 namespace da {
 
@@ -65,6 +68,11 @@ int validate_policy(const decode_attn_shape_t& s, const decode_attn_policy_t& p)
     if (p.fuse_combine != 0 && p.fuse_combine != 1) return DA_ERR_INVALID_ARG;
     if (p.capacity_batch > 0 && (p.capacity_tokens <= 0 || s.batch > p.capacity_batch))
         return DA_ERR_INVALID_ARG;
+    if (p.shared_prefix_tokens < 0 || p.shared_prefix_tokens % s.page_size != 0) return DA_ERR_INVALID_ARG;
+    if (p.shared_prefix_tokens > 0) {
+        if (p.fuse_combine || p.capacity_batch > 0 || p.split_mode == DA_SPLIT_FIXED_COUNT) return DA_ERR_UNSUPPORTED;
+        if (p.kernel == DA_KERNEL_SIMT || s.num_q_heads / s.num_kv_heads > 4) return DA_ERR_UNSUPPORTED;
+    }
     for (int32_t r : p.reserved)
         if (r != 0) return DA_ERR_INVALID_ARG;
     return DA_OK;
@@ -116,17 +124,22 @@ int64_t units_for_chunk(const std::vector<int64_t>& pages, int64_t c, int max_sp
 }  // namespace
 
 int make_layout(const decode_attn_shape_t& s, const decode_attn_policy_t& p, const int32_t* seq_lens,
-                int sm_count, int ctas_per_sm, Layout& out)
+                int sm_count, int ctas_per_sm, Layout& out, int max_bins)
 {
     if (sm_count <= 0 || ctas_per_sm <= 0) return DA_ERR_INVALID_ARG;
     if (s.batch > 0 && seq_lens == nullptr) return DA_ERR_INVALID_ARG;
     const int B = s.batch, P = s.page_size, H = s.num_kv_heads;
     const int max_splits = max_splits_of(p);
+    // With a shared prefix the ordinary units cover only what follows it; the prefix itself is
+    // cut into chunks attended once for a block of sequences at a time (see below).
+    const int64_t prefix_tokens = p.shared_prefix_tokens;
+    const int64_t prefix_pages = prefix_tokens / P;
     std::vector<int64_t> pages(B);
     for (int b = 0; b < B; ++b) {
         if (seq_lens[b] < 0) return DA_ERR_INVALID_ARG;
-        pages[b] = ceil_div(seq_lens[b], P);
-        if (pages[b] > s.max_pages_per_seq) return DA_ERR_INVALID_ARG;
+        if (ceil_div(seq_lens[b], P) > s.max_pages_per_seq) return DA_ERR_INVALID_ARG;
+        if (seq_lens[b] < prefix_tokens) return DA_ERR_INVALID_ARG;   // every sequence contains the prefix
+        pages[b] = ceil_div(seq_lens[b] - prefix_tokens, P);
     }
 
     std::vector<SeqCut> cuts(B);
@@ -176,22 +189,65 @@ int make_layout(const decode_attn_shape_t& s, const decode_attn_policy_t& p, con
         int64_t cost;
     };
     std::vector<Keyed> keyed;
+
+    // Shared prefix: a unit is (block of sequences, KV head, chunk of the prefix); the query rows
+    // of the block's sequences form the columns of one tensor-core tile, so a prefix page is
+    // fetched once per block instead of once per sequence.
+    const int G = s.num_q_heads / s.num_kv_heads;
+    const int seqs_per_block = prefix_tokens > 0 ? kPrefixColumns / G : 1;
+    int32_t PC = 0;
+    if (prefix_tokens > 0 && B > 0) {
+        const int64_t blocks = ceil_div(B, seqs_per_block);
+        const int64_t slots = (int64_t)sm_count * ctas_per_sm;
+        const int64_t max_chunks = std::max<int64_t>(1, prefix_pages / 8);       // chunks of >= 128 tokens
+        PC = (int32_t)std::min<int64_t>(max_chunks, std::max<int64_t>(1, slots / (H * blocks)));
+        if (p.split_mode == DA_SPLIT_DETERMINISTIC) {
+            const int64_t c = min_chunk_pages(s, p);                             // cuts at multiples of the chunk
+            PC = (int32_t)std::max<int64_t>(1, ceil_div(prefix_pages, c));
+        }
+        PC = std::min<int32_t>(PC, max_splits / 2);
+        for (int64_t j = 0; j < blocks; ++j) {
+            const int b0 = (int)(j * seqs_per_block);
+            const int nseq = std::min(seqs_per_block, B - b0);
+            for (int32_t i = 0; i < PC; ++i) {
+                const int64_t q = prefix_pages / PC, r = prefix_pages % PC;
+                const int64_t pb = i * q + std::min<int64_t>(i, r);
+                const int64_t pe = pb + q + (i < r ? 1 : 0);
+                for (int g = 0; g < H; ++g) {
+                    Keyed k;
+                    k.u.seq = b0;
+                    k.u.kv_head = g | (nseq << 16);          // high half: sequences in the block
+                    k.u.tok_begin = (int32_t)(pb * P);
+                    k.u.tok_end = (int32_t)(pe * P);
+                    k.u.slot = -2;                            // records go to each sequence's own slots
+                    k.u.seq_len = seq_lens[b0];
+                    k.u.split_index = i;
+                    k.u.n_splits = 0;
+                    k.cost = (pe - pb) * 4 + (1LL << 40);     // heavier per page, and first in the launch order
+                    keyed.push_back(k);
+                }
+            }
+        }
+    }
+
     for (int b = 0; b < B; ++b) {
         const SeqCut& cut = cuts[b];
-        const int32_t S = cut.splits;
+        const bool has_suffix = prefix_tokens == 0 || cut.pages > 0;
+        const int32_t S_own = has_suffix ? cut.splits : 0;
+        const int32_t S = PC + S_own;
         out.splits[b] = S;
         out.max_splits_used = std::max(out.max_splits_used, S);
         int64_t base_slot = -1;
-        if (S > 1) {
+        if (S > 1 || prefix_tokens > 0) {
             base_slot = out.n_slots;
             out.slot_base[b] = (int32_t)base_slot;
             out.n_slots += S;
             if (out.n_slots > INT32_MAX) return DA_ERR_UNSUPPORTED;
         }
-        for (int32_t i = 0; i < S; ++i) {
+        for (int32_t i = 0; i < S_own; ++i) {
             int64_t pb, pe;
             if (cut.even) {
-                const int64_t q = cut.pages / S, r = cut.pages % S;
+                const int64_t q = cut.pages / S_own, r = cut.pages % S_own;
                 pb = i * q + std::min<int64_t>(i, r);
                 pe = pb + q + (i < r ? 1 : 0);
             } else {
@@ -202,21 +258,47 @@ int make_layout(const decode_attn_shape_t& s, const decode_attn_policy_t& p, con
                 Keyed k;
                 k.u.seq = b;
                 k.u.kv_head = g;
-                k.u.tok_begin = (int32_t)(pb * P);
-                k.u.tok_end = (int32_t)std::min<int64_t>(pe * P, seq_lens[b]);
+                k.u.tok_begin = (int32_t)((prefix_pages + pb) * P);
+                k.u.tok_end = (int32_t)std::min<int64_t>((prefix_pages + pe) * P, seq_lens[b]);
                 if (k.u.tok_end < k.u.tok_begin) k.u.tok_end = k.u.tok_begin;
-                k.u.slot = S > 1 ? (int32_t)(base_slot + i) : -1;
+                k.u.slot = base_slot >= 0 ? (int32_t)(base_slot + PC + i) : -1;
                 k.u.seq_len = seq_lens[b];
-                k.u.split_index = i;
+                k.u.split_index = PC + i;
                 k.u.n_splits = S;
                 k.cost = pe - pb;
                 keyed.push_back(k);
             }
         }
     }
+    out.prefix_chunks = PC;
     std::stable_sort(keyed.begin(), keyed.end(), [](const Keyed& a, const Keyed& b) { return a.cost > b.cost; });
+    out.units.clear();
     out.units.reserve(keyed.size());
-    for (const Keyed& k : keyed) out.units.push_back(k.u);
+    out.block_begin.clear();
+    if (max_bins <= 0 || keyed.empty()) {
+        for (const Keyed& k : keyed) out.units.push_back(k.u);
+        return DA_OK;
+    }
+    // Longest unit first onto the lightest bin.  A unit costs its pages (a shared-prefix page
+    // counts four times: it is attended for a whole block of sequences) plus a fixed charge for
+    // the hand-over between units.
+    constexpr int64_t kHandOverPages = 24;
+    const int bins = (int)std::min<int64_t>((int64_t)keyed.size(), max_bins);
+    std::vector<std::vector<int32_t>> members(bins);
+    std::priority_queue<std::pair<int64_t, int>, std::vector<std::pair<int64_t, int>>, std::greater<>> heap;
+    for (int i = 0; i < bins; ++i) heap.push({0, i});
+    for (size_t i = 0; i < keyed.size(); ++i) {
+        auto [load, bin] = heap.top();
+        heap.pop();
+        members[bin].push_back((int32_t)i);
+        heap.push({load + (keyed[i].cost & ((1LL << 40) - 1)) + kHandOverPages, bin});
+    }
+    out.block_begin.reserve(bins + 1);
+    for (int b = 0; b < bins; ++b) {
+        out.block_begin.push_back((int32_t)out.units.size());
+        for (int32_t i : members[b]) out.units.push_back(keyed[i].u);
+    }
+    out.block_begin.push_back((int32_t)out.units.size());
     return DA_OK;
 }
 

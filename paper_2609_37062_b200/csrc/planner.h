@@ -14,6 +14,7 @@ constexpr int kDefaultAutoMinChunk = 256;         // tokens
 constexpr int kDefaultMaxSplits = 512;
 constexpr int kMaxSplits = 1024;  // hard bound on the splits of one sequence
 constexpr int kMaxGroup = 8;
+constexpr int kPrefixColumns = 16;  // query rows (sequence x head) one shared-prefix unit attends at once
 
 struct Layout {
     std::vector<decode_attn_unit_t> units;  // launch order: most expensive first
@@ -22,6 +23,8 @@ struct Layout {
     int64_t n_slots = 0;
     int32_t chunk_tokens = 0;
     int32_t max_splits_used = 0;
+    int32_t prefix_chunks = 0;              // chunks the shared prefix is cut into (0: no shared prefix)
+    std::vector<int32_t> block_begin;       // [bins + 1] when the units were packed into bins, else empty
 };
 
 // Validates the fields the planner and the kernels rely on.
@@ -29,8 +32,11 @@ int validate_shape(const decode_attn_shape_t& s);
 int validate_policy(const decode_attn_shape_t& s, const decode_attn_policy_t& p);
 
 // Fills `out` for the given lengths.  sm_count and ctas_per_sm must be > 0.
+// max_bins > 0: the units are additionally packed into min(units, max_bins) bins of about equal
+// cost (longest unit first onto the lightest bin) and stored bin by bin; block b of the persistent
+// kernel walks bin b.
 int make_layout(const decode_attn_shape_t& s, const decode_attn_policy_t& p, const int32_t* seq_lens,
-                int sm_count, int ctas_per_sm, Layout& out);
+                int sm_count, int ctas_per_sm, Layout& out, int max_bins = 0);
 
 // Upper bounds for a capacity plan (any batch <= capacity_batch and
 // sum(seq_lens) <= capacity_tokens).

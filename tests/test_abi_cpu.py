@@ -42,7 +42,7 @@ def test_version_and_strerror():
 
 def test_struct_sizes_match_the_header():
     assert ctypes.sizeof(da.Unit) == 32
-    assert ctypes.sizeof(da.Policy) == 64
+    assert ctypes.sizeof(da.Policy) == 64 and da.Policy.shared_prefix_tokens.offset == 40
     assert ctypes.sizeof(da.Shape) == 96
     assert ctypes.sizeof(da.RunArgs) == 88
 
@@ -213,3 +213,43 @@ def test_compute_entry_points_fail_loudly_without_a_device():
     with pytest.raises(da.DecodeAttnError) as e:
         da.decode_attn_plan(da.shape_of_workload(w), da.make_policy(), w.seq_lens)
     assert e.value.status == da.DA_ERR_CUDA
+
+
+def test_shared_prefix_layout_and_validation():
+    lens = wl.lengths_shared_prefix(37, 3, prefix=1536)
+    lens[5] = 1536                                            # a sequence that is nothing but the prefix
+    pol = da.make_policy(shared_prefix_tokens=1536, kernel=da.DA_KERNEL_MMA_TMA)
+    units, splits, slot_base, n_slots, _ = layout(lens, pol)
+    prefix_units = [u for u in units if u.kv_head >> 16]
+    own = [u for u in units if not (u.kv_head >> 16)]
+    assert units[: len(prefix_units)] == prefix_units          # launched first
+    blocks = (37 + 3) // 4
+    chunks = len({u.split_index for u in prefix_units})
+    assert len(prefix_units) == blocks * 8 * chunks
+    for u in prefix_units:
+        assert u.slot == -2 and 0 <= u.tok_begin < u.tok_end <= 1536 and 1 <= (u.kv_head >> 16) <= 4
+    assert sorted({u.kv_head >> 16 for u in prefix_units}) == [1, 4]          # the last block holds one sequence
+    # the prefix chunks tile [0, 1536) and every sequence's own units tile [1536, L)
+    cuts = sorted({(u.tok_begin, u.tok_end) for u in prefix_units})
+    assert cuts[0][0] == 0 and cuts[-1][1] == 1536 and all(a[1] == b[0] for a, b in zip(cuts, cuts[1:]))
+    for b, L in enumerate(lens):
+        mine = sorted([u for u in own if u.seq == b and u.kv_head == 0], key=lambda u: u.split_index)
+        assert splits[b] == chunks + len(mine) and slot_base[b] >= 0
+        pos = 1536
+        for i, u in enumerate(mine):
+            assert u.tok_begin == pos and u.split_index == chunks + i and u.slot == slot_base[b] + chunks + i
+            pos = u.tok_end
+        assert pos == L
+    assert n_slots == int(sum(splits))
+    with pytest.raises(da.DecodeAttnError):
+        layout([1000, 2000], pol)                             # shorter than the prefix
+    with pytest.raises(da.DecodeAttnError) as e:
+        layout(lens, da.make_policy(shared_prefix_tokens=1536, fuse_combine=1))
+    assert e.value.status == da.DA_ERR_UNSUPPORTED
+    w = wl.config_shared_prefix(batch=6, prefix=64)
+    s = da.shape_of_workload(w)
+    assert da.decode_attn_validate_shared_prefix(s, 64, w.seq_lens, w.block_table) == da.DA_OK
+    bt = w.block_table.clone()
+    bt[3, 2] = bt[3, 5]
+    assert da.decode_attn_validate_shared_prefix(s, 64, w.seq_lens, bt) == da.DA_ERR_BAD_PAGE
+    assert da.decode_attn_validate_shared_prefix(s, 60, w.seq_lens, w.block_table) == da.DA_ERR_INVALID_ARG
