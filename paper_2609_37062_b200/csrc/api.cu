@@ -198,8 +198,9 @@ int pick_kernel(const decode_attn_shape_t& s, const decode_attn_policy_t& p)
     return (G >= 2 && mma_supports(s.head_dim, G)) ? DA_KERNEL_MMA_TMA : DA_KERNEL_SIMT;
 }
 
-// Resident blocks per SM of the kernel a plan will launch.
-int query_occupancy(int kernel, int D, int G, int* block_threads, int* dyn_smem, bool prefix = false)
+// Resident blocks per SM of the kernel a plan will launch (the uncached query; it also opts the
+// kernel in to its dynamic shared memory).
+int query_occupancy_uncached(int kernel, int D, int G, int* block_threads, int* dyn_smem, bool prefix)
 {
     int n = 0;
     if (kernel == DA_KERNEL_SIMT) {
@@ -214,6 +215,60 @@ int query_occupancy(int kernel, int D, int G, int* block_threads, int* dyn_smem,
         return n;
     }
     return mma_query_occupancy(D, G, block_threads, dyn_smem, prefix);
+}
+
+// Plans are made every decode step: the answers that depend only on (device, kernel variant) are
+// kept after the first query.
+struct OccEntry {
+    int device, kernel, D, G, prefix, occ, block_threads, dyn_smem;
+};
+std::mutex g_occ_mu;
+std::vector<OccEntry> g_occ;
+std::vector<std::pair<int, int>> g_sm_counts;   // (device, multiprocessors)
+
+int query_occupancy(int kernel, int D, int G, int* block_threads, int* dyn_smem, bool prefix = false)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return -1;
+    }
+    {
+        std::lock_guard<std::mutex> lock(g_occ_mu);
+        for (const OccEntry& e : g_occ)
+            if (e.device == dev && e.kernel == kernel && e.D == D && e.G == G && e.prefix == (int)prefix) {
+                *block_threads = e.block_threads;
+                *dyn_smem = e.dyn_smem;
+                return e.occ;
+            }
+    }
+    const int occ = query_occupancy_uncached(kernel, D, G, block_threads, dyn_smem, prefix);
+    if (occ > 0) {
+        std::lock_guard<std::mutex> lock(g_occ_mu);
+        g_occ.push_back({dev, kernel, D, G, (int)prefix, occ, *block_threads, *dyn_smem});
+    }
+    return occ;
+}
+
+int device_sm_count(int dev, int* out)
+{
+    {
+        std::lock_guard<std::mutex> lock(g_occ_mu);
+        for (const auto& e : g_sm_counts)
+            if (e.first == dev) {
+                *out = e.second;
+                return DA_OK;
+            }
+    }
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return DA_ERR_CUDA;
+    }
+    std::lock_guard<std::mutex> lock(g_occ_mu);
+    g_sm_counts.push_back({dev, n});
+    *out = n;
+    return DA_OK;
 }
 
 void fill_host_mirror(decode_attn_plan_t* pl)
@@ -311,7 +366,8 @@ int decode_attn_plan(const decode_attn_shape_t* shape, const decode_attn_policy_
     if (policy->sm_count > 0) {
         pl->sm_count = policy->sm_count;
     } else {
-        DA_CUDA_TRY(cudaDeviceGetAttribute(&pl->sm_count, cudaDevAttrMultiProcessorCount, pl->device));
+        rc = device_sm_count(pl->device, &pl->sm_count);
+        if (rc != DA_OK) return rc;
     }
     const bool prefix = policy->shared_prefix_tokens > 0;
     if (prefix && pl->kernel != DA_KERNEL_MMA_TMA) return DA_ERR_UNSUPPORTED;
@@ -356,16 +412,16 @@ int decode_attn_plan(const decode_attn_shape_t* shape, const decode_attn_policy_
     PlanBuffers* pb = new (std::nothrow) PlanBuffers();
     if (!pb) return DA_ERR_INVALID_ARG;
     pl->buffers = pb;
-    rc = acquire_buffers(pl->device, pl->total_bytes, pl->upload_bytes, pb);
+    rc = acquire_buffers(pl->device, pl->total_bytes, pl->total_bytes, pb);
     if (rc != DA_OK) return rc;
     pl->dev = pb->dev;
     pl->pinned = pb->pinned;
     pl->stream = pb->stream;
     pl->upload_done = pb->event;
-    std::memset(pl->pinned, 0, pl->upload_bytes);
+    // one copy: work list, split table, block ranges, and zeros for the status word and tickets
+    std::memset(pl->pinned + pl->off_status, 0, pl->total_bytes - pl->off_status);
     fill_host_mirror(pl);
-    DA_CUDA_TRY(cudaMemsetAsync(pl->dev + pl->off_status, 0, pl->total_bytes - pl->off_status, pl->stream));
-    DA_CUDA_TRY(cudaMemcpyAsync(pl->dev, pl->pinned, pl->upload_bytes, cudaMemcpyHostToDevice, pl->stream));
+    DA_CUDA_TRY(cudaMemcpyAsync(pl->dev, pl->pinned, pl->total_bytes, cudaMemcpyHostToDevice, pl->stream));
     DA_CUDA_TRY(cudaStreamSynchronize(pl->stream));
 
     if (workspace_bytes_out) *workspace_bytes_out = pl->workspace_bytes;
