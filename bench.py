@@ -68,6 +68,8 @@ def parse_args():
     ap.add_argument("--skip-e2e", action="store_true")
     ap.add_argument("--probe", action="store_true", help="also time the gather-only probe")
     ap.add_argument("--copies", type=int, default=0, help="pool copies to rotate over (0: enough for 1 GiB)")
+    ap.add_argument("--alias-after", type=int, default=0,
+                    help="sweep cells too large for memory: sequences i >= K reuse the pages of sequence i mod K")
     ap.add_argument("--prefix-aware", action="store_true",
                     help="shared_prefix workload: tell the planner about the common prefix (attended once per block of sequences)")
     ap.add_argument("--mask-fraction", type=float, default=None,
@@ -75,7 +77,7 @@ def parse_args():
     return ap.parse_args()
 
 
-def make_workload(name, device, table_seed=None, seed_shift=0):
+def make_workload(name, device, table_seed=None, seed_shift=0, alias_after=None):
     from paper_2609_37062_b200 import workloads as wl
     if name == "tiny":
         return wl.config_tiny(device=device)
@@ -87,7 +89,8 @@ def make_workload(name, device, table_seed=None, seed_shift=0):
         return wl.config_shared_prefix(device=device, seed=3 + seed_shift, table_seed=table_seed)
     if name.startswith("sweep_"):
         ctx, batch = name[len("sweep_"):].split("x")
-        return wl.config_sweep_cell(int(ctx), int(batch), device=device, seed=4 + seed_shift, table_seed=table_seed)
+        return wl.config_sweep_cell(int(ctx), int(batch), device=device, seed=4 + seed_shift, table_seed=table_seed,
+                                    alias_after=alias_after)
     raise SystemExit(f"unknown workload {name}")
 
 
@@ -256,14 +259,15 @@ def main():
         torch.cuda.synchronize()
 
     # ---- inputs: R physical copies of the workload, this rank's own sequences
-    first = make_workload(args.workload, dev, table_seed=1000 * rank, seed_shift=100 * rank)
+    alias = args.alias_after or None
+    first = make_workload(args.workload, dev, table_seed=1000 * rank, seed_shift=100 * rank, alias_after=alias)
     kv_bytes = first.logical_kv_bytes
     unique_bytes = first.unique_kv_bytes
     copies = args.copies or max(2, -(-(1 << 30) // max(unique_bytes, 1)) + 1)
     copies = min(copies, 64)
     pools = [first]
     for i in range(1, copies):
-        pools.append(make_workload(args.workload, dev, table_seed=1000 * rank + i, seed_shift=100 * rank))
+        pools.append(make_workload(args.workload, dev, table_seed=1000 * rank + i, seed_shift=100 * rank, alias_after=alias))
 
     kernel = {"auto": da.DA_KERNEL_AUTO, "simt": da.DA_KERNEL_SIMT, "mma": da.DA_KERNEL_MMA_TMA}[args.kernel]
     policy = da.make_policy(
@@ -444,7 +448,7 @@ def main():
                        "split": args.split, "chunk_tokens": info.chunk_tokens, "units": info.n_units,
                        "max_splits": info.max_splits_used, "kernel": kname, "ctas_per_sm": info.ctas_per_sm,
                        "fused_combine": bool(policy.fuse_combine), "cuda_graph": not args.no_graph,
-                       "shared_prefix_tokens": int(policy.shared_prefix_tokens),
+                       "shared_prefix_tokens": int(policy.shared_prefix_tokens), "alias_after": args.alias_after,
                        "l2": f"rotating over {copies} physical pool copies ({copies * unique_bytes / 2**30:.2f} GiB)",
                        "first_plan_us": plan_us, "plan_us": replan_us, "parallelism": f"dp{world} (sequences sharded, no collective)"},
             "pct_of_8tbs": value / world / 8000.0 * 100.0,
