@@ -116,10 +116,14 @@ typedef struct {
     float sm_scale;             /* 0: 1/sqrtf(head_dim) evaluated in fp32                            */
 } decode_attn_shape_t;
 
-/* One unit of work: one KV head of one sequence over one token range. */
+/* One unit of work: one KV head of one sequence over one token range.  With
+ * policy.shared_prefix_tokens a second kind exists: a chunk of the shared
+ * prefix attended for a block of consecutive sequences at once; it has
+ * kv_head = g | (sequences_in_block << 16), seq = the block's first sequence
+ * and slot = -2 (each sequence's record goes to its own slots). */
 typedef struct {
     int32_t seq;          /* b                                                                       */
-    int32_t kv_head;      /* g                                                                       */
+    int32_t kv_head;      /* g (low 16 bits)                                                         */
     int32_t tok_begin;    /* first token, a multiple of page_size                                    */
     int32_t tok_end;      /* one past the last token; tok_end == tok_begin marks an empty split      */
     int32_t slot;         /* index of the partial in the workspace, -1: writes `out` directly        */
@@ -214,6 +218,12 @@ int decode_attn_plan_destroy(decode_attn_plan_t *plan);
  * running maximum and sum into the workspace, and - with fuse_combine - the
  * last block of a (sequence, KV head) to finish merges them into `out`.
  * Rows with seq_len 0 get zeros and lse = -inf.  Capture-safe.
+ *
+ * The kernel is launched with a programmatic dependency on whatever precedes
+ * it on `stream`: its blocks may become resident and fetch the plan's work
+ * list while that work drains, but q, K/V, seq_lens, block_table and run_mask
+ * are read only after it has completed, so ordinary stream order holds for
+ * every caller-visible buffer.
  * ------------------------------------------------------------------------- */
 int decode_attn_run(const decode_attn_plan_t *plan, const void *q, const void *k_cache,
                     const void *v_cache, const int32_t *block_table, const int32_t *seq_lens, void *out,
