@@ -84,7 +84,8 @@ typedef struct {
     int32_t sm_count;       /* 0: the current device's multiprocessor count                          */
     int32_t kernel;         /* da_kernel_t                                                           */
     int32_t fuse_combine;   /* 0: decode_attn_combine must follow decode_attn_run.
-                               1: the last partition of a sequence to finish merges inside run       */
+                               1: run's launch carries merge blocks behind the attending ones; they
+                               wait (bounded, DA_ERR_TIMEOUT) for a sequence's records and merge them  */
     int32_t capacity_batch; /* > 0: the plan can be refreshed in place for any batch <= this value
                                (decode_attn_plan_update) and launches a fixed grid whose surplus
                                blocks exit at once (Algorithm 1 step 6, "grid exit")                  */
@@ -216,7 +217,8 @@ int decode_attn_plan_destroy(decode_attn_plan_t *plan);
  * One launch on `stream`.  Sequences with a single split write `out` (and
  * lse) directly; the others write unnormalised fp32 partials with their
  * running maximum and sum into the workspace, and - with fuse_combine - the
- * last block of a (sequence, KV head) to finish merges them into `out`.
+ * merge blocks at the end of the same launch merge them into `out` as soon
+ * as the records of a (sequence, KV head) have all been published.
  * Rows with seq_len 0 get zeros and lse = -inf.  Capture-safe.
  *
  * The kernel is launched with a programmatic dependency on whatever precedes

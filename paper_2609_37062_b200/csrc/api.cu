@@ -45,7 +45,8 @@ struct decode_attn_plan {
     int64_t max_units = 0;   // capacity of the device work list
     int64_t max_batch = 0;
     int64_t max_slots = 0;   // what the workspace is sized for
-    int64_t grid = 0;
+    int64_t grid = 0;        // blocks launched by run: work_grid attending blocks (+ merge blocks when fused)
+    int64_t work_grid = 0;
     size_t workspace_bytes = 0;
     // device buffer (views into the cached allocation the plan holds)
     char* dev = nullptr;
@@ -314,6 +315,9 @@ KernelParams make_params(const decode_attn_plan_t* pl, const decode_attn_run_arg
     kp.seq_info = reinterpret_cast<const SeqInfo*>(pl->dev + pl->off_seq_info);
     kp.block_begin = pl->max_bins > 0 ? reinterpret_cast<const int32_t*>(pl->dev + pl->off_block_begin) : nullptr;
     kp.tickets = reinterpret_cast<int32_t*>(pl->dev + pl->off_tickets);
+    kp.ticket_stride = (int32_t)(pl->max_batch * s.num_kv_heads);
+    kp.batch = s.batch;
+    kp.n_work_blocks = (int32_t)pl->work_grid;
     kp.status = reinterpret_cast<int32_t*>(pl->dev + pl->off_status);
     kp.k_stride_page = s.k_stride_page; kp.k_stride_token = s.k_stride_token; kp.k_stride_head = s.k_stride_head;
     kp.v_stride_page = s.v_stride_page; kp.v_stride_token = s.v_stride_token; kp.v_stride_head = s.v_stride_head;
@@ -376,9 +380,8 @@ int decode_attn_plan(const decode_attn_shape_t* shape, const decode_attn_policy_
     pl->ctas_per_sm = policy->ctas_per_sm > 0 ? policy->ctas_per_sm : occ;
 
     pl->seq_lens.assign(seq_lens_host, seq_lens_host + shape->batch);
-    // The tensor-core kernel walks the work list with a fixed set of resident blocks unless the
-    // merge is fused, which needs one unit per block (its scratch is the stage ring).
-    if (pl->kernel == DA_KERNEL_MMA_TMA && !policy->fuse_combine) pl->max_bins = pl->sm_count * pl->ctas_per_sm;
+    // The tensor-core kernel walks the work list with a fixed set of resident blocks.
+    if (pl->kernel == DA_KERNEL_MMA_TMA) pl->max_bins = pl->sm_count * pl->ctas_per_sm;
     rc = make_layout(*shape, *policy, pl->seq_lens.data(), pl->sm_count, pl->ctas_per_sm, pl->layout, pl->max_bins);
     if (rc != DA_OK) return rc;
 
@@ -397,6 +400,12 @@ int decode_attn_plan(const decode_attn_shape_t* shape, const decode_attn_policy_
     }
     if (pl->grid > 0x7fffffffLL) return DA_ERR_UNSUPPORTED;
     if (pl->max_bins > 0) pl->grid = std::min<int64_t>(pl->grid, pl->max_bins);
+    pl->work_grid = pl->grid;
+    if (policy->fuse_combine && pl->max_slots > 0) {
+        // merge blocks ride behind the attending ones: one per merge task, at most one wave of them
+        const int64_t tasks = pl->max_batch * shape->num_kv_heads * combine_slices(shape->head_dim, pl->group);
+        pl->grid += std::min<int64_t>(tasks, (int64_t)pl->sm_count * pl->ctas_per_sm);
+    }
 
     pl->workspace_bytes = (size_t)pl->max_slots * shape->num_kv_heads * rec_floats(pl->group, shape->head_dim) * sizeof(float);
 
@@ -407,7 +416,7 @@ int decode_attn_plan(const decode_attn_shape_t* shape, const decode_attn_policy_
     pl->off_status = pl->upload_bytes;
     pl->off_tickets = pl->off_status + 32;
     pl->total_bytes = pl->off_tickets +
-                      align_up((size_t)std::max<int64_t>(pl->max_batch, 1) * shape->num_kv_heads * sizeof(int32_t), 32);
+                      align_up(2 * (size_t)std::max<int64_t>(pl->max_batch, 1) * shape->num_kv_heads * sizeof(int32_t), 32);
 
     PlanBuffers* pb = new (std::nothrow) PlanBuffers();
     if (!pb) return DA_ERR_INVALID_ARG;
@@ -629,7 +638,7 @@ int decode_attn_debug_gather(const decode_attn_plan_t* pl, int32_t seq, const vo
     std::memset(&a, 0, sizeof a);
     a.k_cache = k_cache; a.v_cache = v_cache; a.block_table = block_table;
     const KernelParams kp = make_params(pl, a);
-    return mma_debug_gather(pl->shape, pl->group, kp, seq, k_out, v_out, (unsigned)pl->grid, stream);
+    return mma_debug_gather(pl->shape, pl->group, kp, seq, k_out, v_out, (unsigned)pl->work_grid, stream);
 }
 
 int decode_attn_gather_probe(const decode_attn_plan_t* pl, const void* k_cache, const void* v_cache,
@@ -643,7 +652,7 @@ int decode_attn_gather_probe(const decode_attn_plan_t* pl, const void* k_cache, 
     std::memset(&a, 0, sizeof a);
     a.k_cache = k_cache; a.v_cache = v_cache; a.block_table = block_table;
     const KernelParams kp = make_params(pl, a);
-    return mma_gather_probe(pl->shape, pl->group, kp, checksum_out, (unsigned)pl->layout.units.size(), (unsigned)pl->grid,
+    return mma_gather_probe(pl->shape, pl->group, kp, checksum_out, (unsigned)pl->layout.units.size(), (unsigned)pl->work_grid,
                             stream);
 }
 
@@ -819,7 +828,7 @@ constexpr size_t kStaticOffUnits = 256;                                         
 constexpr size_t kStaticOffSeqInfo = kStaticOffUnits + sizeof(decode_attn_unit_t) * kStaticMaxUnits;
 constexpr size_t kStaticOffStatus = kStaticOffSeqInfo + sizeof(SeqInfo) * kStaticMaxBatch;
 constexpr size_t kStaticOffTickets = kStaticOffStatus + 256;
-constexpr size_t kStaticOffRecords = (kStaticOffTickets + sizeof(int32_t) * kStaticMaxBatch * 8 + 255) / 256 * 256;
+constexpr size_t kStaticOffRecords = (kStaticOffTickets + 2 * sizeof(int32_t) * kStaticMaxBatch * 8 + 255) / 256 * 256;
 static_assert(kStaticOffRecords < kStaticScratchBytes, "static scratch layout");
 
 struct StaticSetup {
@@ -926,6 +935,9 @@ int decode_attn_step_static(const decode_attn_shape_t* shape, const int32_t* seq
     kp.fused = 0;
     kp.grid_exit = 0;
     kp.n_units = (int32_t)lay.units.size();
+    kp.n_work_blocks = (int32_t)lay.units.size();
+    kp.batch = shape->batch;
+    kp.ticket_stride = kStaticMaxBatch * 8;
 
     const unsigned grid = (unsigned)lay.units.size();
     if (kernel == DA_KERNEL_SIMT) {

@@ -40,17 +40,19 @@ struct KernelParams {
     const decode_attn_unit_t* units;
     const SeqInfo* seq_info;
     const int32_t* block_begin;  // [grid + 1]: block b walks units block_begin[b] .. block_begin[b+1]; NULL: unit b
-    int32_t* tickets;  // [batch][Hkv], zero between launches
+    int32_t* tickets;  // [2][batch][Hkv], zero between launches: records published / slices merged per (sequence, KV head)
     int32_t* status;   // worst da_status_t seen by any block (0 = ok)
     int64_t k_stride_page, k_stride_token, k_stride_head;
     int64_t v_stride_page, v_stride_token, v_stride_head;
     int64_t num_pages;
-    int32_t num_q_heads, num_kv_heads, max_pages_per_seq;
+    int32_t num_q_heads, num_kv_heads, max_pages_per_seq, batch;
     float scale_log2;  // sm_scale * log2(e): logits are kept in the base-2 domain
     int32_t out_bf16;
     int32_t fused;
     int32_t grid_exit;  // capacity plans: the unit count is read from header->n_units, surplus blocks leave at once
     int32_t n_units;    // otherwise: the unit count
+    int32_t n_work_blocks;  // fused plans: blocks at or beyond this index merge records instead of attending
+    int32_t ticket_stride;  // elements between the two ticket arrays
 #ifdef DA_TRACE
     unsigned long long* trace;  // debug builds: 32 stamps per block, or NULL
 #endif
@@ -143,12 +145,6 @@ __device__ __forceinline__ void block_sync(int id, int nthreads)
 // a record can be moved with one bulk copy.  Record r = slot * Hkv + kv_head.
 __host__ __device__ constexpr int rec_floats(int G, int D) { return (G * D + 2 * G + 3) / 4 * 4; }
 
-// Shared memory merge_group needs to stage `cap` records at a time.
-__host__ __device__ constexpr int merge_stage_bytes(int G, int D, int cap)
-{
-    return cap * rec_floats(G, D) * 4 + cap * G * 4 + 64;
-}
-
 // ---------------------------------------------------------------- mbarrier / bulk copy
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -200,154 +196,169 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
     return true;
 }
 
-// 1-D bulk copy global -> shared, completion counted in bytes on `bar`.
-// Addresses 16-byte aligned, size a multiple of 16.
-__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar)
-{
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
-                 : "memory");
-}
-
-// ---------------------------------------------------------------- LSE merge
+// ---------------------------------------------------------------- LSE merge of one slice
 //
-// Merge of the splits of one (sequence, KV head): all G query heads of the
-// group, ascending split order, by the `nthreads` threads of one block.  Used
-// by the combine kernel and by the last block to finish in a fused launch, so
-// both give the same bits: every output column is the sum of four chains,
-// chain k taking the splits with index k (mod 4) in ascending order, added as
-// ((c0 + c1) + c2) + c3; the sums of exponentials follow the same scheme.
-// The records (written by other SMs) are pulled
-// into shared memory `cap` at a time by bulk copies, one per record, issued
-// by as many threads in parallel as there are records (a bulk copy costs its
-// issuer about one round trip to L2); warp w reduces the running maxima of
-// heads w, w + nwarps, ... by shuffles and leaves the weights e^{m_i - M} in
-// shared memory.  The result does not depend on `cap` (a multiple of 4).
-// The `nthreads` threads synchronise on hardware barrier `bar_id`.
-// `stage`: merge_stage_bytes(G, D, cap) bytes of shared
-// memory, 16-byte aligned, that no thread still reads.  `bar`: an initialised
-// mbarrier (count 1) whose current phase parity is `parity` (updated).
+// Merge of the records of one (sequence, KV head) for a slice of 32 output
+// columns (a column is four consecutive output dims of one query head), by
+// 128 threads = four chains x 32 columns: chain k of a column sums the splits
+// with index k (mod 4) in ascending order, the four chains are added as
+// ((c0 + c1) + c2) + c3.  All of a thread's loads (its column of up to
+// kCombineBatch records and their (max, sum) pairs) are in flight before
+// anything is used, so up to 4 * kCombineBatch splits cost one round trip to
+// L2.  The combine kernel and the merge blocks of a fused launch both call
+// this, so both paths give the same bits.  sm: 4 * 32 * 6 floats of shared
+// memory; the 128 threads synchronise on hardware barrier `bar_id`.
+constexpr int kCombineThreads = 128;
+constexpr int kCombineBatch = 12;
+constexpr int kCombineSmemFloats = 4 * 32 * 6;
+
 template <int D>
-__device__ __forceinline__ void merge_group(const KernelParams& p, int b, int g, int G, int slot_base, int S,
-                                            int tid, int nthreads, int bar_id, uint8_t* stage, int cap, uint32_t bar,
-                                            uint32_t& parity)
+__device__ __forceinline__ void combine_slice(const KernelParams& p, int b, int g, int slice, int G, int slot_base,
+                                              int S, int tid, float* sm, int bar_id)
 {
     constexpr int D4 = D / 4;
-    constexpr int kMaxTasks = 2;                        // G * D4 <= 256 tasks over >= 128 threads
-    const int Hq = p.num_q_heads, Hkv = p.num_kv_heads;
-    const int RF = rec_floats(G, D), RF4 = RF / 4;
-    const int GD4 = G * D4;
-    const int lane = tid & 31, warp = tid >> 5, nwarps = nthreads >> 5;
-    float* const st_rec = reinterpret_cast<float*>(stage);          // [cap][RF]
-    float* const st_w = st_rec + (size_t)cap * RF;                  // [cap][G] weights
-    float* const st_M = st_w + cap * G;                             // [8] maxima
-    const float* const recs = p.ws + ((int64_t)slot_base * Hkv + g) * RF;
-    const int64_t rec_stride = (int64_t)Hkv * RF;                   // next split of the same KV head
+    float* const sm_m = sm;                                    // [4][32]
+    float* const sm_l = sm + 128;                              // [4][32]
+    float4* const sm_acc = reinterpret_cast<float4*>(sm + 256);   // [4][32]
+    const int q = tid >> 5, lane = tid & 31;
+    const int col = slice * 32 + lane;
+    const bool live = col < G * D4;
+    const int h = live ? col / D4 : 0;
+    const int RF = rec_floats(G, D);
+    const float* const recs = p.ws + ((int64_t)slot_base * p.num_kv_heads + g) * RF;
+    const int64_t rec_stride = (int64_t)p.num_kv_heads * RF;
+    const float4* const colp = reinterpret_cast<const float4*>(recs) + (live ? col : 0);
+    const float2* const mlp = reinterpret_cast<const float2*>(recs + G * D) + h;
 
-    float4 acc[kMaxTasks][4];                                       // four chains per column
-    float lch[kMaxTasks][4];                                        // and per head (kept by every column thread)
+    float2 ml[kCombineBatch];
+    float4 v[kCombineBatch];
 #pragma unroll
-    for (int k = 0; k < kMaxTasks; ++k)
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            acc[k][q] = make_float4(0.f, 0.f, 0.f, 0.f);
-            lch[k][q] = 0.f;
+    for (int t = 0; t < kCombineBatch; ++t) {
+        const int j = q + 4 * t;
+        ml[t] = make_float2(-INFINITY, 0.f);
+        v[t] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (j < S) {
+            ml[t] = __ldcg(mlp + j * (rec_stride / 2));
+            v[t] = __ldcg(colp + j * (rec_stride / 4));
         }
-
-    for (int i0 = 0; i0 < S; i0 += cap) {
-        const int n = min(cap, S - i0);
-        // The proxy fence orders the generic-proxy accesses made so far (this block's use of the
-        // stage memory, other blocks' record stores seen through the ticket) before the copies.
-        if (tid < n) asm volatile("fence.proxy.async;" ::: "memory");
-        if (tid == 0) mbar_arrive_expect_tx(bar, (uint32_t)(n * RF * 4));
-        for (int j = tid; j < n; j += nthreads)
-            bulk_copy_g2s(smem_u32(st_rec + (size_t)j * RF), recs + (i0 + j) * rec_stride, (uint32_t)(RF * 4), bar);
-        if (i0 == 0 && S > cap) {
-            // several batches: the maximum of every head over ALL splits must be known before the
-            // first weight, so read the maxima from global memory while the first batch flies
-            for (int h = warp; h < G; h += nwarps) {
-                float m = -INFINITY;
-                for (int i = lane; i < S; i += 32) m = fmaxf(m, __ldcg(recs + i * rec_stride + G * D + 2 * h));
-#pragma unroll
-                for (int off = 16; off >= 1; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
-                if (lane == 0) st_M[h] = m;
-            }
-        }
-        if (!mbar_wait(bar, parity) && tid == 0) record_status(p.status, DA_ERR_TIMEOUT);
-        parity ^= 1u;
-        if (S <= cap) {
-            // one batch: every record is here, take the maxima from shared memory
-            for (int h = warp; h < G; h += nwarps) {
-                float m = -INFINITY;
-                for (int j = lane; j < n; j += 32) m = fmaxf(m, st_rec[(size_t)j * RF + G * D + 2 * h]);
-#pragma unroll
-                for (int off = 16; off >= 1; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
-                if (lane == 0) st_M[h] = m;
-            }
-        }
-        block_sync(bar_id, nthreads);
-        // weights e^{m_i - M}, once per (split, head)
-        for (int c = tid; c < n * G; c += nthreads) {
-            const int j = c / G, h = c % G;
-            const float M = st_M[h];
-            st_w[c] = (M == -INFINITY) ? 0.f : ex2f(st_rec[(size_t)j * RF + G * D + 2 * h] - M);   // empty split: 0
-        }
-        block_sync(bar_id, nthreads);
-#pragma unroll
-        for (int k = 0; k < kMaxTasks; ++k) {
-            const int task = tid + k * nthreads;
-            if (task < GD4) {
-                const int h = task / D4;
-                const float4* o = reinterpret_cast<const float4*>(st_rec) + task;
-                const float* wp = st_w + h;
-                const float* lp = st_rec + G * D + 2 * h + 1;
-                int j = 0;
-                for (; j + 4 <= n; j += 4) {       // i0 and cap are multiples of 4: chain q takes j + q
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const float w = wp[(j + q) * G];
-                        const float4 v = o[(j + q) * RF4];
-                        acc[k][q].x = fmaf(w, v.x, acc[k][q].x);
-                        acc[k][q].y = fmaf(w, v.y, acc[k][q].y);
-                        acc[k][q].z = fmaf(w, v.z, acc[k][q].z);
-                        acc[k][q].w = fmaf(w, v.w, acc[k][q].w);
-                        lch[k][q] = fmaf(w, lp[(size_t)(j + q) * RF], lch[k][q]);
-                    }
-                }
-#pragma unroll
-                for (int q = 0; q < 3; ++q) {
-                    if (j + q < n) {
-                        const float w = wp[(j + q) * G];
-                        const float4 v = o[(j + q) * RF4];
-                        acc[k][q].x = fmaf(w, v.x, acc[k][q].x);
-                        acc[k][q].y = fmaf(w, v.y, acc[k][q].y);
-                        acc[k][q].z = fmaf(w, v.z, acc[k][q].z);
-                        acc[k][q].w = fmaf(w, v.w, acc[k][q].w);
-                        lch[k][q] = fmaf(w, lp[(size_t)(j + q) * RF], lch[k][q]);
-                    }
-                }
-            }
-        }
-        block_sync(bar_id, nthreads);
     }
+    float mloc = -INFINITY;
 #pragma unroll
-    for (int k = 0; k < kMaxTasks; ++k) {
-        const int task = tid + k * nthreads;
-        if (task < GD4) {
-            const int h = task / D4, d4 = task % D4;
-            const float M = st_M[h];
-            const float ls = ((lch[k][0] + lch[k][1]) + lch[k][2]) + lch[k][3];
-            float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (M != -INFINITY && ls > 0.f) {
-                const float inv = 1.0f / ls;
-                o.x = (((acc[k][0].x + acc[k][1].x) + acc[k][2].x) + acc[k][3].x) * inv;
-                o.y = (((acc[k][0].y + acc[k][1].y) + acc[k][2].y) + acc[k][3].y) * inv;
-                o.z = (((acc[k][0].z + acc[k][1].z) + acc[k][2].z) + acc[k][3].z) * inv;
-                o.w = (((acc[k][0].w + acc[k][1].w) + acc[k][2].w) + acc[k][3].w) * inv;
+    for (int t = 0; t < kCombineBatch; ++t) mloc = fmaxf(mloc, ml[t].x);
+    for (int j = q + 4 * kCombineBatch; j < S; j += 4) mloc = fmaxf(mloc, __ldcg(mlp + j * (rec_stride / 2)).x);
+    sm_m[q * 32 + lane] = mloc;
+    block_sync(bar_id, kCombineThreads);
+    const float M = fmaxf(fmaxf(sm_m[lane], sm_m[32 + lane]), fmaxf(sm_m[64 + lane], sm_m[96 + lane]));
+
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    float lch = 0.f;
+    for (int t0 = 0; q + 4 * t0 < S; t0 += kCombineBatch) {
+        if (t0 > 0) {
+#pragma unroll
+            for (int t = 0; t < kCombineBatch; ++t) {
+                const int j = q + 4 * (t0 + t);
+                ml[t] = make_float2(-INFINITY, 0.f);
+                v[t] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (j < S) {
+                    ml[t] = __ldcg(mlp + j * (rec_stride / 2));
+                    v[t] = __ldcg(colp + j * (rec_stride / 4));
+                }
             }
-            store_out4(p.out, ((int64_t)b * Hq + g * G + h) * D + d4 * 4, o, p.out_bf16);
-            if (p.lse != nullptr && d4 == 0)
-                p.lse[(int64_t)b * Hq + g * G + h] = (M != -INFINITY && ls > 0.f) ? (M + log2f(ls)) * kLn2 : -INFINITY;
+        }
+#pragma unroll
+        for (int t = 0; t < kCombineBatch; ++t) {
+            if (q + 4 * (t0 + t) < S) {
+                const float w = (M == -INFINITY) ? 0.f : ex2f(ml[t].x - M);   // empty split: m = -inf, w = 0
+                acc.x = fmaf(w, v[t].x, acc.x);
+                acc.y = fmaf(w, v[t].y, acc.y);
+                acc.z = fmaf(w, v[t].z, acc.z);
+                acc.w = fmaf(w, v[t].w, acc.w);
+                lch = fmaf(w, ml[t].y, lch);
+            }
+        }
+    }
+    sm_acc[q * 32 + lane] = acc;
+    sm_l[q * 32 + lane] = lch;
+    block_sync(bar_id, kCombineThreads);
+    if (q == 0 && live) {
+        const int d4 = col % D4;
+        const float ls = ((sm_l[lane] + sm_l[32 + lane]) + sm_l[64 + lane]) + sm_l[96 + lane];
+        float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (M != -INFINITY && ls > 0.f) {
+            const float inv = 1.0f / ls;
+            const float4 a0 = sm_acc[lane], a1 = sm_acc[32 + lane], a2 = sm_acc[64 + lane], a3 = sm_acc[96 + lane];
+            o.x = (((a0.x + a1.x) + a2.x) + a3.x) * inv;
+            o.y = (((a0.y + a1.y) + a2.y) + a3.y) * inv;
+            o.z = (((a0.z + a1.z) + a2.z) + a3.z) * inv;
+            o.w = (((a0.w + a1.w) + a2.w) + a3.w) * inv;
+        }
+        store_out4(p.out, ((int64_t)b * p.num_q_heads + g * G + h) * D + d4 * 4, o, p.out_bf16);
+        if (p.lse != nullptr && d4 == 0)
+            p.lse[(int64_t)b * p.num_q_heads + g * G + h] = (M != -INFINITY && ls > 0.f) ? (M + log2f(ls)) * kLn2 : -INFINITY;
+    }
+    block_sync(bar_id, kCombineThreads);                       // the scratch may be reused by the next slice
+}
+
+__host__ __device__ inline int combine_slices(int D, int G) { return (G * (D / 4) + 31) / 32; }
+
+__device__ __forceinline__ int32_t ld_acquire(const int32_t* ptr)
+{
+    int32_t v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(ptr) : "memory");
+    return v;
+}
+
+// ---------------------------------------------------------------- merge blocks of a fused launch
+//
+// With fuse_combine the launch carries extra blocks behind the attending ones
+// (blockIdx.x >= n_work_blocks).  They are dispatched after every attending
+// block has been dispatched, take the merge tasks (sequence, KV head, slice)
+// round-robin, and for each task poll the group's arrival counter - every
+// attending block adds one after publishing a record - until all the group's
+// records are in, then merge the slice exactly as the combine kernel would.
+// The poll is bounded (about a second); giving up records DA_ERR_TIMEOUT.
+// The block that merges a group's last slice resets the group's counters, so
+// the plan can be launched again (or replayed from a graph) as it is.
+template <int D>
+__device__ __forceinline__ void fused_merge_blocks(const KernelParams& p, int G, int nthreads, float* sm, int* sm_flag)
+{
+    const int tid = threadIdx.x;
+    const int n_slices = combine_slices(D, G);
+    const int batch = p.grid_exit ? p.header->batch : p.batch;
+    const int n_tasks = batch * p.num_kv_heads * n_slices;
+    const int n_merge_blocks = gridDim.x - p.n_work_blocks;
+    for (int t = blockIdx.x - p.n_work_blocks; t < n_tasks; t += n_merge_blocks) {
+        const int slice = t % n_slices, bg = t / n_slices;
+        const int b = bg / p.num_kv_heads, g = bg % p.num_kv_heads;
+        const SeqInfo si = p.seq_info[b];
+        if (si.slot_base < 0) continue;                        // a single split: written directly
+        if (tid == 0) {
+            const int32_t* arrivals = p.tickets + bg;
+            const long long t0 = clock64();
+            int ok = 1;
+            while (ld_acquire(arrivals) < si.n_splits) {
+                // give up after the limit, or at once when an attending block already gave up
+                // on a wait of its own (it will not publish the rest of its records)
+                if (clock64() - t0 > kWaitLimitCycles || ld_acquire(p.status) <= DA_ERR_TIMEOUT) {
+                    ok = 0;
+                    break;
+                }
+                __nanosleep(100);
+            }
+            if (!ok) record_status(p.status, DA_ERR_TIMEOUT);
+            *sm_flag = ok;
+        }
+        block_sync(0, nthreads);
+        const int ok = *sm_flag;
+        if (ok && tid < kCombineThreads) combine_slice<D>(p, b, g, slice, G, si.slot_base, si.n_splits, tid, sm, 2);
+        block_sync(0, nthreads);
+        if (tid == 0) {
+            // count this slice; whoever completes the group puts its counters back to zero
+            int32_t* done = p.tickets + p.ticket_stride + bg;
+            if (atomicAdd(done, 1) == n_slices - 1) {
+                *done = 0;
+                p.tickets[bg] = 0;
+            }
         }
     }
 }
@@ -358,20 +369,17 @@ __device__ __forceinline__ void merge_group(const KernelParams& p, int b, int g,
 // memory: src_o [R][COLS][D] unnormalised accumulators, src_m / src_l
 // [R][COLS] running maxima (log2 domain, -inf if nothing was attended) and
 // sums.  With DUP, columns h and h + 4 hold the high and low parts of the
-// same head and are added.  All threads call this after a __syncthreads()
-// that made the sources visible.  The states are merged in the fixed order
-// r = 0..R-1 and the result goes straight to `out` (single split) or to the
-// unit's record; with a fused plan the block then draws a ticket and, if it
-// is the last of its (sequence, KV head), merges all records.  The calling
-// threads (`nthreads`, ids 0..nthreads-1) synchronise on hardware barrier
-// `bar_id`.  `stage` / `cap`: shared memory the merge may overwrite (it may
-// alias the sources); cap == 0 means none is available (the block still has
-// units to stream) and a fused plan must not get here.
+// same head and are added.  The calling threads (`nthreads`, ids
+// 0..nthreads-1) call this after a barrier that made the sources visible and
+// synchronise on hardware barrier `bar_id`.  The states are merged in the
+// fixed order r = 0..R-1 and the result goes straight to `out` (single
+// split) or to the unit's record; with a fused plan the block then publishes
+// the record: a device-wide fence and one more arrival on the counter of its
+// (sequence, KV head), which the merge blocks of the launch poll.
 template <int D, int R, int COLS, bool DUP>
 __device__ __forceinline__ void block_finish(const KernelParams& p, const decode_attn_unit_t& u, int G,
-                                             const float* src_o, const float* src_m, const float* src_l,
-                                             int* sm_ticket, uint32_t merge_bar, uint32_t* merge_parity, int tid,
-                                             int nthreads, int bar_id, uint8_t* stage, int cap)
+                                             const float* src_o, const float* src_m, const float* src_l, int tid,
+                                             int nthreads, int bar_id)
 {
     constexpr int D4 = D / 4;
     constexpr int kUnroll = R <= 4 ? R : 1;     // many row groups: keep the loop rolled, registers matter more
@@ -418,31 +426,13 @@ __device__ __forceinline__ void block_finish(const KernelParams& p, const decode
         }
     }
     if (rec == nullptr || !p.fused) return;
-    // Ticket: nobody waits.  The block barrier orders every thread's record
-    // stores before thread 0's fence, which publishes them device-wide ahead
-    // of the ticket; the block that draws the last ticket of its (sequence,
-    // KV head) therefore sees all the other records.
+    // The barrier orders every thread's record stores before thread 0's fence, which publishes
+    // them device-wide ahead of the arrival.
     block_sync(bar_id, nthreads);
-    if (tid == 0) DA_TRACE_CLOCK(blockIdx.x, 13);
-    int32_t* ticket = p.tickets + (int64_t)u.seq * p.num_kv_heads + u.kv_head;
     if (tid == 0) {
         __threadfence();
-        *sm_ticket = atomicAdd(ticket, 1);
-        __threadfence();
+        atomicAdd(p.tickets + (int64_t)u.seq * p.num_kv_heads + u.kv_head, 1);
     }
-    block_sync(bar_id, nthreads);
-    if (tid == 0) DA_TRACE_CLOCK(blockIdx.x, 14);
-    if (*sm_ticket != u.n_splits - 1) return;
-    if (cap <= 0) {                              // host-side contract broken: fused plans run one unit per block
-        if (tid == 0) record_status(p.status, DA_ERR_UNSUPPORTED);
-        return;
-    }
-    uint32_t parity = *merge_parity;
-    merge_group<D>(p, u.seq, u.kv_head, G, u.slot - u.split_index, u.n_splits, tid, nthreads, bar_id, stage, cap, merge_bar,
-                   parity);
-    *merge_parity = parity;
-    if (tid == 0) DA_TRACE_CLOCK(blockIdx.x, 19);
-    if (tid == 0) *ticket = 0;  // ready for the next launch
 }
 
 }  // namespace da

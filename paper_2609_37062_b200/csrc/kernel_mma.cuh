@@ -154,13 +154,20 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;             // 1 KB aligned: the swizzle atom
     uint8_t* const gbase = smem_raw + (base - raw);
-    const uint32_t bar_base = base + NS * Cfg::kStageBytes;   // full[NS], empty[NS], merge
+    const uint32_t bar_base = base + NS * Cfg::kStageBytes;   // full[NS], empty[NS]
     volatile int* const sm_flags = reinterpret_cast<volatile int*>(gbase + NS * Cfg::kStageBytes + 256);
     int* const sm_ticket = reinterpret_cast<int*>(gbase + NS * Cfg::kStageBytes + 256 + 16);
     float* const sm_wo = reinterpret_cast<float*>(gbase + NS * Cfg::kStageBytes + Cfg::kBarrierBytes);   // [4][COLS][D]
     float* const sm_wm = sm_wo + kMmaConsumerWarps * COLS * D;                                           // [4][COLS]
     float* const sm_wl = sm_wm + kMmaConsumerWarps * COLS;                                               // [4][COLS]
 
+    if (MODE == kModeAttend && p.fused && (int)blockIdx.x >= p.n_work_blocks) {
+        // a merge block of a fused launch: no tiles, no pipeline
+        pdl_launch_dependents();
+        pdl_wait_primary();                                   // `out` may still be in use by the kernel before
+        fused_merge_blocks<D>(p, G, kMmaThreads, sm_wo, sm_ticket);
+        return;
+    }
     // this block's units: a range of the work list (the planner's packing), or just unit blockIdx.x
     int ubeg, uend;
     if (p.block_begin != nullptr) {
@@ -182,7 +189,6 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
             mbar_init(bar_base + 8 * s, 1);                             // full: the producer's expect_tx arrival
             mbar_init(bar_base + 8 * (NS + s), kMmaConsumerWarps);      // empty: one arrival per consumer warp
         }
-        mbar_init(bar_base + 8 * 2 * NS, 1);                            // the in-kernel merge's copies
         sm_flags[0] = 0;
         mbar_init_fence();
     }
@@ -290,7 +296,6 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
     const int r = lane >> 2, c = lane & 3;
     const bool lo_role = DUP && (c >= 2);
     uint32_t git = 0;                                         // stages consumed so far, over all units
-    uint32_t merge_parity = 0;
     // what a unit needs before its first tile: lengths / mask of its sequence and Q^T as B
     // fragments (column n = r is query head r, or r mod 4 when duplicated); fetched one unit ahead
     struct Pre {
@@ -703,10 +708,7 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
             }
         }
         block_sync(1, kConsumerThreads);
-        // the in-kernel merge may take the stage ring as scratch only when nothing more will land in it
-        const int cap = last_unit ? (((NS * Cfg::kStageBytes - 64 - 4 * G) / (rec_floats(G, D) * 4 + 4 * G)) & ~3) : 0;
-        block_finish<D, kMmaConsumerWarps, COLS, false>(p, u, G, sm_wo, sm_wm, sm_wl, sm_ticket, bar_base + 8 * 2 * NS,
-                                                        &merge_parity, tid, kConsumerThreads, 1, gbase, cap);
+        block_finish<D, kMmaConsumerWarps, COLS, false>(p, u, G, sm_wo, sm_wm, sm_wl, tid, kConsumerThreads, 1);
         if (uid == ubeg && tid == 0) DA_TRACE_STAMP(blockIdx.x, 6);
         if (failed && sm_flags[0] != 0) return;
         u = nu;

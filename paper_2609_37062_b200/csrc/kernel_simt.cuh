@@ -48,15 +48,20 @@ __global__ void __launch_bounds__(kSimtThreads) decode_attn_simt_kernel(const Ke
 
     // one raw block so the in-kernel merge can reuse it as its staging area
     constexpr int kOwnBytes = ROWS * G * D * 4 + 2 * ROWS * G * 4;
-    constexpr int kRawBytes = kOwnBytes > merge_stage_bytes(G, D, ROWS) ? kOwnBytes : merge_stage_bytes(G, D, ROWS);
+    constexpr int kRawBytes = kOwnBytes > kCombineSmemFloats * 4 ? kOwnBytes : kCombineSmemFloats * 4;
     __shared__ __align__(16) uint8_t sm_raw[kRawBytes];
     float (*sm_acc)[G][D] = reinterpret_cast<float (*)[G][D]>(sm_raw);
     float (*sm_rm)[G] = reinterpret_cast<float (*)[G]>(sm_raw + ROWS * G * D * 4);
     float (*sm_rl)[G] = reinterpret_cast<float (*)[G]>(sm_raw + ROWS * G * D * 4 + ROWS * G * 4);
-    __shared__ __align__(8) uint64_t sm_merge_bar;
-    __shared__ int sm_ticket;
+    __shared__ int sm_flag;
 
     const int uid = blockIdx.x;
+    if (p.fused && uid >= p.n_work_blocks) {    // a merge block of a fused launch
+        pdl_launch_dependents();
+        pdl_wait_primary();
+        fused_merge_blocks<D>(p, G, kSimtThreads, reinterpret_cast<float*>(sm_raw), &sm_flag);
+        return;
+    }
     if (uid >= (p.grid_exit ? p.header->n_units : p.n_units)) return;   // surplus blocks of a capacity launch
     const decode_attn_unit_t u = load_unit(p.units, uid);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -66,10 +71,6 @@ __global__ void __launch_bounds__(kSimtThreads) decode_attn_simt_kernel(const Ke
 
     const int t0 = u.tok_begin;
     int t1 = u.tok_end;
-    if (tid == 0) {
-        mbar_init(smem_u32(&sm_merge_bar), 1);
-        mbar_init_fence();
-    }
     // Only the plan's work list was read so far; what the kernel launched before this one may
     // have produced (q, new K/V rows, lengths, page mappings) is read past this point.
     pdl_wait_primary();
@@ -194,9 +195,7 @@ __global__ void __launch_bounds__(kSimtThreads) decode_attn_simt_kernel(const Ke
         dst[1] = make_float4(acc[h][4], acc[h][5], acc[h][6], acc[h][7]);
     }
     __syncthreads();
-    uint32_t merge_parity = 0;
-    block_finish<D, ROWS, G, false>(p, u, G, &sm_acc[0][0][0], &sm_rm[0][0], &sm_rl[0][0], &sm_ticket,
-                                    smem_u32(&sm_merge_bar), &merge_parity, tid, kSimtThreads, 0, sm_raw, ROWS);
+    block_finish<D, ROWS, G, false>(p, u, G, &sm_acc[0][0][0], &sm_rm[0][0], &sm_rl[0][0], tid, kSimtThreads, 0);
 }
 
 }  // namespace da
