@@ -14,12 +14,16 @@ __global__ void __launch_bounds__(kCombineThreads) decode_attn_combine_kernel(co
 {
     __shared__ __align__(16) float sm[kCombineSmemFloats];
     pdl_launch_dependents();                              // the next kernel may start its prologue
-    pdl_wait_primary();                                   // the records of the launch before this one are complete
+    // The plan's own tables (live batch, split table) do not depend on the launch before this
+    // one: fetch them while it drains, and wait only before touching its records.
     const int slice = blockIdx.x % n_slices;
     const int bg = blockIdx.x / n_slices;
     const int b = bg / p.num_kv_heads, g = bg % p.num_kv_heads;
-    if (b >= p.header->batch) return;                     // rows past the live batch of a capacity plan
-    const SeqInfo si = p.seq_info[b];
+    const bool in_batch = b < p.header->batch;            // rows past the live batch of a capacity plan
+    SeqInfo si;
+    si.slot_base = -1;
+    if (in_batch) si = p.seq_info[b];
+    pdl_wait_primary();                                   // the records of the launch before this one are complete
     if (si.slot_base < 0) return;                         // a single split, written directly by the partial kernel
     combine_slice<D>(p, b, g, slice, G, si.slot_base, si.n_splits, threadIdx.x, sm, 0);
 }

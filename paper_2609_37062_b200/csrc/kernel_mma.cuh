@@ -178,7 +178,12 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
         ubeg = blockIdx.x;
         uend = min(n_units, (int)blockIdx.x + 1);
     }
-    if (ubeg >= uend) return;                                 // surplus blocks of a capacity launch
+    if (ubeg >= uend) {                                       // surplus blocks of a capacity launch
+        // Stream order reaches the kernels behind this one through the waits of this launch's
+        // blocks; should every block be surplus, block 0 still carries it.
+        if (blockIdx.x == 0) pdl_wait_primary();
+        return;
+    }
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     if (tid == 0) DA_TRACE_STAMP(blockIdx.x, 0);
 

@@ -62,7 +62,10 @@ __global__ void __launch_bounds__(kSimtThreads) decode_attn_simt_kernel(const Ke
         fused_merge_blocks<D>(p, G, kSimtThreads, reinterpret_cast<float*>(sm_raw), &sm_flag);
         return;
     }
-    if (uid >= (p.grid_exit ? p.header->n_units : p.n_units)) return;   // surplus blocks of a capacity launch
+    if (uid >= (p.grid_exit ? p.header->n_units : p.n_units)) {   // surplus blocks of a capacity launch
+        if (uid == 0) pdl_wait_primary();       // an empty launch still hands stream order on to its successors
+        return;
+    }
     const decode_attn_unit_t u = load_unit(p.units, uid);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int rg = warp * RPW + lane / LPR;     // row group of this thread
