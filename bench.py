@@ -57,7 +57,7 @@ def parse_args():
                     help="long_32k | short_chat | shared_prefix | sweep_<context>x<batch> | tiny")
     ap.add_argument("--split", default="auto", choices=["auto", "deterministic"])
     ap.add_argument("--chunk-tokens", type=int, default=0)
-    ap.add_argument("--kernel", default="auto", choices=["auto", "simt", "mma"])
+    ap.add_argument("--kernel", default="auto", choices=["auto", "simt", "mma", "umma"])
     ap.add_argument("--fuse", action="store_true",
                     help="merge inside the partial kernel (one launch per step) instead of the combine kernel")
     ap.add_argument("--no-graph", action="store_true", help="launch every step from the host")
@@ -269,7 +269,8 @@ def main():
     for i in range(1, copies):
         pools.append(make_workload(args.workload, dev, table_seed=1000 * rank + i, seed_shift=100 * rank, alias_after=alias))
 
-    kernel = {"auto": da.DA_KERNEL_AUTO, "simt": da.DA_KERNEL_SIMT, "mma": da.DA_KERNEL_MMA_TMA}[args.kernel]
+    kernel = {"auto": da.DA_KERNEL_AUTO, "simt": da.DA_KERNEL_SIMT, "mma": da.DA_KERNEL_MMA_TMA,
+              "umma": da.DA_KERNEL_UMMA_PREFIX}[args.kernel]
     policy = da.make_policy(
         split_mode=da.DA_SPLIT_DETERMINISTIC if args.split == "deterministic" else da.DA_SPLIT_AUTO,
         chunk_tokens=args.chunk_tokens, kernel=kernel, fuse_combine=1 if args.fuse else 0,
@@ -436,7 +437,8 @@ def main():
     if rank == 0:
         peak, peak_kind = peak_hbm()
         achieved = kv_bytes / sec_per_step / 1e9
-        kname = {da.DA_KERNEL_SIMT: "decode_attn_simt_kernel", da.DA_KERNEL_MMA_TMA: "decode_attn_mma_kernel"}[info.kernel]
+        kname = {da.DA_KERNEL_SIMT: "decode_attn_simt_kernel", da.DA_KERNEL_MMA_TMA: "decode_attn_mma_kernel",
+                 da.DA_KERNEL_UMMA_PREFIX: "decode_attn_mma_kernel"}[info.kernel]
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": sec_per_step * 1e3, "us_per_step": sec_per_step * 1e6,

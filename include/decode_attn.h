@@ -71,7 +71,10 @@ typedef enum {
 typedef enum {
     DA_KERNEL_AUTO = 0,     /* tensor-core kernel when the GQA group has >= 2 heads, else SIMT       */
     DA_KERNEL_SIMT = 1,     /* CUDA-core kernel, 16-byte vectorised global loads                      */
-    DA_KERNEL_MMA_TMA = 2   /* TMA-staged pages in shared memory, mma.sync bf16 for QK^T and PV       */
+    DA_KERNEL_MMA_TMA = 2,  /* TMA-staged pages in shared memory, mma.sync bf16 for QK^T and PV       */
+    DA_KERNEL_UMMA_PREFIX = 3 /* shared-prefix plans only (head_dim 128, group 1, 2, 4 or 8): the prefix
+                               units run on the tcgen05 tensor cores, 128 query rows at a time with
+                               accumulators in tensor memory; what follows the prefix runs as MMA_TMA */
 } da_kernel_t;
 
 /* Split policy.  Zero-initialise for the defaults. */

@@ -43,6 +43,7 @@ DA_SPLIT_DETERMINISTIC = 2
 DA_KERNEL_AUTO = 0
 DA_KERNEL_SIMT = 1
 DA_KERNEL_MMA_TMA = 2
+DA_KERNEL_UMMA_PREFIX = 3
 
 EXPORTED = [
     "decode_attn_plan_layout", "decode_attn_plan", "decode_attn_plan_update", "decode_attn_plan_get_info",

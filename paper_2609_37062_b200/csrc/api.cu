@@ -15,6 +15,7 @@
 #include "common.cuh"
 #include "decode_attn.h"
 #include "kernel_mma.cuh"
+#include "kernel_umma.cuh"
 #include "kernel_simt.cuh"
 #include "planner.h"
 
@@ -196,6 +197,7 @@ int pick_kernel(const decode_attn_shape_t& s, const decode_attn_policy_t& p)
 {
     if (p.kernel != DA_KERNEL_AUTO) return p.kernel;
     const int G = s.num_q_heads / s.num_kv_heads;
+    if (p.shared_prefix_tokens > 0 && umma_supports(s.head_dim, G)) return DA_KERNEL_UMMA_PREFIX;
     return (G >= 2 && mma_supports(s.head_dim, G)) ? DA_KERNEL_MMA_TMA : DA_KERNEL_SIMT;
 }
 
@@ -364,7 +366,10 @@ int decode_attn_plan(const decode_attn_shape_t* shape, const decode_attn_policy_
     pl->group = shape->num_q_heads / shape->num_kv_heads;
     pl->scale = shape->sm_scale > 0.f ? shape->sm_scale : 1.0f / sqrtf((float)shape->head_dim);
     pl->kernel = pick_kernel(*shape, *policy);
-    if (pl->kernel == DA_KERNEL_MMA_TMA && !mma_supports(shape->head_dim, pl->group)) return DA_ERR_UNSUPPORTED;
+    if (pl->kernel != DA_KERNEL_SIMT && !mma_supports(shape->head_dim, pl->group)) return DA_ERR_UNSUPPORTED;
+    const bool umma = pl->kernel == DA_KERNEL_UMMA_PREFIX;
+    if (umma && (!umma_supports(shape->head_dim, pl->group) || policy->shared_prefix_tokens <= 0)) return DA_ERR_UNSUPPORTED;
+    pl->policy.kernel = pl->kernel;        // the planner cuts the prefix for the kernel that will run it
 
     DA_CUDA_TRY(cudaGetDevice(&pl->device));
     if (policy->sm_count > 0) {
@@ -374,15 +379,17 @@ int decode_attn_plan(const decode_attn_shape_t* shape, const decode_attn_policy_
         if (rc != DA_OK) return rc;
     }
     const bool prefix = policy->shared_prefix_tokens > 0;
-    if (prefix && pl->kernel != DA_KERNEL_MMA_TMA) return DA_ERR_UNSUPPORTED;
-    int occ = query_occupancy(pl->kernel, shape->head_dim, pl->group, &pl->block_threads, &pl->dyn_smem, prefix);
+    if (prefix && pl->kernel == DA_KERNEL_SIMT) return DA_ERR_UNSUPPORTED;
+    // what follows a tcgen05 prefix runs on the ordinary tensor-core kernel
+    int occ = query_occupancy(DA_KERNEL_MMA_TMA == pl->kernel || umma ? DA_KERNEL_MMA_TMA : pl->kernel, shape->head_dim,
+                              pl->group, &pl->block_threads, &pl->dyn_smem, prefix && !umma);
     if (occ <= 0) return DA_ERR_CUDA;
     pl->ctas_per_sm = policy->ctas_per_sm > 0 ? policy->ctas_per_sm : occ;
 
     pl->seq_lens.assign(seq_lens_host, seq_lens_host + shape->batch);
     // The tensor-core kernel walks the work list with a fixed set of resident blocks.
-    if (pl->kernel == DA_KERNEL_MMA_TMA) pl->max_bins = pl->sm_count * pl->ctas_per_sm;
-    rc = make_layout(*shape, *policy, pl->seq_lens.data(), pl->sm_count, pl->ctas_per_sm, pl->layout, pl->max_bins);
+    if (pl->kernel != DA_KERNEL_SIMT) pl->max_bins = pl->sm_count * pl->ctas_per_sm;
+    rc = make_layout(*shape, pl->policy, pl->seq_lens.data(), pl->sm_count, pl->ctas_per_sm, pl->layout, pl->max_bins);
     if (rc != DA_OK) return rc;
 
     if (policy->capacity_batch > 0) {
@@ -396,7 +403,7 @@ int decode_attn_plan(const decode_attn_shape_t* shape, const decode_attn_policy_
         pl->max_batch = shape->batch;
         pl->max_slots = pl->layout.n_slots;
         pl->max_units = (int64_t)pl->layout.units.size();
-        pl->grid = pl->max_units;
+        pl->grid = pl->max_units - pl->layout.n_front_units;   // front units have a launch of their own
     }
     if (pl->grid > 0x7fffffffLL) return DA_ERR_UNSUPPORTED;
     if (pl->max_bins > 0) pl->grid = std::min<int64_t>(pl->grid, pl->max_bins);
@@ -526,7 +533,8 @@ int decode_attn_run_ex(const decode_attn_plan_t* pl, const decode_attn_run_args_
         if (!a->workspace || !aligned(a->workspace, 256)) return DA_ERR_INVALID_ARG;
         if (a->workspace_bytes < pl->workspace_bytes) return DA_ERR_WORKSPACE_TOO_SMALL;
     }
-    if (pl->grid == 0) return DA_OK;
+    const bool umma = pl->kernel == DA_KERNEL_UMMA_PREFIX;
+    if (pl->grid == 0 && !(umma && pl->layout.n_front_units > 0)) return DA_OK;
     const KernelParams kp = make_params(pl, *a);
     if (pl->kernel == DA_KERNEL_SIMT) {
         simt_kernel_t fn = simt_kernel_for(pl->shape.head_dim, pl->group);
@@ -534,8 +542,15 @@ int decode_attn_run_ex(const decode_attn_plan_t* pl, const decode_attn_run_args_
         int rc = simt_launch(fn, kp, (unsigned)pl->grid, stream);
         if (rc != DA_OK) return rc;
     } else {
-        int rc = mma_launch(pl->shape, pl->group, kp, (unsigned)pl->grid, stream, pl->policy.shared_prefix_tokens > 0);
-        if (rc != DA_OK) return rc;
+        if (umma) {   // the shared prefix first, one block per unit at the front of the work list
+            int rc = umma_prefix_launch(pl->shape, pl->group, kp, (unsigned)pl->layout.n_front_units, stream);
+            if (rc != DA_OK) return rc;
+        }
+        if (pl->grid > 0) {
+            int rc = mma_launch(pl->shape, pl->group, kp, (unsigned)pl->grid, stream,
+                                pl->policy.shared_prefix_tokens > 0 && !umma);
+            if (rc != DA_OK) return rc;
+        }
     }
     DA_CUDA_TRY(cudaGetLastError());
     return DA_OK;
@@ -638,6 +653,7 @@ int decode_attn_debug_gather(const decode_attn_plan_t* pl, int32_t seq, const vo
     std::memset(&a, 0, sizeof a);
     a.k_cache = k_cache; a.v_cache = v_cache; a.block_table = block_table;
     const KernelParams kp = make_params(pl, a);
+    if (pl->kernel == DA_KERNEL_UMMA_PREFIX) return DA_ERR_UNSUPPORTED;
     return mma_debug_gather(pl->shape, pl->group, kp, seq, k_out, v_out, (unsigned)pl->work_grid, stream);
 }
 

@@ -57,7 +57,7 @@ int validate_shape(const decode_attn_shape_t& s)
 int validate_policy(const decode_attn_shape_t& s, const decode_attn_policy_t& p)
 {
     if (p.split_mode < DA_SPLIT_AUTO || p.split_mode > DA_SPLIT_DETERMINISTIC) return DA_ERR_INVALID_ARG;
-    if (p.kernel < DA_KERNEL_AUTO || p.kernel > DA_KERNEL_MMA_TMA) return DA_ERR_INVALID_ARG;
+    if (p.kernel < DA_KERNEL_AUTO || p.kernel > DA_KERNEL_UMMA_PREFIX) return DA_ERR_INVALID_ARG;
     if (p.split_mode == DA_SPLIT_FIXED_COUNT && p.fixed_count < 1) return DA_ERR_INVALID_ARG;
     if (p.chunk_tokens < 0 || p.max_splits < 0 || p.sm_count < 0 || p.ctas_per_sm < 0 ||
         p.capacity_batch < 0 || p.capacity_tokens < 0)
@@ -71,7 +71,14 @@ int validate_policy(const decode_attn_shape_t& s, const decode_attn_policy_t& p)
     if (p.shared_prefix_tokens < 0 || p.shared_prefix_tokens % s.page_size != 0) return DA_ERR_INVALID_ARG;
     if (p.shared_prefix_tokens > 0) {
         if (p.fuse_combine || p.capacity_batch > 0 || p.split_mode == DA_SPLIT_FIXED_COUNT) return DA_ERR_UNSUPPORTED;
-        if (p.kernel == DA_KERNEL_SIMT || s.num_q_heads / s.num_kv_heads > 4) return DA_ERR_UNSUPPORTED;
+        const int G = s.num_q_heads / s.num_kv_heads;
+        if (p.kernel == DA_KERNEL_UMMA_PREFIX) {
+            if (s.head_dim != 128 || kUmmaPrefixRows % G != 0) return DA_ERR_UNSUPPORTED;
+        } else if (p.kernel == DA_KERNEL_SIMT || G > 4) {
+            return DA_ERR_UNSUPPORTED;
+        }
+    } else if (p.kernel == DA_KERNEL_UMMA_PREFIX) {
+        return DA_ERR_UNSUPPORTED;   // that kernel serves shared-prefix plans only
     }
     for (int32_t r : p.reserved)
         if (r != 0) return DA_ERR_INVALID_ARG;
@@ -194,17 +201,21 @@ int make_layout(const decode_attn_shape_t& s, const decode_attn_policy_t& p, con
     // of the block's sequences form the columns of one tensor-core tile, so a prefix page is
     // fetched once per block instead of once per sequence.
     const int G = s.num_q_heads / s.num_kv_heads;
-    const int seqs_per_block = prefix_tokens > 0 ? kPrefixColumns / G : 1;
+    const bool umma = p.kernel == DA_KERNEL_UMMA_PREFIX && prefix_tokens > 0;
+    const int seqs_per_block = prefix_tokens > 0 ? (umma ? kUmmaPrefixRows : kPrefixColumns) / G : 1;
     int32_t PC = 0;
     if (prefix_tokens > 0 && B > 0) {
         const int64_t blocks = ceil_div(B, seqs_per_block);
-        const int64_t slots = (int64_t)sm_count * ctas_per_sm;
+        // the mma.sync kernel runs ctas_per_sm blocks on an SM, the tcgen05 kernel one
+        const int64_t slots = umma ? sm_count : (int64_t)sm_count * ctas_per_sm;
         const int64_t max_chunks = std::max<int64_t>(1, prefix_pages / 8);       // chunks of >= 128 tokens
         PC = (int32_t)std::min<int64_t>(max_chunks, std::max<int64_t>(1, slots / (H * blocks)));
         if (p.split_mode == DA_SPLIT_DETERMINISTIC) {
             const int64_t c = min_chunk_pages(s, p);                             // cuts at multiples of the chunk
             PC = (int32_t)std::max<int64_t>(1, ceil_div(prefix_pages, c));
         }
+        if (umma) PC = (int32_t)std::max<int64_t>(PC, ceil_div(prefix_pages, kUmmaPrefixChunkPages));
+        if (umma && PC > max_splits / 2) return DA_ERR_UNSUPPORTED;              // chunks would outgrow tensor memory
         PC = std::min<int32_t>(PC, max_splits / 2);
         for (int64_t j = 0; j < blocks; ++j) {
             const int b0 = (int)(j * seqs_per_block);
@@ -275,19 +286,25 @@ int make_layout(const decode_attn_shape_t& s, const decode_attn_policy_t& p, con
     out.units.clear();
     out.units.reserve(keyed.size());
     out.block_begin.clear();
-    if (max_bins <= 0 || keyed.empty()) {
-        for (const Keyed& k : keyed) out.units.push_back(k.u);
+    out.n_front_units = 0;
+    size_t first = 0;                       // units before this one stay out of the bins
+    if (umma) {
+        while (first < keyed.size() && keyed[first].u.slot == -2) out.units.push_back(keyed[first++].u);
+        out.n_front_units = (int32_t)first;
+    }
+    if (max_bins <= 0 || first == keyed.size()) {
+        for (size_t i = first; i < keyed.size(); ++i) out.units.push_back(keyed[i].u);
         return DA_OK;
     }
     // Longest unit first onto the lightest bin.  A unit costs its pages (a shared-prefix page
     // counts four times: it is attended for a whole block of sequences) plus a fixed charge for
     // the hand-over between units.
     constexpr int64_t kHandOverPages = 24;
-    const int bins = (int)std::min<int64_t>((int64_t)keyed.size(), max_bins);
+    const int bins = (int)std::min<int64_t>((int64_t)(keyed.size() - first), max_bins);
     std::vector<std::vector<int32_t>> members(bins);
     std::priority_queue<std::pair<int64_t, int>, std::vector<std::pair<int64_t, int>>, std::greater<>> heap;
     for (int i = 0; i < bins; ++i) heap.push({0, i});
-    for (size_t i = 0; i < keyed.size(); ++i) {
+    for (size_t i = first; i < keyed.size(); ++i) {
         auto [load, bin] = heap.top();
         heap.pop();
         members[bin].push_back((int32_t)i);

@@ -15,6 +15,8 @@ constexpr int kDefaultMaxSplits = 512;
 constexpr int kMaxSplits = 1024;  // hard bound on the splits of one sequence
 constexpr int kMaxGroup = 8;
 constexpr int kPrefixColumns = 16;  // query rows (sequence x head) one shared-prefix unit attends at once
+constexpr int kUmmaPrefixRows = 128;       // the same for the tcgen05 prefix kernel (the M dimension of its MMAs)
+constexpr int kUmmaPrefixChunkPages = 24;  // and its longest prefix chunk: 384 tokens of logits fit tensor memory
 
 struct Layout {
     std::vector<decode_attn_unit_t> units;  // launch order: most expensive first
@@ -24,6 +26,8 @@ struct Layout {
     int32_t chunk_tokens = 0;
     int32_t max_splits_used = 0;
     int32_t prefix_chunks = 0;              // chunks the shared prefix is cut into (0: no shared prefix)
+    int32_t n_front_units = 0;              // shared-prefix units kept at the front, outside the bins, for a
+                                            // kernel of their own (policy kernel DA_KERNEL_UMMA_PREFIX)
     std::vector<int32_t> block_begin;       // [bins + 1] when the units were packed into bins, else empty
 };
 
@@ -34,7 +38,9 @@ int validate_policy(const decode_attn_shape_t& s, const decode_attn_policy_t& p)
 // Fills `out` for the given lengths.  sm_count and ctas_per_sm must be > 0.
 // max_bins > 0: the units are additionally packed into min(units, max_bins) bins of about equal
 // cost (longest unit first onto the lightest bin) and stored bin by bin; block b of the persistent
-// kernel walks bin b.
+// kernel walks bin b.  With policy kernel DA_KERNEL_UMMA_PREFIX the shared-prefix units are cut for the
+// tcgen05 kernel (128 query rows, chunks of at most 384 tokens), come first in `units` and stay out of
+// the bins; block_begin then indexes the units behind them.
 int make_layout(const decode_attn_shape_t& s, const decode_attn_policy_t& p, const int32_t* seq_lens,
                 int sm_count, int ctas_per_sm, Layout& out, int max_bins = 0);
 
