@@ -542,8 +542,11 @@ int decode_attn_run_ex(const decode_attn_plan_t* pl, const decode_attn_run_args_
         int rc = simt_launch(fn, kp, (unsigned)pl->grid, stream);
         if (rc != DA_OK) return rc;
     } else {
-        if (umma) {   // the shared prefix first, one block per unit at the front of the work list
-            int rc = umma_prefix_launch(pl->shape, pl->group, kp, (unsigned)pl->layout.n_front_units, stream);
+        if (umma) {
+            // the shared prefix first: the units at the front of the work list, dealt to one block per SM
+            const unsigned n_front = (unsigned)pl->layout.n_front_units;
+            int rc = umma_prefix_launch(pl->shape, pl->group, kp, n_front, std::min<unsigned>(n_front, (unsigned)pl->sm_count),
+                                        stream);
             if (rc != DA_OK) return rc;
         }
         if (pl->grid > 0) {
@@ -584,7 +587,9 @@ int decode_attn_combine(const decode_attn_plan_t* pl, const void* workspace, voi
     const KernelParams kp = make_params(pl, a);
     const unsigned grid = (unsigned)(pl->max_batch * pl->shape.num_kv_heads);
     if (grid == 0) return DA_OK;
-    int rc = combine_launch(pl->shape.head_dim, pl->group, kp, grid, stream);
+    // a capacity plan may be refreshed to any split count its policy allows
+    const int max_splits = pl->policy.capacity_batch > 0 ? kMaxSplits : pl->layout.max_splits_used;
+    int rc = combine_launch(pl->shape.head_dim, pl->group, kp, grid, stream, max_splits);
     if (rc != DA_OK) return rc;
     DA_CUDA_TRY(cudaGetLastError());
     return DA_OK;
@@ -967,7 +972,8 @@ int decode_attn_step_static(const decode_attn_shape_t* shape, const int32_t* seq
     }
     DA_CUDA_TRY(cudaGetLastError());
     if (lay.n_slots > 0) {
-        rc = combine_launch(shape->head_dim, G, kp, (unsigned)(shape->batch * shape->num_kv_heads), stream);
+        rc = combine_launch(shape->head_dim, G, kp, (unsigned)(shape->batch * shape->num_kv_heads), stream,
+                            lay.max_splits_used);
         if (rc != DA_OK) return rc;
         DA_CUDA_TRY(cudaGetLastError());
     }

@@ -154,6 +154,12 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
 }
 
+// A location that holds a live barrier must be invalidated before it is initialised again.
+__device__ __forceinline__ void mbar_inval(uint32_t bar)
+{
+    asm volatile("mbarrier.inval.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
+}
+
 __device__ __forceinline__ void mbar_init_fence()
 {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -212,10 +218,11 @@ constexpr int kCombineThreads = 128;
 constexpr int kCombineBatch = 12;
 constexpr int kCombineSmemFloats = 4 * 32 * 6;
 
-template <int D>
+template <int D, int BATCH = kCombineBatch>
 __device__ __forceinline__ void combine_slice(const KernelParams& p, int b, int g, int slice, int G, int slot_base,
                                               int S, int tid, float* sm, int bar_id)
 {
+    constexpr int kCombineBatch = BATCH;    // loads in flight per thread; does not change the order of the sums
     constexpr int D4 = D / 4;
     float* const sm_m = sm;                                    // [4][32]
     float* const sm_l = sm + 128;                              // [4][32]
