@@ -289,6 +289,8 @@ def main():
     lse = torch.empty((first.batch, first.num_q_heads), dtype=torch.float32, device=dev)
     ws = torch.empty(max(plan.workspace_bytes, 256), dtype=torch.uint8, device=dev)
     launches_per_step = 1 if (policy.fuse_combine or info.n_slots == 0) else 2
+    if info.kernel == da.DA_KERNEL_UMMA_PREFIX:
+        launches_per_step += 1      # the tcgen05 prefix kernel, then the kernel for what follows the prefix
 
     run_mask = None
     masked_bytes = 0
@@ -436,9 +438,13 @@ def main():
 
     if rank == 0:
         peak, peak_kind = peak_hbm()
-        achieved = kv_bytes / sec_per_step / 1e9
+        # With a shared-prefix plan a prefix page is fetched once for the whole batch: the bytes the
+        # step has to move are the unique ones.
+        prefix_plan = int(policy.shared_prefix_tokens) > 0
+        algo_bytes = unique_bytes if prefix_plan else kv_bytes
+        achieved = algo_bytes / sec_per_step / 1e9
         kname = {da.DA_KERNEL_SIMT: "decode_attn_simt_kernel", da.DA_KERNEL_MMA_TMA: "decode_attn_mma_kernel",
-                 da.DA_KERNEL_UMMA_PREFIX: "decode_attn_mma_kernel"}[info.kernel]
+                 da.DA_KERNEL_UMMA_PREFIX: "decode_attn_umma_prefix_kernel + decode_attn_mma_kernel"}[info.kernel]
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": sec_per_step * 1e3, "us_per_step": sec_per_step * 1e6,
@@ -458,8 +464,9 @@ def main():
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                          "frac": (achieved / peak) if achieved else None, "peak_kind": f"of {peak_kind}",
                          "kernel": kname, "traffic": NCU_TRAFFIC_BYTES.get(args.workload),
-                         "algorithmic_bytes_per_launch": kv_bytes,
-                         "how": "logical K+V bytes of the batch / (event time of the timed region / steps): the "
+                         "algorithmic_bytes_per_launch": algo_bytes,
+                         "how": ("unique" if prefix_plan else "logical") +
+                                " K+V bytes of the batch / (event time of the timed region / steps): the "
                                 "step's combine launch and launch gaps are charged to the partial kernel"},
             "gpu_launches": args.steps * launches_per_step,
             "clocks": clocks,

@@ -253,3 +253,34 @@ def test_shared_prefix_layout_and_validation():
     bt[3, 2] = bt[3, 5]
     assert da.decode_attn_validate_shared_prefix(s, 64, w.seq_lens, bt) == da.DA_ERR_BAD_PAGE
     assert da.decode_attn_validate_shared_prefix(s, 60, w.seq_lens, w.block_table) == da.DA_ERR_INVALID_ARG
+
+
+def test_tcgen05_prefix_layout():
+    """The plan for the tcgen05 prefix kernel: 128 query rows per unit (128 / G sequences), chunks
+    of at most 384 tokens, prefix units first; what follows the prefix is planned as before."""
+    for hq, hkv, batch, prefix in ((32, 8, 70, 1536), (8, 8, 300, 1024), (16, 2, 40, 112 * 16)):
+        G = hq // hkv
+        lens = wl.lengths_shared_prefix(batch, 5, prefix=prefix)
+        for mode, chunk in ((da.DA_SPLIT_AUTO, 0), (da.DA_SPLIT_DETERMINISTIC, 0), (da.DA_SPLIT_DETERMINISTIC, 128)):
+            pol = da.make_policy(shared_prefix_tokens=prefix, kernel=da.DA_KERNEL_UMMA_PREFIX, split_mode=mode,
+                                 chunk_tokens=chunk)
+            units, splits, slot_base, n_slots, _ = layout(lens, pol, Hq=hq, Hkv=hkv, D=128)
+            prefix_units = [u for u in units if u.kv_head >> 16]
+            assert units[: len(prefix_units)] == prefix_units
+            per_block = 128 // G
+            blocks = -(-batch // per_block)
+            chunks = len({u.split_index for u in prefix_units})
+            assert len(prefix_units) == blocks * hkv * chunks
+            for u in prefix_units:
+                assert u.slot == -2 and u.seq % per_block == 0 and 1 <= (u.kv_head >> 16) <= per_block
+                assert 0 < u.tok_end - u.tok_begin <= 384 and u.tok_begin % 16 == 0 and u.tok_end % 16 == 0
+            cuts = sorted({(u.tok_begin, u.tok_end) for u in prefix_units})
+            assert cuts[0][0] == 0 and cuts[-1][1] == prefix and all(a[1] == b[0] for a, b in zip(cuts, cuts[1:]))
+            assert n_slots == int(sum(splits)) and all(s >= chunks for s in splits)
+    # head_dim 64, or no shared prefix at all: not this kernel's
+    with pytest.raises(da.DecodeAttnError) as e:
+        layout([300, 400], da.make_policy(shared_prefix_tokens=256, kernel=da.DA_KERNEL_UMMA_PREFIX), Hq=8, Hkv=2, D=64)
+    assert e.value.status == da.DA_ERR_UNSUPPORTED
+    with pytest.raises(da.DecodeAttnError) as e:
+        layout([300, 400], da.make_policy(kernel=da.DA_KERNEL_UMMA_PREFIX))
+    assert e.value.status == da.DA_ERR_UNSUPPORTED
