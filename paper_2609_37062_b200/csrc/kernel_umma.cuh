@@ -2,40 +2,47 @@
 //
 // A prefix every sequence of the batch shares (few-shot prompts served from a
 // prefix cache) is a dense contraction: for one KV head, the query rows of
-// many sequences meet the same K/V pages.  One unit = (KV head, chunk of up to
-// 384 prefix tokens, block of 128 / G sequences): the 128 query rows form the
-// M dimension of the MMAs, so a prefix page is fetched once for 128 rows.
+// many sequences meet the same K/V pages.  One unit = (KV head, block of
+// 128 / G sequences, a range of prefix tokens): the 128 query rows form the M
+// dimension of the MMAs, so a prefix page is fetched once for 128 rows.  The
+// range is walked in tiles of 128 tokens, pipelined over two logit buffers and
+// two output buffers in tensor memory:
 //
-//   S = Q K^T   up to three 128 x 128 x 128 tiles, accumulators in tensor
-//               memory columns [0, 384): row r of S in lane r, token t in
-//               column t
-//   softmax     thread r owns row r: exact maximum over the chunk first (tile
-//               by tile as the MMAs finish), then p = 2^(s * scale * log2 e -
-//               m); no running rescale is needed because the whole chunk's
-//               logits are resident
-//   P           must keep more than bf16 precision: the upper 16 bits of p and
-//               the upper 16 bits of the (exact) remainder are written back
-//               over the logits, two bf16 per column: the 32 logit columns of
-//               32 tokens become 16 columns of high parts and 16 of low
-//               parts.  What is dropped is below 2^-16 of p.
-//   O = P V     A = P from tensor memory, B = V tile from shared memory with
-//               the head dimension contiguous; high and low parts accumulate
-//               into the same 128 x 128 fp32 tile in columns [384, 512); the
-//               MMAs of a tile start as soon as that tile's P is written
-//   records     row r = (sequence r / G, head r mod G) goes to that
-//               sequence's record of this prefix chunk, unnormalised, with
-//               (m, l), exactly like any other split; the combine kernel
-//               merges prefix and suffix splits.  Each thread stages its row
-//               in shared memory and sends it with one bulk copy.
+//   S_j = Q K_j^T  128 x 128 x 128, accumulators in tensor memory columns
+//                  [128 b, 128 b + 128), b = j mod 2: row r of S in lane r,
+//                  token t of the tile in column t
+//   softmax        two threads per row.  Each takes the exact maximum m_j of
+//                  the row over the tile, then turns its 64 logits into
+//                  p = 2^(s * scale * log2 e - m_j)
+//   P_j            must keep more than bf16 precision: the upper 16 bits of p
+//                  and the upper 16 bits of the (exact) remainder are written
+//                  back over the logits, two bf16 per column: the 32 logit
+//                  columns of 32 tokens become 16 columns of high parts and
+//                  16 of low parts.  What is dropped is below 2^-16 of p.
+//   O_j = P_j V_j  A = P_j from tensor memory, B = V tile from shared memory
+//                  with the head dimension contiguous; high and low parts
+//                  accumulate into one 128 x 128 fp32 tile in columns
+//                  [256 + 128 b, 256 + 128 b + 128)
+//   merge          while the tensor core works on tile j + 1, the softmax
+//                  threads fetch O_j and fold it into their running state
+//                  (M, L, acc[64]) in registers with the usual log-sum-exp
+//                  rescale, in ascending tile order
+//   record         row r = (sequence r / G, head r mod G) goes to that
+//                  sequence's record of this prefix chunk, unnormalised, with
+//                  (M, L), exactly like any other split; the combine kernel
+//                  merges prefix and suffix splits.  Each thread stages its
+//                  half row in shared memory and sends it with one bulk copy.
 //
-// Threads: eight warps for softmax and epilogue, two per 32 lanes of tensor
-// memory (one takes the even, one the odd 32-token groups of a row);
-// a ninth warp issues the TMA boxes and, from one lane, the MMAs.  The 2 n tiles of a
-// chunk of n token tiles (K_0 .. K_n-1, V_0 .. V_n-1) go through two stages of
-// shared memory in that order; a stage is refilled when the MMAs that read
-// its tile have completed.  Every barrier is used once.  Every wait is
-// bounded; a wait that gives up records DA_ERR_TIMEOUT, and the block still
-// frees its tensor memory.
+// Threads: eight warps for softmax, merge and epilogue, two per 32 lanes of
+// tensor memory (one takes the even, one the odd 32-token groups of a row and
+// one half of the output columns); one warp whose first lane issues the MMAs;
+// one warp that issues the TMA boxes.  K_0, V_0, K_1, V_1, ... go through a
+// ring of four 32 KB stages; a stage is handed back by the tcgen05.commit of
+// the MMAs that read it.  Blocks are persistent (one per SM: the buffers fill
+// tensor memory); the barriers are invalidated and set up again for every
+// unit.  Every wait is bounded and also ends when another thread of the block
+// has given up; the block then records DA_ERR_TIMEOUT, skips its records and
+// still frees its tensor memory.
 #pragma once
 
 #include "kernel_mma.cuh"
@@ -44,24 +51,21 @@
 namespace da {
 
 constexpr int kUmmaTraceBase = 2048;              // debug timelines: rows of this kernel's units
-constexpr int kUmmaSoftmaxWarps = 8;              // two per 32 lanes of tensor memory
+constexpr int kUmmaSoftmaxWarps = 8;
 constexpr int kUmmaSoftmaxThreads = kUmmaSoftmaxWarps * 32;
-constexpr int kUmmaThreads = kUmmaSoftmaxThreads + 32;   // + the warp that issues loads and MMAs
+constexpr int kUmmaMmaWarp = kUmmaSoftmaxWarps;       // lane 0 issues the MMAs
+constexpr int kUmmaLoadWarp = kUmmaSoftmaxWarps + 1;  // issues the TMA boxes
+constexpr int kUmmaThreads = kUmmaSoftmaxThreads + 64;
 constexpr int kUmmaRows = 128;                    // query rows of a unit
 constexpr int kUmmaTileTokens = 128;
-constexpr int kUmmaMaxTiles = 3;
-constexpr int kUmmaMaxTokens = kUmmaTileTokens * kUmmaMaxTiles;
 constexpr int kUmmaHalfBytes = 128 * 128;         // 128 rows x 64 dims of bf16
 constexpr int kUmmaTileBytes = 2 * kUmmaHalfBytes;   // [half of the head dim][row][64 dims]
-constexpr int kUmmaStages = 2;
-constexpr int kUmmaBarrierBytes = 2048;           // barriers, page ids, the halves' maxima and sums
-constexpr int kUmmaSmemUsed = (1 + kUmmaStages) * kUmmaTileBytes + kUmmaBarrierBytes + 1024 /* alignment */;
-// Asked for: more than half an SM's shared memory, so that two of these blocks, each of which
-// wants all of tensor memory, never share an SM.
-constexpr int kUmmaSmemBytes = 116 * 1024;
-static_assert(kUmmaSmemUsed <= kUmmaSmemBytes, "shared memory of the tcgen05 prefix kernel");
+constexpr int kUmmaStages = 4;
+constexpr int kUmmaMiscBytes = 4096;              // barriers, small state, the halves' row maxima and sums
+constexpr int kUmmaSmemBytes = (1 + kUmmaStages) * kUmmaTileBytes + kUmmaMiscBytes + 1024 /* alignment */;
+static_assert(kUmmaSmemBytes > 114 * 1024, "two of these blocks, each wanting all of tensor memory, must not share an SM");
 constexpr int kUmmaTmemCols = 512;
-constexpr int kUmmaOutCol = kUmmaMaxTokens;       // first column of the output tile
+constexpr int kUmmaOutCol = 256;                  // first column of the output buffers
 constexpr int kUmmaOutRowBytes = 128 * 4 + 16;    // a staged output row; the pad spreads the rows over the banks
 
 inline bool umma_supports(int D, int G) { return D == 128 && (G == 1 || G == 2 || G == 4 || G == 8); }
@@ -76,27 +80,49 @@ __device__ __forceinline__ void bulk_store_commit_and_wait_read()
     asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
 }
 
+// Bounded wait that also ends when the block has given up elsewhere.  The first thread to run
+// out of time raises the flag.
+__device__ __forceinline__ bool umma_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if (*abort_flag != 0) return false;
+        if (clock64() - t0 > kWaitLimitCycles) {
+            *abort_flag = 1;
+            return false;
+        }
+    }
+    return true;
+}
+
 // Shared-prefix units first_unit, first_unit + unit_stride, ... < n_units, one after the other, by
-// the 288 threads of a block.  smem_raw: at least kUmmaSmemUsed bytes of dynamic shared memory.
+// the 320 threads of a block.  smem_raw: at least kUmmaSmemBytes of dynamic shared memory.
 __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const CUtensorMap* k_map, const CUtensorMap* v_map,
                                                   const int G, const int first_unit, const int unit_stride,
                                                   const int n_units, uint8_t* smem_raw)
 {
     constexpr int D = 128;
+    constexpr int NS = kUmmaStages;
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t* const gbase = smem_raw + (base - raw);
     const uint32_t q_base = base;
-    const uint32_t tile_base = base + kUmmaTileBytes;                       // stage s at tile_base + s * tile bytes
-    const uint32_t bar_base = base + (1 + kUmmaStages) * kUmmaTileBytes;
-    // single-use barriers: full[6] (a tile has landed), done[6] (the MMAs reading it have completed;
-    // for a K tile that also means its logits are ready), p_ready[3], o_ready
-    const uint32_t bar_full = bar_base, bar_done = bar_base + 48, bar_p = bar_base + 96, bar_o = bar_base + 120;
+    const uint32_t ring_base = base + kUmmaTileBytes;                       // stage s at ring_base + s * tile bytes
+    uint8_t* const ring_ptr = gbase + kUmmaTileBytes;
+    const uint32_t bar_base = base + (1 + NS) * kUmmaTileBytes;
+    // full[4]: a tile has landed; empty[4]: the MMAs reading it have completed; s_ready[2]: the logits
+    // of a tile are complete; p_ready[2]: its weights are written (all softmax threads); o_ready[2]:
+    // its output tile is complete (and its weights consumed); o_free[2]: the output tile was read;
+    // m_ready[2]: both halves of every row have published their maximum of the tile
+    const uint32_t bar_full = bar_base, bar_empty = bar_base + 32, bar_s = bar_base + 64, bar_p = bar_base + 80;
+    const uint32_t bar_o = bar_base + 96, bar_ofree = bar_base + 112, bar_m = bar_base + 128;
+    constexpr int kBarriers = 18;
     uint8_t* const sm_misc = gbase + (bar_base - base);
-    volatile uint32_t* const sm_tmem = reinterpret_cast<volatile uint32_t*>(sm_misc + 128);
-    volatile int* const sm_abort = reinterpret_cast<volatile int*>(sm_misc + 132);
-    int32_t* const sm_pages = reinterpret_cast<int32_t*>(sm_misc + 256);    // [24] page ids of the chunk
-    float* const sm_part = reinterpret_cast<float*>(sm_misc + 512);         // [2][128]: the column halves' maxima, then sums
+    volatile uint32_t* const sm_tmem = reinterpret_cast<volatile uint32_t*>(sm_misc + 160);
+    volatile int* const sm_abort = reinterpret_cast<volatile int*>(sm_misc + 164);
+    volatile float* const sm_max = reinterpret_cast<volatile float*>(sm_misc + 512);   // [2 buffers][2 halves][128 rows]
+    float* const sm_l = reinterpret_cast<float*>(sm_misc + 512 + 2048);     // [2][128]: the column halves' row sums
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     if (first_unit >= n_units) {
@@ -108,7 +134,7 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
         tma_prefetch_descriptor(v_map);
         *sm_abort = 0;
     }
-    if (warp == kUmmaSoftmaxWarps) umma::tmem_alloc(smem_u32(const_cast<uint32_t*>(sm_tmem)), kUmmaTmemCols);
+    if (warp == kUmmaMmaWarp) umma::tmem_alloc(smem_u32(const_cast<uint32_t*>(sm_tmem)), kUmmaTmemCols);
     umma::fence_before_thread_sync();
     __syncthreads();
     umma::fence_after_thread_sync();
@@ -116,271 +142,275 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
     // Only this block's own state was touched so far.
     pdl_wait_primary();
 
-  for (int unit_index = first_unit; unit_index < n_units && *sm_abort == 0; unit_index += unit_stride) {
-    const decode_attn_unit_t u = load_unit(p.units, unit_index);
-    const int g = u.kv_head & 0xffff, nseq = u.kv_head >> 16;
-    const int n_tok = u.tok_end - u.tok_begin;                              // whole pages, at most 384 tokens
-    const int n_pages = n_tok >> 4;
-    const int n_tiles = (n_tok + kUmmaTileTokens - 1) / kUmmaTileTokens;
-    if (tid == 0) DA_TRACE_STAMP(kUmmaTraceBase + unit_index, 0);
-    if (tid == 0) {
-        // every barrier serves one unit: set up again for each (the block is past a barrier here,
-        // nobody is still waiting on the previous unit's)
-        if (unit_index != first_unit)
-            for (int i = 0; i < 16; ++i) mbar_inval(bar_base + 8 * i);
-        for (int i = 0; i < 12; ++i) mbar_init(bar_base + 8 * i, 1);
-        for (int i = 0; i < 3; ++i) mbar_init(bar_p + 8 * i, kUmmaSoftmaxThreads);
-        mbar_init(bar_o, 1);
-        mbar_init_fence();
-    }
-    __syncthreads();
-    if (tid == 0) DA_TRACE_STAMP(kUmmaTraceBase + unit_index, 1);
+    for (int unit_index = first_unit; unit_index < n_units && *sm_abort == 0; unit_index += unit_stride) {
+        const decode_attn_unit_t u = load_unit(p.units, unit_index);
+        const int g = u.kv_head & 0xffff, nseq = u.kv_head >> 16;
+        const int n_tok = u.tok_end - u.tok_begin;                          // whole pages
+        const int n_pages = n_tok >> 4;
+        const int T = (n_tok + kUmmaTileTokens - 1) / kUmmaTileTokens;      // tiles
+        if (tid == 0) {
+            DA_TRACE_STAMP(kUmmaTraceBase + unit_index, 0);
+            // the barriers serve one unit: set up again for each (the block is past a barrier here,
+            // nobody is still waiting on the previous unit's, and every arrival on them has landed)
+            if (unit_index != first_unit)
+                for (int i = 0; i < kBarriers; ++i) mbar_inval(bar_base + 8 * i);
+            for (int i = 0; i < 2 * NS + 2; ++i) mbar_init(bar_base + 8 * i, 1);      // full, empty, s_ready
+            for (int i = 0; i < 2; ++i) mbar_init(bar_p + 8 * i, kUmmaSoftmaxThreads);
+            for (int i = 0; i < 2; ++i) mbar_init(bar_o + 8 * i, 1);
+            for (int i = 0; i < 2; ++i) mbar_init(bar_ofree + 8 * i, kUmmaSoftmaxThreads);
+            for (int i = 0; i < 2; ++i) mbar_init(bar_m + 8 * i, kUmmaSoftmaxThreads);
+            mbar_init_fence();
+        }
+        __syncthreads();
 
-    if (warp == kUmmaSoftmaxWarps) {
-        // ------------------------------------------------------------ loads and MMAs
-        {
-            // the chunk's page ids, checked once
-            int page_id = (int)p.num_pages;   // a page past the chunk is fetched from outside the pool: zeros
-            if (lane < n_pages) {
-                page_id = __ldg(p.block_table + (int64_t)u.seq * p.max_pages_per_seq + (u.tok_begin >> 4) + lane);
-                if ((unsigned)page_id >= (unsigned)p.num_pages) {           // never hand TMA a page outside the pool
-                    record_status(p.status, DA_ERR_BAD_PAGE);
-                    page_id = 0;
+        if (warp == kUmmaLoadWarp) {
+            // -------------------------------------------------------- TMA: K_0, V_0, K_1, V_1, ...
+            const uint64_t l2_policy = l2_policy_evict_first();
+            const int32_t* bt = p.block_table + (int64_t)u.seq * p.max_pages_per_seq + (u.tok_begin >> 4);
+            const int pg = (lane >> 1) & 7, hf = lane & 1;                  // lane j < 16: box (page j / 2, half j % 2)
+            int page_id = 0;
+            bool ok = true;
+            for (int n = 0; n < 2 * T && ok; ++n) {
+                const int t = n >> 1, st = n % NS;
+                if ((n & 1) == 0) {
+                    // the tile's page ids, checked once, used for K and for V; a page past the
+                    // range is fetched from outside the pool, which the TMA unit fills with zeros
+                    page_id = (int)p.num_pages;
+                    if (t * 8 + pg < n_pages) {
+                        page_id = __ldg(bt + t * 8 + pg);
+                        if ((unsigned)page_id >= (unsigned)p.num_pages) {   // never hand TMA a page outside the pool
+                            record_status(p.status, DA_ERR_BAD_PAGE);
+                            page_id = 0;
+                        }
+                    }
                 }
+                if (n >= NS) {
+                    if (lane == 0) ok = umma_wait(bar_empty + 8 * st, ((n / NS) - 1) & 1, sm_abort);
+                    ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+                    if (!ok) break;
+                }
+                const uint32_t bar = bar_full + 8 * st;
+                if (lane == 0) mbar_arrive_expect_tx(bar, kUmmaTileBytes);
+                __syncwarp();
+                if (lane < 16)
+                    tma_load_4d(ring_base + st * kUmmaTileBytes + hf * kUmmaHalfBytes + pg * 2048, (n & 1) ? v_map : k_map, bar,
+                                hf * 64, 0, g, page_id, l2_policy);
             }
-            if (lane < 24) sm_pages[lane] = page_id;
-            __syncwarp();
-        }
-        const uint64_t l2_policy = l2_policy_evict_first();
-        const int n_loads = 2 * n_tiles;
-        // load i of the chunk: K tile i for i < n_tiles, else V tile i - n_tiles; stage i % 2.
-        // Whole warp: lane j < 16 issues box (page j / 2, half j % 2).
-        auto issue = [&](int i) {
-            const bool is_v = i >= n_tiles;
-            const int t = is_v ? i - n_tiles : i;
-            const uint32_t bar = bar_full + 8 * i;
-            if (lane == 0) mbar_arrive_expect_tx(bar, kUmmaTileBytes);
-            __syncwarp();
-            if (lane < 16) {
-                const int pg = lane >> 1, hf = lane & 1;
-                const uint32_t dst = tile_base + (i % kUmmaStages) * kUmmaTileBytes + hf * kUmmaHalfBytes + pg * 2048;
-                tma_load_4d(dst, is_v ? v_map : k_map, bar, hf * 64, 0, g, sm_pages[t * 8 + pg], l2_policy);
-            }
-        };
-        // lane 0 waits, the warp learns the outcome
-        auto wait = [&](uint32_t bar) {
-            bool r = true;
-            if (lane == 0) r = mbar_wait(bar, 0);
-            return __shfl_sync(0xffffffffu, (int)r, 0) != 0;
-        };
-        issue(0);
-        issue(1);
-        if (lane == 0) DA_TRACE_STAMP(kUmmaTraceBase + unit_index, 2);
-        block_sync(1, kUmmaThreads);                                        // Q is in shared memory
-        constexpr uint32_t idesc_qk = umma::instr_desc_bf16(128, 128, false);
-        constexpr uint32_t idesc_pv = umma::instr_desc_bf16(128, 128, true);
-        bool ok = true;
-        // S_t = Q K_t^T
-        for (int t = 0; t < n_tiles && ok; ++t) {
-            ok = wait(bar_full + 8 * t);
-            if (!ok) break;
+        } else if (warp == kUmmaMmaWarp) {
+            // -------------------------------------------------------- MMAs (one lane)
+            block_sync(1, kUmmaSoftmaxThreads + 32);                        // Q is in shared memory
             if (lane == 0) {
-                if (t == n_tiles - 1) DA_TRACE_STAMP(kUmmaTraceBase + unit_index, 3);
-                umma::fence_after_thread_sync();
-                const uint32_t kt = tile_base + (t % kUmmaStages) * kUmmaTileBytes;
+                constexpr uint32_t idesc_qk = umma::instr_desc_bf16(128, 128, false);
+                constexpr uint32_t idesc_pv = umma::instr_desc_bf16(128, 128, true);
+                bool ok = true;
+                // S_j = Q K_j^T into logit buffer j % 2 (free once tile j - 2's P V has completed)
+                auto qk = [&](int j) {
+                    const int n = 2 * j, st = n % NS, b = j & 1;
+                    ok = umma_wait(bar_full + 8 * st, (n / NS) & 1, sm_abort);
+                    if (ok && j >= 2) ok = umma_wait(bar_o + 8 * b, ((j - 2) >> 1) & 1, sm_abort);
+                    if (!ok) return;
+                    umma::fence_after_thread_sync();
+                    const uint32_t kt = ring_base + st * kUmmaTileBytes;
 #pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks) {
-                    const uint32_t off = (ks >> 2) * kUmmaHalfBytes + (ks & 3) * 32;
-                    umma::mma_ss(tmem + t * kUmmaTileTokens, umma::smem_desc_sw128(q_base + off, 16, 1024),
-                                 umma::smem_desc_sw128(kt + off, 16, 1024), idesc_qk, ks > 0);
-                }
-                umma::commit(bar_done + 8 * t);
-            }
-            __syncwarp();
-            if (t + 2 < n_loads) {                                          // the stage is free once these MMAs are done
-                ok = wait(bar_done + 8 * t);
-                if (ok) issue(t + 2);
-            }
-        }
-        if (lane == 0) DA_TRACE_STAMP(kUmmaTraceBase + unit_index, 4);
-        // O += P_t V_t
-        for (int t = 0; t < n_tiles && ok; ++t) {
-            const int i = n_tiles + t;
-            ok = wait(bar_p + 8 * t);
-            if (lane == 0 && t == 0) DA_TRACE_STAMP(kUmmaTraceBase + unit_index, 9);
-            if (ok) ok = wait(bar_full + 8 * i);
-            if (!ok) break;
-            if (lane == 0) {
-                if (t == n_tiles - 1) DA_TRACE_STAMP(kUmmaTraceBase + unit_index, 10);
-                umma::fence_after_thread_sync();
-                const uint32_t vt = tile_base + (i % kUmmaStages) * kUmmaTileBytes;
-                const int ksteps = min(8, (n_tok - t * kUmmaTileTokens) >> 4);
+                    for (int ks = 0; ks < D / 16; ++ks) {
+                        const uint32_t off = (ks >> 2) * kUmmaHalfBytes + (ks & 3) * 32;
+                        umma::mma_ss(tmem + b * 128, umma::smem_desc_sw128(q_base + off, 16, 1024),
+                                     umma::smem_desc_sw128(kt + off, 16, 1024), idesc_qk, ks > 0);
+                    }
+                    umma::commit(bar_empty + 8 * st);
+                    umma::commit(bar_s + 8 * b);
+                };
+                // O_j = P_j V_j into output buffer j % 2 (free once tile j - 2's output was read)
+                auto pv = [&](int j) {
+                    const int n = 2 * j + 1, st = n % NS, b = j & 1;
+                    ok = umma_wait(bar_p + 8 * b, (j >> 1) & 1, sm_abort);
+                    if (ok) ok = umma_wait(bar_full + 8 * st, (n / NS) & 1, sm_abort);
+                    if (ok && j >= 2) ok = umma_wait(bar_ofree + 8 * b, ((j - 2) >> 1) & 1, sm_abort);
+                    if (!ok) return;
+                    umma::fence_after_thread_sync();
+                    const uint32_t vt = ring_base + st * kUmmaTileBytes;
+                    const int ksteps = min(8, (n_tok - j * kUmmaTileTokens) >> 4);
 #pragma unroll 2
-                for (int j = 0; j < ksteps; ++j) {
-                    // 16 tokens: two groups of 8 rows, 128 bytes a row; the upper 64 dims one half further
-                    const uint64_t b = umma::smem_desc_sw128(vt + j * 2048, kUmmaHalfBytes, 1024);
-                    const int kj = t * 8 + j;                               // 16-token step within the chunk
-                    const uint32_t a_hi = tmem + (kj >> 1) * 32 + (kj & 1) * 8;
-                    umma::mma_ts(tmem + kUmmaOutCol, a_hi, b, idesc_pv, kj > 0);
-                    umma::mma_ts(tmem + kUmmaOutCol, a_hi + 16, b, idesc_pv, true);
+                    for (int k = 0; k < ksteps; ++k) {
+                        // 16 tokens: two groups of 8 rows, 128 bytes a row; the upper 64 dims one half further
+                        const uint64_t bd = umma::smem_desc_sw128(vt + k * 2048, kUmmaHalfBytes, 1024);
+                        const uint32_t a_hi = tmem + b * 128 + (k >> 1) * 32 + (k & 1) * 8;
+                        umma::mma_ts(tmem + kUmmaOutCol + b * 128, a_hi, bd, idesc_pv, k > 0);
+                        umma::mma_ts(tmem + kUmmaOutCol + b * 128, a_hi + 16, bd, idesc_pv, true);
+                    }
+                    umma::commit(bar_empty + 8 * st);
+                    umma::commit(bar_o + 8 * b);
+                };
+                qk(0);
+                if (ok && T > 1) qk(1);
+                for (int j = 0; j < T && ok; ++j) {
+                    pv(j);
+                    if (ok && j + 2 < T) qk(j + 2);
                 }
-                umma::commit(bar_done + 8 * i);
+                // nothing may arrive on a barrier after the unit: the last two stages' hand-backs
+                if (ok) {
+                    const int n1 = 2 * T - 1, n0 = 2 * T - 2;
+                    ok = umma_wait(bar_empty + 8 * (n1 % NS), (n1 / NS) & 1, sm_abort);
+                    if (ok) ok = umma_wait(bar_empty + 8 * (n0 % NS), (n0 / NS) & 1, sm_abort);
+                }
             }
-            __syncwarp();
-            if (lane == 0 && t == 1) DA_TRACE_STAMP(kUmmaTraceBase + unit_index, 15);
-            if (i + 2 < n_loads) {
-                ok = wait(bar_done + 8 * i);
-                if (lane == 0) DA_TRACE_STAMP(kUmmaTraceBase + unit_index, 14);
-                if (ok) issue(i + 2);
-            }
-        }
-        if (lane == 0) {
-            if (ok) {
-                umma::commit(bar_o);
-            } else {
-                record_status(p.status, DA_ERR_TIMEOUT);
-                *sm_abort = 1;
-            }
-        }
-    } else {
-        // ------------------------------------------------------------ query rows, softmax, epilogue
-        // Two threads per row: thread (quarter q, lane) of column half hh = warp / 4 owns row
-        // r = 32 q + lane, the even (hh = 0) or odd (hh = 1) 32-token groups of the logits, and
-        // half of the output columns.
-        const int hh = warp >> 2;
-        const int r = (warp & 3) * 32 + lane;                               // row of the tile = lane of tensor memory
-        const int sl = r / G, h = r % G;
-        const bool valid = sl < nseq;
-        const int seq = u.seq + (valid ? sl : 0);
-        {
-            // 64 dims of row r of Q, 8 chunks of 16 bytes, into the swizzled K-major tile
-            const uint4* src = reinterpret_cast<const uint4*>(p.q + ((int64_t)seq * p.num_q_heads + g * G + h) * D) + hh * 8;
-            uint4 v[8];
+        } else {
+            // -------------------------------------------------------- query rows, softmax, merge, epilogue
+            // Two threads per row: thread (quarter q, lane) of column half hh = warp / 4 owns row
+            // r = 32 q + lane, the even (hh = 0) or odd (hh = 1) 32-token groups of the logits, and
+            // output columns [64 hh, 64 hh + 64).
+            const int hh = warp >> 2;
+            const int r = (warp & 3) * 32 + lane;                           // row of the tile = lane of tensor memory
+            const int sl = r / G, h = r % G;
+            const bool valid = sl < nseq;
+            const int seq = u.seq + (valid ? sl : 0);
+            {
+                // 64 dims of row r of Q, 8 chunks of 16 bytes, into the swizzled K-major tile
+                const uint4* src = reinterpret_cast<const uint4*>(p.q + ((int64_t)seq * p.num_q_heads + g * G + h) * D) + hh * 8;
+                uint4 v[8];
 #pragma unroll
-            for (int c = 0; c < 8; ++c) v[c] = valid ? __ldg(src + c) : make_uint4(0u, 0u, 0u, 0u);
+                for (int c = 0; c < 8; ++c) v[c] = valid ? __ldg(src + c) : make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
-            for (int c = 0; c < 8; ++c) {
-                const uint32_t off = hh * kUmmaHalfBytes + r * 128 + ((c ^ (r & 7)) << 4);
-                *reinterpret_cast<uint4*>(gbase + off) = v[c];
+                for (int c = 0; c < 8; ++c) {
+                    const uint32_t off = hh * kUmmaHalfBytes + r * 128 + ((c ^ (r & 7)) << 4);
+                    *reinterpret_cast<uint4*>(gbase + off) = v[c];
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); // visible to the tensor core's reads
             }
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // visible to the tensor core's reads
-        }
-        if (tid == 0) DA_TRACE_STAMP(kUmmaTraceBase + unit_index, 5);
-        block_sync(1, kUmmaThreads);
+            block_sync(1, kUmmaSoftmaxThreads + 32);
+            if (tid == 0) DA_TRACE_STAMP(kUmmaTraceBase + unit_index, 1);
 
-        const SeqInfo si = p.seq_info[seq];
-        bool dead = p.run_mask != nullptr && __ldg(p.run_mask + seq) == 0;  // masked row: an empty record
-        if (valid && __ldg(p.seq_lens + seq) != si.seq_len) {                // stale plan: void the result, report it
-            dead = true;
-            if (hh == 0) record_status(p.status, DA_ERR_STALE_PLAN);
-        }
+            const SeqInfo si = p.seq_info[seq];
+            bool dead = p.run_mask != nullptr && __ldg(p.run_mask + seq) == 0;   // masked row: an empty record
+            if (valid && __ldg(p.seq_lens + seq) != si.seq_len) {            // stale plan: void the result, report it
+                dead = true;
+                if (hh == 0) record_status(p.status, DA_ERR_STALE_PLAN);
+            }
 
-        const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
-        const int n_chunks = (n_tok + 31) >> 5;
-        uint32_t sa[32], sb[32];
-        bool ok = true;
-        float mx = -INFINITY, l = 0.f;
-        // pass 1: the row maximum, tile by tile as the logits arrive
-        for (int t = 0; t < n_tiles && ok; ++t) {
-            ok = mbar_wait(bar_done + 8 * t, 0);
-            if (!ok) break;
-            if (tid == 0 && t == n_tiles - 1) DA_TRACE_STAMP(kUmmaTraceBase + unit_index, 6);
-            umma::fence_after_thread_sync();
-            const int c0 = 4 * t + hh, c1 = c0 + 2;                          // this thread's two groups of the tile
-            if (c0 < n_chunks) umma::ld32(lane_base + c0 * 32, sa);
-            if (c1 < n_chunks) umma::ld32(lane_base + c1 * 32, sb);
-            umma::wait_ld();
-            if (c0 < n_chunks) {
+            const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+            float acc[64];
 #pragma unroll
-                for (int i = 0; i < 32; ++i)
-                    if (c0 * 32 + i < n_tok) mx = fmaxf(mx, __uint_as_float(sa[i]));
-            }
-            if (c1 < n_chunks) {
+            for (int i = 0; i < 64; ++i) acc[i] = 0.f;
+            float M = -INFINITY, L = 0.f;       // running maximum (log2 domain), this thread's share of the row sum
+            float m_prev = 0.f, l_prev = 0.f;   // of the tile whose output is still to be folded in
+            uint32_t sa[32], sb[32];
+            bool ok = true;
+
+            // folds tile i's output into the running state
+            auto fold = [&](int i) {
+                const int b = i & 1;
+                ok = umma_wait(bar_o + 8 * b, (i >> 1) & 1, sm_abort);
+                if (!ok) return;
+                umma::fence_after_thread_sync();
+                const uint32_t oc = lane_base + kUmmaOutCol + b * 128 + hh * 64;
+                umma::ld32(oc, sa);
+                umma::ld32(oc + 32, sb);
+                umma::wait_ld();
+                umma::fence_before_thread_sync();
+                mbar_arrive(bar_ofree + 8 * b);                              // the buffer may be overwritten
+                const float Mn = fmaxf(M, m_prev);
+                const float a = ex2f(M - Mn), c = ex2f(m_prev - Mn);        // M = -inf at first: a = 0
 #pragma unroll
-                for (int i = 0; i < 32; ++i)
-                    if (c1 * 32 + i < n_tok) mx = fmaxf(mx, __uint_as_float(sb[i]));
-            }
-        }
-        sm_part[hh * 128 + r] = mx;
-        block_sync(2, kUmmaSoftmaxThreads);
-        const float m2 = fmaxf(sm_part[r], sm_part[128 + r]) * p.scale_log2;   // the scale is positive
-        block_sync(2, kUmmaSoftmaxThreads);                                  // sm_part is reused for the sums
-        if (tid == 0) DA_TRACE_STAMP(kUmmaTraceBase + unit_index, 7);
-        // pass 2: weights, written back over the logits as bf16 high and low parts
-        auto weights = [&](const uint32_t (&s)[32], int c) {
-            uint32_t hi[16], lo[16];
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                float p0 = 0.f, p1 = 0.f;
-                if (c * 32 + 2 * i < n_tok) p0 = ex2f(fmaf(__uint_as_float(s[2 * i]), p.scale_log2, -m2));
-                if (c * 32 + 2 * i + 1 < n_tok) p1 = ex2f(fmaf(__uint_as_float(s[2 * i + 1]), p.scale_log2, -m2));
-                l += p0 + p1;
-                const uint32_t b0 = __float_as_uint(p0), b1 = __float_as_uint(p1);
-                const float r0 = p0 - __uint_as_float(b0 & 0xffff0000u);     // exact
-                const float r1 = p1 - __uint_as_float(b1 & 0xffff0000u);
-                hi[i] = __byte_perm(b0, b1, 0x7632);                         // upper halves: element 2i low, 2i+1 high
-                lo[i] = __byte_perm(__float_as_uint(r0), __float_as_uint(r1), 0x7632);
-            }
-            // the group's 32 logit columns become 16 columns of high parts, 16 of low parts
-            umma::st16(lane_base + c * 32, hi);
-            umma::st16(lane_base + c * 32 + 16, lo);
-        };
-        for (int t = 0; t < n_tiles && ok; ++t) {
-            const int c0 = 4 * t + hh, c1 = c0 + 2;
-            if (c0 < n_chunks) umma::ld32(lane_base + c0 * 32, sa);
-            if (c1 < n_chunks) umma::ld32(lane_base + c1 * 32, sb);
-            umma::wait_ld();
-            if (c0 < n_chunks) weights(sa, c0);
-            if (c1 < n_chunks) weights(sb, c1);
-            umma::wait_st();
-            umma::fence_before_thread_sync();
-            mbar_arrive(bar_p + 8 * t);                                       // this tile's P V may start
-            if (tid == 0 && t < 2) DA_TRACE_STAMP(kUmmaTraceBase + unit_index, 16 + t);
-        }
-        if (tid == 0) DA_TRACE_STAMP(kUmmaTraceBase + unit_index, 8);
-        sm_part[hh * 128 + r] = l;
-        if (ok) ok = mbar_wait(bar_o, 0);
-        if (tid == 0) DA_TRACE_STAMP(kUmmaTraceBase + unit_index, 11);
-        block_sync(2, kUmmaSoftmaxThreads);                                  // the sums of both halves are visible
-        if (ok) {
-            umma::fence_after_thread_sync();
-            // Every MMA has completed: the Q tile and the stages are free.  This thread's half
-            // of the row is staged there and leaves with one bulk copy.
-            const int RF = rec_floats(G, D);
-            float* const rec = p.ws + ((int64_t)(si.slot_base + u.split_index) * p.num_kv_heads + g) * RF;
-            uint8_t* const row = gbase + r * kUmmaOutRowBytes + hh * 256;
-#pragma unroll 1
-            for (int c = 0; c < 2; ++c) {
-                umma::ld32(lane_base + kUmmaOutCol + hh * 64 + c * 32, sa);
+                for (int k = 0; k < 32; ++k) {
+                    acc[k] = fmaf(acc[k], a, __uint_as_float(sa[k]) * c);
+                    acc[32 + k] = fmaf(acc[32 + k], a, __uint_as_float(sb[k]) * c);
+                }
+                L = fmaf(L, a, l_prev * c);
+                M = Mn;
+            };
+
+            for (int j = 0; j < T && ok; ++j) {
+                const int b = j & 1;
+                const int tok0 = j * kUmmaTileTokens;                        // first token of the tile within the unit
+                const int n_here = min(kUmmaTileTokens, n_tok - tok0);      // a multiple of 16
+                ok = umma_wait(bar_s + 8 * b, (j >> 1) & 1, sm_abort);
+                if (!ok) break;
+                if (tid == 0 && j == 0) DA_TRACE_STAMP(kUmmaTraceBase + unit_index, 2);
+                umma::fence_after_thread_sync();
+                const uint32_t sc = lane_base + b * 128;
+                // pass 1: the maximum of this thread's 64 logits; the row's other half is exchanged
+                // through shared memory (its logits may not be read once it starts writing weights)
+                float mx = -INFINITY;
+                umma::ld32(sc + hh * 32, sa);
+                umma::ld32(sc + hh * 32 + 64, sb);
                 umma::wait_ld();
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    uint4 v = make_uint4(sa[4 * i], sa[4 * i + 1], sa[4 * i + 2], sa[4 * i + 3]);
-                    if (dead) v = make_uint4(0u, 0u, 0u, 0u);
-                    *reinterpret_cast<uint4*>(row + c * 128 + i * 16) = v;
+                for (int i = 0; i < 32; ++i) {
+                    if (hh * 32 + i < n_here) mx = fmaxf(mx, __uint_as_float(sa[i]));
+                    if (hh * 32 + 64 + i < n_here) mx = fmaxf(mx, __uint_as_float(sb[i]));
                 }
+                sm_max[(b * 2 + hh) * 128 + r] = mx;
+                mbar_arrive(bar_m + 8 * b);
+                ok = umma_wait(bar_m + 8 * b, (j >> 1) & 1, sm_abort);
+                if (!ok) break;
+                mx = fmaxf(mx, sm_max[(b * 2 + (1 - hh)) * 128 + r]);
+                const float m2 = mx * p.scale_log2;                          // the scale is positive
+                // pass 2: this thread's 64 weights, written back over the logits as bf16 high and low parts
+                float lsum = 0.f;
+                auto weights = [&](const uint32_t (&s)[32], int col0) {
+                    uint32_t hi[16], lo[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        float p0 = 0.f, p1 = 0.f;
+                        if (col0 + 2 * i < n_here) p0 = ex2f(fmaf(__uint_as_float(s[2 * i]), p.scale_log2, -m2));
+                        if (col0 + 2 * i + 1 < n_here) p1 = ex2f(fmaf(__uint_as_float(s[2 * i + 1]), p.scale_log2, -m2));
+                        lsum += p0 + p1;
+                        const uint32_t b0 = __float_as_uint(p0), b1 = __float_as_uint(p1);
+                        const float r0 = p0 - __uint_as_float(b0 & 0xffff0000u);   // exact
+                        const float r1 = p1 - __uint_as_float(b1 & 0xffff0000u);
+                        hi[i] = __byte_perm(b0, b1, 0x7632);                 // upper halves: element 2i low, 2i+1 high
+                        lo[i] = __byte_perm(__float_as_uint(r0), __float_as_uint(r1), 0x7632);
+                    }
+                    // the group's 32 logit columns become 16 columns of high parts, 16 of low parts
+                    umma::st16(sc + col0, hi);
+                    umma::st16(sc + col0 + 16, lo);
+                };
+                weights(sa, hh * 32);
+                weights(sb, hh * 32 + 64);
+                umma::wait_st();
+                umma::fence_before_thread_sync();
+                mbar_arrive(bar_p + 8 * b);                                   // this tile's P V may start
+                // while it runs, fold in the tile before
+                if (j >= 1) fold(j - 1);
+                m_prev = m2;
+                l_prev = lsum;
             }
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // visible to the bulk copy's reads
-            if (valid) {
-                bulk_store_s2g(rec + h * D + hh * 64, smem_u32(row), 256);
-                if (hh == 0)
-                    __stcg(reinterpret_cast<float2*>(rec + G * D) + h,
-                           dead ? make_float2(-INFINITY, 0.f) : make_float2(m2, sm_part[r] + sm_part[128 + r]));
+            if (ok) fold(T - 1);
+            if (tid == 0) DA_TRACE_STAMP(kUmmaTraceBase + unit_index, 3);
+            // the row sum is the two halves' sums
+            sm_l[hh * 128 + r] = L;
+            block_sync(2, kUmmaSoftmaxThreads);
+            if (ok) {
+                // Every MMA has completed and every tile was consumed: the ring is free.  This
+                // thread's half of the row is staged there and leaves with one bulk copy.
+                const int RF = rec_floats(G, D);
+                float* const rec = p.ws + ((int64_t)(si.slot_base + u.split_index) * p.num_kv_heads + g) * RF;
+                uint8_t* const row = ring_ptr + r * kUmmaOutRowBytes + hh * 256;
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    float4 v = make_float4(acc[4 * i], acc[4 * i + 1], acc[4 * i + 2], acc[4 * i + 3]);
+                    if (dead) v = make_float4(0.f, 0.f, 0.f, 0.f);
+                    *reinterpret_cast<float4*>(row + i * 16) = v;
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); // visible to the bulk copy's reads
+                if (valid) {
+                    bulk_store_s2g(rec + h * D + hh * 64, smem_u32(row), 256);
+                    if (hh == 0)
+                        __stcg(reinterpret_cast<float2*>(rec + G * D) + h,
+                               dead ? make_float2(-INFINITY, 0.f) : make_float2(M, sm_l[r] + sm_l[128 + r]));
+                }
+                bulk_store_commit_and_wait_read();
             }
-            bulk_store_commit_and_wait_read();
-        } else if (lane == 0 && *sm_abort == 0) {
-            record_status(p.status, DA_ERR_TIMEOUT);
+            if (tid == 0) DA_TRACE_STAMP(kUmmaTraceBase + unit_index, 4);
         }
-        if (tid == 0) DA_TRACE_STAMP(kUmmaTraceBase + unit_index, 12);
+        // the next unit reuses shared memory, tensor memory and the barriers
+        umma::fence_before_thread_sync();
+        __syncthreads();
+        umma::fence_after_thread_sync();
     }
-    // the next unit reuses shared memory, tensor memory and the barriers
-    umma::fence_before_thread_sync();
-    __syncthreads();
-    umma::fence_after_thread_sync();
-    if (tid == 0) DA_TRACE_STAMP(kUmmaTraceBase + unit_index, 13);
-  }
+    if (tid == 0 && *sm_abort != 0) record_status(p.status, DA_ERR_TIMEOUT);
     pdl_launch_dependents();
-    if (warp == kUmmaSoftmaxWarps) umma::tmem_dealloc(tmem, kUmmaTmemCols);
+    if (warp == kUmmaMmaWarp) umma::tmem_dealloc(tmem, kUmmaTmemCols);
 }
 
 __global__ void __launch_bounds__(kUmmaThreads, 1)

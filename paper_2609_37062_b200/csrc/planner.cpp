@@ -208,22 +208,30 @@ int make_layout(const decode_attn_shape_t& s, const decode_attn_policy_t& p, con
         const int64_t blocks = ceil_div(B, seqs_per_block);
         // the mma.sync kernel runs ctas_per_sm blocks on an SM, the tcgen05 kernel one
         const int64_t slots = umma ? sm_count : (int64_t)sm_count * ctas_per_sm;
-        const int64_t max_chunks = std::max<int64_t>(1, prefix_pages / 8);       // chunks of >= 128 tokens
+        // chunks of >= 128 tokens; the tcgen05 kernel works in whole 128-token tiles
+        const int64_t max_chunks = umma ? ceil_div(prefix_pages, 8) : std::max<int64_t>(1, prefix_pages / 8);
         PC = (int32_t)std::min<int64_t>(max_chunks, std::max<int64_t>(1, slots / (H * blocks)));
         if (p.split_mode == DA_SPLIT_DETERMINISTIC) {
             const int64_t c = min_chunk_pages(s, p);                             // cuts at multiples of the chunk
             PC = (int32_t)std::max<int64_t>(1, ceil_div(prefix_pages, c));
         }
-        if (umma) PC = (int32_t)std::max<int64_t>(PC, ceil_div(prefix_pages, kUmmaPrefixChunkPages));
-        if (umma && PC > max_splits / 2) return DA_ERR_UNSUPPORTED;              // chunks would outgrow tensor memory
         PC = std::min<int32_t>(PC, max_splits / 2);
         for (int64_t j = 0; j < blocks; ++j) {
             const int b0 = (int)(j * seqs_per_block);
             const int nseq = std::min(seqs_per_block, B - b0);
             for (int32_t i = 0; i < PC; ++i) {
-                const int64_t q = prefix_pages / PC, r = prefix_pages % PC;
-                const int64_t pb = i * q + std::min<int64_t>(i, r);
-                const int64_t pe = pb + q + (i < r ? 1 : 0);
+                int64_t pb, pe;
+                if (umma && p.split_mode != DA_SPLIT_DETERMINISTIC) {
+                    // whole 128-token tiles (8 pages), dealt evenly; the last chunk takes the ragged end
+                    const int64_t tiles = ceil_div(prefix_pages, 8);
+                    const int64_t q = tiles / PC, r = tiles % PC;
+                    pb = std::min<int64_t>(prefix_pages, (i * q + std::min<int64_t>(i, r)) * 8);
+                    pe = std::min<int64_t>(prefix_pages, pb + (q + (i < r ? 1 : 0)) * 8);
+                } else {
+                    const int64_t q = prefix_pages / PC, r = prefix_pages % PC;
+                    pb = i * q + std::min<int64_t>(i, r);
+                    pe = pb + q + (i < r ? 1 : 0);
+                }
                 for (int g = 0; g < H; ++g) {
                     Keyed k;
                     k.u.seq = b0;

@@ -16,7 +16,6 @@ constexpr int kMaxSplits = 1024;  // hard bound on the splits of one sequence
 constexpr int kMaxGroup = 8;
 constexpr int kPrefixColumns = 16;  // query rows (sequence x head) one shared-prefix unit attends at once
 constexpr int kUmmaPrefixRows = 128;       // the same for the tcgen05 prefix kernel (the M dimension of its MMAs)
-constexpr int kUmmaPrefixChunkPages = 24;  // and its longest prefix chunk: 384 tokens of logits fit tensor memory
 
 struct Layout {
     std::vector<decode_attn_unit_t> units;  // launch order: most expensive first
@@ -39,7 +38,7 @@ int validate_policy(const decode_attn_shape_t& s, const decode_attn_policy_t& p)
 // max_bins > 0: the units are additionally packed into min(units, max_bins) bins of about equal
 // cost (longest unit first onto the lightest bin) and stored bin by bin; block b of the persistent
 // kernel walks bin b.  With policy kernel DA_KERNEL_UMMA_PREFIX the shared-prefix units are cut for the
-// tcgen05 kernel (128 query rows, chunks of at most 384 tokens), come first in `units` and stay out of
+// tcgen05 kernel (128 query rows, chunks of whole 128-token tiles), come first in `units` and stay out of
 // the bins; block_begin then indexes the units behind them.
 int make_layout(const decode_attn_shape_t& s, const decode_attn_policy_t& p, const int32_t* seq_lens,
                 int sm_count, int ctas_per_sm, Layout& out, int max_bins = 0);

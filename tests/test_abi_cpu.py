@@ -257,7 +257,7 @@ def test_shared_prefix_layout_and_validation():
 
 def test_tcgen05_prefix_layout():
     """The plan for the tcgen05 prefix kernel: 128 query rows per unit (128 / G sequences), chunks
-    of at most 384 tokens, prefix units first; what follows the prefix is planned as before."""
+    of whole 128-token tiles (AUTO), prefix units first; what follows the prefix is planned as before."""
     for hq, hkv, batch, prefix in ((32, 8, 70, 1536), (8, 8, 300, 1024), (16, 2, 40, 112 * 16)):
         G = hq // hkv
         lens = wl.lengths_shared_prefix(batch, 5, prefix=prefix)
@@ -273,7 +273,9 @@ def test_tcgen05_prefix_layout():
             assert len(prefix_units) == blocks * hkv * chunks
             for u in prefix_units:
                 assert u.slot == -2 and u.seq % per_block == 0 and 1 <= (u.kv_head >> 16) <= per_block
-                assert 0 < u.tok_end - u.tok_begin <= 384 and u.tok_begin % 16 == 0 and u.tok_end % 16 == 0
+                assert 0 < u.tok_end - u.tok_begin and u.tok_begin % 16 == 0 and u.tok_end % 16 == 0
+                if mode == da.DA_SPLIT_AUTO:
+                    assert u.tok_begin % 128 == 0 and (u.tok_end % 128 == 0 or u.tok_end == prefix)
             cuts = sorted({(u.tok_begin, u.tok_end) for u in prefix_units})
             assert cuts[0][0] == 0 and cuts[-1][1] == prefix and all(a[1] == b[0] for a, b in zip(cuts, cuts[1:]))
             assert n_slots == int(sum(splits)) and all(s >= chunks for s in splits)
