@@ -227,6 +227,7 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
                     if (ok) ok = umma_wait(bar_full + 8 * st, (n / NS) & 1, sm_abort);
                     if (ok && j >= 2) ok = umma_wait(bar_ofree + 8 * b, ((j - 2) >> 1) & 1, sm_abort);
                     if (!ok) return;
+                    if (j < 6) DA_TRACE_STAMP(kUmmaTraceBase + unit_index, 16 + j);
                     umma::fence_after_thread_sync();
                     const uint32_t vt = ring_base + st * kUmmaTileBytes;
                     const int ksteps = min(8, (n_tok - j * kUmmaTileTokens) >> 4);
@@ -301,6 +302,7 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
                 const int b = i & 1;
                 ok = umma_wait(bar_o + 8 * b, (i >> 1) & 1, sm_abort);
                 if (!ok) return;
+                if (tid == 0 && i < 6) DA_TRACE_STAMP(kUmmaTraceBase + unit_index, 22 + i);
                 umma::fence_after_thread_sync();
                 const uint32_t oc = lane_base + kUmmaOutCol + b * 128 + hh * 64;
                 umma::ld32(oc, sa);
@@ -326,6 +328,7 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
                 ok = umma_wait(bar_s + 8 * b, (j >> 1) & 1, sm_abort);
                 if (!ok) break;
                 if (tid == 0 && j == 0) DA_TRACE_STAMP(kUmmaTraceBase + unit_index, 2);
+                if (tid == 0 && j >= 1 && j <= 5) DA_TRACE_STAMP(kUmmaTraceBase + unit_index, 9 + j);
                 umma::fence_after_thread_sync();
                 const uint32_t sc = lane_base + b * 128;
                 // pass 1: the maximum of this thread's 64 logits; the row's other half is exchanged
@@ -370,6 +373,7 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
                 umma::wait_st();
                 umma::fence_before_thread_sync();
                 mbar_arrive(bar_p + 8 * b);                                   // this tile's P V may start
+                if (tid == 0 && j < 3) DA_TRACE_STAMP(kUmmaTraceBase + unit_index, 5 + j);
                 // while it runs, fold in the tile before
                 if (j >= 1) fold(j - 1);
                 m_prev = m2;

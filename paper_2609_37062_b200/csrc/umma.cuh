@@ -39,7 +39,8 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr, uint32_t lbo,
     return d;
 }
 
-// Instruction descriptor of a dense bf16 x bf16 -> fp32 MMA of shape M x N x 16.
+// Instruction descriptor of a dense bf16 x bf16 -> fp32 MMA of shape M x N x 16.  (Both
+// operands have to be of the same 16-bit type: an fp16 A with a bf16 B is rejected by the GPU.)
 // b_mn_major: operand B is stored with N contiguous (else K contiguous); A is K-major.
 __host__ __device__ constexpr uint32_t instr_desc_bf16(int M, int N, bool b_mn_major)
 {
