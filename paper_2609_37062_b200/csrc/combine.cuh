@@ -9,9 +9,7 @@
 
 namespace da {
 
-// BATCH: records a thread keeps in flight (see combine_slice).  Plans with few splits per
-// sequence launch the small variant, whose lower register count lets four times as many blocks
-// be resident; the sums are the same either way.
+// BATCH: records a thread keeps in flight (see combine_slice).
 template <int D, int BATCH>
 __global__ void __launch_bounds__(kCombineThreads) decode_attn_combine_kernel(const KernelParams p, int G, int n_slices)
 {
@@ -31,14 +29,33 @@ __global__ void __launch_bounds__(kCombineThreads) decode_attn_combine_kernel(co
     combine_slice<D, BATCH>(p, b, g, slice, G, si.slot_base, si.n_splits, threadIdx.x, sm, 0);
 }
 
+// Plans whose sequences have at most MAXS (4 or 8) splits: one thread per output column, 128
+// columns per block, nothing shared between threads (see combine_column).
+template <int D, int MAXS>
+__global__ void __launch_bounds__(kCombineThreads) decode_attn_combine_few_kernel(const KernelParams p, int G, int blocks_per_group)
+{
+    pdl_launch_dependents();
+    const int bg = blockIdx.x / blocks_per_group;
+    const int col = (blockIdx.x % blocks_per_group) * kCombineThreads + threadIdx.x;
+    const int b = bg / p.num_kv_heads, g = bg % p.num_kv_heads;
+    const bool in_batch = b < p.header->batch;
+    SeqInfo si;
+    si.slot_base = -1;
+    if (in_batch) si = p.seq_info[b];
+    pdl_wait_primary();
+    if (si.slot_base < 0 || col >= G * (D / 4)) return;
+    combine_column<D, MAXS>(p, b, g, col, G, si.slot_base, si.n_splits);
+}
+
 // Launches the combine kernel with a programmatic dependency on whatever was
 // launched before it on `stream` (the partial kernel).
 template <int D>
-inline int combine_launch_dim(int G, const KernelParams& kp, unsigned groups, cudaStream_t stream, bool few_splits)
+inline int combine_launch_dim(int G, const KernelParams& kp, unsigned groups, cudaStream_t stream, int max_splits)
 {
     const int n_slices = combine_slices(D, G);
+    const int blocks_per_group = (G * (D / 4) + kCombineThreads - 1) / kCombineThreads;
     cudaLaunchConfig_t cfg;
-    cfg.gridDim = dim3(groups * (unsigned)n_slices, 1, 1);
+    cfg.gridDim = dim3(groups * (unsigned)(max_splits <= 8 ? blocks_per_group : n_slices), 1, 1);
     cfg.blockDim = dim3(kCombineThreads, 1, 1);
     cfg.dynamicSmemBytes = 0;
     cfg.stream = stream;
@@ -47,8 +64,10 @@ inline int combine_launch_dim(int G, const KernelParams& kp, unsigned groups, cu
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    const cudaError_t e = few_splits ? cudaLaunchKernelEx(&cfg, decode_attn_combine_kernel<D, 2>, kp, G, n_slices)
-                                     : cudaLaunchKernelEx(&cfg, decode_attn_combine_kernel<D, kCombineBatch>, kp, G, n_slices);
+    const cudaError_t e =
+        max_splits <= 4   ? cudaLaunchKernelEx(&cfg, decode_attn_combine_few_kernel<D, 4>, kp, G, blocks_per_group)
+        : max_splits <= 8 ? cudaLaunchKernelEx(&cfg, decode_attn_combine_few_kernel<D, 8>, kp, G, blocks_per_group)
+                          : cudaLaunchKernelEx(&cfg, decode_attn_combine_kernel<D, kCombineBatch>, kp, G, n_slices);
     if (e != cudaSuccess) {
         (void)cudaGetLastError();
         return DA_ERR_CUDA;
@@ -59,9 +78,8 @@ inline int combine_launch_dim(int G, const KernelParams& kp, unsigned groups, cu
 // max_splits: the most splits any sequence of the plan (or of its capacity) can have.
 inline int combine_launch(int D, int G, const KernelParams& kp, unsigned groups, cudaStream_t stream, int max_splits)
 {
-    const bool few = max_splits <= 8;
-    if (D == 64) return combine_launch_dim<64>(G, kp, groups, stream, few);
-    if (D == 128) return combine_launch_dim<128>(G, kp, groups, stream, few);
+    if (D == 64) return combine_launch_dim<64>(G, kp, groups, stream, max_splits);
+    if (D == 128) return combine_launch_dim<128>(G, kp, groups, stream, max_splits);
     return DA_ERR_UNSUPPORTED;
 }
 

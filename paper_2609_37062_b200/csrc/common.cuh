@@ -306,6 +306,65 @@ __device__ __forceinline__ void combine_slice(const KernelParams& p, int b, int 
     block_sync(bar_id, kCombineThreads);                       // the scratch may be reused by the next slice
 }
 
+// The same merge for sequences of at most MAXS (<= 8) splits, one thread per output column and no
+// shared memory: the thread keeps the four chains in registers and adds them in the same order,
+// so the bits equal combine_slice's.  All of the thread's loads are in flight at once.
+template <int D, int MAXS>
+__device__ __forceinline__ void combine_column(const KernelParams& p, int b, int g, int col, int G, int slot_base, int S)
+{
+    constexpr int D4 = D / 4;
+    const int h = col / D4, d4 = col % D4;
+    const int RF = rec_floats(G, D);
+    const float* const recs = p.ws + ((int64_t)slot_base * p.num_kv_heads + g) * RF;
+    const int64_t rec_stride = (int64_t)p.num_kv_heads * RF;
+    const float4* const colp = reinterpret_cast<const float4*>(recs) + col;
+    const float2* const mlp = reinterpret_cast<const float2*>(recs + G * D) + h;
+    float2 ml[MAXS];
+    float4 v[MAXS];
+#pragma unroll
+    for (int j = 0; j < MAXS; ++j) {
+        ml[j] = make_float2(-INFINITY, 0.f);
+        v[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (j < S) {
+            ml[j] = __ldcg(mlp + j * (rec_stride / 2));
+            v[j] = __ldcg(colp + j * (rec_stride / 4));
+        }
+    }
+    float M = -INFINITY;
+#pragma unroll
+    for (int j = 0; j < MAXS; ++j) M = fmaxf(M, ml[j].x);
+    float4 acc[4];
+    float lch[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+        lch[k] = 0.f;
+    }
+#pragma unroll
+    for (int j = 0; j < MAXS; ++j) {
+        if (j < S) {
+            const float w = (M == -INFINITY) ? 0.f : ex2f(ml[j].x - M);   // empty split: m = -inf, w = 0
+            acc[j & 3].x = fmaf(w, v[j].x, acc[j & 3].x);
+            acc[j & 3].y = fmaf(w, v[j].y, acc[j & 3].y);
+            acc[j & 3].z = fmaf(w, v[j].z, acc[j & 3].z);
+            acc[j & 3].w = fmaf(w, v[j].w, acc[j & 3].w);
+            lch[j & 3] = fmaf(w, ml[j].y, lch[j & 3]);
+        }
+    }
+    const float ls = ((lch[0] + lch[1]) + lch[2]) + lch[3];
+    float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (M != -INFINITY && ls > 0.f) {
+        const float inv = 1.0f / ls;
+        o.x = (((acc[0].x + acc[1].x) + acc[2].x) + acc[3].x) * inv;
+        o.y = (((acc[0].y + acc[1].y) + acc[2].y) + acc[3].y) * inv;
+        o.z = (((acc[0].z + acc[1].z) + acc[2].z) + acc[3].z) * inv;
+        o.w = (((acc[0].w + acc[1].w) + acc[2].w) + acc[3].w) * inv;
+    }
+    store_out4(p.out, ((int64_t)b * p.num_q_heads + g * G + h) * D + d4 * 4, o, p.out_bf16);
+    if (p.lse != nullptr && d4 == 0)
+        p.lse[(int64_t)b * p.num_q_heads + g * G + h] = (M != -INFINITY && ls > 0.f) ? (M + log2f(ls)) * kLn2 : -INFINITY;
+}
+
 __host__ __device__ inline int combine_slices(int D, int G) { return (G * (D / 4) + 31) / 32; }
 
 __device__ __forceinline__ int32_t ld_acquire(const int32_t* ptr)
