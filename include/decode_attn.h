@@ -268,6 +268,26 @@ int decode_attn_append_kv(const decode_attn_shape_t *shape, const void *new_k, c
                           const int32_t *block_table, const int32_t *seq_lens, void *k_cache, void *v_cache,
                           cudaStream_t stream);
 
+/* Merge of KV-range shards (context parallelism; the paper has no multi-GPU
+ * path - this is the one exchange step the decode path has when a single
+ * long sequence is sharded by token range).  Every shard attended its own
+ * token range of the same (sequence, query head) rows with plan / run /
+ * combine and holds a normalised output with its log-sum-exp; after the
+ * shards' results were gathered (torch.distributed all_gather over NCCL, or
+ * one process that ran the shards one after the other), this call writes
+ *   M = max_r lse_r;  w_r = e^{lse_r - M};  out = sum_r w_r out_r / sum_r w_r;
+ *   lse = M + log(sum_r w_r)
+ * in ascending shard order (fixed: the result does not depend on timing).
+ *   out_shards  device, fp32 [n_shards, batch, num_q_heads, head_dim], 16-byte aligned
+ *   lse_shards  device, fp32 [n_shards, batch, num_q_heads]; -inf marks a shard
+ *               whose range was empty for that row (it weighs exactly zero)
+ *   out         device, [batch, num_q_heads, head_dim] in shape.out_dtype, 16-byte aligned
+ *   lse_or_null device, fp32 [batch, num_q_heads] or NULL
+ * Rows that are empty in every shard get zeros and lse = -inf.  1 <= n_shards
+ * <= 1024.  One launch on `stream`, nothing is allocated, capture-safe. */
+int decode_attn_merge_shards(const decode_attn_shape_t *shape, int32_t n_shards, const float *out_shards,
+                             const float *lse_shards, void *out, float *lse_or_null, cudaStream_t stream);
+
 /* LSE combine: merges the partials `run` left in the workspace, per
  * (sequence, query head), in ascending split order:
  *   M = max_i m_i;  out = sum_i e^{m_i-M} o_i / sum_i e^{m_i-M} l_i;  lse = M + log(sum_i e^{m_i-M} l_i)

@@ -53,6 +53,7 @@ EXPORTED = [
     "decode_attn_host_step", "decode_attn_host_release", "decode_attn_strerror", "decode_attn_version",
     "decode_attn_step_static", "decode_attn_append_kv", "decode_attn_breakeven_tokens",
     "decode_attn_switch_thresholds", "decode_attn_switch_next", "decode_attn_validate_shared_prefix",
+    "decode_attn_merge_shards",
 ]
 
 
@@ -124,6 +125,7 @@ _lib.decode_attn_host_step.argtypes = [ctypes.POINTER(Shape), ctypes.POINTER(Pol
 _lib.decode_attn_host_release.argtypes = []
 _lib.decode_attn_step_static.argtypes = [ctypes.POINTER(Shape), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.decode_attn_append_kv.argtypes = [ctypes.POINTER(Shape), _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.decode_attn_merge_shards.argtypes = [ctypes.POINTER(Shape), ctypes.c_int32, _vp, _vp, _vp, _vp, _vp]
 _lib.decode_attn_breakeven_tokens.argtypes = [ctypes.c_double, ctypes.c_double, ctypes.c_double, ctypes.c_int32,
                                               ctypes.c_double, ctypes.POINTER(ctypes.c_double)]
 _lib.decode_attn_switch_thresholds.argtypes = [ctypes.c_double, ctypes.c_double, ctypes.POINTER(ctypes.c_double),
@@ -372,6 +374,15 @@ def decode_attn_append_kv(shape: Shape, new_k, new_v, block_table, seq_lens, k_c
                                     _ptr(k_cache), _ptr(v_cache), _stream(stream))
     if check:
         _check(rc, "decode_attn_append_kv")
+    return rc
+
+
+def decode_attn_merge_shards(shape: Shape, n_shards: int, out_shards, lse_shards, out, lse=None, stream=None,
+                             check: bool = True) -> int:
+    rc = _lib.decode_attn_merge_shards(ctypes.byref(shape), int(n_shards), _ptr(out_shards), _ptr(lse_shards), _ptr(out),
+                                       _ptr(lse), _stream(stream))
+    if check:
+        _check(rc, "decode_attn_merge_shards")
     return rc
 
 

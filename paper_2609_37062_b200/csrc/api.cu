@@ -595,6 +595,26 @@ int decode_attn_combine(const decode_attn_plan_t* pl, const void* workspace, voi
     return DA_OK;
 }
 
+int decode_attn_merge_shards(const decode_attn_shape_t* shape, int32_t n_shards, const float* out_shards,
+                             const float* lse_shards, void* out, float* lse_or_null, cudaStream_t stream)
+{
+    if (!shape || !out_shards || !lse_shards || !out) return DA_ERR_INVALID_ARG;
+    int rc = validate_shape(*shape);
+    if (rc != DA_OK) return rc;
+    if (n_shards < 1 || n_shards > kMaxSplits) return DA_ERR_INVALID_ARG;
+    if (!aligned(out_shards, 16) || !aligned(out, 16) || !aligned(lse_shards, 4)) return DA_ERR_INVALID_ARG;
+    const int64_t rows = (int64_t)shape->batch * shape->num_q_heads;
+    if (rows == 0) return DA_OK;
+    const int D4 = shape->head_dim / 4;
+    const int64_t threads = rows * D4;
+    const int64_t blocks = (threads + 127) / 128;
+    if (blocks > 0x7fffffffLL) return DA_ERR_UNSUPPORTED;
+    decode_attn_merge_shards_kernel<<<(unsigned)blocks, 128, 0, stream>>>(out_shards, lse_shards, n_shards, rows, D4, out,
+                                                                            lse_or_null, shape->out_dtype == DA_DTYPE_BF16);
+    DA_CUDA_TRY(cudaGetLastError());
+    return DA_OK;
+}
+
 int decode_attn_last_device_status(const decode_attn_plan_t* pl, cudaStream_t stream)
 {
     if (!pl) return DA_ERR_INVALID_ARG;

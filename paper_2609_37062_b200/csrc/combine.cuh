@@ -47,6 +47,37 @@ __global__ void __launch_bounds__(kCombineThreads) decode_attn_combine_few_kerne
     combine_column<D, MAXS>(p, b, g, col, G, si.slot_base, si.n_splits);
 }
 
+// Merge of KV-range shards: every shard holds a normalised output and its log-sum-exp (natural
+// log) for each row; one thread per four output dims, shards in ascending order.
+__global__ void __launch_bounds__(128) decode_attn_merge_shards_kernel(const float* out_shards, const float* lse_shards,
+                                                                       int n_shards, int64_t rows, int D4, void* out,
+                                                                       float* lse, int out_bf16)
+{
+    const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= rows * D4) return;
+    const int64_t row = idx / D4;
+    const int d4 = (int)(idx % D4);
+    float M = -INFINITY;
+    for (int r = 0; r < n_shards; ++r) M = fmaxf(M, __ldg(lse_shards + (int64_t)r * rows + row));
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    float ws = 0.f;
+    if (M != -INFINITY) {
+        for (int r = 0; r < n_shards; ++r) {
+            const float w = ex2f((__ldg(lse_shards + (int64_t)r * rows + row) - M) * kLog2e);   // empty shard: w = 0
+            const float4 v = __ldg(reinterpret_cast<const float4*>(out_shards) + ((int64_t)r * rows + row) * D4 + d4);
+            acc.x = fmaf(w, v.x, acc.x);
+            acc.y = fmaf(w, v.y, acc.y);
+            acc.z = fmaf(w, v.z, acc.z);
+            acc.w = fmaf(w, v.w, acc.w);
+            ws += w;
+        }
+        const float inv = 1.0f / ws;                          // ws >= 1: the shard that holds the maximum weighs 1
+        acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+    }
+    store_out4(out, idx * 4, acc, out_bf16);
+    if (lse != nullptr && d4 == 0) lse[row] = (M != -INFINITY) ? M + log2f(ws) * kLn2 : -INFINITY;
+}
+
 // Launches the combine kernel with a programmatic dependency on whatever was
 // launched before it on `stream` (the partial kernel).
 template <int D>

@@ -65,6 +65,20 @@ def _worker(rank, world, port, result_dir):
             parts = torch.stack([g[h] for g in gathered]).numpy()        # rank order = ascending token order
             merged, lse = oracle.merge_partials(parts[:, :D], parts[:, D], parts[:, D + 1])
             assert np.max(np.abs(merged - full[0, h])) < 1e-12 and abs(lse - full_lse[0, h]) < 1e-12
+        # ---- the same through the helpers the GPU path uses: local tables per rank, normalised
+        # outputs with their log-sum-exp, one gather; the merge is the oracle's here (no GPU)
+        mix = wl.make_workload("cp", [1000, 40, 16, 333], 8, 2, 64, seed=11)
+        bt, lens = sharding.shard_kv_tables(mix.block_table, mix.seq_lens, 16, world, rank)
+        import dataclasses
+        local = dataclasses.replace(mix, block_table=bt, seq_lens=lens, max_pages_per_seq=bt.shape[1])
+        o_loc, lse_loc = oracle.paged_decode_attention(oracle.PagedInputs.from_workload(local), num_threads=2)
+        outs, lses = sharding.gather_shards(torch.from_numpy(o_loc), torch.from_numpy(lse_loc))
+        assert outs.shape == (world, 4, 8, 64) and lses.shape == (world, 4, 8)
+        ref, ref_lse = oracle.paged_decode_attention(oracle.PagedInputs.from_workload(mix), num_threads=2)
+        for b in range(4):
+            for h in range(8):
+                merged, lse = oracle.merge_partials(outs[:, b, h].numpy(), lses[:, b, h].numpy(), np.ones(world))
+                assert np.max(np.abs(merged - ref[b, h])) < 1e-12 and abs(lse - ref_lse[b, h]) < 1e-12
     finally:
         dist.destroy_process_group()
 
