@@ -56,6 +56,19 @@ def test_tcgen05_prefix_groups(hq, hkv):
     check(w, policy(prefix, da.DA_KERNEL_UMMA_PREFIX))
 
 
+def test_tcgen05_prefix_long_units_and_few_blocks():
+    """A planner told of 8 SMs leaves the whole 6,400-token prefix to one unit (50 tiles: the stage
+    ring and the tensor-memory buffers wrap many times) and runs the 16 units of the two sequence
+    blocks on 8 persistent thread blocks (two units each, barriers set up again in between)."""
+    w = wl.config_shared_prefix(batch=40, prefix=6400)
+    pol = policy(6400, da.DA_KERNEL_UMMA_PREFIX, sm_count=8)
+    plan = da.decode_attn_plan(da.shape_of_workload(w), pol, w.seq_lens)
+    front = [u for u in da.decode_attn_plan_get_units(plan) if u.kv_head >> 16]
+    assert len(front) == 16 and all(u.tok_end - u.tok_begin == 6400 for u in front)
+    plan.destroy()
+    check(w, pol)
+
+
 def test_tcgen05_prefix_refuses_what_it_cannot_run():
     w = wl.make_workload("p", [300, 400], 8, 2, 64, seed=1, shared_prefix_tokens=256)      # head_dim 64
     with pytest.raises(da.DecodeAttnError) as e:
