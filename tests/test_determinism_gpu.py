@@ -79,3 +79,15 @@ def test_fused_and_separate_merge_give_the_same_bits(kernel):
     b, lb = da.run_workload(w, da.make_policy(kernel=kernel, split_mode=da.DA_SPLIT_DETERMINISTIC, chunk_tokens=512,
                                               fuse_combine=1))
     assert torch.equal(a, b) and torch.equal(la, lb)
+
+
+@pytest.mark.parametrize("splits", [2, 3, 4, 5, 8, 9, 13, 49])
+def test_every_merge_kernel_gives_the_fused_path_its_bits(splits):
+    """The combine launch picks a kernel by the plan's largest split count (one thread per column
+    up to 4 and up to 8 splits, the slice kernel beyond); all of them and the merge blocks of a
+    fused launch add the same four chains in the same order."""
+    w = to_device(wl.make_workload("m", [4000, 17, 900, 2500, 64], 32, 8, 128, seed=41))
+    pol = dict(split_mode=da.DA_SPLIT_FIXED_COUNT, fixed_count=splits)
+    a, la = da.run_workload(w, da.make_policy(fuse_combine=0, **pol))
+    b, lb = da.run_workload(w, da.make_policy(fuse_combine=1, **pol))
+    assert torch.equal(a, b) and torch.equal(la, lb)
