@@ -196,6 +196,11 @@ int make_layout(const decode_attn_shape_t& s, const decode_attn_policy_t& p, con
         int64_t cost;
     };
     std::vector<Keyed> keyed;
+    {
+        size_t expect = 0;
+        for (int b = 0; b < B; ++b) expect += (size_t)cuts[b].splits;
+        keyed.reserve((expect + (size_t)B) * (size_t)H + 64);
+    }
 
     // Shared prefix: a unit is (block of sequences, KV head, chunk of the prefix); the query rows
     // of the block's sequences form the columns of one tensor-core tile, so a prefix page is
@@ -290,39 +295,73 @@ int make_layout(const decode_attn_shape_t& s, const decode_attn_policy_t& p, con
         }
     }
     out.prefix_chunks = PC;
-    std::stable_sort(keyed.begin(), keyed.end(), [](const Keyed& a, const Keyed& b) { return a.cost > b.cost; });
+    // Launch order: most expensive unit first, ties in creation order.  Sorting 4-byte indices is
+    // much cheaper than moving the units (this runs every decode step).
+    const size_t n = keyed.size();
+    std::vector<uint32_t> order(n);
+    for (size_t i = 0; i < n; ++i) order[i] = (uint32_t)i;
+    bool sorted = true;
+    for (size_t i = 1; i < n && sorted; ++i) sorted = keyed[i - 1].cost >= keyed[i].cost;
+    if (!sorted)
+        std::stable_sort(order.begin(), order.end(),
+                         [&keyed](uint32_t x, uint32_t y) { return keyed[x].cost > keyed[y].cost; });
     out.units.clear();
-    out.units.reserve(keyed.size());
+    out.units.resize(n);
     out.block_begin.clear();
     out.n_front_units = 0;
     size_t first = 0;                       // units before this one stay out of the bins
     if (umma) {
-        while (first < keyed.size() && keyed[first].u.slot == -2) out.units.push_back(keyed[first++].u);
+        while (first < n && keyed[order[first]].u.slot == -2) {
+            out.units[first] = keyed[order[first]].u;
+            ++first;
+        }
         out.n_front_units = (int32_t)first;
     }
-    if (max_bins <= 0 || first == keyed.size()) {
-        for (size_t i = first; i < keyed.size(); ++i) out.units.push_back(keyed[i].u);
+    if (max_bins <= 0 || first == n) {
+        for (size_t i = first; i < n; ++i) out.units[i] = keyed[order[i]].u;
         return DA_OK;
     }
     // Longest unit first onto the lightest bin.  A unit costs its pages (a shared-prefix page
     // counts four times: it is attended for a whole block of sequences) plus a fixed charge for
     // the hand-over between units.
     constexpr int64_t kHandOverPages = 24;
-    const int bins = (int)std::min<int64_t>((int64_t)(keyed.size() - first), max_bins);
-    std::vector<std::vector<int32_t>> members(bins);
-    std::priority_queue<std::pair<int64_t, int>, std::vector<std::pair<int64_t, int>>, std::greater<>> heap;
-    for (int i = 0; i < bins; ++i) heap.push({0, i});
-    for (size_t i = first; i < keyed.size(); ++i) {
-        auto [load, bin] = heap.top();
-        heap.pop();
-        members[bin].push_back((int32_t)i);
-        heap.push({load + (keyed[i].cost & ((1LL << 40) - 1)) + kHandOverPages, bin});
+    const int bins = (int)std::min<int64_t>((int64_t)(n - first), max_bins);
+    std::vector<int32_t> bin_of(n), count(bins + 1, 0);
+    const bool equal_costs = keyed[order[first]].cost == keyed[order[n - 1]].cost;     // (sorted: first is the largest)
+    if ((size_t)bins == n - first) {
+        for (size_t i = first; i < n; ++i) bin_of[i] = (int32_t)(i - first);      // a bin for every unit
+    } else if (equal_costs) {
+        for (size_t i = first; i < n; ++i) bin_of[i] = (int32_t)((i - first) % bins);   // what the rule below would do
+    } else {
+        // binary min-heap of (load, bin) in an array; the top is replaced in place and sifted down
+        std::vector<std::pair<int64_t, int32_t>> heap(bins);
+        for (int i = 0; i < bins; ++i) heap[i] = {0, i};
+        for (size_t i = first; i < n; ++i) {
+            bin_of[i] = heap[0].second;
+            std::pair<int64_t, int32_t> top = {heap[0].first + (keyed[order[i]].cost & ((1LL << 40) - 1)) + kHandOverPages,
+                                               heap[0].second};
+            int k = 0;
+            for (;;) {
+                int c = 2 * k + 1;
+                if (c >= bins) break;
+                if (c + 1 < bins && heap[c + 1] < heap[c]) ++c;
+                if (!(heap[c] < top)) break;
+                heap[k] = heap[c];
+                k = c;
+            }
+            heap[k] = top;
+        }
     }
-    out.block_begin.reserve(bins + 1);
+    // counting sort by bin, keeping the order within a bin
+    for (size_t i = first; i < n; ++i) ++count[bin_of[i] + 1];
+    out.block_begin.resize(bins);
+    int32_t run = (int32_t)first;
     for (int b = 0; b < bins; ++b) {
-        out.block_begin.push_back((int32_t)out.units.size());
-        for (int32_t i : members[b]) out.units.push_back(keyed[i].u);
+        out.block_begin[b] = run;
+        run += count[b + 1];
+        count[b + 1] = out.block_begin[b];      // becomes the bin's write cursor
     }
+    for (size_t i = first; i < n; ++i) out.units[count[bin_of[i] + 1]++] = keyed[order[i]].u;
     out.block_begin.push_back((int32_t)out.units.size());
     return DA_OK;
 }
