@@ -277,14 +277,15 @@ def main():
         ctas_per_sm=args.ctas_per_sm,
         shared_prefix_tokens=first.shared_prefix_tokens if args.prefix_aware else 0)
     shape = da.shape_of_workload(first)
+    lens_host = first.seq_lens.cpu().numpy()            # the planner takes the lengths from host memory
     t0 = time.perf_counter()
-    plan = da.decode_attn_plan(shape, policy, first.seq_lens)
+    plan = da.decode_attn_plan(shape, policy, lens_host)
     plan_us = (time.perf_counter() - t0) * 1e6
     info = plan.info()
     t0 = time.perf_counter()
-    for _ in range(20):                      # steady state: buffers come from the library's cache
-        da.decode_attn_plan(shape, policy, first.seq_lens).destroy()
-    replan_us = (time.perf_counter() - t0) * 1e6 / 20
+    for _ in range(50):                      # steady state: buffers come from the library's cache
+        da.decode_attn_plan(shape, policy, lens_host).destroy()
+    replan_us = (time.perf_counter() - t0) * 1e6 / 50
     out = torch.empty((first.batch, first.num_q_heads, first.head_dim), dtype=torch.float32, device=dev)
     lse = torch.empty((first.batch, first.num_q_heads), dtype=torch.float32, device=dev)
     ws = torch.empty(max(plan.workspace_bytes, 256), dtype=torch.uint8, device=dev)
