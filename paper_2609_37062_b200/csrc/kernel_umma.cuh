@@ -11,8 +11,9 @@
 //   S_j = Q K_j^T  128 x 128 x 128, accumulators in tensor memory columns
 //                  [128 b, 128 b + 128), b = j mod 2: row r of S in lane r,
 //                  token t of the tile in column t
-//   softmax        two threads per row.  Each takes the exact maximum m_j of
-//                  the row over the tile, then turns its 64 logits into
+//   softmax        two threads per row.  They exchange the maxima of their
+//                  halves, so each has the exact maximum m_j of the row over
+//                  the tile, then turns its 64 logits into
 //                  p = 2^(s * scale * log2 e - m_j)
 //   P_j            must keep more than bf16 precision: the upper 16 bits of p
 //                  and the upper 16 bits of the (exact) remainder are written
@@ -35,7 +36,8 @@
 //
 // Threads: eight warps for softmax, merge and epilogue, two per 32 lanes of
 // tensor memory (one takes the even, one the odd 32-token groups of a row and
-// one half of the output columns); one warp whose first lane issues the MMAs;
+// one half of the output columns); one warp whose first lane issues the MMAs,
+// always the one - the next Q K^T or the next P V - whose inputs are ready;
 // one warp that issues the TMA boxes.  K_0, V_0, K_1, V_1, ... go through a
 // ring of four 32 KB stages; a stage is handed back by the tcgen05.commit of
 // the MMAs that read it.  Blocks are persistent (one per SM: the buffers fill
@@ -51,7 +53,10 @@
 namespace da {
 
 constexpr int kUmmaTraceBase = 2048;              // debug timelines: rows of this kernel's units
-constexpr int kUmmaSoftmaxWarps = 8;
+constexpr int kUmmaSoftmaxWarps = 8;              // a multiple of 4: warps w, w + 4, ... share 32 lanes of tensor memory
+constexpr int kUmmaThreadsPerRow = kUmmaSoftmaxWarps / 4;
+constexpr int kUmmaGroupsPerThread = 4 / kUmmaThreadsPerRow;     // 32-token groups of a tile a thread owns
+constexpr int kUmmaOutColsPerThread = 128 / kUmmaThreadsPerRow;  // output columns a thread owns
 constexpr int kUmmaSoftmaxThreads = kUmmaSoftmaxWarps * 32;
 constexpr int kUmmaMmaWarp = kUmmaSoftmaxWarps;       // lane 0 issues the MMAs
 constexpr int kUmmaLoadWarp = kUmmaSoftmaxWarps + 1;  // issues the TMA boxes
@@ -61,7 +66,7 @@ constexpr int kUmmaTileTokens = 128;
 constexpr int kUmmaHalfBytes = 128 * 128;         // 128 rows x 64 dims of bf16
 constexpr int kUmmaTileBytes = 2 * kUmmaHalfBytes;   // [half of the head dim][row][64 dims]
 constexpr int kUmmaStages = 4;
-constexpr int kUmmaMiscBytes = 4096;              // barriers, small state, the halves' row maxima and sums
+constexpr int kUmmaMiscBytes = 8192;              // barriers, small state, the threads' row maxima and sums
 constexpr int kUmmaSmemBytes = (1 + kUmmaStages) * kUmmaTileBytes + kUmmaMiscBytes + 1024 /* alignment */;
 static_assert(kUmmaSmemBytes > 114 * 1024, "two of these blocks, each wanting all of tensor memory, must not share an SM");
 constexpr int kUmmaTmemCols = 512;
@@ -97,7 +102,7 @@ __device__ __forceinline__ bool umma_wait(uint32_t bar, uint32_t parity, volatil
 }
 
 // Shared-prefix units first_unit, first_unit + unit_stride, ... < n_units, one after the other, by
-// the 320 threads of a block.  smem_raw: at least kUmmaSmemBytes of dynamic shared memory.
+// the threads of a block (kUmmaThreads).  smem_raw: at least kUmmaSmemBytes of dynamic shared memory.
 __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const CUtensorMap* k_map, const CUtensorMap* v_map,
                                                   const int G, const int first_unit, const int unit_stride,
                                                   const int n_units, uint8_t* smem_raw)
@@ -121,8 +126,9 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
     uint8_t* const sm_misc = gbase + (bar_base - base);
     volatile uint32_t* const sm_tmem = reinterpret_cast<volatile uint32_t*>(sm_misc + 160);
     volatile int* const sm_abort = reinterpret_cast<volatile int*>(sm_misc + 164);
-    volatile float* const sm_max = reinterpret_cast<volatile float*>(sm_misc + 512);   // [2 buffers][2 halves][128 rows]
-    float* const sm_l = reinterpret_cast<float*>(sm_misc + 512 + 2048);     // [2][128]: the column halves' row sums
+    constexpr int TPR = kUmmaThreadsPerRow, GP = kUmmaGroupsPerThread, OC = kUmmaOutColsPerThread;
+    volatile float* const sm_max = reinterpret_cast<volatile float*>(sm_misc + 512);   // [2 buffers][TPR][128 rows]
+    float* const sm_l = reinterpret_cast<float*>(sm_misc + 512 + 2 * TPR * 128 * 4);   // [TPR][128]: the threads' shares of the row sums
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     if (first_unit >= n_units) {
@@ -203,50 +209,81 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
                 constexpr uint32_t idesc_qk = umma::instr_desc_bf16(128, 128, false);
                 constexpr uint32_t idesc_pv = umma::instr_desc_bf16(128, 128, true);
                 bool ok = true;
-                // S_j = Q K_j^T into logit buffer j % 2 (free once tile j - 2's P V has completed)
+                // Descriptors differ only in their address field (16-byte units, the low 14 bits):
+                // stepping through a tile adds a constant to the low word.
+                const uint64_t q_desc = umma::smem_desc_sw128(q_base, 16, 1024);
+                const uint64_t k_desc0 = umma::smem_desc_sw128(ring_base, 16, 1024);
+                const uint64_t v_desc0 = umma::smem_desc_sw128(ring_base, kUmmaHalfBytes, 1024);
+                constexpr uint32_t kStageUnits = kUmmaTileBytes >> 4, kHalfUnits = kUmmaHalfBytes >> 4;
+                // S_j = Q K_j^T into logit buffer j % 2
                 auto qk = [&](int j) {
-                    const int n = 2 * j, st = n % NS, b = j & 1;
-                    ok = umma_wait(bar_full + 8 * st, (n / NS) & 1, sm_abort);
-                    if (ok && j >= 2) ok = umma_wait(bar_o + 8 * b, ((j - 2) >> 1) & 1, sm_abort);
-                    if (!ok) return;
+                    const int st = (2 * j) % NS, b = j & 1;
+                    if (j < 8) DA_TRACE_STAMP(kUmmaTraceBase + 512 + unit_index, j);
                     umma::fence_after_thread_sync();
-                    const uint32_t kt = ring_base + st * kUmmaTileBytes;
+                    const uint64_t kd = k_desc0 + (uint64_t)(st * kStageUnits);
 #pragma unroll
                     for (int ks = 0; ks < D / 16; ++ks) {
-                        const uint32_t off = (ks >> 2) * kUmmaHalfBytes + (ks & 3) * 32;
-                        umma::mma_ss(tmem + b * 128, umma::smem_desc_sw128(q_base + off, 16, 1024),
-                                     umma::smem_desc_sw128(kt + off, 16, 1024), idesc_qk, ks > 0);
+                        const uint32_t off = (ks >> 2) * kHalfUnits + (ks & 3) * 2;      // 32 bytes a step, then the other half
+                        umma::mma_ss(tmem + b * 128, q_desc + off, kd + off, idesc_qk, ks > 0);
                     }
                     umma::commit(bar_empty + 8 * st);
                     umma::commit(bar_s + 8 * b);
                 };
-                // O_j = P_j V_j into output buffer j % 2 (free once tile j - 2's output was read)
+                // O_j = P_j V_j into output buffer j % 2
                 auto pv = [&](int j) {
-                    const int n = 2 * j + 1, st = n % NS, b = j & 1;
-                    ok = umma_wait(bar_p + 8 * b, (j >> 1) & 1, sm_abort);
-                    if (ok) ok = umma_wait(bar_full + 8 * st, (n / NS) & 1, sm_abort);
-                    if (ok && j >= 2) ok = umma_wait(bar_ofree + 8 * b, ((j - 2) >> 1) & 1, sm_abort);
-                    if (!ok) return;
-                    if (j < 6) DA_TRACE_STAMP(kUmmaTraceBase + unit_index, 16 + j);
+                    const int st = (2 * j + 1) % NS, b = j & 1;
+                    if (j < 8) DA_TRACE_STAMP(kUmmaTraceBase + 512 + unit_index, 8 + j);
                     umma::fence_after_thread_sync();
-                    const uint32_t vt = ring_base + st * kUmmaTileBytes;
+                    const uint64_t vd = v_desc0 + (uint64_t)(st * kStageUnits);
                     const int ksteps = min(8, (n_tok - j * kUmmaTileTokens) >> 4);
-#pragma unroll 2
-                    for (int k = 0; k < ksteps; ++k) {
-                        // 16 tokens: two groups of 8 rows, 128 bytes a row; the upper 64 dims one half further
-                        const uint64_t bd = umma::smem_desc_sw128(vt + k * 2048, kUmmaHalfBytes, 1024);
-                        const uint32_t a_hi = tmem + b * 128 + (k >> 1) * 32 + (k & 1) * 8;
-                        umma::mma_ts(tmem + kUmmaOutCol + b * 128, a_hi, bd, idesc_pv, k > 0);
-                        umma::mma_ts(tmem + kUmmaOutCol + b * 128, a_hi + 16, bd, idesc_pv, true);
+                    const uint32_t pd = tmem + b * 128, od = tmem + kUmmaOutCol + b * 128;
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        if (k < ksteps) {
+                            // 16 tokens: two groups of 8 rows, 128 bytes a row (2 KB a step); the weights'
+                            // high parts 8 columns a step within a 32-column group, the low parts 16 further
+                            const uint32_t a_hi = pd + (k >> 1) * 32 + (k & 1) * 8;
+                            umma::mma_ts(od, a_hi, vd + k * 128, idesc_pv, k > 0);
+                            umma::mma_ts(od, a_hi + 16, vd + k * 128, idesc_pv, true);
+                        }
                     }
+                    if (j < 8) DA_TRACE_STAMP(kUmmaTraceBase + 512 + unit_index, 16 + j);
                     umma::commit(bar_empty + 8 * st);
                     umma::commit(bar_o + 8 * b);
                 };
-                qk(0);
-                if (ok && T > 1) qk(1);
-                for (int j = 0; j < T && ok; ++j) {
-                    pv(j);
-                    if (ok && j + 2 < T) qk(j + 2);
+                // Whichever of the next P V and the next Q K^T has its inputs is issued; the tensor
+                // core never waits for this thread to finish waiting for something else.
+                //   Q K^T of tile j: K_j landed; logit buffer free = P V of tile j - 2 complete
+                //   P V of tile j:   its weights written; V_j landed; output buffer read (tile j - 2 folded in)
+                int nq = 0, np = 0;
+                long long t_idle = clock64();
+                while (np < T) {
+                    bool did = false;
+                    if (np < nq) {
+                        const int j = np, n = 2 * j + 1, b = j & 1;
+                        if (mbar_test_wait(bar_p + 8 * b, (j >> 1) & 1) && mbar_test_wait(bar_full + 8 * (n % NS), (n / NS) & 1) &&
+                            (j < 2 || mbar_test_wait(bar_ofree + 8 * b, ((j - 2) >> 1) & 1))) {
+                            pv(j);
+                            ++np;
+                            did = true;
+                        }
+                    }
+                    if (!did && nq < T) {
+                        const int j = nq, n = 2 * j, b = j & 1;
+                        if (mbar_test_wait(bar_full + 8 * (n % NS), (n / NS) & 1) &&
+                            (j < 2 || (np > j - 2 && mbar_test_wait(bar_o + 8 * b, ((j - 2) >> 1) & 1)))) {
+                            qk(j);
+                            ++nq;
+                            did = true;
+                        }
+                    }
+                    if (did) {
+                        t_idle = clock64();
+                    } else if (*sm_abort != 0 || clock64() - t_idle > kWaitLimitCycles) {
+                        *sm_abort = 1;
+                        ok = false;
+                        break;
+                    }
                 }
                 // nothing may arrive on a barrier after the unit: the last two stages' hand-backs
                 if (ok) {
@@ -257,23 +294,25 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
             }
         } else {
             // -------------------------------------------------------- query rows, softmax, merge, epilogue
-            // Two threads per row: thread (quarter q, lane) of column half hh = warp / 4 owns row
-            // r = 32 q + lane, the even (hh = 0) or odd (hh = 1) 32-token groups of the logits, and
-            // output columns [64 hh, 64 hh + 64).
+            // TPR threads per row: thread (quarter q, lane) of part hh = warp / 4 owns row r = 32 q +
+            // lane, the 32-token groups hh, hh + TPR, ... of a tile's logits, and output columns
+            // [OC hh, OC hh + OC).
             const int hh = warp >> 2;
             const int r = (warp & 3) * 32 + lane;                           // row of the tile = lane of tensor memory
             const int sl = r / G, h = r % G;
             const bool valid = sl < nseq;
             const int seq = u.seq + (valid ? sl : 0);
             {
-                // 64 dims of row r of Q, 8 chunks of 16 bytes, into the swizzled K-major tile
-                const uint4* src = reinterpret_cast<const uint4*>(p.q + ((int64_t)seq * p.num_q_heads + g * G + h) * D) + hh * 8;
-                uint4 v[8];
+                // this thread's share of row r of Q, chunks of 16 bytes, into the swizzled K-major tile
+                constexpr int NC = 16 / TPR;
+                const uint4* src = reinterpret_cast<const uint4*>(p.q + ((int64_t)seq * p.num_q_heads + g * G + h) * D) + hh * NC;
+                uint4 v[NC];
 #pragma unroll
-                for (int c = 0; c < 8; ++c) v[c] = valid ? __ldg(src + c) : make_uint4(0u, 0u, 0u, 0u);
+                for (int c = 0; c < NC; ++c) v[c] = valid ? __ldg(src + c) : make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    const uint32_t off = hh * kUmmaHalfBytes + r * 128 + ((c ^ (r & 7)) << 4);
+                for (int c = 0; c < NC; ++c) {
+                    const int ci = hh * NC + c;                                 // chunk of the row: half ci / 8, chunk ci % 8
+                    const uint32_t off = (ci >> 3) * kUmmaHalfBytes + r * 128 + (((ci & 7) ^ (r & 7)) << 4);
                     *reinterpret_cast<uint4*>(gbase + off) = v[c];
                 }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); // visible to the tensor core's reads
@@ -289,12 +328,12 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
             }
 
             const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
-            float acc[64];
+            float acc[OC];
 #pragma unroll
-            for (int i = 0; i < 64; ++i) acc[i] = 0.f;
+            for (int i = 0; i < OC; ++i) acc[i] = 0.f;
             float M = -INFINITY, L = 0.f;       // running maximum (log2 domain), this thread's share of the row sum
             float m_prev = 0.f, l_prev = 0.f;   // of the tile whose output is still to be folded in
-            uint32_t sa[32], sb[32];
+            uint32_t sg[GP < 2 ? 2 : GP][32];      // logits of the thread's groups; also the output tile on its way in
             bool ok = true;
 
             // folds tile i's output into the running state
@@ -302,23 +341,24 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
                 const int b = i & 1;
                 ok = umma_wait(bar_o + 8 * b, (i >> 1) & 1, sm_abort);
                 if (!ok) return;
-                if (tid == 0 && i < 6) DA_TRACE_STAMP(kUmmaTraceBase + unit_index, 22 + i);
+                if (tid == 0 && i < 8) DA_TRACE_STAMP(kUmmaTraceBase + 1024 + unit_index, 16 + i);
                 umma::fence_after_thread_sync();
-                const uint32_t oc = lane_base + kUmmaOutCol + b * 128 + hh * 64;
-                umma::ld32(oc, sa);
-                umma::ld32(oc + 32, sb);
+                const uint32_t oc = lane_base + kUmmaOutCol + b * 128 + hh * OC;
+#pragma unroll
+                for (int q = 0; q < OC / 32; ++q) umma::ld32(oc + 32 * q, sg[q]);
                 umma::wait_ld();
                 umma::fence_before_thread_sync();
                 mbar_arrive(bar_ofree + 8 * b);                              // the buffer may be overwritten
                 const float Mn = fmaxf(M, m_prev);
                 const float a = ex2f(M - Mn), c = ex2f(m_prev - Mn);        // M = -inf at first: a = 0
 #pragma unroll
-                for (int k = 0; k < 32; ++k) {
-                    acc[k] = fmaf(acc[k], a, __uint_as_float(sa[k]) * c);
-                    acc[32 + k] = fmaf(acc[32 + k], a, __uint_as_float(sb[k]) * c);
-                }
+                for (int q = 0; q < OC / 32; ++q)
+#pragma unroll
+                    for (int k = 0; k < 32; ++k)
+                        acc[32 * q + k] = fmaf(acc[32 * q + k], a, __uint_as_float(sg[q][k]) * c);
                 L = fmaf(L, a, l_prev * c);
                 M = Mn;
+                if (tid == 0 && i < 8) DA_TRACE_STAMP(kUmmaTraceBase + 1024 + unit_index, 24 + i);
             };
 
             for (int j = 0; j < T && ok; ++j) {
@@ -328,27 +368,28 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
                 ok = umma_wait(bar_s + 8 * b, (j >> 1) & 1, sm_abort);
                 if (!ok) break;
                 if (tid == 0 && j == 0) DA_TRACE_STAMP(kUmmaTraceBase + unit_index, 2);
-                if (tid == 0 && j >= 1 && j <= 5) DA_TRACE_STAMP(kUmmaTraceBase + unit_index, 9 + j);
+                if (tid == 0 && j < 8) DA_TRACE_STAMP(kUmmaTraceBase + 1024 + unit_index, j);
                 umma::fence_after_thread_sync();
                 const uint32_t sc = lane_base + b * 128;
-                // pass 1: the maximum of this thread's 64 logits; the row's other half is exchanged
-                // through shared memory (its logits may not be read once it starts writing weights)
+                // pass 1: the maximum of this thread's logits; the row's other parts are exchanged
+                // through shared memory (their logits may not be read once they start writing weights)
                 float mx = -INFINITY;
-                umma::ld32(sc + hh * 32, sa);
-                umma::ld32(sc + hh * 32 + 64, sb);
+#pragma unroll
+                for (int q = 0; q < GP; ++q) umma::ld32(sc + (hh + q * TPR) * 32, sg[q]);
                 umma::wait_ld();
 #pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    if (hh * 32 + i < n_here) mx = fmaxf(mx, __uint_as_float(sa[i]));
-                    if (hh * 32 + 64 + i < n_here) mx = fmaxf(mx, __uint_as_float(sb[i]));
-                }
-                sm_max[(b * 2 + hh) * 128 + r] = mx;
+                for (int q = 0; q < GP; ++q)
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        if ((hh + q * TPR) * 32 + i < n_here) mx = fmaxf(mx, __uint_as_float(sg[q][i]));
+                sm_max[(b * TPR + hh) * 128 + r] = mx;
                 mbar_arrive(bar_m + 8 * b);
                 ok = umma_wait(bar_m + 8 * b, (j >> 1) & 1, sm_abort);
                 if (!ok) break;
-                mx = fmaxf(mx, sm_max[(b * 2 + (1 - hh)) * 128 + r]);
+#pragma unroll
+                for (int q = 0; q < TPR; ++q) mx = fmaxf(mx, sm_max[(b * TPR + q) * 128 + r]);
                 const float m2 = mx * p.scale_log2;                          // the scale is positive
-                // pass 2: this thread's 64 weights, written back over the logits as bf16 high and low parts
+                // pass 2: this thread's weights, written back over the logits as bf16 high and low parts
                 float lsum = 0.f;
                 auto weights = [&](const uint32_t (&s)[32], int col0) {
                     uint32_t hi[16], lo[16];
@@ -368,12 +409,12 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
                     umma::st16(sc + col0, hi);
                     umma::st16(sc + col0 + 16, lo);
                 };
-                weights(sa, hh * 32);
-                weights(sb, hh * 32 + 64);
+#pragma unroll
+                for (int q = 0; q < GP; ++q) weights(sg[q], (hh + q * TPR) * 32);
                 umma::wait_st();
                 umma::fence_before_thread_sync();
                 mbar_arrive(bar_p + 8 * b);                                   // this tile's P V may start
-                if (tid == 0 && j < 3) DA_TRACE_STAMP(kUmmaTraceBase + unit_index, 5 + j);
+                if (tid == 0 && j < 8) DA_TRACE_STAMP(kUmmaTraceBase + 1024 + unit_index, 8 + j);
                 // while it runs, fold in the tile before
                 if (j >= 1) fold(j - 1);
                 m_prev = m2;
@@ -381,7 +422,7 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
             }
             if (ok) fold(T - 1);
             if (tid == 0) DA_TRACE_STAMP(kUmmaTraceBase + unit_index, 3);
-            // the row sum is the two halves' sums
+            // the row sum is the sum of the threads' shares, added in a fixed order
             sm_l[hh * 128 + r] = L;
             block_sync(2, kUmmaSoftmaxThreads);
             if (ok) {
@@ -389,19 +430,22 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
                 // thread's half of the row is staged there and leaves with one bulk copy.
                 const int RF = rec_floats(G, D);
                 float* const rec = p.ws + ((int64_t)(si.slot_base + u.split_index) * p.num_kv_heads + g) * RF;
-                uint8_t* const row = ring_ptr + r * kUmmaOutRowBytes + hh * 256;
+                uint8_t* const row = ring_ptr + r * kUmmaOutRowBytes + hh * (OC * 4);
 #pragma unroll
-                for (int i = 0; i < 16; ++i) {
+                for (int i = 0; i < OC / 4; ++i) {
                     float4 v = make_float4(acc[4 * i], acc[4 * i + 1], acc[4 * i + 2], acc[4 * i + 3]);
                     if (dead) v = make_float4(0.f, 0.f, 0.f, 0.f);
                     *reinterpret_cast<float4*>(row + i * 16) = v;
                 }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); // visible to the bulk copy's reads
                 if (valid) {
-                    bulk_store_s2g(rec + h * D + hh * 64, smem_u32(row), 256);
-                    if (hh == 0)
-                        __stcg(reinterpret_cast<float2*>(rec + G * D) + h,
-                               dead ? make_float2(-INFINITY, 0.f) : make_float2(M, sm_l[r] + sm_l[128 + r]));
+                    bulk_store_s2g(rec + h * D + hh * OC, smem_u32(row), OC * 4);
+                    if (hh == 0) {
+                        float ls = sm_l[r];
+#pragma unroll
+                        for (int q = 1; q < TPR; ++q) ls += sm_l[q * 128 + r];
+                        __stcg(reinterpret_cast<float2*>(rec + G * D) + h, dead ? make_float2(-INFINITY, 0.f) : make_float2(M, ls));
+                    }
                 }
                 bulk_store_commit_and_wait_read();
             }
