@@ -69,7 +69,8 @@ typedef enum {
 } da_split_mode_t;
 
 typedef enum {
-    DA_KERNEL_AUTO = 0,     /* tensor-core kernel when the GQA group has >= 2 heads, else SIMT       */
+    DA_KERNEL_AUTO = 0,     /* tensor-core kernel when the GQA group has >= 2 heads, else SIMT; with
+                               shared_prefix_tokens: UMMA_PREFIX where it applies, else MMA_TMA       */
     DA_KERNEL_SIMT = 1,     /* CUDA-core kernel, 16-byte vectorised global loads                      */
     DA_KERNEL_MMA_TMA = 2,  /* TMA-staged pages in shared memory, mma.sync bf16 for QK^T and PV       */
     DA_KERNEL_UMMA_PREFIX = 3 /* shared-prefix plans only (head_dim 128, group 1, 2, 4 or 8): the prefix
@@ -99,8 +100,9 @@ typedef struct {
                                their first shared_prefix_tokens / page_size entries, as with few-shot
                                prompts served from a prefix cache).  A multiple of page_size, at most
                                every seq_len.  The prefix is then attended once per block of
-                               sequences instead of once per sequence.  Tensor-core kernel, groups of
-                               up to 4 heads, separate combine, no capacity plan.                    */
+                               sequences instead of once per sequence.  Tensor-core kernels only
+                               (MMA_TMA: groups of up to 4 heads; UMMA_PREFIX: head_dim 128, groups of
+                               1, 2, 4 or 8), separate combine, no capacity plan, not FIXED_COUNT.    */
     int32_t reserved[5];
 } decode_attn_policy_t;
 
