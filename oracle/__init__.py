@@ -3,7 +3,7 @@
 Only tests/, the smoke check and the benchmark's CPU-baseline leg may import
 this package.  It builds `paged_attention_oracle.c` with gcc on first use and
 never touches the CUDA library; inputs are numpy / CPU torch arrays of bf16
-bit patterns (uint16 / int16).
+(or, with in_fp16, fp16) bit patterns (uint16 / int16).
 """
 from __future__ import annotations
 
@@ -36,7 +36,8 @@ class _Shape(ctypes.Structure):
                 ("page_size", ctypes.c_int32), ("max_pages_per_seq", ctypes.c_int32),
                 ("k_stride_page", ctypes.c_int64), ("k_stride_token", ctypes.c_int64),
                 ("k_stride_head", ctypes.c_int64), ("v_stride_page", ctypes.c_int64),
-                ("v_stride_token", ctypes.c_int64), ("v_stride_head", ctypes.c_int64)]
+                ("v_stride_token", ctypes.c_int64), ("v_stride_head", ctypes.c_int64),
+                ("in_fp16", ctypes.c_int32), ("pad", ctypes.c_int32)]
 
 
 def _load():
@@ -73,7 +74,7 @@ class PagedInputs:
     """Host copies of one call's inputs, in the oracle's terms."""
 
     def __init__(self, q_bits, k_pool, v_pool, block_table, seq_lens, page_size: int,
-                 strides: Tuple[int, int, int], num_kv_heads: int, v_strides=None):
+                 strides: Tuple[int, int, int], num_kv_heads: int, v_strides=None, in_fp16: bool = False):
         self.q = _u16(q_bits)
         self.k = _u16(k_pool)
         self.v = _u16(v_pool)
@@ -82,13 +83,22 @@ class PagedInputs:
         B, Hq, D = self.q.shape
         vs = v_strides or strides
         self.shape = _Shape(B, Hq, num_kv_heads, D, page_size, self.block_table.shape[1],
-                            strides[0], strides[1], strides[2], vs[0], vs[1], vs[2])
+                            strides[0], strides[1], strides[2], vs[0], vs[1], vs[2], 1 if in_fp16 else 0, 0)
         self.B, self.Hq, self.Hkv, self.D, self.P = B, Hq, num_kv_heads, D, page_size
 
     @classmethod
     def from_workload(cls, w) -> "PagedInputs":
         return cls(w.q_bits, w.k_pool, w.v_pool, w.block_table, w.seq_lens, w.page_size, w.strides,
-                   w.num_kv_heads)
+                   w.num_kv_heads, in_fp16=getattr(w, "dtype", "bf16") == "fp16")
+
+
+def decode_bits(bits, in_fp16: bool) -> np.ndarray:
+    """The oracle's reading of 16-bit input patterns, as fp64."""
+    lib = _load()
+    b = np.ascontiguousarray(np.asarray(bits).view(np.uint16)).ravel()
+    out = np.empty(b.shape, dtype=np.float64)
+    lib.oracle_decode_bits(ctypes.c_int(1 if in_fp16 else 0), _p(b), ctypes.c_int64(b.size), _p(out))
+    return out
 
 
 def default_scale(head_dim: int) -> float:

@@ -18,7 +18,7 @@
  *   m      = max_t s_t,  p_t = exp(s_t - m),  l = sum_t p_t
  *   out[d] = (sum_t p_t * V[page][slot][g][d]) / l,   lse = m + log(l)
  *
- * Two passes, ascending t, fp64 throughout (bf16 -> fp64 is exact).  A row
+ * Two passes, ascending t, fp64 throughout (bf16 -> fp64 and fp16 -> fp64 are exact).  A row
  * with seq_len 0, or a row whose RUN mask byte is 0 (a Project-Only row of
  * Algorithm 1 step 2), reads no KV and emits zeros, lse = -inf.
  *
@@ -47,11 +47,33 @@ static double bf16_bits_to_f64(uint16_t bits)
     return (double)f;
 }
 
+/* IEEE binary16: 1 sign, 5 exponent (bias 15), 10 fraction bits; exact in fp64. */
+static double fp16_bits_to_f64(uint16_t bits)
+{
+    const int sign = bits >> 15, e = (bits >> 10) & 31, m = bits & 1023;
+    double v;
+    if (e == 0)
+        v = ldexp((double)m, -24);                      /* subnormal: m / 1024 * 2^-14 */
+    else if (e == 31)
+        v = m ? NAN : INFINITY;
+    else
+        v = ldexp(1.0 + (double)m / 1024.0, e - 15);
+    return sign ? -v : v;
+}
+
 typedef struct {
     int32_t batch, num_q_heads, num_kv_heads, head_dim, page_size, max_pages_per_seq;
     int64_t k_stride_page, k_stride_token, k_stride_head;   /* elements */
     int64_t v_stride_page, v_stride_token, v_stride_head;
+    int32_t in_fp16;   /* q, K and V are fp16 bit patterns (the paper serves Llama in fp16 and Qwen in
+                          bf16, Section 4.1); 0: bf16 */
+    int32_t pad;
 } oracle_shape_t;
+
+static double in_bits_to_f64(const oracle_shape_t *s, uint16_t bits)
+{
+    return s->in_fp16 ? fp16_bits_to_f64(bits) : bf16_bits_to_f64(bits);
+}
 
 int oracle_max_threads(void)
 {
@@ -60,6 +82,14 @@ int oracle_max_threads(void)
 #else
     return 1;
 #endif
+}
+
+/* The input decoding by itself: n 16-bit patterns to fp64 (pinned against a
+ * library's view of the same bits in tests/test_oracle_pins.py). */
+int oracle_decode_bits(int in_fp16, const uint16_t *bits, int64_t n, double *out)
+{
+    for (int64_t i = 0; i < n; ++i) out[i] = in_fp16 ? fp16_bits_to_f64(bits[i]) : bf16_bits_to_f64(bits[i]);
+    return 0;
 }
 
 /* Address of row (token t, kv head g) of sequence b in a pool, in elements. */
@@ -96,7 +126,7 @@ static void attend_range(const oracle_shape_t *s, const uint16_t *q, const uint1
         const uint16_t *krow = k_pool + row_offset(s, block_table, b, t, g, s->k_stride_page,
                                                    s->k_stride_token, s->k_stride_head);
         double dot = 0.0;
-        for (int d = 0; d < D; ++d) dot += bf16_bits_to_f64(qrow[d]) * bf16_bits_to_f64(krow[d]);
+        for (int d = 0; d < D; ++d) dot += in_bits_to_f64(s, qrow[d]) * in_bits_to_f64(s, krow[d]);
         logit[t - t_begin] = scale * dot;
         if (logit[t - t_begin] > m) m = logit[t - t_begin];
     }
@@ -106,7 +136,7 @@ static void attend_range(const oracle_shape_t *s, const uint16_t *q, const uint1
                                                    s->v_stride_token, s->v_stride_head);
         double p = exp(logit[t - t_begin] - m);
         l += p;
-        for (int d = 0; d < D; ++d) o[d] += p * bf16_bits_to_f64(vrow[d]);
+        for (int d = 0; d < D; ++d) o[d] += p * in_bits_to_f64(s, vrow[d]);
         if (probs_or_null) probs_or_null[t - t_begin] = p;
     }
     for (int d = 0; d < D; ++d) o[d] /= l;

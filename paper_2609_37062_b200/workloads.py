@@ -144,6 +144,7 @@ class PagedWorkload:
     seq_uids: List[int] = field(default_factory=list)
     shared_prefix_tokens: int = 0
     unique_tokens: int = 0
+    dtype: str = "bf16"          # what the 16-bit patterns of q, k_pool and v_pool are: "bf16" or "fp16"
 
     @property
     def strides(self):
@@ -217,8 +218,12 @@ def make_workload(name: str, seq_lens: Sequence[int], num_q_heads: int, num_kv_h
                   layout: str = "token_major", device="cpu", seq_uids: Optional[Sequence[int]] = None,
                   shared_prefix_tokens: int = 0, shuffle_pages: bool = True,
                   unused_fill_bits: int = 0x7FC0, max_pages_per_seq: Optional[int] = None,
-                  alias_after: Optional[int] = None, table_seed: Optional[int] = None) -> PagedWorkload:
+                  alias_after: Optional[int] = None, table_seed: Optional[int] = None,
+                  dtype: str = "bf16") -> PagedWorkload:
     """Build pools, block table and q for the given lengths.
+
+    * `dtype` "fp16": the same values (and the same poison in unused slots) stored as fp16 bit
+      patterns instead of bf16 (each bf16 sample converted, round to nearest);
 
     * physical pages: a seeded random permutation of the pool's page ids dealt
       to the sequences in order (prefix pages first when a prefix is shared);
@@ -293,12 +298,16 @@ def make_workload(name: str, seq_lens: Sequence[int], num_q_heads: int, num_kv_h
         src_uid = uids[i if i < n_own else i % n_own]
         q[i] = normal_bf16_bits(stream_key(seed, TENSOR_Q, src_uid), 0, num_q_heads * D, device).view(num_q_heads, D)
 
+    assert dtype in ("bf16", "fp16")
+    if dtype == "fp16":
+        as_fp16 = lambda t: t.view(torch.bfloat16).to(torch.float16).view(torch.int16)
+        q, k_pool, v_pool = as_fp16(q), as_fp16(k_pool), as_fp16(v_pool)
     return PagedWorkload(
         name=name, batch=B, num_q_heads=num_q_heads, num_kv_heads=H, head_dim=D, page_size=P,
         num_pages=num_pages, max_pages_per_seq=mpp,
         seq_lens=torch.tensor(list(seq_lens), dtype=torch.int32).to(device),
         block_table=block_table.to(device), q_bits=q, k_pool=k_pool, v_pool=v_pool, layout=layout,
-        seq_uids=uids, shared_prefix_tokens=shared_prefix_tokens, unique_tokens=unique_tokens)
+        seq_uids=uids, shared_prefix_tokens=shared_prefix_tokens, unique_tokens=unique_tokens, dtype=dtype)
 
 
 # ----------------------------------------------------------------------------

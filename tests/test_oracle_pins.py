@@ -357,3 +357,36 @@ def test_append_writes_the_last_position_and_nothing_else():
             gk, gv = oracle.gather_kv(inp2, b)
             assert np.array_equal(gk[L - 1].view(np.int16), new_k[b].numpy())
             assert np.array_equal(gv[L - 1].view(np.int16), new_v[b].numpy())
+
+
+def test_input_decoding_matches_the_library_for_every_bit_pattern():
+    """bf16 and fp16 patterns -> fp64, all 65,536 of each, against numpy / torch's reading of the
+    same bits (subnormals, signed zeros, infinities included; NaNs as NaNs)."""
+    import torch
+    bits = np.arange(65536, dtype=np.uint16)
+    want16 = bits.view(np.float16).astype(np.float64)
+    got16 = oracle.decode_bits(bits, in_fp16=True)
+    nan = np.isnan(want16)
+    assert np.array_equal(np.isnan(got16), nan) and np.array_equal(got16[~nan], want16[~nan])
+    assert np.array_equal(np.signbit(got16[~nan]), np.signbit(want16[~nan]))
+    wantb = torch.from_numpy(bits.view(np.int16).copy()).view(torch.bfloat16).to(torch.float64).numpy()
+    gotb = oracle.decode_bits(bits, in_fp16=False)
+    nan = np.isnan(wantb)
+    assert np.array_equal(np.isnan(gotb), nan) and np.array_equal(gotb[~nan], wantb[~nan])
+
+
+def test_fp16_inputs_go_through_the_same_definition():
+    """The attention of fp16 inputs equals dense attention over the decoded values (brute force)."""
+    w = wl.make_workload("h", [37, 5], 4, 2, 64, seed=21, dtype="fp16")
+    inp = oracle.PagedInputs.from_workload(w)
+    out, lse = oracle.paged_decode_attention(inp)
+    q = w.q_bits.numpy().view(np.float16).astype(np.float64)
+    for b, L in enumerate(w.seq_lens.tolist()):
+        k, v = oracle.gather_kv(inp, b)
+        k = k.view(np.float16).astype(np.float64)
+        v = v.view(np.float16).astype(np.float64)
+        for h in range(4):
+            s = (k[:, h // 2, :] @ q[b, h]) * oracle.default_scale(64)
+            p = np.exp(s - s.max())
+            assert np.max(np.abs(out[b, h] - (p[:, None] * v[:, h // 2, :]).sum(0) / p.sum())) < 1e-12
+            assert abs(lse[b, h] - (s.max() + np.log(p.sum()))) < 1e-12
