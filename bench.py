@@ -70,6 +70,7 @@ def parse_args():
     ap.add_argument("--copies", type=int, default=0, help="pool copies to rotate over (0: enough for 1 GiB)")
     ap.add_argument("--alias-after", type=int, default=0,
                     help="sweep cells too large for memory: sequences i >= K reuse the pages of sequence i mod K")
+    ap.add_argument("--in-dtype", default="bf16", choices=["bf16", "fp16"], help="type of q, K and V")
     ap.add_argument("--prefix-aware", action="store_true",
                     help="shared_prefix workload: tell the planner about the common prefix (attended once per block of sequences)")
     ap.add_argument("--mask-fraction", type=float, default=None,
@@ -77,7 +78,16 @@ def parse_args():
     return ap.parse_args()
 
 
+IN_DTYPE = "bf16"     # set from --in-dtype
+
+
 def make_workload(name, device, table_seed=None, seed_shift=0, alias_after=None):
+    from paper_2609_37062_b200 import workloads as wl
+    w = _make_workload_bf16(name, device, table_seed, seed_shift, alias_after)
+    return wl.as_fp16(w) if IN_DTYPE == "fp16" else w
+
+
+def _make_workload_bf16(name, device, table_seed=None, seed_shift=0, alias_after=None):
     from paper_2609_37062_b200 import workloads as wl
     if name == "tiny":
         return wl.config_tiny(device=device)
@@ -235,6 +245,8 @@ def run_reference(args):
 
 def main():
     args = parse_args()
+    global IN_DTYPE
+    IN_DTYPE = args.in_dtype
     if args.impl == "reference":
         run_reference(args)
         return
@@ -449,7 +461,7 @@ def main():
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": sec_per_step * 1e3, "us_per_step": sec_per_step * 1e6,
-            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16 in, f32 accumulate",
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": f"{IN_DTYPE} in, f32 accumulate",
             "data": "synthetic",
             "config": {"workload": args.workload, "batch": first.batch, "num_q_heads": first.num_q_heads,
                        "num_kv_heads": first.num_kv_heads, "head_dim": first.head_dim, "page_size": first.page_size,

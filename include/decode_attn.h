@@ -60,7 +60,7 @@ typedef enum {
     DA_ERR_TIMEOUT = -7              /* a bounded device-side wait gave up                             */
 } da_status_t;
 
-enum { DA_DTYPE_BF16 = 1, DA_DTYPE_FP32 = 2 };
+enum { DA_DTYPE_BF16 = 1, DA_DTYPE_FP32 = 2, DA_DTYPE_FP16 = 3 };
 
 typedef enum {
     DA_SPLIT_AUTO = 0,          /* chunk length chosen from the length mix and the SM count          */
@@ -116,8 +116,9 @@ typedef struct {
     int64_t num_pages;          /* pages in each pool                                                */
     int64_t k_stride_page, k_stride_token, k_stride_head;   /* elements; multiples of 8              */
     int64_t v_stride_page, v_stride_token, v_stride_head;
-    int32_t kv_dtype;           /* DA_DTYPE_BF16                                                     */
-    int32_t q_dtype;            /* DA_DTYPE_BF16                                                     */
+    int32_t kv_dtype;           /* DA_DTYPE_BF16 or DA_DTYPE_FP16 (the paper serves one model family in
+                                   each, Section 4.1); fp16 not with shared_prefix_tokens             */
+    int32_t q_dtype;            /* the same as kv_dtype                                              */
     int32_t out_dtype;          /* DA_DTYPE_FP32 or DA_DTYPE_BF16                                    */
     float sm_scale;             /* 0: 1/sqrtf(head_dim) evaluated in fp32                            */
 } decode_attn_shape_t;

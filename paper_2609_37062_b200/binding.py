@@ -35,6 +35,7 @@ DA_ERR_TIMEOUT = -7
 
 DA_DTYPE_BF16 = 1
 DA_DTYPE_FP32 = 2
+DA_DTYPE_FP16 = 3
 
 DA_SPLIT_AUTO = 0
 DA_SPLIT_FIXED_COUNT = 1
@@ -195,13 +196,13 @@ def make_policy(split_mode: int = DA_SPLIT_AUTO, fixed_count: int = 0, chunk_tok
 def make_shape(batch: int, num_q_heads: int, num_kv_heads: int, head_dim: int, page_size: int,
                max_pages_per_seq: int, num_pages: int, k_strides: Sequence[int],
                v_strides: Optional[Sequence[int]] = None, out_dtype: int = DA_DTYPE_FP32,
-               sm_scale: float = 0.0) -> Shape:
+               sm_scale: float = 0.0, in_dtype: int = DA_DTYPE_BF16) -> Shape:
     s = Shape()
     s.batch, s.num_q_heads, s.num_kv_heads, s.head_dim = batch, num_q_heads, num_kv_heads, head_dim
     s.page_size, s.max_pages_per_seq, s.num_pages = page_size, max_pages_per_seq, num_pages
     s.k_stride_page, s.k_stride_token, s.k_stride_head = k_strides
     s.v_stride_page, s.v_stride_token, s.v_stride_head = v_strides or k_strides
-    s.kv_dtype = s.q_dtype = DA_DTYPE_BF16
+    s.kv_dtype = s.q_dtype = in_dtype
     s.out_dtype = out_dtype
     s.sm_scale = sm_scale
     return s
@@ -209,7 +210,8 @@ def make_shape(batch: int, num_q_heads: int, num_kv_heads: int, head_dim: int, p
 
 def shape_of_workload(w, out_dtype: int = DA_DTYPE_FP32, sm_scale: float = 0.0) -> Shape:
     return make_shape(w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim, w.page_size, w.max_pages_per_seq,
-                      w.num_pages, w.strides, out_dtype=out_dtype, sm_scale=sm_scale)
+                      w.num_pages, w.strides, out_dtype=out_dtype, sm_scale=sm_scale,
+                      in_dtype=DA_DTYPE_FP16 if getattr(w, "dtype", "bf16") == "fp16" else DA_DTYPE_BF16)
 
 
 def decode_attn_plan_layout(shape: Shape, policy: Policy, seq_lens, sm_count: int, ctas_per_sm: int):

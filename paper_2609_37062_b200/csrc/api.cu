@@ -329,6 +329,7 @@ KernelParams make_params(const decode_attn_plan_t* pl, const decode_attn_run_arg
     kp.max_pages_per_seq = s.max_pages_per_seq;
     kp.scale_log2 = pl->scale * kLog2e;
     kp.out_bf16 = s.out_dtype == DA_DTYPE_BF16;
+    kp.in_f16 = s.kv_dtype == DA_DTYPE_FP16;
     kp.fused = pl->policy.fuse_combine;
     kp.grid_exit = pl->policy.capacity_batch > 0;
     kp.n_units = (int32_t)pl->layout.units.size();
@@ -973,6 +974,7 @@ int decode_attn_step_static(const decode_attn_shape_t* shape, const int32_t* seq
     const float scale = shape->sm_scale > 0.f ? shape->sm_scale : 1.0f / sqrtf((float)shape->head_dim);
     kp.scale_log2 = scale * kLog2e;
     kp.out_bf16 = shape->out_dtype == DA_DTYPE_BF16;
+    kp.in_f16 = shape->kv_dtype == DA_DTYPE_FP16;
     kp.fused = 0;
     kp.grid_exit = 0;
     kp.n_units = (int32_t)lay.units.size();

@@ -48,6 +48,7 @@ struct KernelParams {
     int32_t num_q_heads, num_kv_heads, max_pages_per_seq, batch;
     float scale_log2;  // sm_scale * log2(e): logits are kept in the base-2 domain
     int32_t out_bf16;
+    int32_t in_f16;          // q, K and V are fp16 (else bf16)
     int32_t fused;
     int32_t grid_exit;  // capacity plans: the unit count is read from header->n_units, surplus blocks leave at once
     int32_t n_units;    // otherwise: the unit count

@@ -36,6 +36,7 @@
 #pragma once
 
 #include <cuda.h>
+#include <cuda_fp16.h>
 
 #include "common.cuh"
 
@@ -109,20 +110,46 @@ __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a)
     return d;
 }
 
-__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
-{
+// The 16-bit input type of q, K and V: bf16, or fp16 (template parameter F16 of the kernel).  P
+// takes the same type, because both operands of an mma must have it.
+template <bool F16>
+struct In16;
+
+template <>
+struct In16<false> {
     // a pure function of its register operands: left non-volatile so the compiler may interleave
     // independent mma chains with the surrounding arithmetic
-    asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
+    static __device__ __forceinline__ void mma(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
+    {
+        asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+            : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+            : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+    }
+    static __device__ __forceinline__ uint32_t pack(float lo, float hi)
+    {
+        __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+        return *reinterpret_cast<uint32_t*>(&v);
+    }
+    static __device__ __forceinline__ float low(uint32_t v) { return __uint_as_float(v << 16); }
+    static __device__ __forceinline__ float high(uint32_t v) { return __uint_as_float(v & 0xffff0000u); }
+};
 
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
-{
-    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<uint32_t*>(&v);
-}
+template <>
+struct In16<true> {
+    static __device__ __forceinline__ void mma(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
+    {
+        asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+            : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+            : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+    }
+    static __device__ __forceinline__ uint32_t pack(float lo, float hi)
+    {
+        __half2 v = __floats2half2_rn(lo, hi);
+        return *reinterpret_cast<uint32_t*>(&v);
+    }
+    static __device__ __forceinline__ float low(uint32_t v) { return __low2float(*reinterpret_cast<const __half2*>(&v)); }
+    static __device__ __forceinline__ float high(uint32_t v) { return __high2float(*reinterpret_cast<const __half2*>(&v)); }
+};
 
 // Byte offset, inside one 16 x 128 B box written by TMA with the 128-byte
 // swizzle, of 16-byte chunk `chunk` (0..7) of row `row` (0..15).
@@ -138,13 +165,14 @@ struct MmaExtra {
     int32_t gather_seq;
 };
 
-template <int D, bool DUP, int MODE, bool PREFIX>
+template <int D, bool DUP, int MODE, bool PREFIX, bool F16 = false>
 __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const KernelParams p,
                                                                       const __grid_constant__ CUtensorMap k_map,
                                                                       const __grid_constant__ CUtensorMap v_map,
                                                                       const int G, const MmaExtra ex)
 {
     using Cfg = MmaCfg<D, DUP>;
+    using In = In16<F16>;
     constexpr int NS = Cfg::kStages;
     constexpr int KSTEPS = D / 16;
     constexpr int COLS = Cfg::kColsOut;
@@ -401,7 +429,7 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
                         uint32_t a[4];
                         ldsm_x4(kpage + (ks >> 2) * Cfg::kBoxBytes + swz(arow, (ks & 3) * 2 + achk), a);
 #pragma unroll
-                        for (int nt = 0; nt < NT; ++nt) mma_bf16_16816(sacc[nt], a, pq[ks][nt][0], pq[ks][nt][1]);
+                        for (int nt = 0; nt < NT; ++nt) In::mma(sacc[nt], a, pq[ks][nt][0], pq[ks][nt][1]);
                     }
                     uint32_t bh[NT][2], bl[NT][2];
 #pragma unroll
@@ -429,9 +457,9 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
                                 pacc[mt][nt][2] *= al0; pacc[mt][nt][3] *= al1;
                             }
                         }
-                        const uint32_t hi0 = pack_bf16(p00, p01), hi1 = pack_bf16(p10, p11);
-                        const uint32_t lo0 = pack_bf16(p00 - __uint_as_float(hi0 << 16), p01 - __uint_as_float(hi0 & 0xffff0000u));
-                        const uint32_t lo1 = pack_bf16(p10 - __uint_as_float(hi1 << 16), p11 - __uint_as_float(hi1 & 0xffff0000u));
+                        const uint32_t hi0 = In::pack(p00, p01), hi1 = In::pack(p10, p11);
+                        const uint32_t lo0 = In::pack(p00 - In::low(hi0), p01 - In::high(hi0));
+                        const uint32_t lo1 = In::pack(p10 - In::low(hi1), p11 - In::high(hi1));
                         bh[nt][0] = movmatrix_trans(hi0);
                         bh[nt][1] = movmatrix_trans(hi1);
                         bl[nt][0] = movmatrix_trans(lo0);
@@ -445,8 +473,8 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
                         ldsm_x4_trans(vpage + (mt >> 2) * Cfg::kBoxBytes + swz(vrow, (mt & 3) * 2 + vchk), a);
 #pragma unroll
                         for (int nt = 0; nt < NT; ++nt) {
-                            mma_bf16_16816(pacc[mt][nt], a, bh[nt][0], bh[nt][1]);
-                            mma_bf16_16816(pacc[mt][nt], a, bl[nt][0], bl[nt][1]);
+                            In::mma(pacc[mt][nt], a, bh[nt][0], bh[nt][1]);
+                            In::mma(pacc[mt][nt], a, bl[nt][0], bl[nt][1]);
                         }
                     }
                 }
@@ -599,7 +627,7 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
                     for (int ks = 0; ks < KSTEPS; ++ks) {
                         uint32_t a[4];
                         ldsm_x4(kpage + (ks >> 2) * Cfg::kBoxBytes + swz(arow, (ks & 3) * 2 + achk), a);
-                        mma_bf16_16816(sacc, a, qb[ks][0], qb[ks][1]);
+                        In::mma(sacc, a, qb[ks][0], qb[ks][1]);
                     }
                     // ---- online softmax on the fragment: rows r, r+8 (tokens), columns 2c, 2c+1 (heads)
                     const bool v_lo = r < n_valid, v_hi = (r + 8) < n_valid;
@@ -629,10 +657,10 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
                         }
                     }
                     // ---- P^T as B fragments (high parts; low parts in the duplicated columns or a second set)
-                    uint32_t hi0 = pack_bf16(p00, p01), hi1 = pack_bf16(p10, p11);
-                    const float r00 = p00 - __uint_as_float(hi0 << 16), r01 = p01 - __uint_as_float(hi0 & 0xffff0000u);
-                    const float r10 = p10 - __uint_as_float(hi1 << 16), r11 = p11 - __uint_as_float(hi1 & 0xffff0000u);
-                    const uint32_t lo0 = pack_bf16(r00, r01), lo1 = pack_bf16(r10, r11);
+                    uint32_t hi0 = In::pack(p00, p01), hi1 = In::pack(p10, p11);
+                    const float r00 = p00 - In::low(hi0), r01 = p01 - In::high(hi0);
+                    const float r10 = p10 - In::low(hi1), r11 = p11 - In::high(hi1);
+                    const uint32_t lo0 = In::pack(r00, r01), lo1 = In::pack(r10, r11);
                     uint32_t b0, b1, b0l = 0, b1l = 0;
                     if (DUP) {
                         b0 = movmatrix_trans(lo_role ? lo0 : hi0);
@@ -650,8 +678,8 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
                     for (int mt = 0; mt < D / 16; ++mt) {
                         uint32_t a[4];
                         ldsm_x4_trans(vpage + (mt >> 2) * Cfg::kBoxBytes + swz(vrow, (mt & 3) * 2 + vchk), a);
-                        mma_bf16_16816(oacc[mt], a, b0, b1);
-                        if (!DUP) mma_bf16_16816(oacc[mt], a, b0l, b1l);
+                        In::mma(oacc[mt], a, b0, b1);
+                        if (!DUP) In::mma(oacc[mt], a, b0l, b1l);
                     }
                 }
             }
@@ -748,6 +776,8 @@ inline encode_tiled_fn get_encode_tiled()
 inline int make_pool_map(CUtensorMap* map, const void* pool, const decode_attn_shape_t& s, int64_t stride_page,
                          int64_t stride_token, int64_t stride_head)
 {
+    const CUtensorMapDataType dt =
+        s.kv_dtype == DA_DTYPE_FP16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
     encode_tiled_fn enc = get_encode_tiled();
     if (!enc) return DA_ERR_CUDA;
     const cuuint64_t dims[4] = {(cuuint64_t)s.head_dim, (cuuint64_t)s.page_size, (cuuint64_t)s.num_kv_heads,
@@ -756,7 +786,7 @@ inline int make_pool_map(CUtensorMap* map, const void* pool, const decode_attn_s
                                    (cuuint64_t)stride_page * 2};
     const cuuint32_t box[4] = {64, 16, 1, 1};
     const cuuint32_t estr[4] = {1, 1, 1, 1};
-    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(pool), dims, strides, box, estr,
+    CUresult r = enc(map, dt, 4, const_cast<void*>(pool), dims, strides, box, estr,
                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? DA_OK : DA_ERR_CUDA;
@@ -764,10 +794,19 @@ inline int make_pool_map(CUtensorMap* map, const void* pool, const decode_attn_s
 
 typedef void (*mma_kernel_t)(const KernelParams, const CUtensorMap, const CUtensorMap, const int, const MmaExtra);
 
+// f16: q, K and V are fp16 (attention mode, no shared-prefix units); else bf16.
 template <int MODE>
-inline mma_kernel_t mma_kernel_for(int D, int G, bool prefix = false)
+inline mma_kernel_t mma_kernel_for(int D, int G, bool prefix = false, bool f16 = false)
 {
     const bool dup = G <= 4;
+    if (f16) {
+        if (MODE != kModeAttend || prefix) return nullptr;
+        if (D == 128) return dup ? decode_attn_mma_kernel<128, true, kModeAttend, false, true>
+                                 : decode_attn_mma_kernel<128, false, kModeAttend, false, true>;
+        if (D == 64) return dup ? decode_attn_mma_kernel<64, true, kModeAttend, false, true>
+                                : decode_attn_mma_kernel<64, false, kModeAttend, false, true>;
+        return nullptr;
+    }
     if (prefix) {   // shared-prefix plans: attention mode, groups of up to 4 heads
         if (MODE != kModeAttend || !dup) return nullptr;
         if (D == 128) return decode_attn_mma_kernel<128, true, kModeAttend, true>;
@@ -787,9 +826,9 @@ inline int mma_smem_bytes(int D, int G)
 }
 
 template <int MODE>
-inline int mma_prepare(int D, int G, mma_kernel_t* fn_out, bool prefix = false)
+inline int mma_prepare(int D, int G, mma_kernel_t* fn_out, bool prefix = false, bool f16 = false)
 {
-    mma_kernel_t fn = mma_kernel_for<MODE>(D, G, prefix);
+    mma_kernel_t fn = mma_kernel_for<MODE>(D, G, prefix, f16);
     if (!fn) return DA_ERR_UNSUPPORTED;
     if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, mma_smem_bytes(D, G)) != cudaSuccess) {
         (void)cudaGetLastError();
@@ -799,10 +838,10 @@ inline int mma_prepare(int D, int G, mma_kernel_t* fn_out, bool prefix = false)
     return DA_OK;
 }
 
-inline int mma_query_occupancy(int D, int G, int* block_threads, int* dyn_smem, bool prefix = false)
+inline int mma_query_occupancy(int D, int G, int* block_threads, int* dyn_smem, bool prefix = false, bool f16 = false)
 {
     mma_kernel_t fn;
-    if (mma_prepare<kModeAttend>(D, G, &fn, prefix) != DA_OK) return -1;
+    if (mma_prepare<kModeAttend>(D, G, &fn, prefix, f16) != DA_OK) return -1;
     *block_threads = kMmaThreads;
     *dyn_smem = mma_smem_bytes(D, G);
     int n = 0;
@@ -818,7 +857,8 @@ inline int mma_launch_mode(const decode_attn_shape_t& s, int G, const KernelPara
                            unsigned grid, cudaStream_t stream, bool prefix = false)
 {
     mma_kernel_t fn;
-    int rc = mma_prepare<MODE>(s.head_dim, G, &fn, prefix);
+    // (the probe and gather modes only move 16-bit words: one variant serves both input types)
+    int rc = mma_prepare<MODE>(s.head_dim, G, &fn, prefix, MODE == kModeAttend && s.kv_dtype == DA_DTYPE_FP16);
     if (rc != DA_OK) return rc;
     CUtensorMap kmap, vmap;
     rc = make_pool_map(&kmap, kp.k, s, s.k_stride_page, s.k_stride_token, s.k_stride_head);

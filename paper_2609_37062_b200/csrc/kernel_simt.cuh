@@ -14,6 +14,8 @@
 // do) and is the CUDA-core reference point for the tensor-core kernel.
 #pragma once
 
+#include <cuda_fp16.h>
+
 #include "common.cuh"
 
 namespace da {
@@ -30,8 +32,19 @@ __device__ __forceinline__ uint4 ldg_stream16(const void* ptr)
     return v;
 }
 
-__device__ __forceinline__ void unpack8(const uint4& w, float (&f)[8])
+// Eight 16-bit inputs to fp32: bf16 by shifts, fp16 by conversion (one flag for the whole launch).
+__device__ __forceinline__ void unpack8(const uint4& w, float (&f)[8], int in_f16)
 {
+    if (in_f16) {
+        const __half2* h = reinterpret_cast<const __half2*>(&w);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float2 v = __half22float2(h[i]);
+            f[2 * i] = v.x;
+            f[2 * i + 1] = v.y;
+        }
+        return;
+    }
     f[0] = __uint_as_float(w.x << 16); f[1] = __uint_as_float(w.x & 0xffff0000u);
     f[2] = __uint_as_float(w.y << 16); f[3] = __uint_as_float(w.y & 0xffff0000u);
     f[4] = __uint_as_float(w.z << 16); f[5] = __uint_as_float(w.z & 0xffff0000u);
@@ -86,7 +99,7 @@ __global__ void __launch_bounds__(kSimtThreads) decode_attn_simt_kernel(const Ke
 #pragma unroll
     for (int h = 0; h < G; ++h) {
         const uint4 w = *reinterpret_cast<const uint4*>(p.q + ((int64_t)b * p.num_q_heads + g * G + h) * D + li * 8);
-        unpack8(w, qf[h]);
+        unpack8(w, qf[h], p.in_f16);
 #pragma unroll
         for (int i = 0; i < 8; ++i) qf[h][i] *= p.scale_log2;
     }
@@ -128,7 +141,7 @@ __global__ void __launch_bounds__(kSimtThreads) decode_attn_simt_kernel(const Ke
 #pragma unroll
         for (int j = 0; j < U; ++j) {
             float kf[8];
-            unpack8(kk[j], kf);
+            unpack8(kk[j], kf, p.in_f16);
 #pragma unroll
             for (int h = 0; h < G; ++h) {
                 float d = 0.f;
@@ -169,7 +182,7 @@ __global__ void __launch_bounds__(kSimtThreads) decode_attn_simt_kernel(const Ke
 #pragma unroll
         for (int j = 0; j < U; ++j) {
             float vf[8];
-            unpack8(vv[j], vf);
+            unpack8(vv[j], vf, p.in_f16);
 #pragma unroll
             for (int h = 0; h < G; ++h)
 #pragma unroll

@@ -20,6 +20,7 @@ cached prefix, long runaway generations); no dataset item is used.
 from __future__ import annotations
 
 import math
+import dataclasses
 from dataclasses import dataclass, field
 from typing import List, Optional, Sequence
 
@@ -347,6 +348,15 @@ def config_sweep_cell(context: int, batch: int, device="cpu", layout="token_majo
     tokens; sequence i has the same content in every batch size."""
     return make_workload(f"sweep_{context}x{batch}", [context] * batch, 32, 8, 128, seed=seed,
                          layout=layout, device=device, alias_after=alias_after, table_seed=table_seed)
+
+
+def as_fp16(w: PagedWorkload) -> PagedWorkload:
+    """The same workload with q, K and V stored as fp16 bit patterns (what `dtype="fp16"` of
+    make_workload gives)."""
+    if w.dtype == "fp16":
+        return w
+    cv = lambda t: t.view(torch.bfloat16).to(torch.float16).view(torch.int16)
+    return dataclasses.replace(w, q_bits=cv(w.q_bits), k_pool=cv(w.k_pool), v_pool=cv(w.v_pool), dtype="fp16")
 
 
 def permute_pages(w: PagedWorkload, seed: int) -> PagedWorkload:
