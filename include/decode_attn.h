@@ -72,7 +72,7 @@ typedef enum {
     DA_KERNEL_AUTO = 0,     /* tensor-core kernel when the GQA group has >= 2 heads, else SIMT; with
                                shared_prefix_tokens: UMMA_PREFIX where it applies, else MMA_TMA       */
     DA_KERNEL_SIMT = 1,     /* CUDA-core kernel, 16-byte vectorised global loads                      */
-    DA_KERNEL_MMA_TMA = 2,  /* TMA-staged pages in shared memory, mma.sync bf16 for QK^T and PV       */
+    DA_KERNEL_MMA_TMA = 2,  /* TMA-staged pages in shared memory, mma.sync (bf16 or fp16) for QK^T, PV  */
     DA_KERNEL_UMMA_PREFIX = 3 /* shared-prefix plans only (head_dim 128, group 1, 2, 4 or 8): the prefix
                                units run on the tcgen05 tensor cores, 128 query rows at a time with
                                accumulators in tensor memory; what follows the prefix runs as MMA_TMA */
@@ -210,8 +210,8 @@ int decode_attn_plan_destroy(decode_attn_plan_t *plan);
 /* ---------------------------------------------------------------------------
  * Split-KV partial kernel (Algorithm 1 step 2, the attention read).
  *
- *   q            device, bf16 [batch, num_q_heads, head_dim], contiguous, 16-byte aligned
- *   k_cache      device, bf16 pool addressed by the k_stride_* of the shape, 16-byte aligned
+ *   q            device, shape.q_dtype (bf16 or fp16) [batch, num_q_heads, head_dim], contiguous, 16-byte aligned
+ *   k_cache      device, shape.kv_dtype pool addressed by the k_stride_* of the shape, 16-byte aligned
  *   v_cache      device, same with v_stride_*
  *   block_table  device, int32 [batch, max_pages_per_seq]; entries at or beyond
  *                ceil(seq_len / page_size) are never read; pages may be shared by rows
@@ -262,7 +262,7 @@ int decode_attn_run_ex(const decode_attn_plan_t *plan, const decode_attn_run_arg
  * the row then attends).  Stores row b's new K and V rows at logical position
  * seq_lens[b] - 1: page block_table[b][(L-1) / page_size], slot
  * (L-1) % page_size.  Bit-exact copy; rows with seq_len 0 write nothing.
- *   new_k, new_v  device, bf16 [batch, num_kv_heads, head_dim], 16-byte aligned
+ *   new_k, new_v  device, 16-bit (shape.kv_dtype) [batch, num_kv_heads, head_dim], 16-byte aligned
  *   block_table, seq_lens  device (seq_lens are the lengths INCLUDING the new token)
  *   k_cache, v_cache  device pools of the shape, modified in place
  * One launch on `stream`; a decode_attn_run enqueued after it on the same
@@ -323,7 +323,7 @@ int decode_attn_validate_shared_prefix(const decode_attn_shape_t *shape, int32_t
  * ------------------------------------------------------------------------- */
 
 /* Writes sequence `seq`'s K and V rows in logical token order,
- * k_out / v_out: device bf16 [seq_len, num_kv_heads, head_dim], fetched
+ * k_out / v_out: device, 16-bit like the pools, [seq_len, num_kv_heads, head_dim], fetched
  * through the same tensor maps and page lookups as the MMA/TMA kernel.
  * Must be bit-exact with a host gather. */
 int decode_attn_debug_gather(const decode_attn_plan_t *plan, int32_t seq, const void *k_cache,
