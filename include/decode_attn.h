@@ -117,7 +117,7 @@ typedef struct {
     int64_t k_stride_page, k_stride_token, k_stride_head;   /* elements; multiples of 8              */
     int64_t v_stride_page, v_stride_token, v_stride_head;
     int32_t kv_dtype;           /* DA_DTYPE_BF16 or DA_DTYPE_FP16 (the paper serves one model family in
-                                   each, Section 4.1); fp16 not with shared_prefix_tokens             */
+                                   each, Section 4.1)                                                 */
     int32_t q_dtype;            /* the same as kv_dtype                                              */
     int32_t out_dtype;          /* DA_DTYPE_FP32 or DA_DTYPE_BF16                                    */
     float sm_scale;             /* 0: 1/sqrtf(head_dim) evaluated in fp32                            */

@@ -794,13 +794,19 @@ inline int make_pool_map(CUtensorMap* map, const void* pool, const decode_attn_s
 
 typedef void (*mma_kernel_t)(const KernelParams, const CUtensorMap, const CUtensorMap, const int, const MmaExtra);
 
-// f16: q, K and V are fp16 (attention mode, no shared-prefix units); else bf16.
+// f16: q, K and V are fp16 (attention mode); else bf16.
 template <int MODE>
 inline mma_kernel_t mma_kernel_for(int D, int G, bool prefix = false, bool f16 = false)
 {
     const bool dup = G <= 4;
     if (f16) {
-        if (MODE != kModeAttend || prefix) return nullptr;
+        if (MODE != kModeAttend) return nullptr;
+        if (prefix) {
+            if (!dup) return nullptr;
+            if (D == 128) return decode_attn_mma_kernel<128, true, kModeAttend, true, true>;
+            if (D == 64) return decode_attn_mma_kernel<64, true, kModeAttend, true, true>;
+            return nullptr;
+        }
         if (D == 128) return dup ? decode_attn_mma_kernel<128, true, kModeAttend, false, true>
                                  : decode_attn_mma_kernel<128, false, kModeAttend, false, true>;
         if (D == 64) return dup ? decode_attn_mma_kernel<64, true, kModeAttend, false, true>

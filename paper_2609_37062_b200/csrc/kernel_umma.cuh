@@ -47,6 +47,8 @@
 // still frees its tensor memory.
 #pragma once
 
+#include <cuda_fp16.h>
+
 #include "kernel_mma.cuh"
 #include "umma.cuh"
 
@@ -103,6 +105,7 @@ __device__ __forceinline__ bool umma_wait(uint32_t bar, uint32_t parity, volatil
 
 // Shared-prefix units first_unit, first_unit + unit_stride, ... < n_units, one after the other, by
 // the threads of a block (kUmmaThreads).  smem_raw: at least kUmmaSmemBytes of dynamic shared memory.
+template <bool F16>
 __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const CUtensorMap* k_map, const CUtensorMap* v_map,
                                                   const int G, const int first_unit, const int unit_stride,
                                                   const int n_units, uint8_t* smem_raw)
@@ -206,8 +209,8 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
             // -------------------------------------------------------- MMAs (one lane)
             block_sync(1, kUmmaSoftmaxThreads + 32);                        // Q is in shared memory
             if (lane == 0) {
-                constexpr uint32_t idesc_qk = umma::instr_desc_bf16(128, 128, false);
-                constexpr uint32_t idesc_pv = umma::instr_desc_bf16(128, 128, true);
+                constexpr uint32_t idesc_qk = umma::instr_desc_16(128, 128, false, F16);
+                constexpr uint32_t idesc_pv = umma::instr_desc_16(128, 128, true, F16);
                 bool ok = true;
                 // Descriptors differ only in their address field (16-byte units, the low 14 bits):
                 // stepping through a tile adds a constant to the low word.
@@ -399,11 +402,20 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
                         if (col0 + 2 * i < n_here) p0 = ex2f(fmaf(__uint_as_float(s[2 * i]), p.scale_log2, -m2));
                         if (col0 + 2 * i + 1 < n_here) p1 = ex2f(fmaf(__uint_as_float(s[2 * i + 1]), p.scale_log2, -m2));
                         lsum += p0 + p1;
-                        const uint32_t b0 = __float_as_uint(p0), b1 = __float_as_uint(p1);
-                        const float r0 = p0 - __uint_as_float(b0 & 0xffff0000u);   // exact
-                        const float r1 = p1 - __uint_as_float(b1 & 0xffff0000u);
-                        hi[i] = __byte_perm(b0, b1, 0x7632);                 // upper halves: element 2i low, 2i+1 high
-                        lo[i] = __byte_perm(__float_as_uint(r0), __float_as_uint(r1), 0x7632);
+                        if (F16) {
+                            // fp16 inputs: the weights are fp16 too, rounded, and so is the remainder
+                            const __half2 ph = __floats2half2_rn(p0, p1);
+                            const float2 pf = __half22float2(ph);
+                            const __half2 pl = __floats2half2_rn(p0 - pf.x, p1 - pf.y);
+                            hi[i] = *reinterpret_cast<const uint32_t*>(&ph);
+                            lo[i] = *reinterpret_cast<const uint32_t*>(&pl);
+                        } else {
+                            const uint32_t b0 = __float_as_uint(p0), b1 = __float_as_uint(p1);
+                            const float r0 = p0 - __uint_as_float(b0 & 0xffff0000u);   // exact
+                            const float r1 = p1 - __uint_as_float(b1 & 0xffff0000u);
+                            hi[i] = __byte_perm(b0, b1, 0x7632);             // upper halves: element 2i low, 2i+1 high
+                            lo[i] = __byte_perm(__float_as_uint(r0), __float_as_uint(r1), 0x7632);
+                        }
                     }
                     // the group's 32 logit columns become 16 columns of high parts, 16 of low parts
                     umma::st16(sc + col0, hi);
@@ -461,20 +473,24 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
     if (warp == kUmmaMmaWarp) umma::tmem_dealloc(tmem, kUmmaTmemCols);
 }
 
+template <bool F16>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 decode_attn_umma_prefix_kernel(const KernelParams p, const __grid_constant__ CUtensorMap k_map,
                                const __grid_constant__ CUtensorMap v_map, const int G, const int n_units)
 {
     extern __shared__ uint8_t smem_raw[];
-    umma_prefix_units(p, &k_map, &v_map, G, blockIdx.x, gridDim.x, n_units, smem_raw);
+    umma_prefix_units<F16>(p, &k_map, &v_map, G, blockIdx.x, gridDim.x, n_units, smem_raw);
 }
 
 // ---------------------------------------------------------------- host side
 
-inline int umma_prepare()
+typedef void (*umma_kernel_t)(const KernelParams, const CUtensorMap, const CUtensorMap, const int, const int);
+
+inline int umma_prepare(bool f16, umma_kernel_t* fn_out)
 {
-    if (cudaFuncSetAttribute(decode_attn_umma_prefix_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             kUmmaSmemBytes) != cudaSuccess) {
+    umma_kernel_t fn = f16 ? decode_attn_umma_prefix_kernel<true> : decode_attn_umma_prefix_kernel<false>;
+    *fn_out = fn;
+    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, kUmmaSmemBytes) != cudaSuccess) {
         (void)cudaGetLastError();
         return DA_ERR_CUDA;
     }
@@ -486,7 +502,8 @@ inline int umma_prefix_launch(const decode_attn_shape_t& s, int G, const KernelP
                               unsigned grid, cudaStream_t stream)
 {
     if (n_prefix_units == 0) return DA_OK;
-    int rc = umma_prepare();
+    umma_kernel_t fn;
+    int rc = umma_prepare(s.kv_dtype == DA_DTYPE_FP16, &fn);
     if (rc != DA_OK) return rc;
     CUtensorMap kmap, vmap;
     rc = make_pool_map(&kmap, kp.k, s, s.k_stride_page, s.k_stride_token, s.k_stride_head);
@@ -503,7 +520,7 @@ inline int umma_prefix_launch(const decode_attn_shape_t& s, int G, const KernelP
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, decode_attn_umma_prefix_kernel, kp, kmap, vmap, G, (int)n_prefix_units) != cudaSuccess) {
+    if (cudaLaunchKernelEx(&cfg, fn, kp, kmap, vmap, G, (int)n_prefix_units) != cudaSuccess) {
         (void)cudaGetLastError();
         return DA_ERR_CUDA;
     }

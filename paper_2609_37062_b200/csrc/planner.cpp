@@ -70,7 +70,6 @@ int validate_policy(const decode_attn_shape_t& s, const decode_attn_policy_t& p)
         return DA_ERR_INVALID_ARG;
     if (p.shared_prefix_tokens < 0 || p.shared_prefix_tokens % s.page_size != 0) return DA_ERR_INVALID_ARG;
     if (p.shared_prefix_tokens > 0) {
-        if (s.kv_dtype != DA_DTYPE_BF16) return DA_ERR_UNSUPPORTED;       // the prefix kernels are bf16 only
         if (p.fuse_combine || p.capacity_batch > 0 || p.split_mode == DA_SPLIT_FIXED_COUNT) return DA_ERR_UNSUPPORTED;
         const int G = s.num_q_heads / s.num_kv_heads;
         if (p.kernel == DA_KERNEL_UMMA_PREFIX) {

@@ -39,14 +39,14 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr, uint32_t lbo,
     return d;
 }
 
-// Instruction descriptor of a dense bf16 x bf16 -> fp32 MMA of shape M x N x 16.  (Both
-// operands have to be of the same 16-bit type: an fp16 A with a bf16 B is rejected by the GPU.)
-// b_mn_major: operand B is stored with N contiguous (else K contiguous); A is K-major.
-__host__ __device__ constexpr uint32_t instr_desc_bf16(int M, int N, bool b_mn_major)
+// Instruction descriptor of a dense 16-bit -> fp32 MMA of shape M x N x 16; f16: both operands
+// are fp16, else both bf16 (they have to be of one type: an fp16 A with a bf16 B is rejected by
+// the GPU).  b_mn_major: operand B is stored with N contiguous (else K contiguous); A is K-major.
+__host__ __device__ constexpr uint32_t instr_desc_16(int M, int N, bool b_mn_major, bool f16)
 {
     return (1u << 4)                       // accumulator format: fp32
-           | (1u << 7)                     // A format: bf16
-           | (1u << 10)                    // B format: bf16
+           | ((f16 ? 0u : 1u) << 7)        // A format: 0 fp16, 1 bf16
+           | ((f16 ? 0u : 1u) << 10)       // B format
            | ((b_mn_major ? 1u : 0u) << 16)
            | ((uint32_t)(N >> 3) << 17)
            | ((uint32_t)(M >> 4) << 24);

@@ -1,7 +1,8 @@
 """q, K and V in fp16 instead of bf16 (the paper serves one model family in
 each, Section 4.1): same path, same oracle, same tolerance, on both kernels,
 in every split mode, fused and separate merge, with a run mask, in both pool
-layouts, and with the own-layer KV write; what is bf16-only is refused."""
+layouts, with the own-layer KV write, and in shared-prefix plans on both
+prefix kernels."""
 import numpy as np
 import pytest
 import torch
@@ -70,14 +71,19 @@ def test_fp16_append_then_attend():
     assert np.array_equal(wd.v_pool.cpu().numpy().view(np.uint16), v_ref.reshape(wd.v_pool.shape))
 
 
-def test_fp16_is_refused_where_only_bf16_is_built():
-    w = wl.make_workload("p16", [600, 700], 32, 8, 128, seed=5, shared_prefix_tokens=512, dtype="fp16")
-    for kernel in (da.DA_KERNEL_MMA_TMA, da.DA_KERNEL_UMMA_PREFIX):
-        with pytest.raises(da.DecodeAttnError) as e:
-            da.decode_attn_plan(da.shape_of_workload(w), da.make_policy(shared_prefix_tokens=512, kernel=kernel), w.seq_lens)
-        assert e.value.status == da.DA_ERR_UNSUPPORTED
+@pytest.mark.parametrize("kernel", [da.DA_KERNEL_MMA_TMA, da.DA_KERNEL_UMMA_PREFIX], ids=["mma_sync", "tcgen05"])
+def test_fp16_shared_prefix_plans(kernel):
+    for batch, prefix in ((12, 512), (33, 1536), (5, 208)):
+        w = wl.as_fp16(wl.config_shared_prefix(batch=batch, prefix=prefix))
+        check_workload(w, da.make_policy(shared_prefix_tokens=prefix, kernel=kernel))
+        check_workload(w, da.make_policy(shared_prefix_tokens=prefix, kernel=kernel, split_mode=da.DA_SPLIT_DETERMINISTIC,
+                                         chunk_tokens=128))
+
+
+def test_mixed_input_types_are_refused():
+    w = wl.make_workload("p16", [600, 700], 32, 8, 128, seed=5, dtype="fp16")
     s = da.shape_of_workload(w)
-    s.q_dtype = da.DA_DTYPE_BF16                  # mixed input types
+    s.q_dtype = da.DA_DTYPE_BF16
     with pytest.raises(da.DecodeAttnError) as e:
         da.decode_attn_plan(s, da.make_policy(), w.seq_lens)
     assert e.value.status == da.DA_ERR_UNSUPPORTED
