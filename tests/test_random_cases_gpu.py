@@ -1,6 +1,7 @@
 """Seeded random cases through the C ABI against the oracle: shapes, length
 mixes with the awkward values (0, 1, page boundaries +-1), both kernels, all
-split modes, fused and separate merge, run masks, both pool layouts, and
+split modes, fused and separate merge, run masks, both pool layouts, both
+input types, and
 shared-prefix plans on both prefix kernels.  What a case does not support is
 refused with DA_ERR_UNSUPPORTED, never computed wrongly."""
 import random
@@ -40,7 +41,8 @@ def one_case(rng, index):
             pol["chunk_tokens"] = rng.choice([16, 64, 128, 1024])
     mask = [rng.choice([0, 1]) for _ in range(B)] if rng.random() < 0.3 else None
     layout = rng.choice(["token_major", "head_major"]) if not prefix else "token_major"
-    w = wl.make_workload("r", lens, hkv * G, hkv, D, seed=index, layout=layout, shared_prefix_tokens=prefix)
+    dtype = rng.choice(["bf16", "fp16"])
+    w = wl.make_workload("r", lens, hkv * G, hkv, D, seed=index, layout=layout, shared_prefix_tokens=prefix, dtype=dtype)
     return w, pol, mask
 
 
@@ -58,7 +60,7 @@ def test_random_cases(seed):
             assert e.status == da.DA_ERR_UNSUPPORTED, (index, pol)
             refused += 1
             continue
-        what = f"seed {seed} case {index}: {pol} lens {w.seq_lens.tolist()} mask {mask}"
+        what = f"seed {seed} case {index}: {pol} {w.dtype} lens {w.seq_lens.tolist()} mask {mask}"
         diff = np.abs(out.double().cpu().numpy() - ref)
         assert diff.max() <= MAX_ABS and diff.mean() <= MEAN_ABS, what
         got = lse.double().cpu().numpy()
