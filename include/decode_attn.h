@@ -119,7 +119,7 @@ typedef struct {
     int32_t kv_dtype;           /* DA_DTYPE_BF16 or DA_DTYPE_FP16 (the paper serves one model family in
                                    each, Section 4.1)                                                 */
     int32_t q_dtype;            /* the same as kv_dtype                                              */
-    int32_t out_dtype;          /* DA_DTYPE_FP32 or DA_DTYPE_BF16                                    */
+    int32_t out_dtype;          /* DA_DTYPE_FP32, DA_DTYPE_BF16 or DA_DTYPE_FP16                     */
     float sm_scale;             /* 0: 1/sqrtf(head_dim) evaluated in fp32                            */
 } decode_attn_shape_t;
 

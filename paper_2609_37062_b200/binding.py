@@ -424,7 +424,7 @@ def run_workload(w, policy: Optional[Policy] = None, out_dtype: int = DA_DTYPE_F
     shape = shape_of_workload(w, out_dtype=out_dtype, sm_scale=sm_scale)
     plan = decode_attn_plan(shape, policy, w.seq_lens)
     dev = w.k_pool.device
-    odt = torch.float32 if out_dtype == DA_DTYPE_FP32 else torch.bfloat16
+    odt = {DA_DTYPE_FP32: torch.float32, DA_DTYPE_BF16: torch.bfloat16, DA_DTYPE_FP16: torch.float16}[out_dtype]
     out = torch.full((w.batch, w.num_q_heads, w.head_dim), float("nan"), dtype=odt, device=dev)
     lse = torch.full((w.batch, w.num_q_heads), float("nan"), dtype=torch.float32, device=dev) if want_lse else None
     ws = torch.empty(max(plan.workspace_bytes, 256), dtype=torch.uint8, device=dev)

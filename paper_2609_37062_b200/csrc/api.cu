@@ -67,6 +67,8 @@ namespace {
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+int out_kind_of(int out_dtype) { return out_dtype == DA_DTYPE_BF16 ? 1 : out_dtype == DA_DTYPE_FP16 ? 2 : 0; }
+
 // Device buffer, pinned mirror, stream and event of a plan.  Creating these
 // costs far more than planning a step, so destroyed plans park theirs here
 // and the next plan of a similar size picks them up.
@@ -328,7 +330,7 @@ KernelParams make_params(const decode_attn_plan_t* pl, const decode_attn_run_arg
     kp.num_kv_heads = s.num_kv_heads;
     kp.max_pages_per_seq = s.max_pages_per_seq;
     kp.scale_log2 = pl->scale * kLog2e;
-    kp.out_bf16 = s.out_dtype == DA_DTYPE_BF16;
+    kp.out_kind = out_kind_of(s.out_dtype);
     kp.in_f16 = s.kv_dtype == DA_DTYPE_FP16;
     kp.fused = pl->policy.fuse_combine;
     kp.grid_exit = pl->policy.capacity_batch > 0;
@@ -611,7 +613,7 @@ int decode_attn_merge_shards(const decode_attn_shape_t* shape, int32_t n_shards,
     const int64_t blocks = (threads + 127) / 128;
     if (blocks > 0x7fffffffLL) return DA_ERR_UNSUPPORTED;
     decode_attn_merge_shards_kernel<<<(unsigned)blocks, 128, 0, stream>>>(out_shards, lse_shards, n_shards, rows, D4, out,
-                                                                            lse_or_null, shape->out_dtype == DA_DTYPE_BF16);
+                                                                            lse_or_null, out_kind_of(shape->out_dtype));
     DA_CUDA_TRY(cudaGetLastError());
     return DA_OK;
 }
@@ -792,7 +794,7 @@ int decode_attn_host_step(const decode_attn_shape_t* shape, const decode_attn_po
         ~PlanGuard() { decode_attn_plan_destroy(p); }
     } pg{plan};
 
-    const size_t out_elem = shape->out_dtype == DA_DTYPE_BF16 ? 2 : 4;
+    const size_t out_elem = shape->out_dtype == DA_DTYPE_FP32 ? 4 : 2;
     const size_t q_bytes = (size_t)shape->batch * shape->num_q_heads * shape->head_dim * 2;
     const size_t pool_bytes = (size_t)pool_elems * 2;
     const size_t bt_bytes = (size_t)shape->batch * shape->max_pages_per_seq * 4;
@@ -973,7 +975,7 @@ int decode_attn_step_static(const decode_attn_shape_t* shape, const int32_t* seq
     kp.max_pages_per_seq = shape->max_pages_per_seq;
     const float scale = shape->sm_scale > 0.f ? shape->sm_scale : 1.0f / sqrtf((float)shape->head_dim);
     kp.scale_log2 = scale * kLog2e;
-    kp.out_bf16 = shape->out_dtype == DA_DTYPE_BF16;
+    kp.out_kind = out_kind_of(shape->out_dtype);
     kp.in_f16 = shape->kv_dtype == DA_DTYPE_FP16;
     kp.fused = 0;
     kp.grid_exit = 0;

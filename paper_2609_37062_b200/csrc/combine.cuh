@@ -51,7 +51,7 @@ __global__ void __launch_bounds__(kCombineThreads) decode_attn_combine_few_kerne
 // log) for each row; one thread per four output dims, shards in ascending order.
 __global__ void __launch_bounds__(128) decode_attn_merge_shards_kernel(const float* out_shards, const float* lse_shards,
                                                                        int n_shards, int64_t rows, int D4, void* out,
-                                                                       float* lse, int out_bf16)
+                                                                       float* lse, int out_kind)
 {
     const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= rows * D4) return;
@@ -74,7 +74,7 @@ __global__ void __launch_bounds__(128) decode_attn_merge_shards_kernel(const flo
         const float inv = 1.0f / ws;                          // ws >= 1: the shard that holds the maximum weighs 1
         acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
     }
-    store_out4(out, idx * 4, acc, out_bf16);
+    store_out4(out, idx * 4, acc, out_kind);
     if (lse != nullptr && d4 == 0) lse[row] = (M != -INFINITY) ? M + log2f(ws) * kLn2 : -INFINITY;
 }
 

@@ -4,6 +4,7 @@
 #pragma once
 
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
 #include <cstdint>
@@ -47,7 +48,7 @@ struct KernelParams {
     int64_t num_pages;
     int32_t num_q_heads, num_kv_heads, max_pages_per_seq, batch;
     float scale_log2;  // sm_scale * log2(e): logits are kept in the base-2 domain
-    int32_t out_bf16;
+    int32_t out_kind;
     int32_t in_f16;          // q, K and V are fp16 (else bf16)
     int32_t fused;
     int32_t grid_exit;  // capacity plans: the unit count is read from header->n_units, surplus blocks leave at once
@@ -106,15 +107,23 @@ __device__ __forceinline__ decode_attn_unit_t load_unit(const decode_attn_unit_t
     return u;
 }
 
-__device__ __forceinline__ void store_out4(void* out, int64_t idx, float4 v, int out_bf16)
+// out_kind: 0 fp32, 1 bf16, 2 fp16 (round to nearest even).
+__device__ __forceinline__ void store_out4(void* out, int64_t idx, float4 v, int out_kind)
 {
-    if (out_bf16) {
+    if (out_kind == 1) {
         __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y);
         __nv_bfloat162 hi = __floats2bfloat162_rn(v.z, v.w);
         uint2 w;
         w.x = *reinterpret_cast<uint32_t*>(&lo);
         w.y = *reinterpret_cast<uint32_t*>(&hi);
         *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(out) + idx) = w;
+    } else if (out_kind == 2) {
+        __half2 lo = __floats2half2_rn(v.x, v.y);
+        __half2 hi = __floats2half2_rn(v.z, v.w);
+        uint2 w;
+        w.x = *reinterpret_cast<uint32_t*>(&lo);
+        w.y = *reinterpret_cast<uint32_t*>(&hi);
+        *reinterpret_cast<uint2*>(reinterpret_cast<__half*>(out) + idx) = w;
     } else {
         *reinterpret_cast<float4*>(reinterpret_cast<float*>(out) + idx) = v;
     }
@@ -314,7 +323,7 @@ __device__ __forceinline__ void combine_slice(const KernelParams& p, int b, int 
             o.z = (((a0.z + a1.z) + a2.z) + a3.z) * inv;
             o.w = (((a0.w + a1.w) + a2.w) + a3.w) * inv;
         }
-        store_out4(p.out, ((int64_t)b * p.num_q_heads + g * G + h) * D + d4 * 4, o, p.out_bf16);
+        store_out4(p.out, ((int64_t)b * p.num_q_heads + g * G + h) * D + d4 * 4, o, p.out_kind);
         if (p.lse != nullptr && d4 == 0)
             p.lse[(int64_t)b * p.num_q_heads + g * G + h] = (M != -INFINITY && ls > 0.f) ? (M + log2f(ls)) * kLn2 : -INFINITY;
     }
@@ -375,7 +384,7 @@ __device__ __forceinline__ void combine_column(const KernelParams& p, int b, int
         o.z = (((acc[0].z + acc[1].z) + acc[2].z) + acc[3].z) * inv;
         o.w = (((acc[0].w + acc[1].w) + acc[2].w) + acc[3].w) * inv;
     }
-    store_out4(p.out, ((int64_t)b * p.num_q_heads + g * G + h) * D + d4 * 4, o, p.out_bf16);
+    store_out4(p.out, ((int64_t)b * p.num_q_heads + g * G + h) * D + d4 * 4, o, p.out_kind);
     if (p.lse != nullptr && d4 == 0)
         p.lse[(int64_t)b * p.num_q_heads + g * G + h] = (M != -INFINITY && ls > 0.f) ? (M + log2f(ls)) * kLn2 : -INFINITY;
 }
@@ -498,7 +507,7 @@ __device__ __forceinline__ void block_finish(const KernelParams& p, const decode
             } else {
                 o = make_float4(0.f, 0.f, 0.f, 0.f);
             }
-            store_out4(p.out, ((int64_t)u.seq * Hq + h0 + h) * D + d4 * 4, o, p.out_bf16);
+            store_out4(p.out, ((int64_t)u.seq * Hq + h0 + h) * D + d4 * 4, o, p.out_kind);
             if (p.lse != nullptr && d4 == 0)
                 p.lse[(int64_t)u.seq * Hq + h0 + h] = (ls > 0.f) ? (M + log2f(ls)) * kLn2 : -INFINITY;
         } else {

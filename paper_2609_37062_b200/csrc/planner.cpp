@@ -49,7 +49,7 @@ int validate_shape(const decode_attn_shape_t& s)
     if (s.head_dim != 64 && s.head_dim != 128) return DA_ERR_UNSUPPORTED;
     if (s.page_size != 16) return DA_ERR_UNSUPPORTED;
     if ((s.kv_dtype != DA_DTYPE_BF16 && s.kv_dtype != DA_DTYPE_FP16) || s.q_dtype != s.kv_dtype) return DA_ERR_UNSUPPORTED;
-    if (s.out_dtype != DA_DTYPE_FP32 && s.out_dtype != DA_DTYPE_BF16) return DA_ERR_UNSUPPORTED;
+    if (s.out_dtype != DA_DTYPE_FP32 && s.out_dtype != DA_DTYPE_BF16 && s.out_dtype != DA_DTYPE_FP16) return DA_ERR_UNSUPPORTED;
     if (s.num_pages > (int64_t)INT32_MAX) return DA_ERR_UNSUPPORTED;
     return DA_OK;
 }

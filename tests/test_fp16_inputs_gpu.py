@@ -80,6 +80,21 @@ def test_fp16_shared_prefix_plans(kernel):
                                          chunk_tokens=128))
 
 
+@pytest.mark.parametrize("kernel", KERNELS, ids=KERNEL_IDS)
+@pytest.mark.parametrize("fused", [0, 1])
+def test_fp16_output_is_the_rounded_result(kernel, fused):
+    """An fp16 `out` sits within one fp16 step of the oracle (its own rounding), whether it is
+    written by the attention kernel (single split), the combine kernel or the merge blocks."""
+    w = wl.make_workload("o16", [17, 64, 129, 900], 8, 2, 64, seed=6, dtype="fp16")
+    ref_out, _ = oracle_of(w)
+    out, _ = da.run_workload(to_device(w), da.make_policy(kernel=kernel, fuse_combine=fused, chunk_tokens=64),
+                             out_dtype=da.DA_DTYPE_FP16)
+    assert out.dtype == torch.float16
+    got = out.float().cpu().numpy().astype(np.float64)
+    step = np.maximum(np.abs(ref_out), 2.0 ** -14) * 2.0 ** -10
+    assert (np.abs(got - ref_out) <= step + 1e-6).all()
+
+
 def test_mixed_input_types_are_refused():
     w = wl.make_workload("p16", [600, 700], 32, 8, 128, seed=5, dtype="fp16")
     s = da.shape_of_workload(w)
