@@ -81,7 +81,7 @@ def test_fused_and_separate_merge_give_the_same_bits(kernel):
     assert torch.equal(a, b) and torch.equal(la, lb)
 
 
-@pytest.mark.parametrize("splits", [2, 3, 4, 5, 8, 9, 13, 49])
+@pytest.mark.parametrize("splits", [2, 3, 4, 5, 8, 9, 13, 49, 300, 1024])
 def test_every_merge_kernel_gives_the_fused_path_its_bits(splits):
     """The combine launch picks a kernel by the plan's largest split count (one thread per column
     up to 4 and up to 8 splits, the slice kernel beyond); all of them and the merge blocks of a
