@@ -315,21 +315,21 @@ def main():
         run_mask = keep.to(dev)
         masked_bytes = int((first.seq_lens.cpu().long() * (1 - keep.long())).sum().item()) * first.kv_bytes_per_token
 
-    def step(i):
+    def step(i, combine=True):
         w = pools[i % copies]
         da.decode_attn_run(plan, w.q_bits, w.k_pool, w.v_pool, w.block_table, w.seq_lens, out, lse, ws,
                            plan.workspace_bytes, run_mask=run_mask)
-        if not policy.fuse_combine and not args.partial_only:
+        if combine and not policy.fuse_combine and not args.partial_only:
             da.decode_attn_combine(plan, ws, out, lse)
 
-    def make_runner(n_steps, first_index):
+    def make_runner(n_steps, first_index, combine=True):
         """n_steps consecutive steps starting at rotation index first_index, as one callable."""
         if args.no_graph:
-            return lambda: [step(first_index + j) for j in range(n_steps)]
+            return lambda: [step(first_index + j, combine) for j in range(n_steps)]
         g = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g):
             for j in range(n_steps):
-                step(first_index + j)
+                step(first_index + j, combine)
         return g.replay
 
     stream = torch.cuda.Stream(device=dev)
@@ -364,6 +364,20 @@ def main():
         st = da.decode_attn_last_device_status(plan, stream)
         if st != da.DA_OK:
             raise SystemExit(f"device status after the timed region: {da.decode_attn_strerror(st)}")
+
+        # the dominant kernel by itself: the same replays without the combine launch
+        kernel_only_us = None
+        if not policy.fuse_combine and not args.partial_only and info.n_slots > 0:
+            n_ko = min(chunk, 2048)
+            run_ko = make_runner(n_ko, 0, combine=False)
+            run_ko()
+            stream.synchronize()
+            k0, k1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            k0.record(stream)
+            run_ko()
+            k1.record(stream)
+            stream.synchronize()
+            kernel_only_us = k0.elapsed_time(k1) * 1e3 / n_ko
 
         probe_us = None
         if args.probe and info.kernel == da.DA_KERNEL_MMA_TMA:
@@ -480,7 +494,11 @@ def main():
                          "algorithmic_bytes_per_launch": algo_bytes,
                          "how": ("unique" if prefix_plan else "logical") +
                                 " K+V bytes of the batch / (event time of the timed region / steps): the "
-                                "step's combine launch and launch gaps are charged to the partial kernel"},
+                                "step's combine launch and launch gaps are charged to the partial kernel",
+                         "kernel_only": None if kernel_only_us is None else
+                         {"us_per_launch": kernel_only_us, "achieved": algo_bytes / kernel_only_us / 1e3,
+                          "frac": algo_bytes / kernel_only_us / 1e3 / peak,
+                          "how": "the same graph replays without the combine launch (results are not merged)"}},
             "gpu_launches": args.steps * launches_per_step,
             "clocks": clocks,
             "e2e": e2e,
