@@ -55,7 +55,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         if p.wait() != 0:
             raise RuntimeError(f"nvcc failed on {src}")
     tmp = LIB + f".{os.getpid()}.tmp"
-    subprocess.check_call([nvcc, "-shared", "-o", tmp, *objs, "-lcudart"])
+    subprocess.check_call([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-o", tmp, *objs, "-lcudart"])
     os.replace(tmp, LIB)
     return LIB
 
