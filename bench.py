@@ -71,6 +71,7 @@ def parse_args():
     ap.add_argument("--alias-after", type=int, default=0,
                     help="sweep cells too large for memory: sequences i >= K reuse the pages of sequence i mod K")
     ap.add_argument("--in-dtype", default="bf16", choices=["bf16", "fp16"], help="type of q, K and V")
+    ap.add_argument("--page-size", type=int, default=16, choices=[16, 32, 64, 128, 256], help="tokens per KV page")
     ap.add_argument("--prefix-aware", action="store_true",
                     help="shared_prefix workload: tell the planner about the common prefix (attended once per block of sequences)")
     ap.add_argument("--mask-fraction", type=float, default=None,
@@ -79,6 +80,7 @@ def parse_args():
 
 
 IN_DTYPE = "bf16"     # set from --in-dtype
+PAGE_SIZE = 16        # set from --page-size
 
 
 def make_workload(name, device, table_seed=None, seed_shift=0, alias_after=None):
@@ -92,15 +94,16 @@ def _make_workload_bf16(name, device, table_seed=None, seed_shift=0, alias_after
     if name == "tiny":
         return wl.config_tiny(device=device)
     if name == "long_32k":
-        return wl.config_long(device=device, seed=1 + seed_shift, table_seed=table_seed)
+        return wl.config_long(device=device, seed=1 + seed_shift, table_seed=table_seed, page_size=PAGE_SIZE)
     if name == "short_chat":
-        return wl.config_short_chat(device=device, seed=2 + seed_shift, table_seed=table_seed)
+        return wl.config_short_chat(device=device, seed=2 + seed_shift, table_seed=table_seed, page_size=PAGE_SIZE)
     if name == "shared_prefix":
-        return wl.config_shared_prefix(device=device, seed=3 + seed_shift, table_seed=table_seed)
+        return wl.config_shared_prefix(device=device, seed=3 + seed_shift, table_seed=table_seed,
+                                       page_size=PAGE_SIZE)
     if name.startswith("sweep_"):
         ctx, batch = name[len("sweep_"):].split("x")
         return wl.config_sweep_cell(int(ctx), int(batch), device=device, seed=4 + seed_shift, table_seed=table_seed,
-                                    alias_after=alias_after)
+                                    alias_after=alias_after, page_size=PAGE_SIZE)
     raise SystemExit(f"unknown workload {name}")
 
 
@@ -245,8 +248,9 @@ def run_reference(args):
 
 def main():
     args = parse_args()
-    global IN_DTYPE
+    global IN_DTYPE, PAGE_SIZE
     IN_DTYPE = args.in_dtype
+    PAGE_SIZE = args.page_size
     if args.impl == "reference":
         run_reference(args)
         return

@@ -82,7 +82,7 @@ typedef enum {
 typedef struct {
     int32_t split_mode;     /* da_split_mode_t                                                       */
     int32_t fixed_count;    /* FIXED_COUNT: splits per sequence (>= 1)                               */
-    int32_t chunk_tokens;   /* DETERMINISTIC: chunk length, a multiple of page_size (0: 1024).
+    int32_t chunk_tokens;   /* DETERMINISTIC: chunk length, a multiple of 16 (0: 1024).
                                AUTO: smallest chunk the planner may choose (0: 256)                  */
     int32_t max_splits;     /* upper bound on the splits of one sequence (0: 512; at most 1024)      */
     int32_t sm_count;       /* 0: the current device's multiprocessor count                          */
@@ -111,7 +111,7 @@ typedef struct {
     int32_t num_q_heads;
     int32_t num_kv_heads;       /* divides num_q_heads; group size <= 8                              */
     int32_t head_dim;           /* 64 or 128                                                         */
-    int32_t page_size;          /* tokens per page: 16                                               */
+    int32_t page_size;          /* tokens per page: 16, 32, 64, 128 or 256                           */
     int32_t max_pages_per_seq;  /* row stride of block_table, in entries                             */
     int64_t num_pages;          /* pages in each pool                                                */
     int64_t k_stride_page, k_stride_token, k_stride_head;   /* elements; multiples of 8              */
@@ -131,7 +131,7 @@ typedef struct {
 typedef struct {
     int32_t seq;          /* b                                                                       */
     int32_t kv_head;      /* g (low 16 bits)                                                         */
-    int32_t tok_begin;    /* first token, a multiple of page_size                                    */
+    int32_t tok_begin;    /* first token, a multiple of 16 (of chunk_tokens in DETERMINISTIC mode)  */
     int32_t tok_end;      /* one past the last token; tok_end == tok_begin marks an empty split      */
     int32_t slot;         /* index of the partial in the workspace, -1: writes `out` directly        */
     int32_t seq_len;      /* the length the plan was made for (checked against device seq_lens)      */

@@ -67,6 +67,14 @@ namespace {
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// page_size is a power of two (validate_shape).
+int log2_of(int x)
+{
+    int r = 0;
+    while ((1 << (r + 1)) <= x) ++r;
+    return r;
+}
+
 int out_kind_of(int out_dtype) { return out_dtype == DA_DTYPE_BF16 ? 1 : out_dtype == DA_DTYPE_FP16 ? 2 : 0; }
 
 // Device buffer, pinned mirror, stream and event of a plan.  Creating these
@@ -332,6 +340,7 @@ KernelParams make_params(const decode_attn_plan_t* pl, const decode_attn_run_arg
     kp.scale_log2 = pl->scale * kLog2e;
     kp.out_kind = out_kind_of(s.out_dtype);
     kp.in_f16 = s.kv_dtype == DA_DTYPE_FP16;
+    kp.tile_shift = log2_of(s.page_size) - 4;
     kp.fused = pl->policy.fuse_combine;
     kp.grid_exit = pl->policy.capacity_batch > 0;
     kp.n_units = (int32_t)pl->layout.units.size();
@@ -726,6 +735,7 @@ int decode_attn_append_kv(const decode_attn_shape_t* shape, const void* new_k, c
     ap.num_kv_heads = shape->num_kv_heads;
     ap.head_dim = shape->head_dim;
     ap.max_pages_per_seq = shape->max_pages_per_seq;
+    ap.page_shift = log2_of(shape->page_size);
     const int rows = shape->batch * shape->num_kv_heads;
     const unsigned grid = (unsigned)((rows + kAppendThreads / 32 - 1) / (kAppendThreads / 32));
     cudaLaunchConfig_t cfg;
@@ -977,6 +987,7 @@ int decode_attn_step_static(const decode_attn_shape_t* shape, const int32_t* seq
     kp.scale_log2 = scale * kLog2e;
     kp.out_kind = out_kind_of(shape->out_dtype);
     kp.in_f16 = shape->kv_dtype == DA_DTYPE_FP16;
+    kp.tile_shift = log2_of(shape->page_size) - 4;
     kp.fused = 0;
     kp.grid_exit = 0;
     kp.n_units = (int32_t)lay.units.size();

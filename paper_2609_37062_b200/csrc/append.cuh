@@ -22,6 +22,7 @@ struct AppendParams {
     int64_t v_stride_page, v_stride_token, v_stride_head;
     int64_t num_pages;
     int32_t batch, num_kv_heads, head_dim, max_pages_per_seq;
+    int32_t page_shift;           // log2(page_size)
 };
 
 __global__ void __launch_bounds__(kAppendThreads) decode_attn_append_kernel(const AppendParams p)
@@ -35,16 +36,16 @@ __global__ void __launch_bounds__(kAppendThreads) decode_attn_append_kernel(cons
     const int L = __ldg(p.seq_lens + b);
     if (L <= 0) return;
     const int t = L - 1;
-    if ((t >> 4) >= p.max_pages_per_seq) {
+    if ((t >> p.page_shift) >= p.max_pages_per_seq) {
         if (lane == 0 && p.status) record_status(p.status, DA_ERR_STALE_PLAN);
         return;
     }
-    const int page = __ldg(p.block_table + (int64_t)b * p.max_pages_per_seq + (t >> 4));
+    const int page = __ldg(p.block_table + (int64_t)b * p.max_pages_per_seq + (t >> p.page_shift));
     if ((unsigned)page >= (unsigned)p.num_pages) {
         if (lane == 0 && p.status) record_status(p.status, DA_ERR_BAD_PAGE);
         return;
     }
-    const int slot = t & 15;
+    const int slot = t & ((1 << p.page_shift) - 1);
     const int chunks = p.head_dim / 8;                  // 16-byte chunks per row (<= 16: both rows fit one warp)
     const uint4* sk = reinterpret_cast<const uint4*>(p.new_k + (int64_t)row * p.head_dim);
     const uint4* sv = reinterpret_cast<const uint4*>(p.new_v + (int64_t)row * p.head_dim);

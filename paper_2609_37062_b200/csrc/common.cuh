@@ -50,6 +50,7 @@ struct KernelParams {
     float scale_log2;  // sm_scale * log2(e): logits are kept in the base-2 domain
     int32_t out_kind;
     int32_t in_f16;          // q, K and V are fp16 (else bf16)
+    int32_t tile_shift;      // log2(page_size / 16): the kernels walk the cache in 16-token tiles, 1 << tile_shift per page
     int32_t fused;
     int32_t grid_exit;  // capacity plans: the unit count is read from header->n_units, surplus blocks leave at once
     int32_t n_units;    // otherwise: the unit count

@@ -237,6 +237,7 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
     if (warp == kMmaConsumerWarps) {
         // ------------------------------------------------------------ producer
         const uint64_t l2_policy = l2_policy_evict_first();
+        const int ts = p.tile_shift;                          // 16-token tiles per page, as a shift
         uint32_t git = 0;                                     // stages issued so far, over all units
         bool alive = true;
         // range of a unit as this launch sees it: a masked row (or, in the gather mode, another
@@ -250,8 +251,8 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
         };
         auto first_ids = [&](const decode_attn_unit_t& x, int end) {
             const int np = (end - x.tok_begin + 15) >> 4;
-            const int32_t* t = p.block_table + (int64_t)x.seq * p.max_pages_per_seq + (x.tok_begin >> 4);
-            return (lane < np) ? __ldg(t + lane) : 0;
+            const int32_t* t = p.block_table + (int64_t)x.seq * p.max_pages_per_seq;
+            return (lane < np) ? __ldg(t + (((x.tok_begin >> 4) + lane) >> ts)) : 0;
         };
         int t1 = unit_end(u);
         int ids_first = first_ids(u, t1);
@@ -265,14 +266,15 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
             const int t0 = u.tok_begin;
             const int n_pages = (t1 - t0 + 15) >> 4;
             const int n_iters = (n_pages + kPagesPerStage - 1) / kPagesPerStage;
-            const int32_t* bt = p.block_table + (int64_t)b * p.max_pages_per_seq + (t0 >> 4);
+            const int32_t* bt = p.block_table + (int64_t)b * p.max_pages_per_seq;
+            const int tile0 = t0 >> 4;                                    // first 16-token tile of the unit
             int ids_next = ids_first;
             int ids_cur = 0;
             for (int it = 0; it < n_iters; ++it, ++git) {
                 if ((it & 7) == 0) {                                      // 32 page ids per 8 stages, one batch ahead
                     ids_cur = ids_next;
                     const int nxt = (it + 8) * kPagesPerStage + lane;
-                    ids_next = (nxt < n_pages) ? __ldg(bt + nxt) : 0;
+                    ids_next = (nxt < n_pages) ? __ldg(bt + ((tile0 + nxt) >> ts)) : 0;
                 }
                 const int s = git % NS;
                 if (git >= (uint32_t)NS) {
@@ -305,7 +307,8 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
                     }
                     const uint32_t dst = base + s * Cfg::kStageBytes + which * Cfg::kTensorBytes +
                                          pg * Cfg::kPageBytes + hf * Cfg::kBoxBytes;
-                    tma_load_4d(dst, which ? &v_map : &k_map, full, hf * 64, 0, g, page_id, l2_policy);
+                    const int slot0 = ((tile0 + it * kPagesPerStage + pg) & ((1 << ts) - 1)) << 4;   // of the tile within its page
+                    tma_load_4d(dst, which ? &v_map : &k_map, full, hf * 64, slot0, g, page_id, l2_policy);
                     if (git == 0 && lane == 0) DA_TRACE_STAMP(blockIdx.x, 2);
                 }
                 if (has_next && !next_ready) {                            // this unit is under way: look ahead

@@ -113,6 +113,7 @@ __global__ void __launch_bounds__(kSimtThreads) decode_attn_simt_kernel(const Ke
     }
 
     const int32_t* bt = p.block_table + (int64_t)b * p.max_pages_per_seq;
+    const int page_shift = 4 + p.tile_shift, page_mask = (1 << page_shift) - 1;
     const __nv_bfloat16* kbase = p.k + (int64_t)g * p.k_stride_head + li * 8;
     const __nv_bfloat16* vbase = p.v + (int64_t)g * p.v_stride_head + li * 8;
 
@@ -126,12 +127,12 @@ __global__ void __launch_bounds__(kSimtThreads) decode_attn_simt_kernel(const Ke
             kk[j] = make_uint4(0, 0, 0, 0);
             vv[j] = make_uint4(0, 0, 0, 0);
             if (ok[j]) {
-                const int page = __ldg(bt + (t >> 4));
+                const int page = __ldg(bt + (t >> page_shift));
                 if ((unsigned)page >= (unsigned)p.num_pages) {
                     record_status(p.status, DA_ERR_BAD_PAGE);
                     ok[j] = false;
                 } else {
-                    const int slot = t & 15;
+                    const int slot = t & page_mask;
                     kk[j] = ldg_stream16(kbase + (int64_t)page * p.k_stride_page + (int64_t)slot * p.k_stride_token);
                     vv[j] = ldg_stream16(vbase + (int64_t)page * p.v_stride_page + (int64_t)slot * p.v_stride_token);
                 }

@@ -175,9 +175,10 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
         if (warp == kUmmaLoadWarp) {
             // -------------------------------------------------------- TMA: K_0, V_0, K_1, V_1, ...
             const uint64_t l2_policy = l2_policy_evict_first();
-            const int32_t* bt = p.block_table + (int64_t)u.seq * p.max_pages_per_seq + (u.tok_begin >> 4);
-            const int pg = (lane >> 1) & 7, hf = lane & 1;                  // lane j < 16: box (page j / 2, half j % 2)
-            int page_id = 0;
+            const int32_t* bt = p.block_table + (int64_t)u.seq * p.max_pages_per_seq;
+            const int ts = p.tile_shift, tile0 = u.tok_begin >> 4;         // 16-token tiles: 1 << ts per page
+            const int pg = (lane >> 1) & 7, hf = lane & 1;                  // lane j < 16: box (16 tokens j / 2, half j % 2)
+            int page_id = 0, slot0 = 0;
             bool ok = true;
             for (int n = 0; n < 2 * T && ok; ++n) {
                 const int t = n >> 1, st = n % NS;
@@ -186,7 +187,8 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
                     // range is fetched from outside the pool, which the TMA unit fills with zeros
                     page_id = (int)p.num_pages;
                     if (t * 8 + pg < n_pages) {
-                        page_id = __ldg(bt + t * 8 + pg);
+                        page_id = __ldg(bt + ((tile0 + t * 8 + pg) >> ts));
+                        slot0 = ((tile0 + t * 8 + pg) & ((1 << ts) - 1)) << 4;
                         if ((unsigned)page_id >= (unsigned)p.num_pages) {   // never hand TMA a page outside the pool
                             record_status(p.status, DA_ERR_BAD_PAGE);
                             page_id = 0;
@@ -203,7 +205,7 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
                 __syncwarp();
                 if (lane < 16)
                     tma_load_4d(ring_base + st * kUmmaTileBytes + hf * kUmmaHalfBytes + pg * 2048, (n & 1) ? v_map : k_map, bar,
-                                hf * 64, 0, g, page_id, l2_policy);
+                                hf * 64, slot0, g, page_id, l2_policy);
             }
         } else if (warp == kUmmaMmaWarp) {
             // -------------------------------------------------------- MMAs (one lane)

@@ -47,7 +47,8 @@ int validate_shape(const decode_attn_shape_t& s)
         return DA_ERR_INVALID_ARG;  // rows of head_dim contiguous elements must not overlap
     if (s.num_q_heads / s.num_kv_heads > kMaxGroup) return DA_ERR_UNSUPPORTED;
     if (s.head_dim != 64 && s.head_dim != 128) return DA_ERR_UNSUPPORTED;
-    if (s.page_size != 16) return DA_ERR_UNSUPPORTED;
+    // the kernels walk the cache in 16-token tiles: a page holds a power-of-two number of them
+    if (s.page_size < 16 || s.page_size > 256 || (s.page_size & (s.page_size - 1)) != 0) return DA_ERR_UNSUPPORTED;
     if ((s.kv_dtype != DA_DTYPE_BF16 && s.kv_dtype != DA_DTYPE_FP16) || s.q_dtype != s.kv_dtype) return DA_ERR_UNSUPPORTED;
     if (s.out_dtype != DA_DTYPE_FP32 && s.out_dtype != DA_DTYPE_BF16 && s.out_dtype != DA_DTYPE_FP16) return DA_ERR_UNSUPPORTED;
     if (s.num_pages > (int64_t)INT32_MAX) return DA_ERR_UNSUPPORTED;
@@ -62,7 +63,7 @@ int validate_policy(const decode_attn_shape_t& s, const decode_attn_policy_t& p)
     if (p.chunk_tokens < 0 || p.max_splits < 0 || p.sm_count < 0 || p.ctas_per_sm < 0 ||
         p.capacity_batch < 0 || p.capacity_tokens < 0)
         return DA_ERR_INVALID_ARG;
-    if (p.chunk_tokens % s.page_size != 0) return DA_ERR_INVALID_ARG;
+    if (p.chunk_tokens % kTileTokens != 0) return DA_ERR_INVALID_ARG;
     if (p.max_splits > kMaxSplits || (p.split_mode == DA_SPLIT_FIXED_COUNT && p.fixed_count > kMaxSplits))
         return DA_ERR_INVALID_ARG;
     if (p.fuse_combine != 0 && p.fuse_combine != 1) return DA_ERR_INVALID_ARG;
@@ -94,14 +95,15 @@ static int min_chunk_pages(const decode_attn_shape_t& s, const decode_attn_polic
         tokens = p.chunk_tokens > 0 ? p.chunk_tokens : kDefaultDeterministicChunk;
     else
         tokens = p.chunk_tokens > 0 ? p.chunk_tokens : kDefaultAutoMinChunk;
-    return (int)std::max<int64_t>(1, ceil_div(tokens, s.page_size));
+    (void)s;
+    return (int)std::max<int64_t>(1, ceil_div(tokens, kTileTokens));
 }
 
 int64_t capacity_slots(const decode_attn_shape_t& s, const decode_attn_policy_t& p)
 {
     if (p.capacity_batch <= 0) return 0;
     if (p.split_mode == DA_SPLIT_FIXED_COUNT) return (int64_t)p.fixed_count * p.capacity_batch;
-    const int64_t chunk_tokens = (int64_t)min_chunk_pages(s, p) * s.page_size;
+    const int64_t chunk_tokens = (int64_t)min_chunk_pages(s, p) * kTileTokens;
     return ceil_div(p.capacity_tokens, chunk_tokens) + p.capacity_batch;
 }
 
@@ -135,7 +137,9 @@ int make_layout(const decode_attn_shape_t& s, const decode_attn_policy_t& p, con
 {
     if (sm_count <= 0 || ctas_per_sm <= 0) return DA_ERR_INVALID_ARG;
     if (s.batch > 0 && seq_lens == nullptr) return DA_ERR_INVALID_ARG;
-    const int B = s.batch, P = s.page_size, H = s.num_kv_heads;
+    // Everything below counts in 16-token tiles ("pages" of the planner): what the kernels fetch at
+    // a time.  The pool's page size only bounds the block table, so a plan does not depend on it.
+    const int B = s.batch, P = kTileTokens, H = s.num_kv_heads;
     const int max_splits = max_splits_of(p);
     // With a shared prefix the ordinary units cover only what follows it; the prefix itself is
     // cut into chunks attended once for a block of sequences at a time (see below).
@@ -144,7 +148,7 @@ int make_layout(const decode_attn_shape_t& s, const decode_attn_policy_t& p, con
     std::vector<int64_t> pages(B);
     for (int b = 0; b < B; ++b) {
         if (seq_lens[b] < 0) return DA_ERR_INVALID_ARG;
-        if (ceil_div(seq_lens[b], P) > s.max_pages_per_seq) return DA_ERR_INVALID_ARG;
+        if (ceil_div(seq_lens[b], s.page_size) > s.max_pages_per_seq) return DA_ERR_INVALID_ARG;
         if (seq_lens[b] < prefix_tokens) return DA_ERR_INVALID_ARG;   // every sequence contains the prefix
         pages[b] = ceil_div(seq_lens[b] - prefix_tokens, P);
     }

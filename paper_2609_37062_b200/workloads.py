@@ -323,31 +323,34 @@ def config_tiny(device="cpu", layout="token_major") -> PagedWorkload:
 
 
 def config_long(device="cpu", context: int = 32768, layout="token_major", seed: int = 1,
-                table_seed: Optional[int] = None) -> PagedWorkload:
+                table_seed: Optional[int] = None, page_size: int = 16) -> PagedWorkload:
     """One sequence of `context` tokens, 32 query / 8 KV heads, head_dim 128."""
     return make_workload("long", [context], 32, 8, 128, seed=seed, layout=layout, device=device,
-                         table_seed=table_seed)
+                         table_seed=table_seed, page_size=page_size)
 
 
 def config_short_chat(device="cpu", batch: int = 64, layout="token_major", seed: int = 2,
-                      table_seed: Optional[int] = None) -> PagedWorkload:
+                      table_seed: Optional[int] = None, page_size: int = 16) -> PagedWorkload:
     return make_workload("short_chat", lengths_short_chat(batch, seed), 32, 8, 128, seed=seed,
-                         layout=layout, device=device, table_seed=table_seed)
+                         layout=layout, device=device, table_seed=table_seed, page_size=page_size)
 
 
 def config_shared_prefix(device="cpu", batch: int = 256, layout="token_major", seed: int = 3,
-                         prefix: int = 1536, table_seed: Optional[int] = None) -> PagedWorkload:
+                         prefix: int = 1536, table_seed: Optional[int] = None,
+                         page_size: int = 16) -> PagedWorkload:
     return make_workload("shared_prefix", lengths_shared_prefix(batch, seed, prefix), 32, 8, 128,
                          seed=seed, layout=layout, device=device, shared_prefix_tokens=prefix,
-                         table_seed=table_seed)
+                         table_seed=table_seed, page_size=page_size)
 
 
 def config_sweep_cell(context: int, batch: int, device="cpu", layout="token_major", seed: int = 4,
-                      alias_after: Optional[int] = None, table_seed: Optional[int] = None) -> PagedWorkload:
+                      alias_after: Optional[int] = None, table_seed: Optional[int] = None,
+                      page_size: int = 16) -> PagedWorkload:
     """One cell of the length x batch sweep: `batch` sequences of `context`
     tokens; sequence i has the same content in every batch size."""
     return make_workload(f"sweep_{context}x{batch}", [context] * batch, 32, 8, 128, seed=seed,
-                         layout=layout, device=device, alias_after=alias_after, table_seed=table_seed)
+                         layout=layout, device=device, alias_after=alias_after, table_seed=table_seed,
+                         page_size=page_size)
 
 
 def as_fp16(w: PagedWorkload) -> PagedWorkload:

@@ -177,11 +177,12 @@ def test_invalid_shapes_and_policies_are_rejected():
             assert e.value.status in (da.DA_ERR_INVALID_ARG, da.DA_ERR_UNSUPPORTED)
         else:
             assert e.value.status == code, (kw, e.value.status)
-    s = shape(B=1)
-    s.page_size = 32
-    with pytest.raises(da.DecodeAttnError) as e:
-        da.decode_attn_plan_layout(s, ok, L, 148, 2)
-    assert e.value.status == da.DA_ERR_UNSUPPORTED
+    for ps in (1, 8, 24, 48, 512):                           # pages hold 16, 32, 64, 128 or 256 tokens
+        s = shape(B=1)
+        s.page_size = ps
+        with pytest.raises(da.DecodeAttnError) as e:
+            da.decode_attn_plan_layout(s, ok, L, 148, 2)
+        assert e.value.status == da.DA_ERR_UNSUPPORTED
     s = shape(B=1)
     s.k_stride_token = 100                                   # not a multiple of 8 elements
     with pytest.raises(da.DecodeAttnError) as e:
@@ -189,6 +190,25 @@ def test_invalid_shapes_and_policies_are_rejected():
     assert e.value.status == da.DA_ERR_INVALID_ARG
     with pytest.raises(da.DecodeAttnError):
         layout([-1], ok)
+
+
+def test_layout_does_not_depend_on_the_page_size():
+    """The planner counts in 16-token tiles; the pool's page size only bounds the block table."""
+    lens = [33, 1000, 4097, 0, 257]
+    for pol in (da.make_policy(), da.make_policy(split_mode=da.DA_SPLIT_DETERMINISTIC, chunk_tokens=256),
+                da.make_policy(split_mode=da.DA_SPLIT_FIXED_COUNT, fixed_count=5)):
+        ref = None
+        for ps in (16, 32, 64, 128, 256):
+            s = da.make_shape(len(lens), 32, 8, 128, ps, 8192 * 16 // ps, 1 << 16, (ps * 8 * 128, 8 * 128, 128))
+            units = da.decode_attn_plan_layout(s, pol, lens, 148, 2)[0]
+            key = [(u.seq, u.kv_head, u.tok_begin, u.tok_end, u.slot, u.split_index, u.n_splits) for u in units]
+            ref = ref or key
+            assert key == ref
+    # the block-table bound does use the page size
+    s = da.make_shape(1, 32, 8, 128, 64, 4, 1 << 16, (64 * 8 * 128, 8 * 128, 128))
+    da.decode_attn_plan_layout(s, da.make_policy(), [256], 148, 2)
+    with pytest.raises(da.DecodeAttnError):
+        da.decode_attn_plan_layout(s, da.make_policy(), [257], 148, 2)
 
 
 def test_validate_block_table():
