@@ -8,7 +8,8 @@
 // unit's pages while the consumers finish the previous unit.  With a grid as
 // large as the work list every block has one unit.  The producer turns block-table entries into
 // TMA tile loads (cp.async.bulk.tensor over a 4-D map [dim, slot, head, page]
-// of each pool): one 16-token page of one KV head lands in shared memory as
+// of each pool): one 16-token tile of one KV head - a whole page, or 16 slots
+// of a larger one; "page" below means such a tile - lands in shared memory as
 // 16 rows x 128 bytes per half of the head dimension, 128-byte swizzled, with
 // an mbarrier counting the bytes.  A stage is four pages of K and of V; a
 // ring of stages keeps tens of KB in flight per block with no register cost.
