@@ -38,9 +38,10 @@
 // tensor memory (one takes the even, one the odd 32-token groups of a row and
 // one half of the output columns); one warp whose first lane issues the MMAs,
 // always the one - the next Q K^T or the next P V - whose inputs are ready;
-// one warp that issues the TMA boxes.  K_0, V_0, K_1, V_1, ... go through a
-// ring of four 32 KB stages; a stage is handed back by the tcgen05.commit of
-// the MMAs that read it.  Blocks are persistent (one per SM: the buffers fill
+// one warp that issues the TMA boxes.  K tiles and V tiles each go through a
+// ring of two 32 KB stages, filled independently (a K stage comes back after
+// Q K^T, a V stage only after P V); a stage is handed back by the
+// tcgen05.commit of the MMAs that read it.  Blocks are persistent (one per SM: the buffers fill
 // tensor memory); the barriers are invalidated and set up again for every
 // unit.  Every wait is bounded and also ends when another thread of the block
 // has given up; the block then records DA_ERR_TIMEOUT, skips its records and
@@ -48,6 +49,8 @@
 #pragma once
 
 #include <cuda_fp16.h>
+
+#include <type_traits>
 
 #include "kernel_mma.cuh"
 #include "umma.cuh"
@@ -122,13 +125,13 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
     // full[4]: a tile has landed; empty[4]: the MMAs reading it have completed; s_ready[2]: the logits
     // of a tile are complete; p_ready[2]: its weights are written (all softmax threads); o_ready[2]:
     // its output tile is complete (and its weights consumed); o_free[2]: the output tile was read;
-    // m_ready[2]: both halves of every row have published their maximum of the tile
+    // m_ready[2][4]: the threads that share 32 rows have published their maxima of the tile
     const uint32_t bar_full = bar_base, bar_empty = bar_base + 32, bar_s = bar_base + 64, bar_p = bar_base + 80;
-    const uint32_t bar_o = bar_base + 96, bar_ofree = bar_base + 112, bar_m = bar_base + 128;
-    constexpr int kBarriers = 18;
+    const uint32_t bar_o = bar_base + 96, bar_ofree = bar_base + 112, bar_m = bar_base + 128;   // m_ready: [2][4]
+    constexpr int kBarriers = 24;
     uint8_t* const sm_misc = gbase + (bar_base - base);
-    volatile uint32_t* const sm_tmem = reinterpret_cast<volatile uint32_t*>(sm_misc + 160);
-    volatile int* const sm_abort = reinterpret_cast<volatile int*>(sm_misc + 164);
+    volatile uint32_t* const sm_tmem = reinterpret_cast<volatile uint32_t*>(sm_misc + 320);
+    volatile int* const sm_abort = reinterpret_cast<volatile int*>(sm_misc + 324);
     constexpr int TPR = kUmmaThreadsPerRow, GP = kUmmaGroupsPerThread, OC = kUmmaOutColsPerThread;
     volatile float* const sm_max = reinterpret_cast<volatile float*>(sm_misc + 512);   // [2 buffers][TPR][128 rows]
     float* const sm_l = reinterpret_cast<float*>(sm_misc + 512 + 2 * TPR * 128 * 4);   // [TPR][128]: the threads' shares of the row sums
@@ -158,7 +161,7 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
         const int n_pages = n_tok >> 4;
         const int T = (n_tok + kUmmaTileTokens - 1) / kUmmaTileTokens;      // tiles
         if (tid == 0) {
-            DA_TRACE_STAMP(kUmmaTraceBase + unit_index, 0);
+            DA_TRACE_CLOCK(kUmmaTraceBase + unit_index, 0);
             // the barriers serve one unit: set up again for each (the block is past a barrier here,
             // nobody is still waiting on the previous unit's, and every arrival on them has landed)
             if (unit_index != first_unit)
@@ -167,45 +170,85 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
             for (int i = 0; i < 2; ++i) mbar_init(bar_p + 8 * i, kUmmaSoftmaxThreads);
             for (int i = 0; i < 2; ++i) mbar_init(bar_o + 8 * i, 1);
             for (int i = 0; i < 2; ++i) mbar_init(bar_ofree + 8 * i, kUmmaSoftmaxThreads);
-            for (int i = 0; i < 2; ++i) mbar_init(bar_m + 8 * i, kUmmaSoftmaxThreads);
+            for (int i = 0; i < 8; ++i) mbar_init(bar_m + 8 * i, 32 * kUmmaThreadsPerRow);
             mbar_init_fence();
         }
         __syncthreads();
 
         if (warp == kUmmaLoadWarp) {
-            // -------------------------------------------------------- TMA: K_0, V_0, K_1, V_1, ...
+            // -------------------------------------------------------- TMA: K tiles and V tiles
+            // K_j goes to stage (2j) % 4, V_j to stage (2j + 1) % 4, so K and V each have a ring of
+            // two.  A K stage comes back as soon as Q K^T of its tile has completed, a V stage only
+            // after P V: the two rings are filled independently (K at most two tiles ahead of V), so
+            // that K_{j+2} never queues behind the wait for V_{j+1}'s stage.  Page ids are fetched 32
+            // at a time (four tiles), one batch ahead, off the path of the copies.
             const uint64_t l2_policy = l2_policy_evict_first();
             const int32_t* bt = p.block_table + (int64_t)u.seq * p.max_pages_per_seq;
             const int ts = p.tile_shift, tile0 = u.tok_begin >> 4;         // 16-token tiles: 1 << ts per page
             const int pg = (lane >> 1) & 7, hf = lane & 1;                  // lane j < 16: box (16 tokens j / 2, half j % 2)
-            int page_id = 0, slot0 = 0;
-            bool ok = true;
-            for (int n = 0; n < 2 * T && ok; ++n) {
-                const int t = n >> 1, st = n % NS;
-                if ((n & 1) == 0) {
-                    // the tile's page ids, checked once, used for K and for V; a page past the
-                    // range is fetched from outside the pool, which the TMA unit fills with zeros
+            auto fetch_ids = [&](int batch) {                               // lane l: 16-token tile 32 batch + l
+                const int i = batch * 32 + lane;
+                return i < n_pages ? __ldg(bt + ((tile0 + i) >> ts)) : 0;
+            };
+            int cb = 0;                                                     // batch of the V cursor
+            int ids0 = fetch_ids(0), ids1 = fetch_ids(1);
+            auto issue = [&](int j, int n, const CUtensorMap* map) {
+                const int st = n % NS;
+                const int idx = j * 8 + pg;                                 // 16-token tile of this lane's box
+                int page_id = __shfl_sync(0xffffffffu, (j >> 2) == cb ? ids0 : ids1, ((j & 3) * 8 + pg) & 31);
+                if (idx >= n_pages) {
+                    // past the range: fetched from outside the pool, which the TMA unit fills with zeros
                     page_id = (int)p.num_pages;
-                    if (t * 8 + pg < n_pages) {
-                        page_id = __ldg(bt + ((tile0 + t * 8 + pg) >> ts));
-                        slot0 = ((tile0 + t * 8 + pg) & ((1 << ts) - 1)) << 4;
-                        if ((unsigned)page_id >= (unsigned)p.num_pages) {   // never hand TMA a page outside the pool
-                            record_status(p.status, DA_ERR_BAD_PAGE);
-                            page_id = 0;
-                        }
-                    }
+                } else if ((unsigned)page_id >= (unsigned)p.num_pages) {    // never hand TMA a page outside the pool
+                    record_status(p.status, DA_ERR_BAD_PAGE);
+                    page_id = 0;
                 }
-                if (n >= NS) {
-                    if (lane == 0) ok = umma_wait(bar_empty + 8 * st, ((n / NS) - 1) & 1, sm_abort);
-                    ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
-                    if (!ok) break;
-                }
+                const int slot0 = ((tile0 + idx) & ((1 << ts) - 1)) << 4;
                 const uint32_t bar = bar_full + 8 * st;
                 if (lane == 0) mbar_arrive_expect_tx(bar, kUmmaTileBytes);
                 __syncwarp();
                 if (lane < 16)
-                    tma_load_4d(ring_base + st * kUmmaTileBytes + hf * kUmmaHalfBytes + pg * 2048, (n & 1) ? v_map : k_map, bar,
-                                hf * 64, slot0, g, page_id, l2_policy);
+                    tma_load_4d(ring_base + st * kUmmaTileBytes + hf * kUmmaHalfBytes + pg * 2048, map, bar, hf * 64, slot0, g,
+                                page_id, l2_policy);
+            };
+            auto stage_free = [&](int n) {                                  // the stage of copy n was handed back
+                if (n < NS) return true;
+                bool f = false;
+                if (lane == 0) f = mbar_test_wait(bar_empty + 8 * (n % NS), ((n / NS) - 1) & 1);
+                return __shfl_sync(0xffffffffu, (int)f, 0) != 0;
+            };
+            int jk = 0, jv = 0;                                             // next K tile, next V tile
+            long long t_idle = clock64();
+            while (jv < T) {
+                bool did = false;
+                if (jk < T && jk - jv < 2 && stage_free(2 * jk)) {
+                    issue(jk, 2 * jk, k_map);
+                    ++jk;
+                    did = true;
+                }
+                if (jv < jk && stage_free(2 * jv + 1)) {
+                    issue(jv, 2 * jv + 1, v_map);
+                    ++jv;
+                    did = true;
+                    if ((jv & 3) == 0) {                                    // the V cursor enters the next batch
+                        ids0 = ids1;
+                        ++cb;
+                        ids1 = fetch_ids(cb + 1);
+                    }
+                }
+                if (did) {
+                    t_idle = clock64();
+                } else {
+                    bool stop = false;
+                    if (lane == 0) {
+                        stop = *sm_abort != 0;
+                        if (!stop && clock64() - t_idle > kWaitLimitCycles) {
+                            *sm_abort = 1;
+                            stop = true;
+                        }
+                    }
+                    if (__shfl_sync(0xffffffffu, (int)stop, 0) != 0) break;
+                }
             }
         } else if (warp == kUmmaMmaWarp) {
             // -------------------------------------------------------- MMAs (one lane)
@@ -223,7 +266,7 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
                 // S_j = Q K_j^T into logit buffer j % 2
                 auto qk = [&](int j) {
                     const int st = (2 * j) % NS, b = j & 1;
-                    if (j < 8) DA_TRACE_STAMP(kUmmaTraceBase + 512 + unit_index, j);
+                    if (j < 8) DA_TRACE_CLOCK(kUmmaTraceBase + 512 + unit_index, j);
                     umma::fence_after_thread_sync();
                     const uint64_t kd = k_desc0 + (uint64_t)(st * kStageUnits);
 #pragma unroll
@@ -237,7 +280,7 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
                 // O_j = P_j V_j into output buffer j % 2
                 auto pv = [&](int j) {
                     const int st = (2 * j + 1) % NS, b = j & 1;
-                    if (j < 8) DA_TRACE_STAMP(kUmmaTraceBase + 512 + unit_index, 8 + j);
+                    if (j < 8) DA_TRACE_CLOCK(kUmmaTraceBase + 512 + unit_index, 8 + j);
                     umma::fence_after_thread_sync();
                     const uint64_t vd = v_desc0 + (uint64_t)(st * kStageUnits);
                     const int ksteps = min(8, (n_tok - j * kUmmaTileTokens) >> 4);
@@ -252,7 +295,7 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
                             umma::mma_ts(od, a_hi + 16, vd + k * 128, idesc_pv, true);
                         }
                     }
-                    if (j < 8) DA_TRACE_STAMP(kUmmaTraceBase + 512 + unit_index, 16 + j);
+                    if (j < 8) DA_TRACE_CLOCK(kUmmaTraceBase + 512 + unit_index, 16 + j);
                     umma::commit(bar_empty + 8 * st);
                     umma::commit(bar_o + 8 * b);
                 };
@@ -264,21 +307,23 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
                 long long t_idle = clock64();
                 while (np < T) {
                     bool did = false;
-                    if (np < nq) {
-                        const int j = np, n = 2 * j + 1, b = j & 1;
-                        if (mbar_test_wait(bar_p + 8 * b, (j >> 1) & 1) && mbar_test_wait(bar_full + 8 * (n % NS), (n / NS) & 1) &&
-                            (j < 2 || mbar_test_wait(bar_ofree + 8 * b, ((j - 2) >> 1) & 1))) {
-                            pv(j);
-                            ++np;
-                            did = true;
-                        }
-                    }
-                    if (!did && nq < T) {
+                    // Q K^T first: the logits feed the softmax threads, which are the busier side;
+                    // P V only gates the fold and the logit buffer two tiles on.
+                    if (nq < T) {
                         const int j = nq, n = 2 * j, b = j & 1;
                         if (mbar_test_wait(bar_full + 8 * (n % NS), (n / NS) & 1) &&
                             (j < 2 || (np > j - 2 && mbar_test_wait(bar_o + 8 * b, ((j - 2) >> 1) & 1)))) {
                             qk(j);
                             ++nq;
+                            did = true;
+                        }
+                    }
+                    if (!did && np < nq) {
+                        const int j = np, n = 2 * j + 1, b = j & 1;
+                        if (mbar_test_wait(bar_p + 8 * b, (j >> 1) & 1) && mbar_test_wait(bar_full + 8 * (n % NS), (n / NS) & 1) &&
+                            (j < 2 || mbar_test_wait(bar_ofree + 8 * b, ((j - 2) >> 1) & 1))) {
+                            pv(j);
+                            ++np;
                             did = true;
                         }
                     }
@@ -323,7 +368,7 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); // visible to the tensor core's reads
             }
             block_sync(1, kUmmaSoftmaxThreads + 32);
-            if (tid == 0) DA_TRACE_STAMP(kUmmaTraceBase + unit_index, 1);
+            if (tid == 0) DA_TRACE_CLOCK(kUmmaTraceBase + unit_index, 1);
 
             const SeqInfo si = p.seq_info[seq];
             bool dead = p.run_mask != nullptr && __ldg(p.run_mask + seq) == 0;   // masked row: an empty record
@@ -346,7 +391,7 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
                 const int b = i & 1;
                 ok = umma_wait(bar_o + 8 * b, (i >> 1) & 1, sm_abort);
                 if (!ok) return;
-                if (tid == 0 && i < 8) DA_TRACE_STAMP(kUmmaTraceBase + 1024 + unit_index, 16 + i);
+                if (tid == 0 && i < 8) DA_TRACE_CLOCK(kUmmaTraceBase + 1024 + unit_index, 16 + i);
                 umma::fence_after_thread_sync();
                 const uint32_t oc = lane_base + kUmmaOutCol + b * 128 + hh * OC;
 #pragma unroll
@@ -363,7 +408,7 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
                         acc[32 * q + k] = fmaf(acc[32 * q + k], a, __uint_as_float(sg[q][k]) * c);
                 L = fmaf(L, a, l_prev * c);
                 M = Mn;
-                if (tid == 0 && i < 8) DA_TRACE_STAMP(kUmmaTraceBase + 1024 + unit_index, 24 + i);
+                if (tid == 0 && i < 8) DA_TRACE_CLOCK(kUmmaTraceBase + 1024 + unit_index, 24 + i);
             };
 
             for (int j = 0; j < T && ok; ++j) {
@@ -372,70 +417,80 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
                 const int n_here = min(kUmmaTileTokens, n_tok - tok0);      // a multiple of 16
                 ok = umma_wait(bar_s + 8 * b, (j >> 1) & 1, sm_abort);
                 if (!ok) break;
-                if (tid == 0 && j == 0) DA_TRACE_STAMP(kUmmaTraceBase + unit_index, 2);
-                if (tid == 0 && j < 8) DA_TRACE_STAMP(kUmmaTraceBase + 1024 + unit_index, j);
+                if (tid == 0 && j == 0) DA_TRACE_CLOCK(kUmmaTraceBase + unit_index, 2);
+                if (tid == 0 && j < 8) DA_TRACE_CLOCK(kUmmaTraceBase + 1024 + unit_index, j);
                 umma::fence_after_thread_sync();
                 const uint32_t sc = lane_base + b * 128;
-                // pass 1: the maximum of this thread's logits; the row's other parts are exchanged
-                // through shared memory (their logits may not be read once they start writing weights)
-                float mx = -INFINITY;
+                float m2 = 0.f, lsum = 0.f;
+                // A full tile (all but possibly a unit's last) needs no per-token bounds.
+                auto softmax_tile = [&](auto full_tag) {
+                    constexpr bool FULL = decltype(full_tag)::value;
+                    // pass 1: the maximum of this thread's logits; the row's other parts are exchanged
+                    // through shared memory (their logits may not be read once they start writing weights)
+                    float mx = -INFINITY;
 #pragma unroll
-                for (int q = 0; q < GP; ++q) umma::ld32(sc + (hh + q * TPR) * 32, sg[q]);
-                umma::wait_ld();
+                    for (int q = 0; q < GP; ++q) umma::ld32(sc + (hh + q * TPR) * 32, sg[q]);
+                    umma::wait_ld();
 #pragma unroll
-                for (int q = 0; q < GP; ++q)
+                    for (int q = 0; q < GP; ++q)
 #pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        if ((hh + q * TPR) * 32 + i < n_here) mx = fmaxf(mx, __uint_as_float(sg[q][i]));
-                sm_max[(b * TPR + hh) * 128 + r] = mx;
-                mbar_arrive(bar_m + 8 * b);
-                ok = umma_wait(bar_m + 8 * b, (j >> 1) & 1, sm_abort);
-                if (!ok) break;
+                        for (int i = 0; i < 32; ++i)
+                            if (FULL || (hh + q * TPR) * 32 + i < n_here) mx = fmaxf(mx, __uint_as_float(sg[q][i]));
+                    sm_max[(b * TPR + hh) * 128 + r] = mx;
+                    const uint32_t bm = bar_m + 8 * (b * 4 + (warp & 3));       // of the warps sharing these rows
+                    mbar_arrive(bm);
+                    ok = umma_wait(bm, (j >> 1) & 1, sm_abort);
+                    if (!ok) return;
 #pragma unroll
-                for (int q = 0; q < TPR; ++q) mx = fmaxf(mx, sm_max[(b * TPR + q) * 128 + r]);
-                const float m2 = mx * p.scale_log2;                          // the scale is positive
-                // pass 2: this thread's weights, written back over the logits as bf16 high and low parts
-                float lsum = 0.f;
-                auto weights = [&](const uint32_t (&s)[32], int col0) {
-                    uint32_t hi[16], lo[16];
+                    for (int q = 0; q < TPR; ++q) mx = fmaxf(mx, sm_max[(b * TPR + q) * 128 + r]);
+                    m2 = mx * p.scale_log2;                                      // the scale is positive
+                    // pass 2: this thread's weights, written back over the logits as bf16 high and low parts
+                    auto weights = [&](const uint32_t (&s)[32], int col0) {
+                        uint32_t hi[16], lo[16];
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        float p0 = 0.f, p1 = 0.f;
-                        if (col0 + 2 * i < n_here) p0 = ex2f(fmaf(__uint_as_float(s[2 * i]), p.scale_log2, -m2));
-                        if (col0 + 2 * i + 1 < n_here) p1 = ex2f(fmaf(__uint_as_float(s[2 * i + 1]), p.scale_log2, -m2));
-                        lsum += p0 + p1;
-                        if (F16) {
-                            // fp16 inputs: the weights are fp16 too, rounded, and so is the remainder
-                            const __half2 ph = __floats2half2_rn(p0, p1);
-                            const float2 pf = __half22float2(ph);
-                            const __half2 pl = __floats2half2_rn(p0 - pf.x, p1 - pf.y);
-                            hi[i] = *reinterpret_cast<const uint32_t*>(&ph);
-                            lo[i] = *reinterpret_cast<const uint32_t*>(&pl);
-                        } else {
-                            const uint32_t b0 = __float_as_uint(p0), b1 = __float_as_uint(p1);
-                            const float r0 = p0 - __uint_as_float(b0 & 0xffff0000u);   // exact
-                            const float r1 = p1 - __uint_as_float(b1 & 0xffff0000u);
-                            hi[i] = __byte_perm(b0, b1, 0x7632);             // upper halves: element 2i low, 2i+1 high
-                            lo[i] = __byte_perm(__float_as_uint(r0), __float_as_uint(r1), 0x7632);
+                        for (int i = 0; i < 16; ++i) {
+                            float p0 = 0.f, p1 = 0.f;
+                            if (FULL || col0 + 2 * i < n_here) p0 = ex2f(fmaf(__uint_as_float(s[2 * i]), p.scale_log2, -m2));
+                            if (FULL || col0 + 2 * i + 1 < n_here) p1 = ex2f(fmaf(__uint_as_float(s[2 * i + 1]), p.scale_log2, -m2));
+                            lsum += p0 + p1;
+                            if (F16) {
+                                // fp16 inputs: the weights are fp16 too, rounded, and so is the remainder
+                                const __half2 ph = __floats2half2_rn(p0, p1);
+                                const float2 pf = __half22float2(ph);
+                                const __half2 pl = __floats2half2_rn(p0 - pf.x, p1 - pf.y);
+                                hi[i] = *reinterpret_cast<const uint32_t*>(&ph);
+                                lo[i] = *reinterpret_cast<const uint32_t*>(&pl);
+                            } else {
+                                const uint32_t b0 = __float_as_uint(p0), b1 = __float_as_uint(p1);
+                                const float r0 = p0 - __uint_as_float(b0 & 0xffff0000u);   // exact
+                                const float r1 = p1 - __uint_as_float(b1 & 0xffff0000u);
+                                hi[i] = __byte_perm(b0, b1, 0x7632);             // upper halves: element 2i low, 2i+1 high
+                                lo[i] = __byte_perm(__float_as_uint(r0), __float_as_uint(r1), 0x7632);
+                            }
                         }
-                    }
-                    // the group's 32 logit columns become 16 columns of high parts, 16 of low parts
-                    umma::st16(sc + col0, hi);
-                    umma::st16(sc + col0 + 16, lo);
-                };
+                        // the group's 32 logit columns become 16 columns of high parts, 16 of low parts
+                        umma::st16(sc + col0, hi);
+                        umma::st16(sc + col0 + 16, lo);
+                    };
 #pragma unroll
-                for (int q = 0; q < GP; ++q) weights(sg[q], (hh + q * TPR) * 32);
+                    for (int q = 0; q < GP; ++q) weights(sg[q], (hh + q * TPR) * 32);
+                };
+                if (n_here == kUmmaTileTokens)
+                    softmax_tile(std::true_type());
+                else
+                    softmax_tile(std::false_type());
+                if (!ok) break;
                 umma::wait_st();
                 umma::fence_before_thread_sync();
                 mbar_arrive(bar_p + 8 * b);                                   // this tile's P V may start
-                if (tid == 0 && j < 8) DA_TRACE_STAMP(kUmmaTraceBase + 1024 + unit_index, 8 + j);
+                if (tid == 0 && j < 8) DA_TRACE_CLOCK(kUmmaTraceBase + 1024 + unit_index, 8 + j);
                 // while it runs, fold in the tile before
                 if (j >= 1) fold(j - 1);
                 m_prev = m2;
                 l_prev = lsum;
             }
             if (ok) fold(T - 1);
-            if (tid == 0) DA_TRACE_STAMP(kUmmaTraceBase + unit_index, 3);
+            if (tid == 0) DA_TRACE_CLOCK(kUmmaTraceBase + unit_index, 3);
             // the row sum is the sum of the threads' shares, added in a fixed order
             sm_l[hh * 128 + r] = L;
             block_sync(2, kUmmaSoftmaxThreads);
@@ -463,7 +518,7 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
                 }
                 bulk_store_commit_and_wait_read();
             }
-            if (tid == 0) DA_TRACE_STAMP(kUmmaTraceBase + unit_index, 4);
+            if (tid == 0) DA_TRACE_CLOCK(kUmmaTraceBase + unit_index, 4);
         }
         // the next unit reuses shared memory, tensor memory and the barriers
         umma::fence_before_thread_sync();
