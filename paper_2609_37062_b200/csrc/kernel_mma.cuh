@@ -487,6 +487,8 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
             }
             if (last_unit) pdl_launch_dependents();
             if (!last_unit) prefetch(nu, nxt);
+            // one answer for the whole block on whether a wait was given up (see below)
+            pfailed = block_sync_or(1, kConsumerThreads, pfailed || sm_flags[0] != 0);
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
 #pragma unroll
@@ -707,20 +709,21 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
         }
 
         // ------------------------------------------------------------ end of the unit
-        if (dev_len != u.seq_len) {                               // stale plan: void the result, report it
-            if (tid == 0) record_status(p.status, DA_ERR_STALE_PLAN);
-            failed = true;
-        }
+        const bool stale = dev_len != u.seq_len;                  // stale plan: void the result, report it
+        if (stale && tid == 0) record_status(p.status, DA_ERR_STALE_PLAN);
 #pragma unroll
         for (int off = 4; off <= 16; off <<= 1) {
             l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], off);
             l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], off);
         }
-        if (failed) {
+        // Every warp is done reading the previous unit's results.  A warp may have given up on a
+        // wait just before the others saw the flag: the barrier carries a vote, every warp gets
+        // the same answer, the unit's result is voided and the block leaves together.
+        const bool gave_up = block_sync_or(1, kConsumerThreads, failed || sm_flags[0] != 0);
+        if (gave_up || stale) {
             m_run[0] = m_run[1] = -INFINITY;
             l_run[0] = l_run[1] = 0.f;
         }
-        block_sync(1, kConsumerThreads);          // every warp is done reading the previous unit's results
         if (DUP) {
             // columns 4..7 carried the low parts of P for heads 0..3: lanes c = 2, 3 hand theirs to c = 0, 1
 #pragma unroll
@@ -747,7 +750,7 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
         block_sync(1, kConsumerThreads);
         block_finish<D, kMmaConsumerWarps, COLS, false>(p, u, G, sm_wo, sm_wm, sm_wl, tid, kConsumerThreads, 1);
         if (uid == ubeg && tid == 0) DA_TRACE_STAMP(blockIdx.x, 6);
-        if (failed && sm_flags[0] != 0) return;
+        if (gave_up) return;
         u = nu;
         cur = nxt;
     }
