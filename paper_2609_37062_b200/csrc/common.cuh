@@ -56,6 +56,7 @@ struct KernelParams {
     int32_t n_units;    // otherwise: the unit count
     int32_t n_work_blocks;  // fused plans: blocks at or beyond this index merge records instead of attending
     int32_t ticket_stride;  // elements between the two ticket arrays
+    int32_t hint_first_pages;  // tensor-core kernel: ask a block's first pages into L2 ahead of the dependency wait
 #ifdef DA_TRACE
     unsigned long long* trace;  // debug builds: 32 stamps per block, or NULL
 #endif

@@ -75,6 +75,14 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
         : "memory");
 }
 
+// The same box brought into L2 only: no shared memory, no barrier, nothing to wait for.
+__device__ __forceinline__ void tma_prefetch_l2_4d(const CUtensorMap* map, int c0, int c1, int c2, int c3, uint64_t l2_policy)
+{
+    asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global.tile.L2::cache_hint [%0, {%1, %2, %3, %4}], %5;"
+                 ::"l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "l"(l2_policy)
+                 : "memory");
+}
+
 __device__ __forceinline__ void tma_prefetch_descriptor(const CUtensorMap* map)
 {
     asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
@@ -233,6 +241,28 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
     // kernel launched before this one may have produced (q, new K/V rows, lengths, page
     // mappings) is read only past this point; with a programmatic dependency the lines above
     // overlap that kernel's tail.
+    if (MODE == kModeAttend && warp == 0 && p.hint_first_pages != 0) {
+        // Hints, while the kernel before this one drains (from a consumer warp, which has nothing to do
+        // until the first stage lands; the producer goes straight to its wait): the pages that will fill the ring first
+        // are asked into L2.  The mask and the page ids read here may be about to change; they steer
+        // prefetches only (the loads below read them again, behind the wait), and an L2 prefetch
+        // of the wrong line is harmless.
+        const int np = min((u.tok_end - u.tok_begin + 15) >> 4, NS * kPagesPerStage);
+        const bool masked = p.run_mask != nullptr && (u.kv_head >> 16) == 0 && __ldcg(p.run_mask + u.seq) == 0;
+        if (lane < np && !masked) {
+            const int tile = (u.tok_begin >> 4) + lane;
+            const int id = __ldcg(p.block_table + (int64_t)u.seq * p.max_pages_per_seq + (tile >> p.tile_shift));
+            if ((unsigned)id < (unsigned)p.num_pages) {
+                const int slot0 = (tile & ((1 << p.tile_shift) - 1)) << 4;
+                const uint64_t hint_policy = l2_policy_evict_first();
+#pragma unroll
+                for (int hf = 0; hf < Cfg::kHalves; ++hf) {
+                    tma_prefetch_l2_4d(&k_map, hf * 64, slot0, u.kv_head & 0xffff, id, hint_policy);
+                    tma_prefetch_l2_4d(&v_map, hf * 64, slot0, u.kv_head & 0xffff, id, hint_policy);
+                }
+            }
+        }
+    }
     pdl_wait_primary();
 
     if (warp == kMmaConsumerWarps) {
