@@ -229,9 +229,14 @@ int decode_attn_plan_destroy(decode_attn_plan_t *plan);
  *
  * The kernel is launched with a programmatic dependency on whatever precedes
  * it on `stream`: its blocks may become resident and fetch the plan's work
- * list while that work drains, but q, K/V, seq_lens, block_table and run_mask
- * are read only after it has completed, so ordinary stream order holds for
- * every caller-visible buffer.
+ * list while that work drains, but what it computes with - q, K/V, seq_lens,
+ * block_table and run_mask - is read only after it has completed, so ordinary
+ * stream order holds for every caller-visible buffer.  One thing happens
+ * earlier in plans that give every block a single unit: block_table and
+ * run_mask are also read before that point to choose K/V lines to prefetch
+ * into L2.  Those early values are used for nothing else and are read again
+ * afterwards, so a kernel that is still writing them does no harm; the
+ * buffers only have to be mapped device memory when the launch is enqueued.
  * ------------------------------------------------------------------------- */
 int decode_attn_run(const decode_attn_plan_t *plan, const void *q, const void *k_cache,
                     const void *v_cache, const int32_t *block_table, const int32_t *seq_lens, void *out,
