@@ -559,16 +559,30 @@ int decode_attn_run_ex(const decode_attn_plan_t* pl, const decode_attn_run_args_
         int rc = simt_launch(fn, kp, (unsigned)pl->grid, stream);
         if (rc != DA_OK) return rc;
     } else {
-        if (umma) {
-            // the shared prefix first: the units at the front of the work list, dealt to one block per SM
-            const unsigned n_front = (unsigned)pl->layout.n_front_units;
+        const unsigned n_front = (unsigned)pl->layout.n_front_units;
+        const bool pair = umma && n_front > 0 && pl->grid > 0;
+        if (umma && n_front > 0 && !pair) {
+            // only shared-prefix units: dealt to one block per SM
             int rc = umma_prefix_launch(pl->shape, pl->group, kp, n_front, std::min<unsigned>(n_front, (unsigned)pl->sm_count),
                                         stream);
             if (rc != DA_OK) return rc;
         }
         if (pl->grid > 0) {
-            int rc = mma_launch(pl->shape, pl->group, kp, (unsigned)pl->grid, stream,
+            KernelParams k1 = kp;
+            k1.early_trigger = pair;
+            int rc = mma_launch(pl->shape, pl->group, k1, (unsigned)pl->grid, stream,
                                 pl->policy.shared_prefix_tokens > 0 && !umma);
+            if (rc != DA_OK) return rc;
+        }
+        if (pair) {
+            // The bandwidth-bound kernel goes first and the tcgen05 kernel for the shared prefix
+            // follows as the second of a pair: its blocks (one per SM, each wanting a whole SM's
+            // shared memory) move in as the first kernel's blocks leave, so its start-up and its
+            // first tiles fill the other kernel's ragged end instead of following it.
+            KernelParams k2 = kp;
+            k2.late_wait = 1;
+            int rc = umma_prefix_launch(pl->shape, pl->group, k2, n_front, std::min<unsigned>(n_front, (unsigned)pl->sm_count),
+                                        stream);
             if (rc != DA_OK) return rc;
         }
     }

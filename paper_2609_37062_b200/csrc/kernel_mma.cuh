@@ -264,6 +264,7 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
         }
     }
     pdl_wait_primary();
+    if (p.early_trigger) pdl_launch_dependents();             // first of a pair: see KernelParams
 
     if (warp == kMmaConsumerWarps) {
         // ------------------------------------------------------------ producer

@@ -151,8 +151,10 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
     __syncthreads();
     umma::fence_after_thread_sync();
     const uint32_t tmem = *sm_tmem;
-    // Only this block's own state was touched so far.
-    pdl_wait_primary();
+    // Only this block's own state was touched so far.  As the second of a pair (see KernelParams)
+    // the kernel was let go only after the first one's own wait, so what precedes the pair is
+    // complete and nothing the first one writes is read here.
+    if (!p.late_wait) pdl_wait_primary();
 
     for (int unit_index = first_unit; unit_index < n_units && *sm_abort == 0; unit_index += unit_stride) {
         const decode_attn_unit_t u = load_unit(p.units, unit_index);
@@ -526,6 +528,7 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
         umma::fence_after_thread_sync();
     }
     if (tid == 0 && *sm_abort != 0) record_status(p.status, DA_ERR_TIMEOUT);
+    if (p.late_wait) pdl_wait_primary();                      // this kernel's end then implies the first one's
     pdl_launch_dependents();
     if (warp == kUmmaMmaWarp) umma::tmem_dealloc(tmem, kUmmaTmemCols);
 }
