@@ -344,11 +344,15 @@ KernelParams make_params(const decode_attn_plan_t* pl, const decode_attn_run_arg
     kp.fused = pl->policy.fuse_combine;
     kp.grid_exit = pl->policy.capacity_batch > 0;
     kp.n_units = (int32_t)pl->layout.units.size();
-    // Plans that give every block a single unit spend a visible share of the step waiting for the
-    // first pages: there the kernel asks for them ahead of the dependency wait (measured: 24.9 ->
-    // 23.4 us on one 32k sequence; plans with several units per block lose 1-3 % and keep it off).
-    kp.hint_first_pages = pl->kernel != DA_KERNEL_SIMT && pl->policy.capacity_batch == 0 &&
-                          (int64_t)pl->layout.units.size() - pl->layout.n_front_units <= pl->work_grid;
+    // The tensor-core kernel asks the first pages of every block into L2 ahead of its dependency
+    // wait.  Two stages' worth when a block has a single unit (the opening burst is then a visible
+    // share of the step: 24.9 -> 23.0 us on one 32k sequence), one stage's worth otherwise
+    // (short_chat 20.0 -> 19.1 us); more than that costs more than it brings.
+    if (pl->kernel != DA_KERNEL_SIMT) {
+        const bool single = pl->policy.capacity_batch == 0 &&
+                            (int64_t)pl->layout.units.size() - pl->layout.n_front_units <= pl->work_grid;
+        kp.hint_first_pages = single ? 8 : 4;
+    }
 #ifdef DA_TRACE
     kp.trace = g_trace_buffer;
 #endif

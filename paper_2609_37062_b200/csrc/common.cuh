@@ -56,7 +56,7 @@ struct KernelParams {
     int32_t n_units;    // otherwise: the unit count
     int32_t n_work_blocks;  // fused plans: blocks at or beyond this index merge records instead of attending
     int32_t ticket_stride;  // elements between the two ticket arrays
-    int32_t hint_first_pages;  // tensor-core kernel: ask a block's first pages into L2 ahead of the dependency wait
+    int32_t hint_first_pages;  // tensor-core kernel: pages of a block's first unit asked into L2 ahead of the dependency wait
     // A plan that runs two partial kernels (shared prefix on tcgen05 + everything else) launches them as a
     // pair whose members do not depend on each other: the first lets its successor go as soon as its own
     // dependency wait is over (early_trigger), the second starts without waiting and waits before it exits

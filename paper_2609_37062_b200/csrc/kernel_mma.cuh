@@ -247,7 +247,7 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
         // are asked into L2.  The mask and the page ids read here may be about to change; they steer
         // prefetches only (the loads below read them again, behind the wait), and an L2 prefetch
         // of the wrong line is harmless.
-        const int np = min((u.tok_end - u.tok_begin + 15) >> 4, NS * kPagesPerStage);
+        const int np = min((u.tok_end - u.tok_begin + 15) >> 4, p.hint_first_pages);
         const bool masked = p.run_mask != nullptr && (u.kv_head >> 16) == 0 && __ldcg(p.run_mask + u.seq) == 0;
         if (lane < np && !masked) {
             const int tile = (u.tok_begin >> 4) + lane;
