@@ -232,9 +232,9 @@ int decode_attn_plan_destroy(decode_attn_plan_t *plan);
  * list while that work drains, but what it computes with - q, K/V, seq_lens,
  * block_table and run_mask - is read only after it has completed, so ordinary
  * stream order holds for every caller-visible buffer.  One thing happens
- * earlier in plans that give every block a single unit: block_table and
- * run_mask are also read before that point to choose K/V lines to prefetch
- * into L2.  Those early values are used for nothing else and are read again
+ * earlier in the tensor-core kernel: block_table and run_mask are also read
+ * before that point to choose a few K/V lines to prefetch into L2.  Those
+ * early values are used for nothing else and are read again
  * afterwards, so a kernel that is still writing them does no harm; the
  * buffers only have to be mapped device memory when the launch is enqueued.
  * ------------------------------------------------------------------------- */
