@@ -69,7 +69,7 @@ typedef enum {
 } da_split_mode_t;
 
 typedef enum {
-    DA_KERNEL_AUTO = 0,     /* tensor-core kernel when the GQA group has >= 2 heads, else SIMT; with
+    DA_KERNEL_AUTO = 0,     /* MMA_TMA (every supported head_dim and group size); with
                                shared_prefix_tokens: UMMA_PREFIX where it applies, else MMA_TMA       */
     DA_KERNEL_SIMT = 1,     /* CUDA-core kernel, 16-byte vectorised global loads                      */
     DA_KERNEL_MMA_TMA = 2,  /* TMA-staged pages in shared memory, mma.sync (bf16 or fp16) for QK^T, PV  */
