@@ -492,16 +492,19 @@ __device__ __forceinline__ void fused_merge_blocks(const KernelParams& p, int G,
 template <int D, int R, int COLS, bool DUP>
 __device__ __forceinline__ void block_finish(const KernelParams& p, const decode_attn_unit_t& u, int G,
                                              const float* src_o, const float* src_m, const float* src_l, int tid,
-                                             int nthreads, int bar_id)
+                                             int nthreads, int bar_id, int head_first = 0, int head_count = -1,
+                                             bool publish = true)
 {
+    // heads [head_first, head_first + head_count) of the group, held in source columns 0 .. head_count - 1
+    if (head_count < 0) head_count = G;
     constexpr int D4 = D / 4;
     constexpr int kUnroll = R <= 4 ? R : 1;     // many row groups: keep the loop rolled, registers matter more
     const int Hq = p.num_q_heads;
     const int h0 = u.kv_head * G;
     const int RF = rec_floats(G, D);
     float* const rec = (u.slot >= 0) ? p.ws + ((int64_t)u.slot * p.num_kv_heads + u.kv_head) * RF : nullptr;
-    for (int task = tid; task < G * D4; task += nthreads) {
-        const int h = task / D4, d4 = task % D4;
+    for (int task = tid; task < head_count * D4; task += nthreads) {
+        const int h = task / D4, d4 = task % D4;          // source column h is head head_first + h
         float M = -INFINITY;
 #pragma unroll kUnroll
         for (int r = 0; r < R; ++r) M = fmaxf(M, src_m[r * COLS + h]);
@@ -530,15 +533,15 @@ __device__ __forceinline__ void block_finish(const KernelParams& p, const decode
             } else {
                 o = make_float4(0.f, 0.f, 0.f, 0.f);
             }
-            store_out4(p.out, ((int64_t)u.seq * Hq + h0 + h) * D + d4 * 4, o, p.out_kind);
+            store_out4(p.out, ((int64_t)u.seq * Hq + h0 + head_first + h) * D + d4 * 4, o, p.out_kind);
             if (p.lse != nullptr && d4 == 0)
-                p.lse[(int64_t)u.seq * Hq + h0 + h] = (ls > 0.f) ? (M + log2f(ls)) * kLn2 : -INFINITY;
+                p.lse[(int64_t)u.seq * Hq + h0 + head_first + h] = (ls > 0.f) ? (M + log2f(ls)) * kLn2 : -INFINITY;
         } else {
-            __stcg(reinterpret_cast<float4*>(rec) + task, o);
-            if (d4 == 0) __stcg(reinterpret_cast<float2*>(rec + G * D) + h, make_float2(M, ls));
+            __stcg(reinterpret_cast<float4*>(rec) + head_first * D4 + task, o);
+            if (d4 == 0) __stcg(reinterpret_cast<float2*>(rec + G * D) + head_first + h, make_float2(M, ls));
         }
     }
-    if (rec == nullptr || !p.fused) return;
+    if (rec == nullptr || !p.fused || !publish) return;
     // The barrier orders every thread's record stores before thread 0's fence, which publishes
     // them device-wide ahead of the arrival.
     block_sync(bar_id, nthreads);

@@ -56,8 +56,8 @@ struct MmaCfg {
     static constexpr int kPageBytes = kHalves * kBoxBytes;      // one page of one tensor
     static constexpr int kTensorBytes = kPagesPerStage * kPageBytes;
     static constexpr int kStageBytes = 2 * kTensorBytes;        // K then V
-    static constexpr int kColsOut = DUP ? 4 : 8;                // output columns a warp hands to the block merge
-    static constexpr int kStages = (D == 128) ? (DUP ? 3 : 2) : 6;   // two blocks per SM must fit
+    static constexpr int kColsOut = 4;                          // output columns a warp hands to the block merge at a time
+    static constexpr int kStages = (D == 128) ? 3 : 6;         // two blocks per SM must fit
     static constexpr int kBarrierBytes = 1024;                  // barriers + small state, keeps tiles 1 KB aligned
     static constexpr int kScratchBytes = kMmaConsumerWarps * kColsOut * D * 4 + 256;   // warps' results for the merge
     static constexpr int kSmemBytes = kStages * kStageBytes + kBarrierBytes + kScratchBytes + 1024;  // + alignment slack
@@ -762,24 +762,33 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
 #pragma unroll
                 for (int i = 0; i < 4; ++i) oacc[mt][i] += __shfl_down_sync(0xffffffffu, oacc[mt][i], 2);
         }
-        if (!DUP || c < 2) {
-            if (r == 0) {
-                sm_wm[warp * COLS + 2 * c] = m_run[0];
-                sm_wm[warp * COLS + 2 * c + 1] = m_run[1];
-                sm_wl[warp * COLS + 2 * c] = l_run[0];
-                sm_wl[warp * COLS + 2 * c + 1] = l_run[1];
-            }
-            float* wo = sm_wo + warp * COLS * D;
+        // The warps' states meet in the block's scratch four heads at a time (it holds [4 warps][4
+        // columns][D]): heads 4q .. 4q+3 live in lanes c = 2q, 2q+1 (all of a duplicated group in c = 0, 1).
 #pragma unroll
-            for (int mt = 0; mt < D / 16; ++mt) {
-                wo[(2 * c) * D + mt * 16 + r] = oacc[mt][0];
-                wo[(2 * c + 1) * D + mt * 16 + r] = oacc[mt][1];
-                wo[(2 * c) * D + mt * 16 + r + 8] = oacc[mt][2];
-                wo[(2 * c + 1) * D + mt * 16 + r + 8] = oacc[mt][3];
+        for (int q = 0; q < (DUP ? 1 : 2); ++q) {
+            if (4 * q >= G) break;
+            if (q > 0) block_sync(1, kConsumerThreads);                     // the scratch is free again
+            if ((c >> 1) == q) {
+                const int lc = 2 * (c & 1);                                 // local columns lc, lc + 1
+                if (r == 0) {
+                    sm_wm[warp * COLS + lc] = m_run[0];
+                    sm_wm[warp * COLS + lc + 1] = m_run[1];
+                    sm_wl[warp * COLS + lc] = l_run[0];
+                    sm_wl[warp * COLS + lc + 1] = l_run[1];
+                }
+                float* wo = sm_wo + (warp * COLS + lc) * D;
+#pragma unroll
+                for (int mt = 0; mt < D / 16; ++mt) {
+                    wo[mt * 16 + r] = oacc[mt][0];
+                    wo[D + mt * 16 + r] = oacc[mt][1];
+                    wo[mt * 16 + r + 8] = oacc[mt][2];
+                    wo[D + mt * 16 + r + 8] = oacc[mt][3];
+                }
             }
+            block_sync(1, kConsumerThreads);
+            block_finish<D, kMmaConsumerWarps, COLS, false>(p, u, G, sm_wo, sm_wm, sm_wl, tid, kConsumerThreads, 1, 4 * q,
+                                                            min(4, G - 4 * q), DUP || 4 * (q + 1) >= G);
         }
-        block_sync(1, kConsumerThreads);
-        block_finish<D, kMmaConsumerWarps, COLS, false>(p, u, G, sm_wo, sm_wm, sm_wl, tid, kConsumerThreads, 1);
         if (uid == ubeg && tid == 0) DA_TRACE_STAMP(blockIdx.x, 6);
         if (gave_up) return;
         u = nu;
