@@ -74,7 +74,7 @@ int validate_policy(const decode_attn_shape_t& s, const decode_attn_policy_t& p)
         if (p.fuse_combine || p.capacity_batch > 0 || p.split_mode == DA_SPLIT_FIXED_COUNT) return DA_ERR_UNSUPPORTED;
         const int G = s.num_q_heads / s.num_kv_heads;
         if (p.kernel == DA_KERNEL_UMMA_PREFIX) {
-            if (s.head_dim != 128 || kUmmaPrefixRows % G != 0) return DA_ERR_UNSUPPORTED;
+            if (s.head_dim != 128) return DA_ERR_UNSUPPORTED;
         } else if (p.kernel == DA_KERNEL_SIMT || G > 4) {
             return DA_ERR_UNSUPPORTED;
         }

@@ -33,7 +33,7 @@ def one_case(rng, index, any_page_size=False):
     if mode == da.DA_SPLIT_DETERMINISTIC:
         pol["chunk_tokens"] = rng.choice([16, 32, 64, 256, 1024])
     prefix = 0
-    if rng.random() < 0.25 and G in (1, 2, 4):
+    if rng.random() < 0.25:                       # (groups of 5+ heads: the tcgen05 prefix kernel only)
         prefix = (rng.choice([16, 128, 160, 512, 1040]) + ps - 1) // ps * ps
         lens = [prefix + n for n in lens]
         pol = dict(shared_prefix_tokens=prefix, split_mode=rng.choice([da.DA_SPLIT_AUTO, da.DA_SPLIT_DETERMINISTIC]),
