@@ -35,8 +35,9 @@
 //                  half row in shared memory and sends it with one bulk copy.
 //
 // Threads: eight warps for softmax, merge and epilogue, two per 32 lanes of
-// tensor memory (one takes the even, one the odd 32-token groups of a row and
-// one half of the output columns); one warp whose first lane issues the MMAs,
+// tensor memory (each takes one half of a row's 128 tokens and one half of
+// the output columns, and moves them with few, large tensor-memory accesses:
+// a 64-column load, two 32-column stores); one warp whose first lane issues the MMAs,
 // always the one - the next Q K^T or the next P V - whose inputs are ready;
 // one warp that issues the TMA boxes.  K tiles and V tiles each go through a
 // ring of two 32 KB stages, filled independently (a K stage comes back after
@@ -348,7 +349,7 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
         } else {
             // -------------------------------------------------------- query rows, softmax, merge, epilogue
             // TPR threads per row: thread (quarter q, lane) of part hh = warp / 4 owns row r = 32 q +
-            // lane, the 32-token groups hh, hh + TPR, ... of a tile's logits, and output columns
+            // lane, tokens [64 hh, 64 hh + 64) of a tile's logits, and output columns
             // [OC hh, OC hh + OC).
             const int hh = warp >> 2;
             const int r = (warp & 3) * 32 + lane;                           // row of the tile = lane of tensor memory
@@ -386,7 +387,8 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
             for (int i = 0; i < OC; ++i) acc[i] = 0.f;
             float M = -INFINITY, L = 0.f;       // running maximum (log2 domain), this thread's share of the row sum
             float m_prev = 0.f, l_prev = 0.f;   // of the tile whose output is still to be folded in
-            uint32_t sg[GP < 2 ? 2 : GP][32];      // logits of the thread's groups; also the output tile on its way in
+            static_assert(GP == 2 && OC == 64, "a thread owns 64 consecutive logit columns and 64 output columns");
+            uint32_t sg[64];                        // logits of the thread's columns; also the output tile on its way in
             bool ok = true;
 
             // folds tile i's output into the running state
@@ -398,7 +400,7 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
                 umma::fence_after_thread_sync();
                 const uint32_t oc = lane_base + kUmmaOutCol + b * 128 + hh * OC;
 #pragma unroll
-                for (int q = 0; q < OC / 32; ++q) umma::ld32(oc + 32 * q, sg[q]);
+                umma::ld64(oc, sg);
                 umma::wait_ld();
                 umma::fence_before_thread_sync();
                 mbar_arrive(bar_ofree + 8 * b);                              // the buffer may be overwritten
@@ -408,7 +410,7 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
                 for (int q = 0; q < OC / 32; ++q)
 #pragma unroll
                     for (int k = 0; k < 32; ++k)
-                        acc[32 * q + k] = fmaf(acc[32 * q + k], a, __uint_as_float(sg[q][k]) * c);
+                        acc[32 * q + k] = fmaf(acc[32 * q + k], a, __uint_as_float(sg[32 * q + k]) * c);
                 L = fmaf(L, a, l_prev * c);
                 M = Mn;
                 if (tid == 0 && i < 8) DA_TRACE_CLOCK(kUmmaTraceBase + 1024 + unit_index, 24 + i);
@@ -432,13 +434,13 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
                     // through shared memory (their logits may not be read once they start writing weights)
                     float mx = -INFINITY;
 #pragma unroll
-                    for (int q = 0; q < GP; ++q) umma::ld32(sc + (hh + q * TPR) * 32, sg[q]);
+                    umma::ld64(sc + hh * 64, sg);                           // columns 64 hh .. 64 hh + 63
                     umma::wait_ld();
 #pragma unroll
                     for (int q = 0; q < GP; ++q)
 #pragma unroll
                         for (int i = 0; i < 32; ++i)
-                            if (FULL || (hh + q * TPR) * 32 + i < n_here) mx = fmaxf(mx, __uint_as_float(sg[q][i]));
+                            if (FULL || (hh * GP + q) * 32 + i < n_here) mx = fmaxf(mx, __uint_as_float(sg[32 * q + i]));
                     sm_max[(b * TPR + hh) * 128 + r] = mx;
                     const uint32_t bm = bar_m + 8 * (b * 4 + (warp & 3));       // of the warps sharing these rows
                     mbar_arrive(bm);
@@ -448,8 +450,8 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
                     for (int q = 0; q < TPR; ++q) mx = fmaxf(mx, sm_max[(b * TPR + q) * 128 + r]);
                     m2 = mx * p.scale_log2;                                      // the scale is positive
                     // pass 2: this thread's weights, written back over the logits as bf16 high and low parts
-                    auto weights = [&](const uint32_t (&s)[32], int col0) {
-                        uint32_t hi[16], lo[16];
+                    auto weights = [&](const uint32_t* s, int col0) {
+                        uint32_t hl[32];                                     // 16 high parts, then 16 low parts
 #pragma unroll
                         for (int i = 0; i < 16; ++i) {
                             float p0 = 0.f, p1 = 0.f;
@@ -461,22 +463,23 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
                                 const __half2 ph = __floats2half2_rn(p0, p1);
                                 const float2 pf = __half22float2(ph);
                                 const __half2 pl = __floats2half2_rn(p0 - pf.x, p1 - pf.y);
-                                hi[i] = *reinterpret_cast<const uint32_t*>(&ph);
-                                lo[i] = *reinterpret_cast<const uint32_t*>(&pl);
+                                hl[i] = *reinterpret_cast<const uint32_t*>(&ph);
+                                hl[16 + i] = *reinterpret_cast<const uint32_t*>(&pl);
                             } else {
                                 const uint32_t b0 = __float_as_uint(p0), b1 = __float_as_uint(p1);
                                 const float r0 = p0 - __uint_as_float(b0 & 0xffff0000u);   // exact
                                 const float r1 = p1 - __uint_as_float(b1 & 0xffff0000u);
-                                hi[i] = __byte_perm(b0, b1, 0x7632);             // upper halves: element 2i low, 2i+1 high
-                                lo[i] = __byte_perm(__float_as_uint(r0), __float_as_uint(r1), 0x7632);
+                                hl[i] = __byte_perm(b0, b1, 0x7632);             // upper halves: element 2i low, 2i+1 high
+                                hl[16 + i] = __byte_perm(__float_as_uint(r0), __float_as_uint(r1), 0x7632);
                             }
                         }
-                        // the group's 32 logit columns become 16 columns of high parts, 16 of low parts
-                        umma::st16(sc + col0, hi);
-                        umma::st16(sc + col0 + 16, lo);
+                        // the group's 32 logit columns become 16 columns of high parts, 16 of low parts, in one
+                        // store: fewer, larger accesses to tensor memory disturb the MMAs less (four stores of
+                        // 16 columns per thread and tile instead of two of 32 cost the kernel 2 us of 20)
+                        umma::st32(sc + col0, hl);
                     };
 #pragma unroll
-                    for (int q = 0; q < GP; ++q) weights(sg[q], (hh + q * TPR) * 32);
+                    for (int q = 0; q < GP; ++q) weights(sg + 32 * q, (hh * GP + q) * 32);
                 };
                 if (n_here == kUmmaTileTokens)
                     softmax_tile(std::true_type());
