@@ -42,7 +42,7 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the partial kernel, from the
 # ncu capture summarised under profiles/ (null until a capture of that workload exists).
 NCU_TRAFFIC_BYTES = {
-    "long_32k": 134_292_000 + 4_551_000,          # profiles/decode_attn_mma_kernel_long_32k.md
+    "long_32k": 134_293_000 + 3_623_000,          # profiles/decode_attn_mma_kernel_long_32k.md
     "sweep_8192x64": 2_148_308_000 + 4_320_000,   # profiles/decode_attn_mma_kernel_sweep_8192x64.md
 }
 
