@@ -53,7 +53,8 @@ struct decode_attn_plan {
     char* dev = nullptr;
     char* pinned = nullptr;
     size_t upload_bytes = 0;
-    size_t off_units = 0, off_seq_info = 0, off_block_begin = 0, off_status = 0, off_tickets = 0, total_bytes = 0;
+    size_t off_units = 0, off_seq_info = 0, off_block_begin = 0, off_unit_rank = 0, off_status = 0, off_tickets = 0,
+           total_bytes = 0;
     int max_bins = 0;        // > 0: the units are packed into per-block ranges (persistent tensor-core kernel)
     cudaStream_t stream = nullptr;
     cudaEvent_t upload_done = nullptr;  // last refresh of the device work list
@@ -286,6 +287,15 @@ int device_sm_count(int dev, int* out)
     return DA_OK;
 }
 
+// The kernel's redistribution under a RUN mask reads the binned units by cost rank, packed into a
+// word each: work lists of up to kMaxRanked units and batches below 2^20 - 1 sequences.
+constexpr int kMaxRanked = 2560;
+bool ranked_fits(const decode_attn_plan_t* pl)
+{
+    return pl->max_bins > 0 && !pl->layout.rank_pos.empty() && pl->layout.rank_pos.size() <= (size_t)kMaxRanked &&
+           pl->shape.batch < 0xfffff;
+}
+
 void fill_host_mirror(decode_attn_plan_t* pl)
 {
     DevHeader* hdr = reinterpret_cast<DevHeader*>(pl->pinned);
@@ -307,6 +317,18 @@ void fill_host_mirror(decode_attn_plan_t* pl)
         const std::vector<int32_t>& src = pl->layout.block_begin;
         const int32_t end = (int32_t)pl->layout.units.size();
         for (int64_t i = 0; i <= pl->grid; ++i) bb[i] = i < (int64_t)src.size() ? src[i] : end;
+        // every binned unit by cost rank: its 16-token tiles, its sequence (-1: no RUN mask applies,
+        // a shared-prefix unit) and where it sits in the work list
+        uint32_t* ur = reinterpret_cast<uint32_t*>(pl->pinned + pl->off_unit_rank);
+        if (ranked_fits(pl)) {
+            const int32_t first = pl->layout.n_front_units;
+            for (size_t j = 0; j < pl->layout.rank_pos.size(); ++j) {
+                const int32_t pos = pl->layout.rank_pos[j];
+                const decode_attn_unit_t& u = pl->layout.units[pos];
+                const uint32_t seq = (u.kv_head >> 16) ? 0xfffffu : (uint32_t)u.seq;
+                ur[j] = seq << 12 | (uint32_t)(pos - first);
+            }
+        }
     }
 }
 
@@ -328,6 +350,9 @@ KernelParams make_params(const decode_attn_plan_t* pl, const decode_attn_run_arg
     kp.units = reinterpret_cast<const decode_attn_unit_t*>(pl->dev + pl->off_units);
     kp.seq_info = reinterpret_cast<const SeqInfo*>(pl->dev + pl->off_seq_info);
     kp.block_begin = pl->max_bins > 0 ? reinterpret_cast<const int32_t*>(pl->dev + pl->off_block_begin) : nullptr;
+    kp.unit_rank = reinterpret_cast<const uint32_t*>(pl->dev + pl->off_unit_rank);
+    kp.n_ranked = ranked_fits(pl) ? (int32_t)pl->layout.rank_pos.size() : 0;
+    kp.first_binned = pl->layout.n_front_units;
     kp.tickets = reinterpret_cast<int32_t*>(pl->dev + pl->off_tickets);
     kp.ticket_stride = (int32_t)(pl->max_batch * s.num_kv_heads);
     kp.batch = s.batch;
@@ -442,7 +467,10 @@ int decode_attn_plan(const decode_attn_shape_t* shape, const decode_attn_policy_
     pl->off_units = align_up(sizeof(DevHeader), 32);
     pl->off_seq_info = pl->off_units + align_up((size_t)std::max<int64_t>(pl->max_units, 1) * sizeof(decode_attn_unit_t), 32);
     pl->off_block_begin = pl->off_seq_info + align_up((size_t)std::max<int64_t>(pl->max_batch, 1) * sizeof(SeqInfo), 32);
-    pl->upload_bytes = pl->off_block_begin + align_up((size_t)(pl->grid + 1) * sizeof(int32_t), 32);
+    pl->off_unit_rank = pl->off_block_begin + align_up((size_t)(pl->grid + 1) * sizeof(int32_t), 32);
+    // the binned units by cost rank, for the kernel's redistribution under a RUN mask
+    pl->upload_bytes = pl->off_unit_rank +
+                       (pl->max_bins > 0 ? align_up((size_t)kMaxRanked * sizeof(uint32_t), 32) : 0);
     pl->off_status = pl->upload_bytes;
     pl->off_tickets = pl->off_status + 32;
     pl->total_bytes = pl->off_tickets +

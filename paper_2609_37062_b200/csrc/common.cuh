@@ -41,6 +41,10 @@ struct KernelParams {
     const decode_attn_unit_t* units;
     const SeqInfo* seq_info;
     const int32_t* block_begin;  // [grid + 1]: block b walks units block_begin[b] .. block_begin[b+1]; NULL: unit b
+    const uint32_t* unit_rank;   // [n_ranked] the binned units by cost rank: sequence << 12 | position behind the first
+                                 // binned unit (sequence 0xfffff: no RUN mask applies); work lists of <= 2,560 units
+    int32_t n_ranked;            // entries of unit_rank (0: none)
+    int32_t first_binned;        // position of the first binned unit in the work list
     int32_t* tickets;  // [2][batch][Hkv], zero between launches: records published / slices merged per (sequence, KV head)
     int32_t* status;   // worst da_status_t seen by any block (0 = ok)
     int64_t k_stride_page, k_stride_token, k_stride_head;
@@ -545,6 +549,38 @@ __device__ __forceinline__ void block_finish(const KernelParams& p, const decode
     // The barrier orders every thread's record stores before thread 0's fence, which publishes
     // them device-wide ahead of the arrival.
     block_sync(bar_id, nthreads);
+    if (tid == 0) {
+        __threadfence();
+        atomicAdd(p.tickets + (int64_t)u.seq * p.num_kv_heads + u.kv_head, 1);
+    }
+}
+
+// The result of a unit that read nothing: zeros (and lse = -inf) for a sequence with a single split,
+// an empty record (maximum -inf, sum 0) otherwise; published like any other record in fused plans.
+template <int D>
+__device__ __forceinline__ void block_finish_empty(const KernelParams& p, const decode_attn_unit_t& u, int G, int tid,
+                                                   int nthreads)
+{
+    constexpr int D4 = D / 4;
+    const int Hq = p.num_q_heads;
+    const int h0 = u.kv_head * G;
+    const int RF = rec_floats(G, D);
+    float* const rec = (u.slot >= 0) ? p.ws + ((int64_t)u.slot * p.num_kv_heads + u.kv_head) * RF : nullptr;
+    const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int task = tid; task < G * D4; task += nthreads) {
+        const int h = task / D4, d4 = task % D4;
+        if (rec == nullptr) {
+            store_out4(p.out, ((int64_t)u.seq * Hq + h0 + h) * D + d4 * 4, zero, p.out_kind);
+            if (p.lse != nullptr && d4 == 0) p.lse[(int64_t)u.seq * Hq + h0 + h] = -INFINITY;
+        } else {
+            __stcg(reinterpret_cast<float4*>(rec) + task, zero);
+            if (d4 == 0) __stcg(reinterpret_cast<float2*>(rec + G * D) + h, make_float2(-INFINITY, 0.f));
+        }
+    }
+    if (rec == nullptr || !p.fused) return;
+    // fused plans: the record is published; the named barrier orders every thread's stores before
+    // thread 0's fence (the same barrier id the ordinary finish uses, by the same threads)
+    block_sync(1, nthreads);
     if (tid == 0) {
         __threadfence();
         atomicAdd(p.tickets + (int64_t)u.seq * p.num_kv_heads + u.kv_head, 1);

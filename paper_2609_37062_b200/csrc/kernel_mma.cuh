@@ -174,7 +174,9 @@ struct MmaExtra {
     int32_t gather_seq;
 };
 
-template <int D, bool DUP, int MODE, bool PREFIX, bool F16 = false>
+// MASKED: the variant launched when a RUN mask is given (ordinary attention plans): it can deal the
+// work list out again among the blocks; kept apart so that launches without a mask carry none of it.
+template <int D, bool DUP, int MODE, bool PREFIX, bool F16 = false, bool MASKED = false>
 __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const KernelParams p,
                                                                       const __grid_constant__ CUtensorMap k_map,
                                                                       const __grid_constant__ CUtensorMap v_map,
@@ -194,6 +196,9 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
     const uint32_t bar_base = base + NS * Cfg::kStageBytes;   // full[NS], empty[NS]
     volatile int* const sm_flags = reinterpret_cast<volatile int*>(gbase + NS * Cfg::kStageBytes + 256);
     int* const sm_ticket = reinterpret_cast<int*>(gbase + NS * Cfg::kStageBytes + 256 + 16);
+    constexpr int kListMax = 160;                             // units a block can own after a redistribution
+    int* const sm_list = reinterpret_cast<int*>(gbase + NS * Cfg::kStageBytes + 384);   // [kListMax], 640 bytes
+    static_assert(384 + 4 * kListMax <= Cfg::kBarrierBytes, "the unit list overlaps the scratch");
     float* const sm_wo = reinterpret_cast<float*>(gbase + NS * Cfg::kStageBytes + Cfg::kBarrierBytes);   // [4][COLS][D]
     float* const sm_wm = sm_wo + kMmaConsumerWarps * COLS * D;                                           // [4][COLS]
     float* const sm_wl = sm_wm + kMmaConsumerWarps * COLS;                                               // [4][COLS]
@@ -241,6 +246,7 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
     // kernel launched before this one may have produced (q, new K/V rows, lengths, page
     // mappings) is read only past this point; with a programmatic dependency the lines above
     // overlap that kernel's tail.
+    const bool redistribute = MASKED && MODE == kModeAttend && p.run_mask != nullptr && p.n_ranked > 0 && !p.grid_exit;
     if (MODE == kModeAttend && warp == 0 && p.hint_first_pages != 0) {
         // Hints, while the kernel before this one drains (from a consumer warp, which has nothing to do
         // until the first stage lands; the producer goes straight to its wait): the pages that will fill the ring first
@@ -265,6 +271,90 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
     }
     pdl_wait_primary();
     if (p.early_trigger) pdl_launch_dependents();             // first of a pair: see KernelParams
+
+    bool listed = false;                                      // the block walks sm_list instead of its range
+    if (redistribute) {
+        // With a RUN mask the planner's packing is off: it could not know which rows read nothing,
+        // and a block whose rows all run sets the step's time.  So every block deals the units out
+        // again, the same way: in cost order the units that run go to the blocks in turn (back and
+        // forth, so that no block always gets the largest of a round), and likewise the masked ones,
+        // which cost next to nothing, behind them.  Consecutive units of the order - the KV heads
+        // of one sequence - still go to different blocks at the same time, every unit has one
+        // owner, and no block depends on another.  A block's list lives in shared memory.
+        const int n = p.n_ranked, nb = p.n_work_blocks, b = blockIdx.x;
+        // Work lists of up to 2,560 units (16 a thread, a word each, read in rank order so that a
+        // warp's loads are adjacent); longer ones keep the planner's packing: with that many units a
+        // block the masked rows even out by themselves.  Every block reads the same words at the same
+        // moment, which costs a few microseconds, so a look at the first rows' mask bytes decides
+        // first whether enough rows are masked for the new deal to pay (about three in ten).
+        constexpr int CH = 16;
+        const int n_seen = min(p.batch, kMmaThreads);
+        const int seen_masked = __syncthreads_count(tid < n_seen && __ldg(p.run_mask + tid) == 0);
+        if (seen_masked * 10 >= n_seen * 3) {
+            uint32_t* const words = reinterpret_cast<uint32_t*>(sm_wo);      // [CH * 5] which units run, in rank order
+            int* const before = reinterpret_cast<int*>(sm_wo) + CH * 5;      // [CH * 5 + 1] running units before each word
+            int pos_held[CH], seq_held[CH];
+#pragma unroll
+            for (int i = 0; i < CH; ++i) {
+                const int j = i * kMmaThreads + tid;
+                const uint32_t e = (j < n) ? __ldg(p.unit_rank + j) : 0xfffff000u;
+                seq_held[i] = (e >> 12) == 0xfffffu ? -1 : (int)(e >> 12);
+                pos_held[i] = p.first_binned + (int)(e & 0xfffu);
+            }
+            uint32_t my_bits = 0;
+#pragma unroll
+            for (int i = 0; i < CH; ++i) {
+                const int j = i * kMmaThreads + tid;
+                const bool r = j < n && (seq_held[i] < 0 || __ldg(p.run_mask + seq_held[i]) != 0);
+                const uint32_t w = __ballot_sync(0xffffffffu, r);
+                if (lane == 0) words[i * (kMmaThreads / 32) + warp] = w;
+                my_bits |= (r ? 1u : 0u) << i;
+            }
+            __syncthreads();
+            constexpr int NW = CH * (kMmaThreads / 32);
+            if (tid <= NW) {
+                int acc = 0;
+                for (int w = 0; w < tid; ++w) acc += __popc(words[w]);
+                before[tid] = acc;                                            // before[NW]: all running units
+            }
+            __syncthreads();
+            const int total = before[NW];
+            // the k-th unit of a kind (running / masked): round k / nb, block k % nb or, in odd rounds,
+            // nb - 1 - k % nb; how many of `count` a block gets follows in closed form
+            auto owner = [&](int k) { return ((k / nb) & 1) ? nb - 1 - k % nb : k % nb; };
+            auto share = [&](int count) {
+                const int full = count / nb, rem = count % nb;
+                const bool extra = (full & 1) ? b >= nb - rem : b < rem;
+                return full + (extra ? 1 : 0);
+            };
+            const int n_run = share(total), n_all = n_run + share(n - total);
+            if (n_all <= kListMax) {
+#pragma unroll
+                for (int i = 0; i < CH; ++i) {
+                    const int j = i * kMmaThreads + tid;
+                    if (j < n) {
+                        const int w = i * (kMmaThreads / 32) + warp;
+                        const int kr = before[w] + __popc(words[w] & ((1u << lane) - 1u));   // running units before j
+                        if ((my_bits >> i) & 1u) {
+                            if (owner(kr) == b) sm_list[kr / nb] = pos_held[i];
+                        } else {
+                            const int km = j - kr;                                            // masked units before j
+                            if (owner(km) == b) sm_list[n_run + km / nb] = pos_held[i];
+                        }
+                    }
+                }
+                listed = true;
+                ubeg = 0;
+                uend = n_all;
+            }
+        }
+        __syncthreads();                                      // the list is written, the scratch goes back to its use
+        if (listed) {
+            if (ubeg >= uend) return;
+            u = load_unit(p.units, sm_list[0]);
+        }
+    }
+    auto unit_at = [&](int k) { return (MASKED && listed) ? sm_list[k] : k; };   // position in the work list of the block's k-th unit
 
     if (warp == kMmaConsumerWarps) {
         // ------------------------------------------------------------ producer
@@ -291,7 +381,7 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
         for (int uid = ubeg; uid < uend && alive; ++uid) {
             const bool has_next = uid + 1 < uend;
             decode_attn_unit_t nu = u;
-            if (has_next) nu = load_unit(p.units, uid + 1);               // lands while this unit streams
+            if (has_next) nu = load_unit(p.units, unit_at(uid + 1));      // lands while this unit streams
             int nt1 = 0, nids_first = 0;
             bool next_ready = false;
             const int b = u.seq, g = u.kv_head & 0xffff;   // (a shared-prefix unit keeps its block size in the high half)
@@ -393,7 +483,7 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
     for (int uid = ubeg; uid < uend; ++uid) {
         const bool last_unit = uid + 1 >= uend;
         decode_attn_unit_t nu = u;
-        if (!last_unit) nu = load_unit(p.units, uid + 1);                 // lands while this unit is consumed
+        if (!last_unit) nu = load_unit(p.units, unit_at(uid + 1));        // lands while this unit is consumed
         Pre nxt = cur;
         const int b = u.seq, g = u.kv_head & 0xffff;
         const int nseq = u.kv_head >> 16;                                  // > 0: a shared-prefix unit
@@ -742,6 +832,15 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
         // ------------------------------------------------------------ end of the unit
         const bool stale = dev_len != u.seq_len;                  // stale plan: void the result, report it
         if (stale && tid == 0) record_status(p.status, DA_ERR_STALE_PLAN);
+        if (n_pages == 0) {
+            // Nothing was read (a masked row, an empty split, a sequence of length 0): the empty
+            // result is written straight away - no states to merge, no barrier, the scratch untouched.
+            block_finish_empty<D>(p, u, G, tid, kConsumerThreads);
+            if (uid == ubeg && tid == 0) DA_TRACE_STAMP(blockIdx.x, 6);
+            u = nu;
+            cur = nxt;
+            continue;
+        }
 #pragma unroll
         for (int off = 4; off <= 16; off <<= 1) {
             l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], off);
@@ -843,9 +942,22 @@ typedef void (*mma_kernel_t)(const KernelParams, const CUtensorMap, const CUtens
 
 // f16: q, K and V are fp16 (attention mode); else bf16.
 template <int MODE>
-inline mma_kernel_t mma_kernel_for(int D, int G, bool prefix = false, bool f16 = false)
+inline mma_kernel_t mma_kernel_for(int D, int G, bool prefix = false, bool f16 = false, bool masked = false)
 {
     const bool dup = G <= 4;
+    if (masked && MODE == kModeAttend && !prefix) {
+        if (D == 128)
+            return f16 ? (dup ? decode_attn_mma_kernel<128, true, kModeAttend, false, true, true>
+                              : decode_attn_mma_kernel<128, false, kModeAttend, false, true, true>)
+                       : (dup ? decode_attn_mma_kernel<128, true, kModeAttend, false, false, true>
+                              : decode_attn_mma_kernel<128, false, kModeAttend, false, false, true>);
+        if (D == 64)
+            return f16 ? (dup ? decode_attn_mma_kernel<64, true, kModeAttend, false, true, true>
+                              : decode_attn_mma_kernel<64, false, kModeAttend, false, true, true>)
+                       : (dup ? decode_attn_mma_kernel<64, true, kModeAttend, false, false, true>
+                              : decode_attn_mma_kernel<64, false, kModeAttend, false, false, true>);
+        return nullptr;
+    }
     if (f16) {
         if (MODE != kModeAttend) return nullptr;
         if (prefix) {
@@ -879,9 +991,9 @@ inline int mma_smem_bytes(int D, int G)
 }
 
 template <int MODE>
-inline int mma_prepare(int D, int G, mma_kernel_t* fn_out, bool prefix = false, bool f16 = false)
+inline int mma_prepare(int D, int G, mma_kernel_t* fn_out, bool prefix = false, bool f16 = false, bool masked = false)
 {
-    mma_kernel_t fn = mma_kernel_for<MODE>(D, G, prefix, f16);
+    mma_kernel_t fn = mma_kernel_for<MODE>(D, G, prefix, f16, masked);
     if (!fn) return DA_ERR_UNSUPPORTED;
     if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, mma_smem_bytes(D, G)) != cudaSuccess) {
         (void)cudaGetLastError();
@@ -911,7 +1023,8 @@ inline int mma_launch_mode(const decode_attn_shape_t& s, int G, const KernelPara
 {
     mma_kernel_t fn;
     // (the probe and gather modes only move 16-bit words: one variant serves both input types)
-    int rc = mma_prepare<MODE>(s.head_dim, G, &fn, prefix, MODE == kModeAttend && s.kv_dtype == DA_DTYPE_FP16);
+    const bool masked = MODE == kModeAttend && !prefix && kp.run_mask != nullptr && kp.n_ranked > 0 && !kp.grid_exit;
+    int rc = mma_prepare<MODE>(s.head_dim, G, &fn, prefix, MODE == kModeAttend && s.kv_dtype == DA_DTYPE_FP16, masked);
     if (rc != DA_OK) return rc;
     CUtensorMap kmap, vmap;
     rc = make_pool_map(&kmap, kp.k, s, s.k_stride_page, s.k_stride_token, s.k_stride_head);

@@ -312,6 +312,7 @@ int make_layout(const decode_attn_shape_t& s, const decode_attn_policy_t& p, con
     out.units.clear();
     out.units.resize(n);
     out.block_begin.clear();
+    out.rank_pos.clear();
     out.n_front_units = 0;
     size_t first = 0;                       // units before this one stay out of the bins
     if (umma) {
@@ -365,7 +366,12 @@ int make_layout(const decode_attn_shape_t& s, const decode_attn_policy_t& p, con
         run += count[b + 1];
         count[b + 1] = out.block_begin[b];      // becomes the bin's write cursor
     }
-    for (size_t i = first; i < n; ++i) out.units[count[bin_of[i] + 1]++] = keyed[order[i]].u;
+    out.rank_pos.resize(n - first);
+    for (size_t i = first; i < n; ++i) {
+        const int32_t pos = count[bin_of[i] + 1]++;
+        out.units[pos] = keyed[order[i]].u;
+        out.rank_pos[i - first] = pos;
+    }
     out.block_begin.push_back((int32_t)out.units.size());
     return DA_OK;
 }

@@ -29,6 +29,8 @@ struct Layout {
     int32_t n_front_units = 0;              // shared-prefix units kept at the front, outside the bins, for a
                                             // kernel of their own (policy kernel DA_KERNEL_UMMA_PREFIX)
     std::vector<int32_t> block_begin;       // [bins + 1] when the units were packed into bins, else empty
+    std::vector<int32_t> rank_pos;          // binned layouts: position in `units` of the binned unit with cost rank j
+                                            // (j = 0: most expensive; ties in creation order)
 };
 
 // Validates the fields the planner and the kernels rely on.
