@@ -183,3 +183,29 @@ def test_page_permutation_changes_nothing_within_tolerance(kernel):
 def test_block_table_rows_may_be_wider_than_needed(kernel):
     w = wl.make_workload("wide", [40, 333], 8, 2, 64, seed=3, max_pages_per_seq=77)
     check_workload(w, da.make_policy(kernel=kernel, fuse_combine=1, chunk_tokens=64))
+
+
+@pytest.mark.parametrize("fused", [0, 1])
+@pytest.mark.parametrize("frac", [0.1, 0.5, 0.9])
+def test_run_mask_on_a_work_list_of_several_rounds(fused, frac):
+    """More units than resident blocks and many masked rows: the masked variant of the tensor-core
+    kernel deals the work list out again among its blocks (from three masked rows in ten); the
+    result must not depend on which block attends which unit."""
+    rng = np.random.default_rng(7)
+    lens = [int(x) for x in rng.integers(1, 700, size=300)]
+    w = wl.make_workload("m", lens, 32, 8, 128, seed=31)
+    mask = (rng.random(len(lens)) >= frac).astype(np.uint8)
+    ref_out, ref_lse = oracle_of(w, run_mask=mask)
+    wd = to_device(w)
+    dmask = torch.from_numpy(mask).cuda()
+    pol = da.make_policy(kernel=da.DA_KERNEL_MMA_TMA, fuse_combine=fused, chunk_tokens=64)
+    out, lse = da.run_workload(wd, pol, run_mask=dmask)
+    assert_parity(out, lse, ref_out, ref_lse)
+    # the same bits as row by row: a row's result does not depend on the mask of the others
+    det = da.make_policy(kernel=da.DA_KERNEL_MMA_TMA, split_mode=da.DA_SPLIT_DETERMINISTIC, chunk_tokens=128)
+    out_m, _ = da.run_workload(wd, det, run_mask=dmask)
+    out_all, _ = da.run_workload(wd, det)
+    keep = torch.from_numpy(mask.astype(bool)).cuda()
+    assert torch.equal(out_m[keep], out_all[keep])
+    assert not out_m[~keep].any()
+
