@@ -301,7 +301,8 @@ void fill_host_mirror(decode_attn_plan_t* pl)
     DevHeader* hdr = reinterpret_cast<DevHeader*>(pl->pinned);
     hdr->n_units = (int32_t)pl->layout.units.size();
     hdr->batch = pl->shape.batch;
-    hdr->pad[0] = hdr->pad[1] = 0;
+    hdr->n_ranked = ranked_fits(pl) ? (int32_t)pl->layout.rank_pos.size() : 0;
+    hdr->first_binned = pl->layout.n_front_units;
     std::memcpy(pl->pinned + pl->off_units, pl->layout.units.data(),
                 pl->layout.units.size() * sizeof(decode_attn_unit_t));
     SeqInfo* si = reinterpret_cast<SeqInfo*>(pl->pinned + pl->off_seq_info);
@@ -353,6 +354,7 @@ KernelParams make_params(const decode_attn_plan_t* pl, const decode_attn_run_arg
     kp.unit_rank = reinterpret_cast<const uint32_t*>(pl->dev + pl->off_unit_rank);
     kp.n_ranked = ranked_fits(pl) ? (int32_t)pl->layout.rank_pos.size() : 0;
     kp.first_binned = pl->layout.n_front_units;
+    kp.may_rank = pl->max_bins > 0 && pl->policy.capacity_batch > 0;
     kp.tickets = reinterpret_cast<int32_t*>(pl->dev + pl->off_tickets);
     kp.ticket_stride = (int32_t)(pl->max_batch * s.num_kv_heads);
     kp.batch = s.batch;
@@ -1000,7 +1002,8 @@ int decode_attn_step_static(const decode_attn_shape_t* shape, const int32_t* seq
     DevHeader* hdr = reinterpret_cast<DevHeader*>(g_static.staging);
     hdr->n_units = (int32_t)lay.units.size();
     hdr->batch = shape->batch;
-    hdr->pad[0] = hdr->pad[1] = 0;
+    hdr->n_ranked = 0;
+    hdr->first_binned = 0;
     std::memcpy(g_static.staging + kStaticOffUnits, lay.units.data(), lay.units.size() * sizeof(decode_attn_unit_t));
     SeqInfo* si = reinterpret_cast<SeqInfo*>(g_static.staging + kStaticOffSeqInfo);
     for (int b = 0; b < shape->batch; ++b) {

@@ -17,7 +17,8 @@ namespace da {
 struct DevHeader {
     int32_t n_units;
     int32_t batch;
-    int32_t pad[2];
+    int32_t n_ranked;       // entries of the rank-ordered unit list (0: none), see KernelParams::unit_rank
+    int32_t first_binned;   // position of the first binned unit in the work list
 };
 
 struct SeqInfo {
@@ -43,8 +44,9 @@ struct KernelParams {
     const int32_t* block_begin;  // [grid + 1]: block b walks units block_begin[b] .. block_begin[b+1]; NULL: unit b
     const uint32_t* unit_rank;   // [n_ranked] the binned units by cost rank: sequence << 12 | position behind the first
                                  // binned unit (sequence 0xfffff: no RUN mask applies); work lists of <= 2,560 units
-    int32_t n_ranked;            // entries of unit_rank (0: none)
+    int32_t n_ranked;            // entries of unit_rank (0: none); capacity plans read both from the header,
     int32_t first_binned;        // position of the first binned unit in the work list
+    int32_t may_rank;            // capacity plans: the rank list exists (how long it is changes with every refresh)
     int32_t* tickets;  // [2][batch][Hkv], zero between launches: records published / slices merged per (sequence, KV head)
     int32_t* status;   // worst da_status_t seen by any block (0 = ok)
     int64_t k_stride_page, k_stride_token, k_stride_head;

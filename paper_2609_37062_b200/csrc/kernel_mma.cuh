@@ -220,7 +220,11 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
         ubeg = blockIdx.x;
         uend = min(n_units, (int)blockIdx.x + 1);
     }
-    if (ubeg >= uend) {                                       // surplus blocks of a capacity launch
+    // (with a RUN mask the masked variant may deal the units out again, to every block of the launch)
+    const bool may_redistribute = MASKED && MODE == kModeAttend && p.run_mask != nullptr &&
+                                  (p.grid_exit ? p.may_rank != 0 : p.n_ranked > 0);
+    const bool idle = ubeg >= uend;                           // no units from the planner's packing
+    if (idle && !may_redistribute) {                          // surplus blocks of a capacity launch
         // Stream order reaches the kernels behind this one through the waits of this launch's
         // blocks; should every block be surplus, block 0 still carries it.
         if (blockIdx.x == 0) pdl_wait_primary();
@@ -239,15 +243,16 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
         sm_flags[0] = 0;
         mbar_init_fence();
     }
-    decode_attn_unit_t u = load_unit(p.units, ubeg);
+    decode_attn_unit_t u = load_unit(p.units, idle ? 0 : ubeg);
     __syncthreads();
     if (tid == 0) DA_TRACE_STAMP(blockIdx.x, 1);
     // Everything above touched only the plan's own work list and kernel parameters.  What the
     // kernel launched before this one may have produced (q, new K/V rows, lengths, page
     // mappings) is read only past this point; with a programmatic dependency the lines above
     // overlap that kernel's tail.
-    const bool redistribute = MASKED && MODE == kModeAttend && p.run_mask != nullptr && p.n_ranked > 0 && !p.grid_exit;
-    if (MODE == kModeAttend && warp == 0 && p.hint_first_pages != 0) {
+    const int n_ranked = p.grid_exit ? p.header->n_ranked : p.n_ranked;
+    const bool redistribute = may_redistribute && n_ranked > 0;
+    if (MODE == kModeAttend && warp == 0 && p.hint_first_pages != 0 && !idle) {
         // Hints, while the kernel before this one drains (from a consumer warp, which has nothing to do
         // until the first stage lands; the producer goes straight to its wait): the pages that will fill the ring first
         // are asked into L2.  The mask and the page ids read here may be about to change; they steer
@@ -281,7 +286,8 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
         // which cost next to nothing, behind them.  Consecutive units of the order - the KV heads
         // of one sequence - still go to different blocks at the same time, every unit has one
         // owner, and no block depends on another.  A block's list lives in shared memory.
-        const int n = p.n_ranked, nb = p.n_work_blocks, b = blockIdx.x;
+        const int n = n_ranked, nb = p.n_work_blocks, b = blockIdx.x;
+        const int first_binned = p.grid_exit ? p.header->first_binned : p.first_binned;
         // Work lists of up to 2,560 units (16 a thread, a word each, read in rank order so that a
         // warp's loads are adjacent); longer ones keep the planner's packing: with that many units a
         // block the masked rows even out by themselves.  Every block reads the same words at the same
@@ -299,7 +305,7 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
                 const int j = i * kMmaThreads + tid;
                 const uint32_t e = (j < n) ? __ldg(p.unit_rank + j) : 0xfffff000u;
                 seq_held[i] = (e >> 12) == 0xfffffu ? -1 : (int)(e >> 12);
-                pos_held[i] = p.first_binned + (int)(e & 0xfffu);
+                pos_held[i] = first_binned + (int)(e & 0xfffu);
             }
             uint32_t my_bits = 0;
 #pragma unroll
@@ -354,6 +360,7 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
             u = load_unit(p.units, sm_list[0]);
         }
     }
+    if (idle && !listed) return;                              // a surplus block that stayed for nothing
     auto unit_at = [&](int k) { return (MASKED && listed) ? sm_list[k] : k; };   // position in the work list of the block's k-th unit
 
     if (warp == kMmaConsumerWarps) {
@@ -1023,7 +1030,8 @@ inline int mma_launch_mode(const decode_attn_shape_t& s, int G, const KernelPara
 {
     mma_kernel_t fn;
     // (the probe and gather modes only move 16-bit words: one variant serves both input types)
-    const bool masked = MODE == kModeAttend && !prefix && kp.run_mask != nullptr && kp.n_ranked > 0 && !kp.grid_exit;
+    const bool masked = MODE == kModeAttend && !prefix && kp.run_mask != nullptr &&
+                        (kp.grid_exit ? kp.may_rank != 0 : kp.n_ranked > 0);
     int rc = mma_prepare<MODE>(s.head_dim, G, &fn, prefix, MODE == kModeAttend && s.kv_dtype == DA_DTYPE_FP16, masked);
     if (rc != DA_OK) return rc;
     CUtensorMap kmap, vmap;

@@ -98,3 +98,58 @@ def test_updates_beyond_the_capacity_are_refused():
     with pytest.raises(da.DecodeAttnError) as e:
         da.decode_attn_plan_update(plain, [100, 200])
     assert e.value.status == da.DA_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("fused", [0, 1])
+def test_run_mask_in_a_captured_capacity_graph(fused):
+    """The paper's deployment: one captured launch for the capacity, a RUN mask that changes every
+    step.  With many rows masked the kernel deals the (refreshed) work list out again among all
+    blocks of the fixed grid, surplus ones included; rows past the live batch stay untouched."""
+    cap_b, cap_tok = 96, 90000
+    steps = [([700] * 60, 0.6), ([300, 5, 1200, 64] * 12, 0.5), ([900] * 96, 0.0), ([100] * 7, 0.9), ([500] * 90, 1.0)]
+    first = wl.make_workload("capm", steps[0][0], 32, 8, 128, seed=60, pool_pages=6000, max_pages_per_seq=80)
+    shape = da.shape_of_workload(first)
+    pol = da.make_policy(kernel=da.DA_KERNEL_MMA_TMA, chunk_tokens=128, fuse_combine=fused, capacity_batch=cap_b,
+                         capacity_tokens=cap_tok)
+    plan = da.decode_attn_plan(shape, pol, first.seq_lens)
+    k_pool, v_pool = first.k_pool.cuda(), first.v_pool.cuda()
+    q = padded(first.q_bits, cap_b)
+    bt = padded(first.block_table, cap_b)
+    sl = padded(first.seq_lens, cap_b)
+    mask = torch.ones((cap_b,), dtype=torch.uint8, device="cuda")
+    out = torch.zeros((cap_b, 32, 128), dtype=torch.float32, device="cuda")
+    lse = torch.zeros((cap_b, 32), dtype=torch.float32, device="cuda")
+    ws = torch.empty(max(plan.workspace_bytes, 256), dtype=torch.uint8, device="cuda")
+
+    def launch():
+        da.decode_attn_run(plan, q, k_pool, v_pool, bt, sl, out, lse, ws, plan.workspace_bytes, run_mask=mask)
+        if not fused:
+            da.decode_attn_combine(plan, ws, out, lse)
+
+    stream = torch.cuda.Stream()
+    rng = torch.Generator().manual_seed(5)
+    with torch.cuda.stream(stream):
+        launch()
+        stream.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            launch()
+        for i, (lens, frac) in enumerate(steps):
+            w = wl.make_workload("capm", lens, 32, 8, 128, seed=61 + i, pool_pages=6000, max_pages_per_seq=80)
+            host_mask = (torch.rand(len(lens), generator=rng) >= frac).to(torch.uint8)
+            k_pool.copy_(w.k_pool)
+            v_pool.copy_(w.v_pool)
+            q.zero_(); bt.zero_(); sl.zero_(); mask.fill_(1)
+            q[: len(lens)] = w.q_bits.cuda()
+            bt[: len(lens)] = w.block_table.cuda()
+            sl[: len(lens)] = w.seq_lens.cuda()
+            mask[: len(lens)] = host_mask.cuda()
+            out.fill_(float("nan"))
+            da.decode_attn_plan_update(plan, w.seq_lens, stream)
+            graph.replay()
+            stream.synchronize()
+            assert da.decode_attn_last_device_status(plan, stream) == da.DA_OK
+            ref_out, ref_lse = oracle_of(w, run_mask=host_mask.numpy())
+            assert_parity(out[: len(lens)], lse[: len(lens)], ref_out, ref_lse, f"step {i}")
+            assert torch.isnan(out[len(lens):]).all()
+    plan.destroy()
