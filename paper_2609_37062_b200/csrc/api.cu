@@ -288,12 +288,11 @@ int device_sm_count(int dev, int* out)
 }
 
 // The kernel's redistribution under a RUN mask reads the binned units by cost rank, packed into a
-// word each: work lists of up to kMaxRanked units and batches below 2^20 - 1 sequences.
-constexpr int kMaxRanked = 2560;
+// word each: work lists of up to kMaxRanked units and batches below kRankNoSeq sequences.
 bool ranked_fits(const decode_attn_plan_t* pl)
 {
     return pl->max_bins > 0 && !pl->layout.rank_pos.empty() && pl->layout.rank_pos.size() <= (size_t)kMaxRanked &&
-           pl->shape.batch < 0xfffff;
+           (uint32_t)pl->shape.batch < kRankNoSeq;
 }
 
 void fill_host_mirror(decode_attn_plan_t* pl)
@@ -326,8 +325,8 @@ void fill_host_mirror(decode_attn_plan_t* pl)
             for (size_t j = 0; j < pl->layout.rank_pos.size(); ++j) {
                 const int32_t pos = pl->layout.rank_pos[j];
                 const decode_attn_unit_t& u = pl->layout.units[pos];
-                const uint32_t seq = (u.kv_head >> 16) ? 0xfffffu : (uint32_t)u.seq;
-                ur[j] = seq << 12 | (uint32_t)(pos - first);
+                const uint32_t seq = (u.kv_head >> 16) ? kRankNoSeq : (uint32_t)u.seq;
+                ur[j] = seq << kRankPosBits | (uint32_t)(pos - first);
             }
         }
     }
@@ -472,7 +471,9 @@ int decode_attn_plan(const decode_attn_shape_t* shape, const decode_attn_policy_
     pl->off_unit_rank = pl->off_block_begin + align_up((size_t)(pl->grid + 1) * sizeof(int32_t), 32);
     // the binned units by cost rank, for the kernel's redistribution under a RUN mask
     pl->upload_bytes = pl->off_unit_rank +
-                       (pl->max_bins > 0 ? align_up((size_t)kMaxRanked * sizeof(uint32_t), 32) : 0);
+                       (pl->max_bins > 0
+                            ? align_up((size_t)std::min<int64_t>(std::max<int64_t>(pl->max_units, 1), kMaxRanked) * sizeof(uint32_t), 32)
+                            : 0);
     pl->off_status = pl->upload_bytes;
     pl->off_tickets = pl->off_status + 32;
     pl->total_bytes = pl->off_tickets +

@@ -288,40 +288,42 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
         // owner, and no block depends on another.  A block's list lives in shared memory.
         const int n = n_ranked, nb = p.n_work_blocks, b = blockIdx.x;
         const int first_binned = p.grid_exit ? p.header->first_binned : p.first_binned;
-        // Work lists of up to 2,560 units (16 a thread, a word each, read in rank order so that a
-        // warp's loads are adjacent); longer ones keep the planner's packing: with that many units a
-        // block the masked rows even out by themselves.  Every block reads the same words at the same
+        // Work lists of up to 10,240 units (a word each, read in rank order, 16 a thread at a time, so
+        // that a warp's loads are adjacent); longer ones keep the planner's packing: with that many
+        // units a block the masked rows even out by themselves.  Every block reads the same words at the same
         // moment, which costs a few microseconds, so a look at the first rows' mask bytes decides
         // first whether enough rows are masked for the new deal to pay (about three in ten).
-        constexpr int CH = 16;
+        constexpr int CH = 16;                                // units a thread holds at a time
+        constexpr int WPP = CH * (kMmaThreads / 32);          // ballot words of a pass of CH * threads units
+        const int passes = (n + CH * kMmaThreads - 1) / (CH * kMmaThreads);     // <= kRankPasses
         const int n_seen = min(p.batch, kMmaThreads);
         const int seen_masked = __syncthreads_count(tid < n_seen && __ldg(p.run_mask + tid) == 0);
         if (seen_masked * 10 >= n_seen * 3) {
-            uint32_t* const words = reinterpret_cast<uint32_t*>(sm_wo);      // [CH * 5] which units run, in rank order
-            int* const before = reinterpret_cast<int*>(sm_wo) + CH * 5;      // [CH * 5 + 1] running units before each word
-            int pos_held[CH], seq_held[CH];
+            uint32_t* const words = reinterpret_cast<uint32_t*>(sm_wo);              // [passes * WPP] which units run, in rank order
+            int* const before = reinterpret_cast<int*>(sm_wo) + kRankPasses * WPP;   // [passes * WPP + 1] running units before each word
+            static_assert((2 * kRankPasses * WPP + 1) * 4 <= Cfg::kScratchBytes, "the ballot words do not fit the scratch");
+            for (int ps = 0; ps < passes; ++ps) {
+                int seq_held[CH];
 #pragma unroll
-            for (int i = 0; i < CH; ++i) {
-                const int j = i * kMmaThreads + tid;
-                const uint32_t e = (j < n) ? __ldg(p.unit_rank + j) : 0xfffff000u;
-                seq_held[i] = (e >> 12) == 0xfffffu ? -1 : (int)(e >> 12);
-                pos_held[i] = first_binned + (int)(e & 0xfffu);
-            }
-            uint32_t my_bits = 0;
+                for (int i = 0; i < CH; ++i) {
+                    const int j = (ps * CH + i) * kMmaThreads + tid;
+                    const uint32_t e = (j < n) ? __ldg(p.unit_rank + j) : 0xffffffffu;
+                    seq_held[i] = (e >> kRankPosBits) == kRankNoSeq ? -1 : (int)(e >> kRankPosBits);
+                }
 #pragma unroll
-            for (int i = 0; i < CH; ++i) {
-                const int j = i * kMmaThreads + tid;
-                const bool r = j < n && (seq_held[i] < 0 || __ldg(p.run_mask + seq_held[i]) != 0);
-                const uint32_t w = __ballot_sync(0xffffffffu, r);
-                if (lane == 0) words[i * (kMmaThreads / 32) + warp] = w;
-                my_bits |= (r ? 1u : 0u) << i;
+                for (int i = 0; i < CH; ++i) {
+                    const int j = (ps * CH + i) * kMmaThreads + tid;
+                    const bool r = j < n && (seq_held[i] < 0 || __ldg(p.run_mask + seq_held[i]) != 0);
+                    const uint32_t w = __ballot_sync(0xffffffffu, r);
+                    if (lane == 0) words[(ps * CH + i) * (kMmaThreads / 32) + warp] = w;
+                }
             }
             __syncthreads();
-            constexpr int NW = CH * (kMmaThreads / 32);
-            if (tid <= NW) {
+            const int NW = passes * WPP;
+            for (int t = tid; t <= NW; t += kMmaThreads) {
                 int acc = 0;
-                for (int w = 0; w < tid; ++w) acc += __popc(words[w]);
-                before[tid] = acc;                                            // before[NW]: all running units
+                for (int w = 0; w < t; ++w) acc += __popc(words[w]);
+                before[t] = acc;                                              // before[NW]: all running units
             }
             __syncthreads();
             const int total = before[NW];
@@ -335,17 +337,21 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
             };
             const int n_run = share(total), n_all = n_run + share(n - total);
             if (n_all <= kListMax) {
+                for (int ps = 0; ps < passes; ++ps) {
 #pragma unroll
-                for (int i = 0; i < CH; ++i) {
-                    const int j = i * kMmaThreads + tid;
-                    if (j < n) {
-                        const int w = i * (kMmaThreads / 32) + warp;
-                        const int kr = before[w] + __popc(words[w] & ((1u << lane) - 1u));   // running units before j
-                        if ((my_bits >> i) & 1u) {
-                            if (owner(kr) == b) sm_list[kr / nb] = pos_held[i];
-                        } else {
-                            const int km = j - kr;                                            // masked units before j
-                            if (owner(km) == b) sm_list[n_run + km / nb] = pos_held[i];
+                    for (int i = 0; i < CH; ++i) {
+                        const int j = (ps * CH + i) * kMmaThreads + tid;
+                        if (j < n) {
+                            const int pos = first_binned + (int)(__ldg(p.unit_rank + j) & ((1u << kRankPosBits) - 1u));
+                            const int w = (ps * CH + i) * (kMmaThreads / 32) + warp;
+                            const uint32_t bits = words[w];
+                            const int kr = before[w] + __popc(bits & ((1u << lane) - 1u));       // running units before j
+                            if ((bits >> lane) & 1u) {
+                                if (owner(kr) == b) sm_list[kr / nb] = pos;
+                            } else {
+                                const int km = j - kr;                                            // masked units before j
+                                if (owner(km) == b) sm_list[n_run + km / nb] = pos;
+                            }
                         }
                     }
                 }
