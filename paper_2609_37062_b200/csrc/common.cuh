@@ -585,9 +585,13 @@ __device__ __forceinline__ void block_finish_empty(const KernelParams& p, const 
         }
     }
     if (rec == nullptr || !p.fused) return;
-    // fused plans: the record is published; the named barrier orders every thread's stores before
-    // thread 0's fence (the same barrier id the ordinary finish uses, by the same threads)
-    block_sync(1, nthreads);
+    // fused plans: the record is published; the barrier orders every thread's stores before
+    // thread 0's fence (the named barrier the ordinary finish uses, by the same threads; a single
+    // warp synchronises by itself)
+    if (nthreads == 32)
+        __syncwarp();
+    else
+        block_sync(1, nthreads);
     if (tid == 0) {
         __threadfence();
         atomicAdd(p.tickets + (int64_t)u.seq * p.num_kv_heads + u.kv_head, 1);

@@ -357,7 +357,13 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
                 }
                 listed = true;
                 ubeg = 0;
-                uend = n_all;
+                uend = n_run;
+                // The masked units of the list are done with here, a warp each: an empty result costs
+                // a descriptor read and a few stores, and going through the pipeline for it would
+                // cost a block about a microsecond of dependent reads per unit.
+                __syncthreads();                              // the list is complete
+                for (int k = n_run + warp; k < n_all; k += kMmaThreads / 32)
+                    block_finish_empty<D>(p, load_unit(p.units, sm_list[k]), G, lane, 32);
             }
         }
         __syncthreads();                                      // the list is written, the scratch goes back to its use
