@@ -399,7 +399,6 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
                 if (tid == 0 && i < 8) DA_TRACE_CLOCK(kUmmaTraceBase + 1024 + unit_index, 16 + i);
                 umma::fence_after_thread_sync();
                 const uint32_t oc = lane_base + kUmmaOutCol + b * 128 + hh * OC;
-#pragma unroll
                 umma::ld64(oc, sg);
                 umma::wait_ld();
                 umma::fence_before_thread_sync();
@@ -433,7 +432,6 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
                     // pass 1: the maximum of this thread's logits; the row's other parts are exchanged
                     // through shared memory (their logits may not be read once they start writing weights)
                     float mx = -INFINITY;
-#pragma unroll
                     umma::ld64(sc + hh * 64, sg);                           // columns 64 hh .. 64 hh + 63
                     umma::wait_ld();
 #pragma unroll
