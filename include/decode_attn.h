@@ -71,8 +71,9 @@ typedef enum {
 typedef enum {
     DA_KERNEL_AUTO = 0,     /* MMA_TMA (every supported head_dim and group size); with
                                shared_prefix_tokens: UMMA_PREFIX where it applies, else MMA_TMA       */
-    DA_KERNEL_SIMT = 1,     /* CUDA-core kernel, 16-byte vectorised global loads                      */
-    DA_KERNEL_MMA_TMA = 2,  /* TMA-staged pages in shared memory, mma.sync (bf16 or fp16) for QK^T, PV  */
+    DA_KERNEL_SIMT = 1,     /* CUDA-core kernel, 16-byte vectorised global loads; groups of up to 8   */
+    DA_KERNEL_MMA_TMA = 2,  /* TMA-staged pages in shared memory, mma.sync (bf16 or fp16) for QK^T, PV;
+                               groups of up to 16 heads (two 8-column tiles of heads above 8)         */
     DA_KERNEL_UMMA_PREFIX = 3 /* shared-prefix plans only (head_dim 128, groups of 1 to 8 heads): the prefix
                                units run on the tcgen05 tensor cores, 128 query rows at a time with
                                accumulators in tensor memory; what follows the prefix runs as MMA_TMA */
@@ -109,7 +110,7 @@ typedef struct {
 typedef struct {
     int32_t batch;              /* live sequences B (rows of q, out, block_table)                    */
     int32_t num_q_heads;
-    int32_t num_kv_heads;       /* divides num_q_heads; group size <= 8                              */
+    int32_t num_kv_heads;       /* divides num_q_heads; group size <= 16 (DA_ERR_UNSUPPORTED above)  */
     int32_t head_dim;           /* 64 or 128                                                         */
     int32_t page_size;          /* tokens per page: 16, 32, 64, 128 or 256                           */
     int32_t max_pages_per_seq;  /* row stride of block_table, in entries                             */

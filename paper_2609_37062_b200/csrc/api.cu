@@ -416,6 +416,7 @@ int decode_attn_plan(const decode_attn_shape_t* shape, const decode_attn_policy_
     pl->scale = shape->sm_scale > 0.f ? shape->sm_scale : 1.0f / sqrtf((float)shape->head_dim);
     pl->kernel = pick_kernel(*shape, *policy);
     if (pl->kernel != DA_KERNEL_SIMT && !mma_supports(shape->head_dim, pl->group)) return DA_ERR_UNSUPPORTED;
+    if (pl->kernel == DA_KERNEL_SIMT && !simt_kernel_for(shape->head_dim, pl->group)) return DA_ERR_UNSUPPORTED;
     const bool umma = pl->kernel == DA_KERNEL_UMMA_PREFIX;
     if (umma && (!umma_supports(shape->head_dim, pl->group) || policy->shared_prefix_tokens <= 0)) return DA_ERR_UNSUPPORTED;
     pl->policy.kernel = pl->kernel;        // the planner cuts the prefix for the kernel that will run it

@@ -176,7 +176,8 @@ struct MmaExtra {
 
 // MASKED: the variant launched when a RUN mask is given (ordinary attention plans): it can deal the
 // work list out again among the blocks; kept apart so that launches without a mask carry none of it.
-template <int D, bool DUP, int MODE, bool PREFIX, bool F16 = false, bool MASKED = false>
+// WIDE: groups of 9..16 query heads: two 8-column tiles of heads per K/V tile instead of one.
+template <int D, bool DUP, int MODE, bool PREFIX, bool F16 = false, bool MASKED = false, bool WIDE = false>
 __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const KernelParams p,
                                                                       const __grid_constant__ CUtensorMap k_map,
                                                                       const __grid_constant__ CUtensorMap v_map,
@@ -188,6 +189,8 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
     constexpr int KSTEPS = D / 16;
     constexpr int COLS = Cfg::kColsOut;
     constexpr int kConsumerThreads = kMmaConsumerWarps * 32;
+    constexpr int NT = WIDE ? 2 : 1;                          // 8-column tiles of query heads
+    static_assert(!(WIDE && (DUP || PREFIX)), "wide groups: ordinary units, low parts of P in a second mma");
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -474,11 +477,12 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
     const bool lo_role = DUP && (c >= 2);
     uint32_t git = 0;                                         // stages consumed so far, over all units
     // what a unit needs before its first tile: lengths / mask of its sequence and Q^T as B
-    // fragments (column n = r is query head r, or r mod 4 when duplicated); fetched one unit ahead
+    // fragments (column n = r of tile nt is query head 8 nt + r, or r mod 4 when duplicated); fetched
+    // one unit ahead
     struct Pre {
         int dev_len;
         int masked;
-        uint32_t qb[KSTEPS][2];
+        uint32_t qb[KSTEPS][NT][2];
     };
     auto prefetch = [&](const decode_attn_unit_t& x, Pre& o) {
         o.dev_len = x.seq_len;
@@ -486,14 +490,17 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
         if (MODE == kModeAttend) {
             o.dev_len = __ldg(p.seq_lens + x.seq);
             if (p.run_mask != nullptr) o.masked = __ldg(p.run_mask + x.seq) == 0;
-            const int head = DUP ? (r & 3) : r;
-            const bool live = head < G;
-            const uint32_t* qrow = reinterpret_cast<const uint32_t*>(
-                p.q + ((int64_t)x.seq * p.num_q_heads + (x.kv_head & 0xffff) * G + (live ? head : 0)) * D);
 #pragma unroll
-            for (int ks = 0; ks < KSTEPS; ++ks) {
-                o.qb[ks][0] = live ? __ldg(qrow + ks * 8 + c) : 0u;         // dims ks*16 + 2c, +1
-                o.qb[ks][1] = live ? __ldg(qrow + ks * 8 + 4 + c) : 0u;     // dims ks*16 + 8 + 2c, +1
+            for (int nt = 0; nt < NT; ++nt) {
+                const int head = DUP ? (r & 3) : nt * 8 + r;
+                const bool live = head < G;
+                const uint32_t* qrow = reinterpret_cast<const uint32_t*>(
+                    p.q + ((int64_t)x.seq * p.num_q_heads + (x.kv_head & 0xffff) * G + (live ? head : 0)) * D);
+#pragma unroll
+                for (int ks = 0; ks < KSTEPS; ++ks) {
+                    o.qb[ks][nt][0] = live ? __ldg(qrow + ks * 8 + c) : 0u;         // dims ks*16 + 2c, +1
+                    o.qb[ks][nt][1] = live ? __ldg(qrow + ks * 8 + 4 + c) : 0u;     // dims ks*16 + 8 + 2c, +1
+                }
             }
         }
     };
@@ -516,7 +523,7 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
         if (MODE == kModeGather && b != ex.gather_seq) t1 = t0;
         const int n_pages = (t1 - t0 + 15) >> 4;
         const int n_iters = (n_pages + kPagesPerStage - 1) / kPagesPerStage;
-        uint32_t (&qb)[KSTEPS][2] = cur.qb;
+        uint32_t (&qb)[KSTEPS][NT][2] = cur.qb;
 
         if (PREFIX && MODE == kModeAttend && nseq > 0) {
             // -------------------------------------------------------- shared-prefix unit
@@ -707,10 +714,15 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
             continue;
         }
 
-        float oacc[D / 16][4];
-        float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+        float oacc[D / 16][NT][4];
+        float m_run[NT][2], l_run[NT][2];
 #pragma unroll
-        for (int i = 0; i < D / 16; ++i) oacc[i][0] = oacc[i][1] = oacc[i][2] = oacc[i][3] = 0.f;
+        for (int nt = 0; nt < NT; ++nt) {
+            m_run[nt][0] = m_run[nt][1] = -INFINITY;
+            l_run[nt][0] = l_run[nt][1] = 0.f;
+#pragma unroll
+            for (int i = 0; i < D / 16; ++i) oacc[i][nt][0] = oacc[i][nt][1] = oacc[i][nt][2] = oacc[i][nt][3] = 0.f;
+        }
         uint32_t probe_sum = 0;
         bool failed = false;
 
@@ -766,56 +778,63 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
                         __syncwarp();
                     }
                     // ---- S^T = K . Q^T
-                    float sacc[4] = {0.f, 0.f, 0.f, 0.f};
+                    float sacc[NT][4];
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) sacc[nt][0] = sacc[nt][1] = sacc[nt][2] = sacc[nt][3] = 0.f;
                     const int arow = (lane & 7) + ((lane >> 3) & 1) * 8;
                     const int achk = lane >> 4;
 #pragma unroll
                     for (int ks = 0; ks < KSTEPS; ++ks) {
                         uint32_t a[4];
                         ldsm_x4(kpage + (ks >> 2) * Cfg::kBoxBytes + swz(arow, (ks & 3) * 2 + achk), a);
-                        In::mma(sacc, a, qb[ks][0], qb[ks][1]);
+#pragma unroll
+                        for (int nt = 0; nt < NT; ++nt) In::mma(sacc[nt], a, qb[ks][nt][0], qb[ks][nt][1]);
                     }
                     // ---- online softmax on the fragment: rows r, r+8 (tokens), columns 2c, 2c+1 (heads)
                     const bool v_lo = r < n_valid, v_hi = (r + 8) < n_valid;
-                    float s00 = v_lo ? sacc[0] * p.scale_log2 : -INFINITY;
-                    float s01 = v_lo ? sacc[1] * p.scale_log2 : -INFINITY;
-                    float s10 = v_hi ? sacc[2] * p.scale_log2 : -INFINITY;
-                    float s11 = v_hi ? sacc[3] * p.scale_log2 : -INFINITY;
-                    float mx0 = fmaxf(s00, s10), mx1 = fmaxf(s01, s11);
+                    uint32_t b0[NT], b1[NT], b0l[NT], b1l[NT];
 #pragma unroll
-                    for (int off = 4; off <= 16; off <<= 1) {
-                        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, off));
-                        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, off));
-                    }
-                    const float mn0 = fmaxf(m_run[0], mx0), mn1 = fmaxf(m_run[1], mx1);   // finite: token 0 of the page is valid
-                    const float al0 = ex2f(m_run[0] - mn0), al1 = ex2f(m_run[1] - mn1);
-                    m_run[0] = mn0;
-                    m_run[1] = mn1;
-                    const float p00 = ex2f(s00 - mn0), p01 = ex2f(s01 - mn1);
-                    const float p10 = ex2f(s10 - mn0), p11 = ex2f(s11 - mn1);
-                    l_run[0] = fmaf(l_run[0], al0, p00 + p10);
-                    l_run[1] = fmaf(l_run[1], al1, p01 + p11);
-                    if (__any_sync(0xffffffffu, al0 != 1.f || al1 != 1.f)) {
+                    for (int nt = 0; nt < NT; ++nt) {
+                        float s00 = v_lo ? sacc[nt][0] * p.scale_log2 : -INFINITY;
+                        float s01 = v_lo ? sacc[nt][1] * p.scale_log2 : -INFINITY;
+                        float s10 = v_hi ? sacc[nt][2] * p.scale_log2 : -INFINITY;
+                        float s11 = v_hi ? sacc[nt][3] * p.scale_log2 : -INFINITY;
+                        float mx0 = fmaxf(s00, s10), mx1 = fmaxf(s01, s11);
 #pragma unroll
-                        for (int mt = 0; mt < D / 16; ++mt) {
-                            oacc[mt][0] *= al0; oacc[mt][1] *= al1;
-                            oacc[mt][2] *= al0; oacc[mt][3] *= al1;
+                        for (int off = 4; off <= 16; off <<= 1) {
+                            mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, off));
+                            mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, off));
                         }
-                    }
-                    // ---- P^T as B fragments (high parts; low parts in the duplicated columns or a second set)
-                    uint32_t hi0 = In::pack(p00, p01), hi1 = In::pack(p10, p11);
-                    const float r00 = p00 - In::low(hi0), r01 = p01 - In::high(hi0);
-                    const float r10 = p10 - In::low(hi1), r11 = p11 - In::high(hi1);
-                    const uint32_t lo0 = In::pack(r00, r01), lo1 = In::pack(r10, r11);
-                    uint32_t b0, b1, b0l = 0, b1l = 0;
-                    if (DUP) {
-                        b0 = movmatrix_trans(lo_role ? lo0 : hi0);
-                        b1 = movmatrix_trans(lo_role ? lo1 : hi1);
-                    } else {
-                        b0 = movmatrix_trans(hi0);
-                        b1 = movmatrix_trans(hi1);
-                        b0l = movmatrix_trans(lo0);
-                        b1l = movmatrix_trans(lo1);
+                        const float mn0 = fmaxf(m_run[nt][0], mx0), mn1 = fmaxf(m_run[nt][1], mx1);   // finite: token 0 of the page is valid
+                        const float al0 = ex2f(m_run[nt][0] - mn0), al1 = ex2f(m_run[nt][1] - mn1);
+                        m_run[nt][0] = mn0;
+                        m_run[nt][1] = mn1;
+                        const float p00 = ex2f(s00 - mn0), p01 = ex2f(s01 - mn1);
+                        const float p10 = ex2f(s10 - mn0), p11 = ex2f(s11 - mn1);
+                        l_run[nt][0] = fmaf(l_run[nt][0], al0, p00 + p10);
+                        l_run[nt][1] = fmaf(l_run[nt][1], al1, p01 + p11);
+                        if (__any_sync(0xffffffffu, al0 != 1.f || al1 != 1.f)) {
+#pragma unroll
+                            for (int mt = 0; mt < D / 16; ++mt) {
+                                oacc[mt][nt][0] *= al0; oacc[mt][nt][1] *= al1;
+                                oacc[mt][nt][2] *= al0; oacc[mt][nt][3] *= al1;
+                            }
+                        }
+                        // ---- P^T as B fragments (high parts; low parts in the duplicated columns or a second set)
+                        uint32_t hi0 = In::pack(p00, p01), hi1 = In::pack(p10, p11);
+                        const float r00 = p00 - In::low(hi0), r01 = p01 - In::high(hi0);
+                        const float r10 = p10 - In::low(hi1), r11 = p11 - In::high(hi1);
+                        const uint32_t lo0 = In::pack(r00, r01), lo1 = In::pack(r10, r11);
+                        b0l[nt] = b1l[nt] = 0;
+                        if (DUP) {
+                            b0[nt] = movmatrix_trans(lo_role ? lo0 : hi0);
+                            b1[nt] = movmatrix_trans(lo_role ? lo1 : hi1);
+                        } else {
+                            b0[nt] = movmatrix_trans(hi0);
+                            b1[nt] = movmatrix_trans(hi1);
+                            b0l[nt] = movmatrix_trans(lo0);
+                            b1l[nt] = movmatrix_trans(lo1);
+                        }
                     }
                     // ---- O^T += V^T . P^T
                     const int vrow = (lane & 7) + (lane >> 4) * 8;
@@ -824,8 +843,11 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
                     for (int mt = 0; mt < D / 16; ++mt) {
                         uint32_t a[4];
                         ldsm_x4_trans(vpage + (mt >> 2) * Cfg::kBoxBytes + swz(vrow, (mt & 3) * 2 + vchk), a);
-                        In::mma(oacc[mt], a, b0, b1);
-                        if (!DUP) In::mma(oacc[mt], a, b0l, b1l);
+#pragma unroll
+                        for (int nt = 0; nt < NT; ++nt) {
+                            In::mma(oacc[mt][nt], a, b0[nt], b1[nt]);
+                            if (!DUP) In::mma(oacc[mt][nt], a, b0l[nt], b1l[nt]);
+                        }
                     }
                 }
             }
@@ -861,46 +883,54 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
             continue;
         }
 #pragma unroll
-        for (int off = 4; off <= 16; off <<= 1) {
-            l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], off);
-            l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], off);
+        for (int nt = 0; nt < NT; ++nt) {
+#pragma unroll
+            for (int off = 4; off <= 16; off <<= 1) {
+                l_run[nt][0] += __shfl_xor_sync(0xffffffffu, l_run[nt][0], off);
+                l_run[nt][1] += __shfl_xor_sync(0xffffffffu, l_run[nt][1], off);
+            }
         }
         // Every warp is done reading the previous unit's results.  A warp may have given up on a
         // wait just before the others saw the flag: the barrier carries a vote, every warp gets
         // the same answer, the unit's result is voided and the block leaves together.
         const bool gave_up = block_sync_or(1, kConsumerThreads, failed || sm_flags[0] != 0);
         if (gave_up || stale) {
-            m_run[0] = m_run[1] = -INFINITY;
-            l_run[0] = l_run[1] = 0.f;
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                m_run[nt][0] = m_run[nt][1] = -INFINITY;
+                l_run[nt][0] = l_run[nt][1] = 0.f;
+            }
         }
         if (DUP) {
             // columns 4..7 carried the low parts of P for heads 0..3: lanes c = 2, 3 hand theirs to c = 0, 1
 #pragma unroll
             for (int mt = 0; mt < D / 16; ++mt)
 #pragma unroll
-                for (int i = 0; i < 4; ++i) oacc[mt][i] += __shfl_down_sync(0xffffffffu, oacc[mt][i], 2);
+                for (int i = 0; i < 4; ++i) oacc[mt][0][i] += __shfl_down_sync(0xffffffffu, oacc[mt][0][i], 2);
         }
         // The warps' states meet in the block's scratch four heads at a time (it holds [4 warps][4
-        // columns][D]): heads 4q .. 4q+3 live in lanes c = 2q, 2q+1 (all of a duplicated group in c = 0, 1).
+        // columns][D]): heads 4q .. 4q+3 live in tile q / 2, lanes c = 2 (q % 2), +1 (all of a duplicated
+        // group in c = 0, 1).
 #pragma unroll
-        for (int q = 0; q < (DUP ? 1 : 2); ++q) {
+        for (int q = 0; q < (DUP ? 1 : 2 * NT); ++q) {
             if (4 * q >= G) break;
+            const int nt = q >> 1;
             if (q > 0) block_sync(1, kConsumerThreads);                     // the scratch is free again
-            if ((c >> 1) == q) {
+            if ((c >> 1) == (q & 1)) {
                 const int lc = 2 * (c & 1);                                 // local columns lc, lc + 1
                 if (r == 0) {
-                    sm_wm[warp * COLS + lc] = m_run[0];
-                    sm_wm[warp * COLS + lc + 1] = m_run[1];
-                    sm_wl[warp * COLS + lc] = l_run[0];
-                    sm_wl[warp * COLS + lc + 1] = l_run[1];
+                    sm_wm[warp * COLS + lc] = m_run[nt][0];
+                    sm_wm[warp * COLS + lc + 1] = m_run[nt][1];
+                    sm_wl[warp * COLS + lc] = l_run[nt][0];
+                    sm_wl[warp * COLS + lc + 1] = l_run[nt][1];
                 }
                 float* wo = sm_wo + (warp * COLS + lc) * D;
 #pragma unroll
                 for (int mt = 0; mt < D / 16; ++mt) {
-                    wo[mt * 16 + r] = oacc[mt][0];
-                    wo[D + mt * 16 + r] = oacc[mt][1];
-                    wo[mt * 16 + r + 8] = oacc[mt][2];
-                    wo[D + mt * 16 + r + 8] = oacc[mt][3];
+                    wo[mt * 16 + r] = oacc[mt][nt][0];
+                    wo[D + mt * 16 + r] = oacc[mt][nt][1];
+                    wo[mt * 16 + r + 8] = oacc[mt][nt][2];
+                    wo[D + mt * 16 + r + 8] = oacc[mt][nt][3];
                 }
             }
             block_sync(1, kConsumerThreads);
@@ -916,7 +946,7 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
 
 // ---------------------------------------------------------------- host side
 
-inline bool mma_supports(int D, int G) { return (D == 64 || D == 128) && G >= 1 && G <= 8; }
+inline bool mma_supports(int D, int G) { return (D == 64 || D == 128) && G >= 1 && G <= 16; }
 
 typedef CUresult (*encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                     const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -964,6 +994,20 @@ template <int MODE>
 inline mma_kernel_t mma_kernel_for(int D, int G, bool prefix = false, bool f16 = false, bool masked = false)
 {
     const bool dup = G <= 4;
+    if (G > 8 && MODE == kModeAttend) {   // two tiles of heads; ordinary plans only
+        if (prefix) return nullptr;
+        if (D == 128)
+            return f16 ? (masked ? decode_attn_mma_kernel<128, false, kModeAttend, false, true, true, true>
+                                 : decode_attn_mma_kernel<128, false, kModeAttend, false, true, false, true>)
+                       : (masked ? decode_attn_mma_kernel<128, false, kModeAttend, false, false, true, true>
+                                 : decode_attn_mma_kernel<128, false, kModeAttend, false, false, false, true>);
+        if (D == 64)
+            return f16 ? (masked ? decode_attn_mma_kernel<64, false, kModeAttend, false, true, true, true>
+                                 : decode_attn_mma_kernel<64, false, kModeAttend, false, true, false, true>)
+                       : (masked ? decode_attn_mma_kernel<64, false, kModeAttend, false, false, true, true>
+                                 : decode_attn_mma_kernel<64, false, kModeAttend, false, false, false, true>);
+        return nullptr;
+    }
     if (masked && MODE == kModeAttend && !prefix) {
         if (D == 128)
             return f16 ? (dup ? decode_attn_mma_kernel<128, true, kModeAttend, false, true, true>

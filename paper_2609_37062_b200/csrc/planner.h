@@ -14,7 +14,7 @@ constexpr int kTileTokens = 16;                  // what the kernels fetch at a 
 constexpr int kDefaultAutoMinChunk = 256;         // tokens
 constexpr int kDefaultMaxSplits = 512;
 constexpr int kMaxSplits = 1024;  // hard bound on the splits of one sequence
-constexpr int kMaxGroup = 8;
+constexpr int kMaxGroup = 16;
 constexpr int kPrefixColumns = 16;  // query rows (sequence x head) one shared-prefix unit attends at once
 constexpr int kUmmaPrefixRows = 128;       // the same for the tcgen05 prefix kernel (the M dimension of its MMAs)
 

@@ -157,12 +157,18 @@ def test_max_splits_caps_the_split_count():
     assert splits[0] == 16
 
 
+def test_groups_of_up_to_16_heads_plan_like_any_other():
+    for hq in (72, 96, 128):                                  # groups of 9, 12, 16
+        units, splits, _, _, _ = layout([5000, 100], da.make_policy(), Hq=hq, Hkv=8)
+        covered_exactly_once(units, [5000, 100], 8)
+
+
 def test_invalid_shapes_and_policies_are_rejected():
     L = [100]
     ok = da.make_policy()
     bad = [
         (dict(Hq=30), ok, da.DA_ERR_INVALID_ARG),           # heads do not divide
-        (dict(Hq=128, Hkv=8), ok, da.DA_ERR_UNSUPPORTED),   # group of 16
+        (dict(Hq=136, Hkv=8), ok, da.DA_ERR_UNSUPPORTED),   # group of 17
         (dict(D=96), ok, da.DA_ERR_INVALID_ARG),            # stride rule holds but dim unsupported
         (dict(mpp=3), ok, da.DA_ERR_INVALID_ARG),           # block table row too short
         ({}, da.make_policy(split_mode=7), da.DA_ERR_INVALID_ARG),

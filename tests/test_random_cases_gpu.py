@@ -1,7 +1,7 @@
 """Seeded random cases through the C ABI against the oracle: shapes, length
 mixes with the awkward values (0, 1, page boundaries +-1), both kernels, all
 split modes, fused and separate merge, run masks, both pool layouts, both
-input types, page sizes, and
+input types, page sizes, groups of up to 16 heads, and
 shared-prefix plans on both prefix kernels.  What a case does not support is
 refused with DA_ERR_UNSUPPORTED, never computed wrongly."""
 import random
@@ -18,11 +18,11 @@ pytestmark = pytest.mark.gpu
 LENGTHS = [0, 1, 15, 16, 17, 31, 33, 64, 100, 255, 256, 257, 500, 1000, 1500, 2049, 3000]
 
 
-def one_case(rng, index, any_page_size=False):
+def one_case(rng, index, any_page_size=False, wide_groups=False):
     ps = rng.choice([16, 32, 64, 128, 256]) if any_page_size else 16
     D = rng.choice([64, 128])
     hkv = rng.choice([1, 2, 4, 8])
-    G = rng.choice([1, 2, 3, 4, 5, 8])
+    G = rng.choice([9, 10, 11, 12, 13, 14, 15, 16, 4, 7]) if wide_groups else rng.choice([1, 2, 3, 4, 5, 8])
     B = rng.choice([1, 2, 3, 5, 9, 17])
     lens = [rng.choice(LENGTHS) for _ in range(B)]
     mode = rng.choice([da.DA_SPLIT_AUTO, da.DA_SPLIT_DETERMINISTIC, da.DA_SPLIT_FIXED_COUNT])
@@ -48,12 +48,12 @@ def one_case(rng, index, any_page_size=False):
     return w, pol, mask
 
 
-@pytest.mark.parametrize("seed", [11, 12, 13, 14, 15])
+@pytest.mark.parametrize("seed", [11, 12, 13, 14, 15, 16, 17])
 def test_random_cases(seed):
     rng = random.Random(seed)
     refused = 0
     for index in range(60):
-        w, pol, mask = one_case(rng, index, any_page_size=seed >= 14)
+        w, pol, mask = one_case(rng, index, any_page_size=seed >= 14, wide_groups=seed >= 16)
         ref, ref_lse = oracle_of(w, run_mask=mask)
         m = None if mask is None else torch.tensor(mask, dtype=torch.uint8, device="cuda")
         try:
@@ -70,4 +70,4 @@ def test_random_cases(seed):
         assert np.array_equal(np.isneginf(got), np.isneginf(ref_lse)), what
         if fin.any():
             assert (np.abs(got[fin] - ref_lse[fin]) <= LSE_ABS + LSE_REL * np.abs(ref_lse[fin])).all(), what
-    assert refused < 30
+    assert refused < (45 if seed >= 16 else 30)      # (wide groups: neither the CUDA-core kernel nor prefix plans)
