@@ -74,7 +74,7 @@ typedef enum {
     DA_KERNEL_SIMT = 1,     /* CUDA-core kernel, 16-byte vectorised global loads; groups of up to 8   */
     DA_KERNEL_MMA_TMA = 2,  /* TMA-staged pages in shared memory, mma.sync (bf16 or fp16) for QK^T, PV;
                                groups of up to 16 heads (two 8-column tiles of heads above 8)         */
-    DA_KERNEL_UMMA_PREFIX = 3 /* shared-prefix plans only (head_dim 128, groups of 1 to 8 heads): the prefix
+    DA_KERNEL_UMMA_PREFIX = 3 /* shared-prefix plans only (head_dim 128, groups of 1 to 16 heads): the prefix
                                units run on the tcgen05 tensor cores, 128 query rows at a time with
                                accumulators in tensor memory; what follows the prefix runs as MMA_TMA */
 } da_kernel_t;
@@ -103,7 +103,7 @@ typedef struct {
                                every seq_len.  The prefix is then attended once per block of
                                sequences instead of once per sequence.  Tensor-core kernels only
                                (MMA_TMA: groups of up to 4 heads; UMMA_PREFIX: head_dim 128, groups of
-                               up to 8), separate combine, no capacity plan, not FIXED_COUNT.         */
+                               up to 16), separate combine, no capacity plan, not FIXED_COUNT.         */
     int32_t reserved[5];
 } decode_attn_policy_t;
 

@@ -79,8 +79,8 @@ constexpr int kUmmaTmemCols = 512;
 constexpr int kUmmaOutCol = 256;                  // first column of the output buffers
 constexpr int kUmmaOutRowBytes = 128 * 4 + 16;    // a staged output row; the pad spreads the rows over the banks
 
-// Any group of up to 8 heads: a unit takes floor(128 / G) sequences, rows past them stay empty.
-inline bool umma_supports(int D, int G) { return D == 128 && G >= 1 && G <= 8; }
+// Any group of up to 16 heads: a unit takes floor(128 / G) sequences, rows past them stay empty.
+inline bool umma_supports(int D, int G) { return D == 128 && G >= 1 && G <= 16; }
 
 __device__ __forceinline__ void bulk_store_s2g(void* dst, uint32_t src, uint32_t bytes)
 {

@@ -44,10 +44,12 @@ def test_full_few_shot_configuration(kernel):
     check(w, policy(1536, kernel))
 
 
-@pytest.mark.parametrize("hq,hkv", [(8, 8), (16, 8), (32, 8), (16, 2), (24, 8), (10, 2), (12, 2), (28, 4)])
+@pytest.mark.parametrize("hq,hkv", [(8, 8), (16, 8), (32, 8), (16, 2), (24, 8), (10, 2), (12, 2), (28, 4), (18, 2), (48, 4),
+                                    (13, 1), (128, 8)])
 def test_tcgen05_prefix_groups(hq, hkv):
-    """Groups of 1 to 8 heads (128 rows hold floor(128 / G) sequences; with 3, 5, 6 or 7 heads the
-    last rows of a unit stay empty); a prefix that is not a whole number of 128-token tiles
+    """Groups of 1 to 16 heads (128 rows hold floor(128 / G) sequences; where G does not divide 128
+    the last rows of a unit stay empty; what follows the prefix runs on the mma.sync kernel, with two
+    tiles of heads above 8); a prefix that is not a whole number of 128-token tiles
     (zero-filled tail pages) and more sequences than one 128-row block holds."""
     prefix = 13 * 16
     lens = [prefix + x for x in ([0, 1, 16, 17, 100, 255, 300, 31, 64] * (3 if hq // hkv >= 5 else 1))]
