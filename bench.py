@@ -42,7 +42,7 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the partial kernel, from the
 # ncu capture summarised under profiles/ (null until a capture of that workload exists).
 NCU_TRAFFIC_BYTES = {
-    "long_32k": 134_293_000 + 3_623_000,          # profiles/decode_attn_mma_kernel_long_32k.md
+    "long_32k": 134_300_000 + 3_362_000,          # profiles/decode_attn_mma_kernel_long_32k.md
     "sweep_8192x64": 2_148_308_000 + 4_320_000,   # profiles/decode_attn_mma_kernel_sweep_8192x64.md
 }
 
@@ -72,6 +72,8 @@ def parse_args():
                     help="sweep cells too large for memory: sequences i >= K reuse the pages of sequence i mod K")
     ap.add_argument("--in-dtype", default="bf16", choices=["bf16", "fp16"], help="type of q, K and V")
     ap.add_argument("--page-size", type=int, default=16, choices=[16, 32, 64, 128, 256], help="tokens per KV page")
+    ap.add_argument("--q-heads", type=int, default=32, choices=[8, 16, 24, 32, 40, 48, 56, 64, 72, 96, 128],
+                    help="query heads over the 8 KV heads of a sweep cell (groups of 1 to 16)")
     ap.add_argument("--prefix-aware", action="store_true",
                     help="shared_prefix workload: tell the planner about the common prefix (attended once per block of sequences)")
     ap.add_argument("--mask-fraction", type=float, default=None,
@@ -81,6 +83,7 @@ def parse_args():
 
 IN_DTYPE = "bf16"     # set from --in-dtype
 PAGE_SIZE = 16        # set from --page-size
+Q_HEADS = 32          # set from --q-heads (sweep cells)
 
 
 def make_workload(name, device, table_seed=None, seed_shift=0, alias_after=None):
@@ -103,7 +106,7 @@ def _make_workload_bf16(name, device, table_seed=None, seed_shift=0, alias_after
     if name.startswith("sweep_"):
         ctx, batch = name[len("sweep_"):].split("x")
         return wl.config_sweep_cell(int(ctx), int(batch), device=device, seed=4 + seed_shift, table_seed=table_seed,
-                                    alias_after=alias_after, page_size=PAGE_SIZE)
+                                    alias_after=alias_after, page_size=PAGE_SIZE, num_q_heads=Q_HEADS)
     raise SystemExit(f"unknown workload {name}")
 
 
@@ -197,7 +200,7 @@ def oracle_sample(name):
     if w is None:
         ctx, batch = (int(x) for x in name[len("sweep_"):].split("x"))
         keep = min(batch, max(1, 262144 // ctx))
-        w = wl.config_sweep_cell(ctx, keep)
+        w = wl.config_sweep_cell(ctx, keep, num_q_heads=Q_HEADS)
         return w, f"{keep} of {batch} sequences, extrapolated per token", 1.0
     return w, "whole batch", 1.0
 
@@ -248,9 +251,10 @@ def run_reference(args):
 
 def main():
     args = parse_args()
-    global IN_DTYPE, PAGE_SIZE
+    global IN_DTYPE, PAGE_SIZE, Q_HEADS
     IN_DTYPE = args.in_dtype
     PAGE_SIZE = args.page_size
+    Q_HEADS = args.q_heads
     if args.impl == "reference":
         run_reference(args)
         return

@@ -345,10 +345,10 @@ def config_shared_prefix(device="cpu", batch: int = 256, layout="token_major", s
 
 def config_sweep_cell(context: int, batch: int, device="cpu", layout="token_major", seed: int = 4,
                       alias_after: Optional[int] = None, table_seed: Optional[int] = None,
-                      page_size: int = 16) -> PagedWorkload:
+                      page_size: int = 16, num_q_heads: int = 32) -> PagedWorkload:
     """One cell of the length x batch sweep: `batch` sequences of `context`
     tokens; sequence i has the same content in every batch size."""
-    return make_workload(f"sweep_{context}x{batch}", [context] * batch, 32, 8, 128, seed=seed,
+    return make_workload(f"sweep_{context}x{batch}", [context] * batch, num_q_heads, 8, 128, seed=seed,
                          layout=layout, device=device, alias_after=alias_after, table_seed=table_seed,
                          page_size=page_size)
 
