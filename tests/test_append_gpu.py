@@ -13,7 +13,7 @@ pytestmark = pytest.mark.gpu
 
 
 @pytest.mark.parametrize("layout", ["token_major", "head_major"])
-@pytest.mark.parametrize("hq,hkv,d", [(8, 2, 64), (32, 8, 128)])
+@pytest.mark.parametrize("hq,hkv,d", [(8, 2, 64), (32, 8, 128), (24, 2, 128)])
 def test_append_then_attend(layout, hq, hkv, d):
     lens = [1, 16, 17, 300, 0, 1024, 1025, 77]
     w = wl.make_workload("append", lens, hq, hkv, d, seed=17, layout=layout, pool_pages=300)

@@ -93,6 +93,49 @@ def test_wide_group_deterministic_mode_is_bit_equal_across_batches():
             assert torch.equal(out[i], full[r]) and torch.equal(lse[i], full_lse[r]), (rows, r)
 
 
+def test_wide_group_static_step_host_step_and_captured_capacity_plan():
+    w = wl.make_workload("wide_s", [900, 40, 333, 0, 2100], 64, 4, 128, seed=49)
+    ref_out, ref_lse = oracle_of(w)
+    wd = to_device(w)
+    s = da.shape_of_workload(wd)
+    out = torch.empty((w.batch, 64, 128), dtype=torch.float32, device="cuda")
+    lse = torch.empty((w.batch, 64), dtype=torch.float32, device="cuda")
+    da.decode_attn_step_static(s, w.seq_lens, wd.q_bits, wd.k_pool, wd.v_pool, wd.block_table, wd.seq_lens, out, lse)
+    torch.cuda.synchronize()
+    assert_parity(out, lse, ref_out, ref_lse, "static step")
+    hout = torch.empty((w.batch, 64, 128), dtype=torch.float32).pin_memory()
+    da.decode_attn_host_step(s, da.make_policy(), w.q_bits, w.k_pool, w.v_pool, w.block_table, w.seq_lens, hout)
+    da.decode_attn_host_release()
+    assert_parity(hout, None, ref_out, ref_lse, "host step")
+    # a capacity plan captured once and replayed (buffers sized for the capacity, fixed addresses)
+    cap = 8
+
+    def padded(t):
+        full = torch.zeros((cap,) + tuple(t.shape[1:]), dtype=t.dtype, device="cuda")
+        full[: t.shape[0]] = t.cuda()
+        return full
+
+    pol = da.make_policy(capacity_batch=cap, capacity_tokens=16384, fuse_combine=1)
+    plan = da.decode_attn_plan(s, pol, w.seq_lens)
+    q, bt, sl = padded(w.q_bits), padded(w.block_table), padded(w.seq_lens)
+    cout = torch.zeros((cap, 64, 128), dtype=torch.float32, device="cuda")
+    clse = torch.zeros((cap, 64), dtype=torch.float32, device="cuda")
+    ws = torch.empty(max(plan.workspace_bytes, 256), dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        da.decode_attn_run(plan, q, wd.k_pool, wd.v_pool, bt, sl, cout, clse, ws, plan.workspace_bytes)
+        stream.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            da.decode_attn_run(plan, q, wd.k_pool, wd.v_pool, bt, sl, cout, clse, ws, plan.workspace_bytes)
+        cout.zero_()
+        graph.replay()
+        stream.synchronize()
+    assert da.decode_attn_last_device_status(plan) == da.DA_OK
+    assert_parity(cout[: w.batch], clse[: w.batch], ref_out, ref_lse, "captured capacity plan")
+    plan.destroy()
+
+
 def test_wide_groups_are_refused_where_unsupported():
     w = wl.make_workload("wide_no", [100, 300], 24, 2, 128, seed=1)
     with pytest.raises(da.DecodeAttnError) as e:
