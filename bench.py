@@ -57,6 +57,7 @@ def parse_args():
                     help="long_32k | short_chat | shared_prefix | sweep_<context>x<batch> | tiny")
     ap.add_argument("--split", default="auto", choices=["auto", "deterministic"])
     ap.add_argument("--chunk-tokens", type=int, default=0)
+    ap.add_argument("--max-splits", type=int, default=0, help="most splits of one sequence (0: the library default)")
     ap.add_argument("--kernel", default="auto", choices=["auto", "simt", "mma", "umma"])
     ap.add_argument("--fuse", action="store_true",
                     help="merge inside the partial kernel (one launch per step) instead of the combine kernel")
@@ -293,7 +294,7 @@ def main():
               "umma": da.DA_KERNEL_UMMA_PREFIX}[args.kernel]
     policy = da.make_policy(
         split_mode=da.DA_SPLIT_DETERMINISTIC if args.split == "deterministic" else da.DA_SPLIT_AUTO,
-        chunk_tokens=args.chunk_tokens, kernel=kernel, fuse_combine=1 if args.fuse else 0,
+        chunk_tokens=args.chunk_tokens, max_splits=args.max_splits, kernel=kernel, fuse_combine=1 if args.fuse else 0,
         ctas_per_sm=args.ctas_per_sm,
         shared_prefix_tokens=first.shared_prefix_tokens if args.prefix_aware else 0)
     shape = da.shape_of_workload(first)

@@ -65,7 +65,8 @@ enum { DA_DTYPE_BF16 = 1, DA_DTYPE_FP32 = 2, DA_DTYPE_FP16 = 3 };
 typedef enum {
     DA_SPLIT_AUTO = 0,          /* chunk length chosen from the length mix and the SM count          */
     DA_SPLIT_FIXED_COUNT = 1,   /* every sequence gets exactly fixed_count splits (some may be empty) */
-    DA_SPLIT_DETERMINISTIC = 2  /* boundaries at multiples of chunk_tokens: a function of seq_len only */
+    DA_SPLIT_DETERMINISTIC = 2  /* boundaries at multiples of chunk_tokens (of the longer chunk that
+                                   max_splits asks for on a long sequence): a function of seq_len only */
 } da_split_mode_t;
 
 typedef enum {
@@ -85,7 +86,8 @@ typedef struct {
     int32_t fixed_count;    /* FIXED_COUNT: splits per sequence (>= 1)                               */
     int32_t chunk_tokens;   /* DETERMINISTIC: chunk length, a multiple of 16 (0: 1024).
                                AUTO: smallest chunk the planner may choose (0: 256)                  */
-    int32_t max_splits;     /* upper bound on the splits of one sequence (0: 512; at most 1024)      */
+    int32_t max_splits;     /* upper bound on the splits of one sequence (0: 512, DETERMINISTIC 32;
+                               at most 1024); a longer sequence gets longer chunks                   */
     int32_t sm_count;       /* 0: the current device's multiprocessor count                          */
     int32_t kernel;         /* da_kernel_t                                                           */
     int32_t fuse_combine;   /* 0: decode_attn_combine must follow decode_attn_run.

@@ -13,6 +13,7 @@ constexpr int kDefaultDeterministicChunk = 1024;  // tokens
 constexpr int kTileTokens = 16;                  // what the kernels fetch at a time; pages hold a power-of-two number of these
 constexpr int kDefaultAutoMinChunk = 256;         // tokens
 constexpr int kDefaultMaxSplits = 512;
+constexpr int kDefaultDeterministicMaxSplits = 32;
 constexpr int kMaxSplits = 1024;  // hard bound on the splits of one sequence
 constexpr int kMaxGroup = 16;
 constexpr int kPrefixColumns = 16;  // query rows (sequence x head) one shared-prefix unit attends at once

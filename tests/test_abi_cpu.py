@@ -152,6 +152,22 @@ def test_fixed_count_gives_empty_trailing_splits():
     assert all(u.tok_end == u.tok_begin for u in mine[3:])
 
 
+def test_deterministic_default_bounds_the_splits_by_the_sequence_alone():
+    """At most 32 splits by default: a longer sequence gets longer chunks, whatever else is in the batch."""
+    det = da.make_policy(split_mode=da.DA_SPLIT_DETERMINISTIC)
+    expect = {32768: (32, 1024), 131072: (32, 4096), 40000: (32, 1264), 5000: (5, 1024), 100: (1, 1024)}
+    for batch in ([131072], [100, 40000, 131072, 5000, 32768], [32768] * 9 + [131072, 40000]):
+        units, splits, _, _, _ = layout(batch, det)
+        covered_exactly_once(units, batch, 8)
+        for b, L in enumerate(batch):
+            n, chunk = expect[L]
+            assert splits[b] == n
+            mine = sorted([u for u in units if u.seq == b and u.kv_head == 0], key=lambda u: u.split_index)
+            assert [u.tok_begin for u in mine] == [min(i * chunk, (L + 15) // 16 * 16) for i in range(n)]
+    units, splits, _, _, _ = layout([131072], da.make_policy(split_mode=da.DA_SPLIT_DETERMINISTIC, max_splits=512))
+    assert splits[0] == 128                                   # the old rule on request
+
+
 def test_max_splits_caps_the_split_count():
     units, splits, _, _, _ = layout([131072], da.make_policy(max_splits=16, chunk_tokens=16))
     assert splits[0] == 16

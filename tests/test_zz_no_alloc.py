@@ -61,8 +61,9 @@ def test_tiny_config_and_limits():
     assert rc == da.DA_ERR_WORKSPACE_TOO_SMALL
     long = wl.make_workload("long", [16], 32, 8, 128, seed=1, max_pages_per_seq=70000)
     s = da.shape_of_workload(long)
-    rc = da.decode_attn_step_static(s, [1_000_000], w.q_bits, w.k_pool, w.v_pool, w.block_table, w.seq_lens, out2,
-                                    check=False)
+    s.batch = 200                                            # 200 x 32 splits x 8 heads: more units than it holds
+    rc = da.decode_attn_step_static(s, [1_000_000] * 200, w.q_bits, w.k_pool, w.v_pool, w.block_table, w.seq_lens,
+                                    out2, check=False)
     assert rc == da.DA_ERR_WORKSPACE_TOO_SMALL
     torch.cuda.synchronize()
     assert not out2.any()
