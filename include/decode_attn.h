@@ -372,8 +372,9 @@ int decode_attn_host_step(const decode_attn_shape_t *shape, const decode_attn_po
  * The work list and the partial records live in a scratch array compiled
  * into the library (8 MiB of device memory, held by every GPU that loads the
  * library until the process exits).  The step is planned with the
- * deterministic split policy at its default chunk length (1,024 tokens), so
- * its result equals plan / run / combine with that policy.
+ * deterministic split policy at its defaults (1,024-token chunks, at most 32
+ * splits per sequence), so its result equals plan / run / combine with that
+ * policy.
  *
  * Limits: batch <= 1,024; at most 4,096 work units (batch x KV heads x
  * splits); the partial records must fit in about 7.8 MiB (e.g. 470 split
