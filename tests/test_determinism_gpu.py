@@ -91,3 +91,17 @@ def test_every_merge_kernel_gives_the_fused_path_its_bits(splits):
     a, la = da.run_workload(w, da.make_policy(fuse_combine=0, **pol))
     b, lb = da.run_workload(w, da.make_policy(fuse_combine=1, **pol))
     assert torch.equal(a, b) and torch.equal(la, lb)
+
+
+@pytest.mark.parametrize("kernel", KERNELS, ids=KERNEL_IDS)
+def test_sequences_beyond_the_default_split_bound(kernel):
+    """Past 32,768 tokens the default bound of 32 splits lengthens the chunks (40,000 tokens: 1,264 each): still a
+    function of the sequence's own length, so its bits do not change with the company it keeps."""
+    pol = da.make_policy(split_mode=da.DA_SPLIT_DETERMINISTIC, kernel=kernel)
+    out_a, lse_a, w = run([40000], [50], pol)
+    ref_out, ref_lse = oracle_of(to_device(w, "cpu"))
+    assert_parity(out_a, lse_a, ref_out, ref_lse)
+    out_b, lse_b, _ = run([700, 40000, 33000, 16], [51, 50, 52, 53], pol, table_seed=3)
+    assert torch.equal(out_a[0], out_b[1]) and torch.equal(lse_a[0], lse_b[1])
+    out_c, lse_c, _ = run([33000, 40000], [52, 50], pol, table_seed=4)
+    assert torch.equal(out_b[2], out_c[0]) and torch.equal(out_a[0], out_c[1])
