@@ -30,8 +30,8 @@
 // bf16(p - bf16(p)), and one PV mma accumulates both; the two halves are
 // added at the end.  For groups of 5..8 heads the low part takes a second
 // mma; groups of 9..16 heads are two such tiles of 8 columns side by side
-// (every K and V fragment feeds both).  P^T reaches the B-operand layout with one movmatrix transpose per
-// 8x8 block.
+// (every K and V fragment feeds both).  P^T reaches the B-operand layout
+// with one movmatrix transpose per 8x8 block.
 //
 // Every wait on an mbarrier is bounded; a wait that gives up records
 // DA_ERR_TIMEOUT and the block drains without touching the tiles.
