@@ -84,7 +84,9 @@ typedef enum {
 typedef struct {
     int32_t split_mode;     /* da_split_mode_t                                                       */
     int32_t fixed_count;    /* FIXED_COUNT: splits per sequence (>= 1)                               */
-    int32_t chunk_tokens;   /* DETERMINISTIC: chunk length, a multiple of 16 (0: 1024).
+    int32_t chunk_tokens;   /* DETERMINISTIC: chunk length, a multiple of 16 (0: 256; with the default
+                               max_splits a sequence of L tokens then gets chunks of
+                               max(256, L / 32 rounded up to 16) tokens).
                                AUTO: smallest chunk the planner may choose (0: 256)                  */
     int32_t max_splits;     /* upper bound on the splits of one sequence (0: 512, DETERMINISTIC 32;
                                at most 1024); a longer sequence gets longer chunks                   */
@@ -179,13 +181,22 @@ int decode_attn_plan_layout(const decode_attn_shape_t *shape, const decode_attn_
                             int32_t *chunk_tokens_out);
 
 /* Builds a plan for one decode step: validates shape and policy, runs the
- * planner on seq_lens_host [batch] (host), uploads the work list to a small
- * device buffer the plan owns (synchronously, on an internal stream) and
- * reports the workspace size run/combine need.  *plan_out is set only on
- * DA_OK.  The device buffer, its pinned mirror and the stream come from a
- * small cache fed by destroyed plans, so re-planning every step does not
- * allocate.  A plan is tied to the CUDA device current at creation and must not
- * be used by two launches that overlap on the GPU. */
+ * planner on seq_lens_host [batch] (host), starts the upload of the work list
+ * to a small device buffer the plan owns (on an internal stream, without
+ * waiting for it: the plan's first launch on a caller's stream is ordered
+ * behind the upload on the device) and reports the workspace size run/combine
+ * need.  *plan_out is set only on DA_OK.  The device buffer, its pinned mirror
+ * and the stream come from a small cache fed by destroyed plans, so
+ * re-planning every step does not allocate.  A plan is tied to the CUDA device
+ * current at creation and must not be used by two launches that overlap on
+ * the GPU.
+ *
+ * Lifetime: plan / run / combine / destroy may follow one another without any
+ * synchronisation - destroying a plan whose kernels are still queued or
+ * running is allowed; its device buffer is handed to a later plan only behind
+ * those kernels.  The one exception is stream capture: launches recorded into
+ * a CUDA graph run when the graph is replayed, so a plan must outlive every
+ * replay of a graph that holds its launches. */
 int decode_attn_plan(const decode_attn_shape_t *shape, const decode_attn_policy_t *policy,
                      const int32_t *seq_lens_host, decode_attn_plan_t **plan_out,
                      size_t *workspace_bytes_out);
@@ -279,6 +290,15 @@ int decode_attn_append_kv(const decode_attn_shape_t *shape, const void *new_k, c
                           const int32_t *block_table, const int32_t *seq_lens, void *k_cache, void *v_cache,
                           cudaStream_t stream);
 
+/* The same write with the device-side checks reported: a row whose page id lies
+ * outside the pool, or whose position lies beyond max_pages_per_seq, is not
+ * written (as above) and records DA_ERR_BAD_PAGE / DA_ERR_STALE_PLAN in the
+ * status word of `plan`, which decode_attn_last_device_status reads.  The
+ * shape is the plan's. */
+int decode_attn_append_kv_checked(const decode_attn_plan_t *plan, const void *new_k, const void *new_v,
+                                  const int32_t *block_table, const int32_t *seq_lens, void *k_cache,
+                                  void *v_cache, cudaStream_t stream);
+
 /* Merge of KV-range shards (context parallelism; the paper has no multi-GPU
  * path - this is the one exchange step the decode path has when a single
  * long sequence is sharded by token range).  Every shard attended its own
@@ -310,7 +330,9 @@ int decode_attn_combine(const decode_attn_plan_t *plan, const void *workspace, v
 
 /* Synchronises `stream`, returns the worst condition the kernels recorded
  * since the last call (DA_OK, DA_ERR_STALE_PLAN, DA_ERR_BAD_PAGE,
- * DA_ERR_TIMEOUT) and clears it.  For tests and debugging. */
+ * DA_ERR_TIMEOUT) and clears it.  For tests and debugging.  plan == NULL
+ * reads the status word of decode_attn_step_static (which has no plan) on the
+ * current device instead. */
 int decode_attn_last_device_status(const decode_attn_plan_t *plan, cudaStream_t stream);
 
 /* Host-only check of a block table against the shape: every entry below
@@ -344,6 +366,19 @@ int decode_attn_debug_gather(const decode_attn_plan_t *plan, int32_t seq, const 
 int decode_attn_gather_probe(const decode_attn_plan_t *plan, const void *k_cache, const void *v_cache,
                              const int32_t *block_table, uint32_t *checksum_out, cudaStream_t stream);
 
+/* Test hook for the bounded waits (failure detection without a fault): launches
+ * the plan's partial kernel exactly as decode_attn_run_ex would, except that
+ * its producer warps withhold their loads and every wait of the launch gives
+ * up after limit_cycles clock cycles (clamped to [100,000, the ordinary limit
+ * of about a second]) instead of the ordinary limit.  Nothing is at fault and
+ * nothing hangs: the waits run out, the blocks void their results and leave,
+ * DA_ERR_TIMEOUT is recorded in the plan's status word, and `out` holds no
+ * valid result.  After decode_attn_last_device_status has read (and cleared)
+ * that status the plan is good for ordinary launches again.  Plans of the
+ * MMA_TMA kernel only (DA_ERR_UNSUPPORTED otherwise). */
+int decode_attn_debug_expire_wait(const decode_attn_plan_t *plan, const decode_attn_run_args_t *args,
+                                  int64_t limit_cycles, cudaStream_t stream);
+
 /* ---------------------------------------------------------------------------
  * Whole step from host buffers: copies q, both pools, block table and
  * lengths to the device (into a grow-only arena the library keeps), plans,
@@ -372,9 +407,8 @@ int decode_attn_host_step(const decode_attn_shape_t *shape, const decode_attn_po
  * The work list and the partial records live in a scratch array compiled
  * into the library (8 MiB of device memory, held by every GPU that loads the
  * library until the process exits).  The step is planned with the
- * deterministic split policy at its defaults (1,024-token chunks, at most 32
- * splits per sequence), so its result equals plan / run / combine with that
- * policy.
+ * deterministic split policy at its defaults, so its result equals
+ * plan / run / combine with that policy.
  *
  * Limits: batch <= 1,024; at most 4,096 work units (batch x KV heads x
  * splits); the partial records must fit in about 7.8 MiB (e.g. 470 split
@@ -382,11 +416,22 @@ int decode_attn_host_step(const decode_attn_shape_t *shape, const decode_attn_po
  * beyond these returns DA_ERR_WORKSPACE_TOO_SMALL and launches nothing.
  *
  * All calls share the one array, which keeps whatever the previous call left
- * there; the call itself clears what has to start at zero.  Two calls whose
+ * there; nothing in it has to start at zero (every call uploads what its
+ * kernels read and writes its records before reading them).  Two calls whose
  * kernels overlap on the GPU (different streams, no ordering) race on it -
- * order them.  The first call on a device looks up the array's device
- * address and sets kernel attributes; make that first call outside any stream
- * capture.  Arguments are those of decode_attn_plan + decode_attn_run:
+ * order them.
+ *
+ * Not for stream capture: every call plans on the host and uploads its own
+ * work list (two small copies from pageable memory, taken by the runtime
+ * before the call returns), so a captured call would replay a stale list; a
+ * call on a capturing stream returns DA_ERR_UNSUPPORTED.  The first call on a
+ * device also looks up the array's device address and sets kernel attributes.
+ *
+ * Conditions its kernels detect on the device (lengths that differ from
+ * seq_lens_host, page ids outside the pool, a wait that gave up) void the
+ * affected rows and are recorded in a status word inside the array:
+ * decode_attn_last_device_status(NULL, stream) returns and clears it.
+ * Arguments are those of decode_attn_plan + decode_attn_run:
  * seq_lens_host [batch] on the host, everything else on the device.
  * ------------------------------------------------------------------------- */
 int decode_attn_step_static(const decode_attn_shape_t *shape, const int32_t *seq_lens_host, const void *q,

@@ -54,7 +54,7 @@ EXPORTED = [
     "decode_attn_host_step", "decode_attn_host_release", "decode_attn_strerror", "decode_attn_version",
     "decode_attn_step_static", "decode_attn_append_kv", "decode_attn_breakeven_tokens",
     "decode_attn_switch_thresholds", "decode_attn_switch_next", "decode_attn_validate_shared_prefix",
-    "decode_attn_merge_shards",
+    "decode_attn_merge_shards", "decode_attn_append_kv_checked", "decode_attn_debug_expire_wait",
 ]
 
 
@@ -126,6 +126,8 @@ _lib.decode_attn_host_step.argtypes = [ctypes.POINTER(Shape), ctypes.POINTER(Pol
 _lib.decode_attn_host_release.argtypes = []
 _lib.decode_attn_step_static.argtypes = [ctypes.POINTER(Shape), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.decode_attn_append_kv.argtypes = [ctypes.POINTER(Shape), _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.decode_attn_append_kv_checked.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.decode_attn_debug_expire_wait.argtypes = [_vp, ctypes.POINTER(RunArgs), ctypes.c_int64, _vp]
 _lib.decode_attn_merge_shards.argtypes = [ctypes.POINTER(Shape), ctypes.c_int32, _vp, _vp, _vp, _vp, _vp]
 _lib.decode_attn_breakeven_tokens.argtypes = [ctypes.c_double, ctypes.c_double, ctypes.c_double, ctypes.c_int32,
                                               ctypes.c_double, ctypes.POINTER(ctypes.c_double)]
@@ -323,8 +325,23 @@ def decode_attn_combine(plan: Plan, workspace, out, lse=None, stream=None, check
     return rc
 
 
-def decode_attn_last_device_status(plan: Plan, stream=None) -> int:
-    return _lib.decode_attn_last_device_status(plan.handle, _stream(stream))
+def decode_attn_last_device_status(plan: Optional[Plan], stream=None) -> int:
+    """plan None: the status word of decode_attn_step_static on the current device."""
+    return _lib.decode_attn_last_device_status(plan.handle if plan is not None else None, _stream(stream))
+
+
+def decode_attn_debug_expire_wait(plan: Plan, q, k_cache, v_cache, block_table, seq_lens, out, lse=None,
+                                  workspace=None, workspace_bytes: Optional[int] = None, limit_cycles: int = 2_000_000,
+                                  stream=None) -> int:
+    """Test hook: the plan's partial kernel with its loads withheld and its waits cut to limit_cycles."""
+    if workspace_bytes is None:
+        workspace_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    a = RunArgs()
+    a.struct_size = ctypes.sizeof(RunArgs)
+    a.q, a.k_cache, a.v_cache = _ptr(q), _ptr(k_cache), _ptr(v_cache)
+    a.block_table, a.seq_lens = _ptr(block_table), _ptr(seq_lens)
+    a.out, a.lse, a.workspace, a.workspace_bytes = _ptr(out), _ptr(lse), _ptr(workspace), workspace_bytes
+    return _lib.decode_attn_debug_expire_wait(plan.handle, ctypes.byref(a), int(limit_cycles), _stream(stream))
 
 
 def decode_attn_validate_block_table(shape: Shape, seq_lens_host, block_table_host) -> int:
@@ -376,6 +393,15 @@ def decode_attn_append_kv(shape: Shape, new_k, new_v, block_table, seq_lens, k_c
                                     _ptr(k_cache), _ptr(v_cache), _stream(stream))
     if check:
         _check(rc, "decode_attn_append_kv")
+    return rc
+
+
+def decode_attn_append_kv_checked(plan: Plan, new_k, new_v, block_table, seq_lens, k_cache, v_cache, stream=None,
+                                  check: bool = True) -> int:
+    rc = _lib.decode_attn_append_kv_checked(plan.handle, _ptr(new_k), _ptr(new_v), _ptr(block_table), _ptr(seq_lens),
+                                            _ptr(k_cache), _ptr(v_cache), _stream(stream))
+    if check:
+        _check(rc, "decode_attn_append_kv_checked")
     return rc
 
 

@@ -58,6 +58,8 @@ struct decode_attn_plan {
     int max_bins = 0;        // > 0: the units are packed into per-block ranges (persistent tensor-core kernel)
     cudaStream_t stream = nullptr;
     cudaEvent_t upload_done = nullptr;  // last refresh of the device work list
+    cudaEvent_t launch_done = nullptr;  // behind the plan's last launch on a caller's stream (not while capturing)
+    mutable bool upload_pending = false;   // the first upload may still be in flight on the plan's own stream
     void* buffers = nullptr;            // PlanBuffers*, returned to the cache on destroy
 };
 
@@ -87,7 +89,8 @@ struct PlanBuffers {
     char* pinned = nullptr;
     size_t dev_bytes = 0, pinned_bytes = 0;
     cudaStream_t stream = nullptr;
-    cudaEvent_t event = nullptr;
+    cudaEvent_t event = nullptr;        // upload of the work list
+    cudaEvent_t launched = nullptr;     // behind the last kernel that reads the device buffer
 };
 
 void free_buffers(PlanBuffers& b)
@@ -95,6 +98,10 @@ void free_buffers(PlanBuffers& b)
     if (b.stream) {
         cudaStreamSynchronize(b.stream);
         cudaStreamDestroy(b.stream);
+    }
+    if (b.launched) {
+        cudaEventSynchronize(b.launched);     // kernels of the plan that held these buffers may still run
+        cudaEventDestroy(b.launched);
     }
     if (b.event) cudaEventDestroy(b.event);
     if (b.dev) cudaFree(b.dev);
@@ -135,6 +142,7 @@ int acquire_buffers(int device, size_t dev_bytes, size_t pinned_bytes, PlanBuffe
     b.pinned_bytes = round_pow2(pinned_bytes);
     if (cudaStreamCreateWithFlags(&b.stream, cudaStreamNonBlocking) != cudaSuccess ||
         cudaEventCreateWithFlags(&b.event, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&b.launched, cudaEventDisableTiming) != cudaSuccess ||
         cudaMalloc(&b.dev, b.dev_bytes) != cudaSuccess || cudaMallocHost(&b.pinned, b.pinned_bytes) != cudaSuccess) {
         (void)cudaGetLastError();
         free_buffers(b);
@@ -144,12 +152,13 @@ int acquire_buffers(int device, size_t dev_bytes, size_t pinned_bytes, PlanBuffe
     return DA_OK;
 }
 
+// Parks the buffers of a destroyed plan without waiting for the device: kernels of that plan may
+// still be running on the caller's stream (a step is plan / run / combine / destroy with no
+// synchronisation in between).  Whoever takes the buffers next orders its upload behind `launched`
+// (see decode_attn_plan) and waits for `event` on the host before it rewrites the pinned mirror.
 void release_buffers(PlanBuffers& b)
 {
     if (!b.dev) return;
-    if (b.stream) cudaStreamSynchronize(b.stream);
-    if (b.event) cudaEventSynchronize(b.event);
-    (void)cudaGetLastError();
     {
         std::lock_guard<std::mutex> lock(g_buffers.mu);
         if (g_buffers.free_list.size() < BufferCache::kMaxParked) {
@@ -372,6 +381,7 @@ KernelParams make_params(const decode_attn_plan_t* pl, const decode_attn_run_arg
     kp.fused = pl->policy.fuse_combine;
     kp.grid_exit = pl->policy.capacity_batch > 0;
     kp.n_units = (int32_t)pl->layout.units.size();
+    kp.wait_limit = kWaitLimitCycles;
     // The tensor-core kernel asks the first pages of every block into L2 ahead of its dependency
     // wait.  Two stages' worth when a block has a single unit (the opening burst is then a visible
     // share of the step: 24.9 -> 23.0 us on one 32k sequence), one stage's worth otherwise
@@ -388,6 +398,56 @@ KernelParams make_params(const decode_attn_plan_t* pl, const decode_attn_run_arg
 }
 
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+bool stream_is_capturing(cudaStream_t stream)
+{
+    cudaStreamCaptureStatus st = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(stream, &st) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return false;
+    }
+    return st != cudaStreamCaptureStatusNone;
+}
+
+// A plan's work list is uploaded on the plan's own stream without waiting for it.  Every launch
+// that reads the device buffer is ordered behind that upload: a device-side wait on the caller's
+// stream while the copy may still be in flight (a host-side one while that stream is being
+// captured, so that no outside event enters the graph), nothing once it is known to be complete.
+int order_behind_upload(const decode_attn_plan_t* pl, cudaStream_t stream)
+{
+    if (!pl->upload_pending) return DA_OK;
+    const cudaError_t q = cudaEventQuery(pl->upload_done);
+    if (q == cudaSuccess) {
+        pl->upload_pending = false;
+        return DA_OK;
+    }
+    (void)cudaGetLastError();
+    if (q != cudaErrorNotReady) return DA_ERR_CUDA;
+    if (stream_is_capturing(stream)) {
+        DA_CUDA_TRY(cudaEventSynchronize(pl->upload_done));
+        pl->upload_pending = false;
+        return DA_OK;
+    }
+    DA_CUDA_TRY(cudaStreamWaitEvent(stream, pl->upload_done, 0));
+    return DA_OK;
+}
+
+// Marks the end of the plan's launches on a caller's stream, so that the plan's device buffer is
+// not handed to another plan's upload while they run (see release_buffers).  Launches that are
+// being captured into a graph run later, at replay: a plan must outlive the replays of a graph
+// that holds its launches, as the header says.
+void mark_launched(const decode_attn_plan_t* pl, cudaStream_t stream)
+{
+    if (pl->launch_done == nullptr || stream_is_capturing(stream)) return;
+    if (cudaEventRecord(pl->launch_done, stream) != cudaSuccess) (void)cudaGetLastError();
+}
+
+// marks the plan's launch on scope exit (for the entry points that return the launch's status)
+struct mma_launch_guard {
+    const decode_attn_plan_t* pl;
+    cudaStream_t stream;
+    ~mma_launch_guard() { mark_launched(pl, stream); }
+};
 
 }  // namespace
 
@@ -489,11 +549,21 @@ int decode_attn_plan(const decode_attn_shape_t* shape, const decode_attn_policy_
     pl->pinned = pb->pinned;
     pl->stream = pb->stream;
     pl->upload_done = pb->event;
+    pl->launch_done = pb->launched;
+    // Buffers that come from a destroyed plan: that plan's last upload has to be out of the pinned
+    // mirror before the host rewrites it (long done in practice; a host wait only if not), and its
+    // kernels, which may still be running on their caller's stream, have to be done with the device
+    // buffer before the new work list lands there (ordered on the device, no host wait).
+    DA_CUDA_TRY(cudaEventSynchronize(pl->upload_done));
+    DA_CUDA_TRY(cudaStreamWaitEvent(pl->stream, pl->launch_done, 0));
     // one copy: work list, split table, block ranges, and zeros for the status word and tickets
     std::memset(pl->pinned + pl->off_status, 0, pl->total_bytes - pl->off_status);
     fill_host_mirror(pl);
+    // The upload is not waited for here: the first launch on a caller's stream is ordered behind it
+    // (order_behind_upload), so planning costs no round trip to the device.
     DA_CUDA_TRY(cudaMemcpyAsync(pl->dev, pl->pinned, pl->total_bytes, cudaMemcpyHostToDevice, pl->stream));
-    DA_CUDA_TRY(cudaStreamSynchronize(pl->stream));
+    DA_CUDA_TRY(cudaEventRecord(pl->upload_done, pl->stream));
+    pl->upload_pending = true;
 
     if (workspace_bytes_out) *workspace_bytes_out = pl->workspace_bytes;
     *plan_out = pl;
@@ -517,6 +587,7 @@ int decode_attn_plan_update(decode_attn_plan_t* pl, int32_t batch, const int32_t
     if ((int64_t)lay.units.size() > pl->max_units || lay.n_slots > pl->max_slots) return DA_ERR_INVALID_ARG;
     // the previous refresh may still be reading the pinned mirror
     DA_CUDA_TRY(cudaEventSynchronize(pl->upload_done));
+    pl->upload_pending = false;
     pl->shape.batch = batch;
     pl->layout = std::move(lay);
     pl->seq_lens.assign(seq_lens_host, seq_lens_host + batch);
@@ -575,7 +646,8 @@ int decode_attn_plan_destroy(decode_attn_plan_t* pl)
     return DA_OK;
 }
 
-int decode_attn_run_ex(const decode_attn_plan_t* pl, const decode_attn_run_args_t* a, cudaStream_t stream)
+// debug_limit > 0: the launch of decode_attn_debug_expire_wait (loads withheld, waits cut short).
+static int run_impl(const decode_attn_plan_t* pl, const decode_attn_run_args_t* a, cudaStream_t stream, long long debug_limit)
 {
     if (!pl || !a) return DA_ERR_INVALID_ARG;
     if (a->struct_size != sizeof(decode_attn_run_args_t) || a->flags != 0) return DA_ERR_INVALID_ARG;
@@ -590,7 +662,17 @@ int decode_attn_run_ex(const decode_attn_plan_t* pl, const decode_attn_run_args_
     }
     const bool umma = pl->kernel == DA_KERNEL_UMMA_PREFIX;
     if (pl->grid == 0 && !(umma && pl->layout.n_front_units > 0)) return DA_OK;
-    const KernelParams kp = make_params(pl, *a);
+    {
+        const int rc = order_behind_upload(pl, stream);
+        if (rc != DA_OK) return rc;
+    }
+    KernelParams kp = make_params(pl, *a);
+    if (debug_limit > 0) {
+        if (pl->kernel != DA_KERNEL_MMA_TMA) return DA_ERR_UNSUPPORTED;
+        kp.wait_limit = debug_limit;
+        kp.debug_drop_loads = 1;
+        kp.hint_first_pages = 0;
+    }
     if (pl->kernel == DA_KERNEL_SIMT) {
         simt_kernel_t fn = simt_kernel_for(pl->shape.head_dim, pl->group);
         if (!fn) return DA_ERR_UNSUPPORTED;
@@ -625,7 +707,22 @@ int decode_attn_run_ex(const decode_attn_plan_t* pl, const decode_attn_run_args_
         }
     }
     DA_CUDA_TRY(cudaGetLastError());
+    mark_launched(pl, stream);
     return DA_OK;
+}
+
+int decode_attn_run_ex(const decode_attn_plan_t* pl, const decode_attn_run_args_t* a, cudaStream_t stream)
+{
+    return run_impl(pl, a, stream, 0);
+}
+
+int decode_attn_debug_expire_wait(const decode_attn_plan_t* pl, const decode_attn_run_args_t* a, int64_t limit_cycles,
+                                  cudaStream_t stream)
+{
+    if (limit_cycles <= 0) return DA_ERR_INVALID_ARG;
+    // between 50 microseconds and the ordinary limit, whatever was asked for
+    const long long limit = std::min<long long>(std::max<long long>(limit_cycles, 100000LL), kWaitLimitCycles);
+    return run_impl(pl, a, stream, limit);
 }
 
 int decode_attn_run(const decode_attn_plan_t* pl, const void* q, const void* k_cache, const void* v_cache,
@@ -656,11 +753,14 @@ int decode_attn_combine(const decode_attn_plan_t* pl, const void* workspace, voi
     const KernelParams kp = make_params(pl, a);
     const unsigned grid = (unsigned)(pl->max_batch * pl->shape.num_kv_heads);
     if (grid == 0) return DA_OK;
+    int rc = order_behind_upload(pl, stream);
+    if (rc != DA_OK) return rc;
     // a capacity plan may be refreshed to any split count its policy allows
     const int max_splits = pl->policy.capacity_batch > 0 ? kMaxSplits : pl->layout.max_splits_used;
-    int rc = combine_launch(pl->shape.head_dim, pl->group, kp, grid, stream, max_splits);
+    rc = combine_launch(pl->shape.head_dim, pl->group, kp, grid, stream, max_splits);
     if (rc != DA_OK) return rc;
     DA_CUDA_TRY(cudaGetLastError());
+    mark_launched(pl, stream);
     return DA_OK;
 }
 
@@ -684,10 +784,14 @@ int decode_attn_merge_shards(const decode_attn_shape_t* shape, int32_t n_shards,
     return DA_OK;
 }
 
+static int static_step_status(cudaStream_t stream);
+
 int decode_attn_last_device_status(const decode_attn_plan_t* pl, cudaStream_t stream)
 {
-    if (!pl) return DA_ERR_INVALID_ARG;
+    if (!pl) return static_step_status(stream);     // the allocation-free step has no plan: its status word
     int32_t st = 0;
+    DA_CUDA_TRY(cudaEventSynchronize(pl->upload_done));
+    pl->upload_pending = false;
     DA_CUDA_TRY(cudaStreamSynchronize(stream));
     DA_CUDA_TRY(cudaMemcpy(&st, pl->dev + pl->off_status, sizeof st, cudaMemcpyDeviceToHost));
     if (st != 0) {
@@ -748,6 +852,8 @@ int decode_attn_debug_gather(const decode_attn_plan_t* pl, int32_t seq, const vo
     a.k_cache = k_cache; a.v_cache = v_cache; a.block_table = block_table;
     const KernelParams kp = make_params(pl, a);
     if (pl->kernel == DA_KERNEL_UMMA_PREFIX) return DA_ERR_UNSUPPORTED;
+    if (order_behind_upload(pl, stream) != DA_OK) return DA_ERR_CUDA;
+    mma_launch_guard guard{pl, stream};
     return mma_debug_gather(pl->shape, pl->group, kp, seq, k_out, v_out, (unsigned)pl->work_grid, stream);
 }
 
@@ -762,13 +868,15 @@ int decode_attn_gather_probe(const decode_attn_plan_t* pl, const void* k_cache, 
     std::memset(&a, 0, sizeof a);
     a.k_cache = k_cache; a.v_cache = v_cache; a.block_table = block_table;
     const KernelParams kp = make_params(pl, a);
+    if (order_behind_upload(pl, stream) != DA_OK) return DA_ERR_CUDA;
+    mma_launch_guard guard{pl, stream};
     return mma_gather_probe(pl->shape, pl->group, kp, checksum_out, (unsigned)pl->layout.units.size(), (unsigned)pl->work_grid,
                             stream);
 }
 
-int decode_attn_append_kv(const decode_attn_shape_t* shape, const void* new_k, const void* new_v,
-                          const int32_t* block_table, const int32_t* seq_lens, void* k_cache, void* v_cache,
-                          cudaStream_t stream)
+static int append_impl(const decode_attn_shape_t* shape, int32_t* status, const void* new_k, const void* new_v,
+                       const int32_t* block_table, const int32_t* seq_lens, void* k_cache, void* v_cache,
+                       cudaStream_t stream)
 {
     if (!shape || !new_k || !new_v || !block_table || !seq_lens || !k_cache || !v_cache) return DA_ERR_INVALID_ARG;
     int rc = validate_shape(*shape);
@@ -784,7 +892,7 @@ int decode_attn_append_kv(const decode_attn_shape_t* shape, const void* new_k, c
     ap.v = static_cast<__nv_bfloat16*>(v_cache);
     ap.block_table = block_table;
     ap.seq_lens = seq_lens;
-    ap.status = nullptr;
+    ap.status = status;
     ap.k_stride_page = shape->k_stride_page; ap.k_stride_token = shape->k_stride_token; ap.k_stride_head = shape->k_stride_head;
     ap.v_stride_page = shape->v_stride_page; ap.v_stride_token = shape->v_stride_token; ap.v_stride_head = shape->v_stride_head;
     ap.num_pages = shape->num_pages;
@@ -810,6 +918,26 @@ int decode_attn_append_kv(const decode_attn_shape_t* shape, const void* new_k, c
         return DA_ERR_CUDA;
     }
     return DA_OK;
+}
+
+int decode_attn_append_kv(const decode_attn_shape_t* shape, const void* new_k, const void* new_v,
+                          const int32_t* block_table, const int32_t* seq_lens, void* k_cache, void* v_cache,
+                          cudaStream_t stream)
+{
+    return append_impl(shape, nullptr, new_k, new_v, block_table, seq_lens, k_cache, v_cache, stream);
+}
+
+int decode_attn_append_kv_checked(const decode_attn_plan_t* pl, const void* new_k, const void* new_v,
+                                  const int32_t* block_table, const int32_t* seq_lens, void* k_cache, void* v_cache,
+                                  cudaStream_t stream)
+{
+    if (!pl) return DA_ERR_INVALID_ARG;
+    int rc = order_behind_upload(pl, stream);      // the upload also zeroes the status word this launch may write
+    if (rc != DA_OK) return rc;
+    rc = append_impl(&pl->shape, reinterpret_cast<int32_t*>(pl->dev + pl->off_status), new_k, new_v, block_table,
+                     seq_lens, k_cache, v_cache, stream);
+    if (rc == DA_OK) mark_launched(pl, stream);
+    return rc;
 }
 
 // ------------------------------------------------------------------ host-buffer step
@@ -935,12 +1063,13 @@ static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBy
 
 namespace {
 
-constexpr size_t kStaticOffUnits = 256;                                                   // header first
-constexpr size_t kStaticOffSeqInfo = kStaticOffUnits + sizeof(decode_attn_unit_t) * kStaticMaxUnits;
-constexpr size_t kStaticOffStatus = kStaticOffSeqInfo + sizeof(SeqInfo) * kStaticMaxBatch;
-constexpr size_t kStaticOffTickets = kStaticOffStatus + 256;
-constexpr size_t kStaticOffRecords = (kStaticOffTickets + 2 * sizeof(int32_t) * kStaticMaxBatch * 8 + 255) / 256 * 256;
-static_assert(kStaticOffRecords < kStaticScratchBytes, "static scratch layout");
+// header | split table | work list | status word | records.  The split table sits in front of the
+// work list so that each of the two uploads is as long as the step needs and no longer.
+constexpr size_t kStaticOffSeqInfo = 256;
+constexpr size_t kStaticOffUnits = kStaticOffSeqInfo + sizeof(SeqInfo) * kStaticMaxBatch;
+constexpr size_t kStaticOffStatus = kStaticOffUnits + sizeof(decode_attn_unit_t) * kStaticMaxUnits;
+constexpr size_t kStaticOffRecords = kStaticOffStatus + 256;
+static_assert(kStaticOffRecords % 256 == 0 && kStaticOffRecords < kStaticScratchBytes, "static scratch layout");
 
 struct StaticSetup {
     std::mutex mu;
@@ -953,6 +1082,27 @@ struct StaticSetup {
 
 }  // namespace
 
+// Status word of decode_attn_step_static on the current device: synchronises `stream`, returns the
+// worst condition its kernels recorded since the last call and clears it.  Copies through the
+// static array's address; allocates nothing.
+static int static_step_status(cudaStream_t stream)
+{
+    int dev = -1;
+    DA_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= StaticSetup::kMaxDevices) return DA_ERR_UNSUPPORTED;
+    unsigned char* base = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_static.mu);
+        base = g_static.base[dev];
+    }
+    if (base == nullptr) return DA_OK;              // no static step has run on this device yet
+    int32_t st = 0;
+    DA_CUDA_TRY(cudaStreamSynchronize(stream));
+    DA_CUDA_TRY(cudaMemcpy(&st, base + kStaticOffStatus, sizeof st, cudaMemcpyDeviceToHost));
+    if (st != 0) DA_CUDA_TRY(cudaMemset(base + kStaticOffStatus, 0, sizeof(int32_t)));
+    return st;
+}
+
 int decode_attn_step_static(const decode_attn_shape_t* shape, const int32_t* seq_lens_host, const void* q,
                             const void* k_cache, const void* v_cache, const int32_t* block_table,
                             const int32_t* seq_lens, void* out, float* lse_or_null, cudaStream_t stream)
@@ -963,7 +1113,10 @@ int decode_attn_step_static(const decode_attn_shape_t* shape, const int32_t* seq
     if (rc != DA_OK) return rc;
     if (!aligned(q, 16) || !aligned(k_cache, 16) || !aligned(v_cache, 16) || !aligned(out, 16)) return DA_ERR_INVALID_ARG;
     if (shape->batch == 0) return DA_OK;
-    if (shape->batch > kStaticMaxBatch || shape->num_kv_heads > 8) return DA_ERR_WORKSPACE_TOO_SMALL;
+    if (shape->batch > kStaticMaxBatch) return DA_ERR_WORKSPACE_TOO_SMALL;
+    // Every call plans on the host and uploads its own work list, so a captured call would replay
+    // a stale one: refuse instead.
+    if (stream_is_capturing(stream)) return DA_ERR_UNSUPPORTED;
 
     decode_attn_policy_t policy;
     std::memset(&policy, 0, sizeof policy);
@@ -985,6 +1138,7 @@ int decode_attn_step_static(const decode_attn_shape_t* shape, const int32_t* seq
         int block_threads = 0, dyn_smem = 0;
         if (query_occupancy(kernel, shape->head_dim, G, &block_threads, &dyn_smem) <= 0) return DA_ERR_CUDA;
         DA_CUDA_TRY(cudaDeviceGetAttribute(&g_static.sm_count[dev], cudaDevAttrMultiProcessorCount, dev));
+        // (a __device__ array without an initialiser starts zeroed: the status word reads DA_OK)
         g_static.base[dev] = static_cast<unsigned char*>(ptr);
     } else if (kernel == DA_KERNEL_MMA_TMA) {
         int block_threads = 0, dyn_smem = 0;       // another head_dim / group may need its own opt-in
@@ -1014,11 +1168,16 @@ int decode_attn_step_static(const decode_attn_shape_t* shape, const int32_t* seq
         si[b].seq_len = seq_lens_host[b];
         si[b].pad = 0;
     }
-    const size_t upload = kStaticOffSeqInfo + sizeof(SeqInfo) * (size_t)shape->batch;
-    // The array keeps the previous call's contents: the status word and tickets must start at zero.
-    DA_CUDA_TRY(cudaMemsetAsync(base + kStaticOffStatus, 0, kStaticOffRecords - kStaticOffStatus, stream));
-    // Pageable source: the runtime stages the bytes before returning, so the staging area may be reused.
-    DA_CUDA_TRY(cudaMemcpyAsync(base, g_static.staging, upload, cudaMemcpyHostToDevice, stream));
+    // The array keeps the previous call's contents.  What the kernels only read is overwritten by
+    // the two uploads below, records are written before they are read, and the status word is
+    // cumulative on purpose (decode_attn_last_device_status(NULL, ...) reads and clears it), so
+    // nothing needs zeroing here.
+    // Pageable source: the runtime has taken the bytes when the call returns, so the staging area
+    // may be reused by the next call.
+    DA_CUDA_TRY(cudaMemcpyAsync(base, g_static.staging, kStaticOffSeqInfo + sizeof(SeqInfo) * (size_t)shape->batch,
+                                cudaMemcpyHostToDevice, stream));
+    DA_CUDA_TRY(cudaMemcpyAsync(base + kStaticOffUnits, g_static.staging + kStaticOffUnits,
+                                lay.units.size() * sizeof(decode_attn_unit_t), cudaMemcpyHostToDevice, stream));
 
     KernelParams kp;
     std::memset(&kp, 0, sizeof kp);
@@ -1033,7 +1192,7 @@ int decode_attn_step_static(const decode_attn_shape_t* shape, const int32_t* seq
     kp.header = reinterpret_cast<const DevHeader*>(base);
     kp.units = reinterpret_cast<const decode_attn_unit_t*>(base + kStaticOffUnits);
     kp.seq_info = reinterpret_cast<const SeqInfo*>(base + kStaticOffSeqInfo);
-    kp.tickets = reinterpret_cast<int32_t*>(base + kStaticOffTickets);
+    kp.tickets = nullptr;                           // only fused plans count arrivals; this step is not one
     kp.status = reinterpret_cast<int32_t*>(base + kStaticOffStatus);
     kp.k_stride_page = shape->k_stride_page; kp.k_stride_token = shape->k_stride_token; kp.k_stride_head = shape->k_stride_head;
     kp.v_stride_page = shape->v_stride_page; kp.v_stride_token = shape->v_stride_token; kp.v_stride_head = shape->v_stride_head;
@@ -1048,10 +1207,10 @@ int decode_attn_step_static(const decode_attn_shape_t* shape, const int32_t* seq
     kp.tile_shift = log2_of(shape->page_size) - 4;
     kp.fused = 0;
     kp.grid_exit = 0;
+    kp.wait_limit = kWaitLimitCycles;
     kp.n_units = (int32_t)lay.units.size();
     kp.n_work_blocks = (int32_t)lay.units.size();
     kp.batch = shape->batch;
-    kp.ticket_stride = kStaticMaxBatch * 8;
 
     const unsigned grid = (unsigned)lay.units.size();
     if (kernel == DA_KERNEL_SIMT) {

@@ -69,6 +69,12 @@ struct KernelParams {
     // (late_wait), so that what follows the pair still sees both complete.
     int32_t early_trigger;
     int32_t late_wait;
+    // Bounded waits of the tensor-core kernel and of the merge blocks give up after this many
+    // clock cycles (kWaitLimitCycles in every ordinary launch).
+    long long wait_limit;
+    // Test hook (decode_attn_debug_expire_wait): the producer withholds its loads, so that the
+    // waits of the launch run out and its give-up path is exercised with nothing at fault.
+    int32_t debug_drop_loads;
 #ifdef DA_TRACE
     unsigned long long* trace;  // debug builds: 32 stamps per block, or NULL
 #endif
@@ -249,13 +255,13 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)
 
 constexpr long long kWaitLimitCycles = 2000000000LL;  // about one second
 
-// Bounded wait: false if the phase did not complete within the limit.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
+// Bounded wait: false if the phase did not complete within `limit` clock cycles.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, long long limit = kWaitLimitCycles)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     while (!mbar_try_wait(bar, parity)) {
-        if (clock64() - t0 > kWaitLimitCycles) return false;
+        if (clock64() - t0 > limit) return false;
     }
     return true;
 }
@@ -463,7 +469,7 @@ __device__ __forceinline__ void fused_merge_blocks(const KernelParams& p, int G,
             while (ld_acquire(arrivals) < si.n_splits) {
                 // give up after the limit, or at once when an attending block already gave up
                 // on a wait of its own (it will not publish the rest of its records)
-                if (clock64() - t0 > kWaitLimitCycles || ld_acquire(p.status) <= DA_ERR_TIMEOUT) {
+                if (clock64() - t0 > p.wait_limit || ld_acquire(p.status) <= DA_ERR_TIMEOUT) {
                     ok = 0;
                     break;
                 }

@@ -424,7 +424,7 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
                 const int s = git % NS;
                 if (git >= (uint32_t)NS) {
                     bool ok = true;
-                    if (lane == 0) ok = mbar_wait(bar_base + 8 * (NS + s), ((git / NS) & 1) ^ 1);
+                    if (lane == 0) ok = mbar_wait(bar_base + 8 * (NS + s), ((git / NS) & 1) ^ 1, p.wait_limit);
                     ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
                     if (!ok) {
                         if (lane == 0) {
@@ -435,6 +435,7 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
                         break;
                     }
                 }
+                if (p.debug_drop_loads) continue;                         // test hook: nothing arrives, the waits run out
                 const int pages_here = min(kPagesPerStage, n_pages - it * kPagesPerStage);
                 const uint32_t full = bar_base + 8 * s;
                 if (lane == 0) mbar_arrive_expect_tx(full, (uint32_t)pages_here * 2u * Cfg::kPageBytes);
@@ -559,7 +560,7 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
             bool pfailed = false;
             for (int it = 0; it < n_iters; ++it, ++git) {
                 const int s = git % NS;
-                if (!mbar_wait(bar_base + 8 * s, (git / NS) & 1) || sm_flags[0] != 0) {
+                if (!mbar_wait(bar_base + 8 * s, (git / NS) & 1, p.wait_limit) || sm_flags[0] != 0) {
                     if (lane == 0) {
                         record_status(p.status, DA_ERR_TIMEOUT);
                         sm_flags[0] = 1;
@@ -729,7 +730,7 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
 
         for (int it = 0; it < n_iters; ++it, ++git) {
             const int s = git % NS;
-            if (!mbar_wait(bar_base + 8 * s, (git / NS) & 1) || sm_flags[0] != 0) {
+            if (!mbar_wait(bar_base + 8 * s, (git / NS) & 1, p.wait_limit) || sm_flags[0] != 0) {
                 if (lane == 0) {
                     record_status(p.status, DA_ERR_TIMEOUT);
                     sm_flags[0] = 1;

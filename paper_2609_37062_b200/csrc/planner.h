@@ -9,7 +9,7 @@
 
 namespace da {
 
-constexpr int kDefaultDeterministicChunk = 1024;  // tokens
+constexpr int kDefaultDeterministicChunk = 256;   // tokens: the floor; the bound of 32 splits lengthens it above 8,192 tokens
 constexpr int kTileTokens = 16;                  // what the kernels fetch at a time; pages hold a power-of-two number of these
 constexpr int kDefaultAutoMinChunk = 256;         // tokens
 constexpr int kDefaultMaxSplits = 512;

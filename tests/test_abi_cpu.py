@@ -140,7 +140,7 @@ def test_deterministic_boundaries_depend_on_the_length_alone():
     assert cuts([77, 5000, 123456], 1) == alone
     assert cuts([5000] * 256, 200) == alone
     assert cuts([5000, 9], 0, sm=16, ctas=1) == alone
-    assert layout([5000], da.make_policy(split_mode=da.DA_SPLIT_DETERMINISTIC))[4] == 1024
+    assert layout([5000], da.make_policy(split_mode=da.DA_SPLIT_DETERMINISTIC))[4] == 256
 
 
 def test_fixed_count_gives_empty_trailing_splits():
@@ -155,8 +155,9 @@ def test_fixed_count_gives_empty_trailing_splits():
 def test_deterministic_default_bounds_the_splits_by_the_sequence_alone():
     """At most 32 splits by default: a longer sequence gets longer chunks, whatever else is in the batch."""
     det = da.make_policy(split_mode=da.DA_SPLIT_DETERMINISTIC)
-    expect = {32768: (32, 1024), 131072: (32, 4096), 40000: (32, 1264), 5000: (5, 1024), 100: (1, 1024)}
-    for batch in ([131072], [100, 40000, 131072, 5000, 32768], [32768] * 9 + [131072, 40000]):
+    expect = {32768: (32, 1024), 131072: (32, 4096), 40000: (32, 1264), 5000: (20, 256), 100: (1, 256),
+              8192: (32, 256), 8200: (31, 272), 2048: (8, 256)}
+    for batch in ([131072], [100, 40000, 131072, 5000, 32768], [32768] * 9 + [131072, 40000], [8192, 8200, 2048, 100]):
         units, splits, _, _, _ = layout(batch, det)
         covered_exactly_once(units, batch, 8)
         for b, L in enumerate(batch):

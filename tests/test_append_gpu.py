@@ -59,3 +59,23 @@ def test_append_rejects_bad_arguments_and_skips_bad_pages():
     da.decode_attn_append_kv(shape, nk, nk, bt, w.seq_lens, w.k_pool, w.v_pool)
     torch.cuda.synchronize()
     assert torch.equal(before, w.k_pool)                 # nothing was written, nothing faulted
+
+
+def test_checked_append_reports_rows_it_could_not_write():
+    """Invariant 1 is only kept if a dropped write is known: with a plan given, a row whose page
+    id lies outside the pool is skipped (nothing faults) and reported through the plan's status."""
+    w = to_device(wl.config_tiny())
+    plan = da.decode_attn_plan(da.shape_of_workload(w), da.make_policy(), w.seq_lens)
+    nk = wl.normal_bf16_bits(wl.stream_key(3, wl.TENSOR_NEW_K, 0), 0, 4 * 2 * 64).view(4, 2, 64).cuda()
+    before = w.k_pool.clone()
+    da.decode_attn_append_kv_checked(plan, nk, nk, w.block_table, w.seq_lens, w.k_pool, w.v_pool)
+    assert da.decode_attn_last_device_status(plan) == da.DA_OK
+    assert not torch.equal(before, w.k_pool)
+    bt = w.block_table.clone()
+    last = (int(w.seq_lens[2]) - 1) // w.page_size
+    bt[2, last] = w.num_pages                                # one row's last page: outside the pool
+    mid = w.k_pool.clone()
+    da.decode_attn_append_kv_checked(plan, nk, nk, bt, w.seq_lens, w.k_pool, w.v_pool)
+    assert da.decode_attn_last_device_status(plan) == da.DA_ERR_BAD_PAGE
+    assert torch.equal(mid, w.k_pool)                        # the other rows rewrote the same bytes, row 2 wrote nothing
+    assert da.decode_attn_last_device_status(plan) == da.DA_OK

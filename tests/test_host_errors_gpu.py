@@ -108,3 +108,67 @@ def test_empty_batch_is_a_no_op():
     out = torch.zeros(4, device="cuda")
     assert da.decode_attn_run(plan, w.q_bits, w.k_pool, w.v_pool, w.block_table, w.seq_lens, out) == da.DA_OK
     assert da.decode_attn_combine(plan, None, out) == da.DA_OK
+
+
+@pytest.mark.parametrize("fused", [0, 1])
+@pytest.mark.parametrize("lens", [[300, 5000, 64, 1200], [40000]])
+def test_a_bounded_wait_that_runs_out_is_reported_and_the_plan_recovers(fused, lens):
+    """The waits of the tensor-core kernel (consumers on a stage's arrival, the producer on its
+    release, the merge blocks on a group's records) all carry a limit.  The test hook withholds
+    the producer's loads and cuts the limit to about a millisecond: nothing is at fault, the waits
+    simply run out.  The launch must come back by itself, report DA_ERR_TIMEOUT, and leave the plan
+    and the context good for the next ordinary launch."""
+    import time
+    from gpu_util import assert_parity, oracle_of
+    w = to_device(wl.make_workload("expire", lens, 32, 8, 128, seed=53))
+    plan = da.decode_attn_plan(da.shape_of_workload(w), da.make_policy(kernel=da.DA_KERNEL_MMA_TMA, fuse_combine=fused),
+                               w.seq_lens)
+    out = torch.zeros((w.batch, w.num_q_heads, w.head_dim), dtype=torch.float32, device="cuda")
+    lse = torch.zeros((w.batch, w.num_q_heads), dtype=torch.float32, device="cuda")
+    ws = torch.empty(max(plan.workspace_bytes, 256), dtype=torch.uint8, device="cuda")
+    args = (w.q_bits, w.k_pool, w.v_pool, w.block_table, w.seq_lens, out, lse, ws, plan.workspace_bytes)
+    t0 = time.perf_counter()
+    assert da.decode_attn_debug_expire_wait(plan, *args, limit_cycles=2_000_000) == da.DA_OK
+    assert da.decode_attn_last_device_status(plan) == da.DA_ERR_TIMEOUT      # synchronises: the launch returned
+    assert time.perf_counter() - t0 < 5.0                                    # long before the ordinary one-second limits add up
+    assert da.decode_attn_last_device_status(plan) == da.DA_OK               # cleared by the read
+    # the very same plan, an ordinary launch: clean status, correct result
+    da.decode_attn_run(plan, *args)
+    if not fused:
+        da.decode_attn_combine(plan, ws, out, lse)
+    assert da.decode_attn_last_device_status(plan) == da.DA_OK
+    ref_out, ref_lse = oracle_of(to_device(w, "cpu"))
+    assert_parity(out, lse, ref_out, ref_lse)
+    # the hook refuses what it does not cover, and a non-positive limit
+    assert da.decode_attn_debug_expire_wait(plan, *args, limit_cycles=0) == da.DA_ERR_INVALID_ARG
+    simt = da.decode_attn_plan(da.shape_of_workload(w), da.make_policy(kernel=da.DA_KERNEL_SIMT), w.seq_lens)
+    assert da.decode_attn_debug_expire_wait(simt, *args[:8], simt.workspace_bytes) in (da.DA_ERR_UNSUPPORTED,
+                                                                                       da.DA_ERR_WORKSPACE_TOO_SMALL)
+
+
+def test_a_plan_may_be_destroyed_while_its_kernels_are_still_queued():
+    """A step is plan / run / combine / destroy with no synchronisation in between.  The next
+    plan takes the destroyed plan's device buffer from the library's cache and uploads its own
+    work list there: that upload has to wait, on the device, for the first plan's kernels."""
+    from gpu_util import oracle_of
+    a = wl.config_sweep_cell(2048, 64, device="cuda")                  # ~80 us of kernel time queued behind one another
+    b = to_device(wl.make_workload("other", [700, 33, 5000, 16, 1800], 32, 8, 128, seed=77))
+    want_a, want_a_lse = da.run_workload(a, da.make_policy())
+    want_b, want_b_lse = da.run_workload(b, da.make_policy())
+    torch.cuda.synchronize()
+    for _ in range(20):
+        outs = []
+        for w in (a, b, a, b):
+            plan = da.decode_attn_plan(da.shape_of_workload(w), da.make_policy(), w.seq_lens)
+            out = torch.full((w.batch, w.num_q_heads, w.head_dim), float("nan"), dtype=torch.float32, device="cuda")
+            lse = torch.full((w.batch, w.num_q_heads), float("nan"), dtype=torch.float32, device="cuda")
+            ws = torch.empty(max(plan.workspace_bytes, 256), dtype=torch.uint8, device="cuda")
+            da.decode_attn_run(plan, w.q_bits, w.k_pool, w.v_pool, w.block_table, w.seq_lens, out, lse, ws,
+                               plan.workspace_bytes)
+            da.decode_attn_combine(plan, ws, out, lse)
+            plan.destroy()                                              # kernels still queued or running
+            outs.append((out, lse, ws))
+        torch.cuda.synchronize()
+        assert torch.equal(outs[0][0], want_a) and torch.equal(outs[2][0], want_a)
+        assert torch.equal(outs[1][0], want_b) and torch.equal(outs[3][0], want_b)
+        assert torch.equal(outs[0][1], want_a_lse) and torch.equal(outs[3][1], want_b_lse)
