@@ -165,8 +165,9 @@ def test_deterministic_default_bounds_the_splits_by_the_sequence_alone():
             assert splits[b] == n
             mine = sorted([u for u in units if u.seq == b and u.kv_head == 0], key=lambda u: u.split_index)
             assert [u.tok_begin for u in mine] == [min(i * chunk, (L + 15) // 16 * 16) for i in range(n)]
-    units, splits, _, _, _ = layout([131072], da.make_policy(split_mode=da.DA_SPLIT_DETERMINISTIC, max_splits=512))
-    assert splits[0] == 128                                   # the old rule on request
+    units, splits, _, _, _ = layout([131072], da.make_policy(split_mode=da.DA_SPLIT_DETERMINISTIC, max_splits=512,
+                                                             chunk_tokens=1024))
+    assert splits[0] == 128                                   # fixed 1,024-token chunks on request
 
 
 def test_max_splits_caps_the_split_count():
