@@ -53,7 +53,7 @@ struct decode_attn_plan {
     char* dev = nullptr;
     char* pinned = nullptr;
     size_t upload_bytes = 0;
-    size_t off_units = 0, off_seq_info = 0, off_block_begin = 0, off_unit_rank = 0, off_status = 0, off_tickets = 0,
+    size_t off_units = 0, off_seq_info = 0, off_block_begin = 0, off_unit_rank = 0, off_status = 0, off_tickets = 0, off_queue = 0,
            total_bytes = 0;
     int max_bins = 0;        // > 0: the units are packed into per-block ranges (persistent tensor-core kernel)
     cudaStream_t stream = nullptr;
@@ -296,12 +296,11 @@ int device_sm_count(int dev, int* out)
     return DA_OK;
 }
 
-// The kernel's redistribution under a RUN mask reads the binned units by cost rank, packed into a
-// word each: work lists of up to kMaxRanked units and batches below kRankNoSeq sequences.
+// Launches with a RUN mask hand the binned units out in cost order (see the kernel's queue): the
+// plan uploads their positions by rank.
 bool ranked_fits(const decode_attn_plan_t* pl)
 {
-    return pl->max_bins > 0 && !pl->layout.rank_pos.empty() && pl->layout.rank_pos.size() <= (size_t)kMaxRanked &&
-           (uint32_t)pl->shape.batch < kRankNoSeq;
+    return pl->max_bins > 0 && !pl->layout.rank_pos.empty();
 }
 
 void fill_host_mirror(decode_attn_plan_t* pl)
@@ -326,16 +325,13 @@ void fill_host_mirror(decode_attn_plan_t* pl)
         const std::vector<int32_t>& src = pl->layout.block_begin;
         const int32_t end = (int32_t)pl->layout.units.size();
         for (int64_t i = 0; i <= pl->grid; ++i) bb[i] = i < (int64_t)src.size() ? src[i] : end;
-        // every binned unit by cost rank: its 16-token tiles, its sequence (-1: no RUN mask applies,
-        // a shared-prefix unit) and where it sits in the work list
-        uint32_t* ur = reinterpret_cast<uint32_t*>(pl->pinned + pl->off_unit_rank);
+        // every binned unit by cost rank: where it sits in the work list and whose row it is
         if (ranked_fits(pl)) {
-            const int32_t first = pl->layout.n_front_units;
+            int2* ur = reinterpret_cast<int2*>(pl->pinned + pl->off_unit_rank);
             for (size_t j = 0; j < pl->layout.rank_pos.size(); ++j) {
                 const int32_t pos = pl->layout.rank_pos[j];
                 const decode_attn_unit_t& u = pl->layout.units[pos];
-                const uint32_t seq = (u.kv_head >> 16) ? kRankNoSeq : (uint32_t)u.seq;
-                ur[j] = seq << kRankPosBits | (uint32_t)(pos - first);
+                ur[j] = make_int2(pos, (u.kv_head >> 16) ? -1 : u.seq);
             }
         }
     }
@@ -359,7 +355,8 @@ KernelParams make_params(const decode_attn_plan_t* pl, const decode_attn_run_arg
     kp.units = reinterpret_cast<const decode_attn_unit_t*>(pl->dev + pl->off_units);
     kp.seq_info = reinterpret_cast<const SeqInfo*>(pl->dev + pl->off_seq_info);
     kp.block_begin = pl->max_bins > 0 ? reinterpret_cast<const int32_t*>(pl->dev + pl->off_block_begin) : nullptr;
-    kp.unit_rank = reinterpret_cast<const uint32_t*>(pl->dev + pl->off_unit_rank);
+    kp.unit_rank = reinterpret_cast<const int2*>(pl->dev + pl->off_unit_rank);
+    kp.queue = pl->max_bins > 0 ? reinterpret_cast<int32_t*>(pl->dev + pl->off_queue) : nullptr;
     kp.n_ranked = ranked_fits(pl) ? (int32_t)pl->layout.rank_pos.size() : 0;
     kp.first_binned = pl->layout.n_front_units;
     kp.may_rank = pl->max_bins > 0 && pl->policy.capacity_batch > 0;
@@ -533,12 +530,13 @@ int decode_attn_plan(const decode_attn_shape_t* shape, const decode_attn_policy_
     // the binned units by cost rank, for the kernel's redistribution under a RUN mask
     pl->upload_bytes = pl->off_unit_rank +
                        (pl->max_bins > 0
-                            ? align_up((size_t)std::min<int64_t>(std::max<int64_t>(pl->max_units, 1), kMaxRanked) * sizeof(uint32_t), 32)
+                            ? align_up((size_t)std::max<int64_t>(pl->max_units, 1) * sizeof(int2), 32)
                             : 0);
     pl->off_status = pl->upload_bytes;
     pl->off_tickets = pl->off_status + 32;
-    pl->total_bytes = pl->off_tickets +
-                      align_up(2 * (size_t)std::max<int64_t>(pl->max_batch, 1) * shape->num_kv_heads * sizeof(int32_t), 32);
+    pl->off_queue = pl->off_tickets +
+                    align_up(2 * (size_t)std::max<int64_t>(pl->max_batch, 1) * shape->num_kv_heads * sizeof(int32_t), 32);
+    pl->total_bytes = pl->off_queue + 32;          // the two counters of the masked launches' queue
 
     PlanBuffers* pb = new (std::nothrow) PlanBuffers();
     if (!pb) return DA_ERR_INVALID_ARG;

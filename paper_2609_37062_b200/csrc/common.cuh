@@ -42,9 +42,12 @@ struct KernelParams {
     const decode_attn_unit_t* units;
     const SeqInfo* seq_info;
     const int32_t* block_begin;  // [grid + 1]: block b walks units block_begin[b] .. block_begin[b+1]; NULL: unit b
-    const uint32_t* unit_rank;   // [n_ranked] the binned units by cost rank: sequence << 14 | position behind the first
-                                 // binned unit (sequence kRankNoSeq: no RUN mask applies); work lists of <= kMaxRanked units
-    int32_t n_ranked;            // entries of unit_rank (0: none); capacity plans read both from the header,
+    const int2* unit_rank;       // [n_ranked] the binned unit with cost rank j (0: the most expensive): its position in the
+                                 // work list and its sequence (-1: no RUN mask applies, a shared-prefix unit); the order
+                                 // in which launches with a RUN mask hand the units out
+    int32_t* queue;              // two counters, zero between launches: units drawn from unit_rank beyond the first of
+                                 // every block, blocks that have drawn their last (NULL: no rank list)
+    int32_t n_ranked;            // entries of unit_rank (0: none); capacity plans read it from the header
     int32_t first_binned;        // position of the first binned unit in the work list
     int32_t may_rank;            // capacity plans: the rank list exists (how long it is changes with every refresh)
     int32_t* tickets;  // [2][batch][Hkv], zero between launches: records published / slices merged per (sequence, KV head)
@@ -100,11 +103,6 @@ struct KernelParams {
 #define DA_TRACE_CLOCK(uid, slot) ((void)0)
 #endif
 
-
-constexpr int kRankPosBits = 14;                    // unit_rank words: position in the low bits, sequence above
-constexpr uint32_t kRankNoSeq = (1u << (32 - kRankPosBits)) - 1u;
-constexpr int kRankPasses = 4;                      // the kernel reads the list 2,560 units at a time
-constexpr int kMaxRanked = kRankPasses * 2560;
 
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kLog2e = 1.4426950408889634f;

@@ -200,9 +200,14 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
     const uint32_t bar_base = base + NS * Cfg::kStageBytes;   // full[NS], empty[NS]
     volatile int* const sm_flags = reinterpret_cast<volatile int*>(gbase + NS * Cfg::kStageBytes + 256);
     int* const sm_ticket = reinterpret_cast<int*>(gbase + NS * Cfg::kStageBytes + 256 + 16);
-    constexpr int kListMax = 160;                             // units a block can own after a redistribution
-    int* const sm_list = reinterpret_cast<int*>(gbase + NS * Cfg::kStageBytes + 384);   // [kListMax], 640 bytes
-    static_assert(384 + 4 * kListMax <= Cfg::kBarrierBytes, "the unit list overlaps the scratch");
+    // Launches with a RUN mask take their units from a queue (see below): the producer warp hands the
+    // consumers the descriptors of the units it drew through a small ring, sm_pub counting the entries
+    // published so far.  The producer is never more than NS + 1 units ahead of the consumers.
+    constexpr int kRing = 8;
+    static_assert(kRing > NS + 1, "the ring of drawn units is too short for the stages in flight");
+    volatile int* const sm_pub = reinterpret_cast<volatile int*>(gbase + NS * Cfg::kStageBytes + 256 + 32);
+    int4* const sm_ring = reinterpret_cast<int4*>(gbase + NS * Cfg::kStageBytes + 384);   // [kRing][2], 256 bytes
+    static_assert(384 + 32 * kRing <= Cfg::kBarrierBytes, "the unit ring overlaps the scratch");
     float* const sm_wo = reinterpret_cast<float*>(gbase + NS * Cfg::kStageBytes + Cfg::kBarrierBytes);   // [4][COLS][D]
     float* const sm_wm = sm_wo + kMmaConsumerWarps * COLS * D;                                           // [4][COLS]
     float* const sm_wl = sm_wm + kMmaConsumerWarps * COLS;                                               // [4][COLS]
@@ -224,11 +229,23 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
         ubeg = blockIdx.x;
         uend = min(n_units, (int)blockIdx.x + 1);
     }
-    // (with a RUN mask the masked variant may deal the units out again, to every block of the launch)
-    const bool may_redistribute = MASKED && MODE == kModeAttend && p.run_mask != nullptr &&
-                                  (p.grid_exit ? p.may_rank != 0 : p.n_ranked > 0);
-    const bool idle = ubeg >= uend;                           // no units from the planner's packing
-    if (idle && !may_redistribute) {                          // surplus blocks of a capacity launch
+    // With a RUN mask the planner's packing is off: it could not know which rows read nothing, and a
+    // block whose rows all run would set the step's time.  Such launches (the MASKED variant) hand
+    // the units out through a queue instead: in cost order, block b starts with the unit of rank b
+    // and then draws the next rank with one atomic add on a counter the plan owns, one unit ahead
+    // of its consumers.  A unit whose row is masked costs the drawing warp a look at the mask byte
+    // and the stores of its empty result.  No block waits for another, and a unit's result does not
+    // depend on which block ran it.  The last block to have drawn puts the counters back to zero,
+    // so the launch can be repeated (or replayed from a graph) as it is.
+    const bool queued = MASKED && MODE == kModeAttend && p.run_mask != nullptr && p.queue != nullptr &&
+                        (p.grid_exit ? p.may_rank != 0 : p.n_ranked > 0);
+    const int n_ranked = queued ? (p.grid_exit ? p.header->n_ranked : p.n_ranked) : 0;
+    if (queued) {
+        ubeg = (int)blockIdx.x < n_ranked ? __ldg(p.unit_rank + blockIdx.x).x : 0;
+        uend = (int)blockIdx.x < n_ranked ? ubeg + 1 : ubeg;
+    }
+    const bool idle = ubeg >= uend;                           // no units: a surplus block of a capacity launch
+    if (idle) {
         // Stream order reaches the kernels behind this one through the waits of this launch's
         // blocks; should every block be surplus, block 0 still carries it.
         if (blockIdx.x == 0) pdl_wait_primary();
@@ -245,18 +262,17 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
             mbar_init(bar_base + 8 * (NS + s), kMmaConsumerWarps);      // empty: one arrival per consumer warp
         }
         sm_flags[0] = 0;
+        sm_pub[0] = 0;
         mbar_init_fence();
     }
-    decode_attn_unit_t u = load_unit(p.units, idle ? 0 : ubeg);
+    decode_attn_unit_t u = load_unit(p.units, ubeg);
     __syncthreads();
     if (tid == 0) DA_TRACE_STAMP(blockIdx.x, 1);
     // Everything above touched only the plan's own work list and kernel parameters.  What the
     // kernel launched before this one may have produced (q, new K/V rows, lengths, page
     // mappings) is read only past this point; with a programmatic dependency the lines above
     // overlap that kernel's tail.
-    const int n_ranked = p.grid_exit ? p.header->n_ranked : p.n_ranked;
-    const bool redistribute = may_redistribute && n_ranked > 0;
-    if (MODE == kModeAttend && warp == 0 && p.hint_first_pages != 0 && !idle) {
+    if (MODE == kModeAttend && warp == 0 && p.hint_first_pages != 0) {
         // Hints, while the kernel before this one drains (from a consumer warp, which has nothing to do
         // until the first stage lands; the producer goes straight to its wait): the pages that will fill the ring first
         // are asked into L2.  The mask and the page ids read here may be about to change; they steer
@@ -281,104 +297,6 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
     pdl_wait_primary();
     if (p.early_trigger) pdl_launch_dependents();             // first of a pair: see KernelParams
 
-    bool listed = false;                                      // the block walks sm_list instead of its range
-    if (redistribute) {
-        // With a RUN mask the planner's packing is off: it could not know which rows read nothing,
-        // and a block whose rows all run sets the step's time.  So every block deals the units out
-        // again, the same way: in cost order the units that run go to the blocks in turn (back and
-        // forth, so that no block always gets the largest of a round), and likewise the masked ones,
-        // which cost next to nothing, behind them.  Consecutive units of the order - the KV heads
-        // of one sequence - still go to different blocks at the same time, every unit has one
-        // owner, and no block depends on another.  A block's list lives in shared memory.
-        const int n = n_ranked, nb = p.n_work_blocks, b = blockIdx.x;
-        const int first_binned = p.grid_exit ? p.header->first_binned : p.first_binned;
-        // Work lists of up to 10,240 units (a word each, read in rank order, 16 a thread at a time, so
-        // that a warp's loads are adjacent); longer ones keep the planner's packing: with that many
-        // units a block the masked rows even out by themselves.  Every block reads the same words at the same
-        // moment, which costs a few microseconds, so a look at the first rows' mask bytes decides
-        // first whether enough rows are masked for the new deal to pay (about three in ten).
-        constexpr int CH = 16;                                // units a thread holds at a time
-        constexpr int WPP = CH * (kMmaThreads / 32);          // ballot words of a pass of CH * threads units
-        const int passes = (n + CH * kMmaThreads - 1) / (CH * kMmaThreads);     // <= kRankPasses
-        const int n_seen = min(p.batch, kMmaThreads);
-        const int seen_masked = __syncthreads_count(tid < n_seen && __ldg(p.run_mask + tid) == 0);
-        if (seen_masked * 10 >= n_seen * 3) {
-            uint32_t* const words = reinterpret_cast<uint32_t*>(sm_wo);              // [passes * WPP] which units run, in rank order
-            int* const before = reinterpret_cast<int*>(sm_wo) + kRankPasses * WPP;   // [passes * WPP + 1] running units before each word
-            static_assert((2 * kRankPasses * WPP + 1) * 4 <= Cfg::kScratchBytes, "the ballot words do not fit the scratch");
-            for (int ps = 0; ps < passes; ++ps) {
-                int seq_held[CH];
-#pragma unroll
-                for (int i = 0; i < CH; ++i) {
-                    const int j = (ps * CH + i) * kMmaThreads + tid;
-                    const uint32_t e = (j < n) ? __ldg(p.unit_rank + j) : 0xffffffffu;
-                    seq_held[i] = (e >> kRankPosBits) == kRankNoSeq ? -1 : (int)(e >> kRankPosBits);
-                }
-#pragma unroll
-                for (int i = 0; i < CH; ++i) {
-                    const int j = (ps * CH + i) * kMmaThreads + tid;
-                    const bool r = j < n && (seq_held[i] < 0 || __ldg(p.run_mask + seq_held[i]) != 0);
-                    const uint32_t w = __ballot_sync(0xffffffffu, r);
-                    if (lane == 0) words[(ps * CH + i) * (kMmaThreads / 32) + warp] = w;
-                }
-            }
-            __syncthreads();
-            const int NW = passes * WPP;
-            for (int t = tid; t <= NW; t += kMmaThreads) {
-                int acc = 0;
-                for (int w = 0; w < t; ++w) acc += __popc(words[w]);
-                before[t] = acc;                                              // before[NW]: all running units
-            }
-            __syncthreads();
-            const int total = before[NW];
-            // the k-th unit of a kind (running / masked): round k / nb, block k % nb or, in odd rounds,
-            // nb - 1 - k % nb; how many of `count` a block gets follows in closed form
-            auto owner = [&](int k) { return ((k / nb) & 1) ? nb - 1 - k % nb : k % nb; };
-            auto share = [&](int count) {
-                const int full = count / nb, rem = count % nb;
-                const bool extra = (full & 1) ? b >= nb - rem : b < rem;
-                return full + (extra ? 1 : 0);
-            };
-            const int n_run = share(total), n_all = n_run + share(n - total);
-            if (n_all <= kListMax) {
-                for (int ps = 0; ps < passes; ++ps) {
-#pragma unroll
-                    for (int i = 0; i < CH; ++i) {
-                        const int j = (ps * CH + i) * kMmaThreads + tid;
-                        if (j < n) {
-                            const int pos = first_binned + (int)(__ldg(p.unit_rank + j) & ((1u << kRankPosBits) - 1u));
-                            const int w = (ps * CH + i) * (kMmaThreads / 32) + warp;
-                            const uint32_t bits = words[w];
-                            const int kr = before[w] + __popc(bits & ((1u << lane) - 1u));       // running units before j
-                            if ((bits >> lane) & 1u) {
-                                if (owner(kr) == b) sm_list[kr / nb] = pos;
-                            } else {
-                                const int km = j - kr;                                            // masked units before j
-                                if (owner(km) == b) sm_list[n_run + km / nb] = pos;
-                            }
-                        }
-                    }
-                }
-                listed = true;
-                ubeg = 0;
-                uend = n_run;
-                // The masked units of the list are done with here, a warp each: an empty result costs
-                // a descriptor read and a few stores, and going through the pipeline for it would
-                // cost a block about a microsecond of dependent reads per unit.
-                __syncthreads();                              // the list is complete
-                for (int k = n_run + warp; k < n_all; k += kMmaThreads / 32)
-                    block_finish_empty<D>(p, load_unit(p.units, sm_list[k]), G, lane, 32);
-            }
-        }
-        __syncthreads();                                      // the list is written, the scratch goes back to its use
-        if (listed) {
-            if (ubeg >= uend) return;
-            u = load_unit(p.units, sm_list[0]);
-        }
-    }
-    if (idle && !listed) return;                              // a surplus block that stayed for nothing
-    auto unit_at = [&](int k) { return (MASKED && listed) ? sm_list[k] : k; };   // position in the work list of the block's k-th unit
-
     if (warp == kMmaConsumerWarps) {
         // ------------------------------------------------------------ producer
         const uint64_t l2_policy = l2_policy_evict_first();
@@ -399,14 +317,99 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
             const int32_t* t = p.block_table + (int64_t)x.seq * p.max_pages_per_seq;
             return (lane < np) ? __ldg(t + (((x.tok_begin >> 4) + lane) >> ts)) : 0;
         };
-        int t1 = unit_end(u);
-        int ids_first = first_ids(u, t1);
-        for (int uid = ubeg; uid < uend && alive; ++uid) {
-            const bool has_next = uid + 1 < uend;
+        // ---- launches with a RUN mask: the queue (see the top of the kernel)
+        const int nb = p.n_work_blocks;
+        int published = 0;
+        // hands a drawn unit (or, with valid = false, the end of the queue) to the consumers
+        auto publish = [&](const decode_attn_unit_t& x, bool valid) {
+            if (lane == 0) {
+                int4* const e = sm_ring + 2 * (published % kRing);
+                e[0] = make_int4(valid ? x.seq : -1, x.kv_head, x.tok_begin, x.tok_end);
+                e[1] = make_int4(x.slot, x.seq_len, x.split_index, x.n_splits);
+                __threadfence_block();
+                sm_pub[0] = published + 1;
+            }
+            ++published;
+        };
+        auto draw = [&]() {
+            int j = 0;
+            if (lane == 0) j = nb + atomicAdd(p.queue, 1);
+            return __shfl_sync(0xffffffffu, j, 0);
+        };
+        // the unit of rank j: 1 if it runs (x, its end and its first page ids are set), 0 if it reads
+        // nothing (its empty result is written here, by this warp), -1 if the queue is exhausted
+        auto candidate = [&](int j, decode_attn_unit_t& x, int& end, int& ids) {
+            if (j >= n_ranked) return -1;
+            x = load_unit(p.units, __ldg(p.unit_rank + j).x);
+            end = unit_end(x);
+            if (end > x.tok_begin) {
+                ids = first_ids(x, end);
+                return 1;
+            }
+            block_finish_empty<D>(p, x, G, lane, 32);
+            return 0;
+        };
+        int t1 = 0, ids_first = 0;
+        bool have = true;
+        if (queued) {
+            // the block's first unit is the one of rank blockIdx.x, whose descriptor is in hand: its mask
+            // byte and its first page ids are asked for together
+            ids_first = first_ids(u, u.tok_end);
+            t1 = unit_end(u);
+            int r = 1;
+            if (t1 <= u.tok_begin) {
+                block_finish_empty<D>(p, u, G, lane, 32);
+                r = 0;
+            }
+            while (r == 0) r = candidate(draw(), u, t1, ids_first);
+            have = r == 1;
+            publish(u, have);
+        } else {
+            t1 = unit_end(u);
+            ids_first = first_ids(u, t1);
+        }
+        for (int uid = ubeg; (queued ? have : uid < uend) && alive; ++uid) {
+            const bool has_next = queued || uid + 1 < uend;
             decode_attn_unit_t nu = u;
-            if (has_next) nu = load_unit(p.units, unit_at(uid + 1));      // lands while this unit streams
+            if (!queued && has_next) nu = load_unit(p.units, uid + 1);    // lands while this unit streams
             int nt1 = 0, nids_first = 0;
             bool next_ready = false;
+            int next_state = 0;                                           // queue: 0 still looking, 1 found, -1 none left
+            // The look for the next unit is a chain of dependent reads (the counter, the rank list,
+            // the descriptor and the mask byte, the first page ids).  It advances one link per stage
+            // issued - each link's loads are asked for in one step and used in the next - so that
+            // the chain's latency passes while the warp waits for stages anyway.
+            int q_link = 0, q_j = 0, q_masked = 0;
+            int2 q_rank = make_int2(0, 0);
+            auto queue_step = [&]() {
+                if (q_link == 0) {
+                    if (lane == 0) q_j = nb + atomicAdd(p.queue, 1);
+                    q_link = 1;
+                } else if (q_link == 1) {
+                    q_j = __shfl_sync(0xffffffffu, q_j, 0);
+                    if (q_j >= n_ranked) {
+                        next_state = -1;
+                        publish(nu, false);
+                    } else {
+                        q_rank = __ldg(p.unit_rank + q_j);
+                        q_link = 2;
+                    }
+                } else if (q_link == 2) {
+                    nu = load_unit(p.units, q_rank.x);
+                    q_masked = q_rank.y >= 0 ? (int)(__ldg(p.run_mask + q_rank.y) == 0) : 0;
+                    q_link = 3;
+                } else {
+                    nt1 = q_masked ? nu.tok_begin : nu.tok_end;
+                    if (nt1 > nu.tok_begin) {
+                        nids_first = first_ids(nu, nt1);
+                        next_state = 1;
+                        publish(nu, true);
+                    } else {
+                        block_finish_empty<D>(p, nu, G, lane, 32);
+                        q_link = 0;
+                    }
+                }
+            };
             const int b = u.seq, g = u.kv_head & 0xffff;   // (a shared-prefix unit keeps its block size in the high half)
             const int t0 = u.tok_begin;
             const int n_pages = (t1 - t0 + 15) >> 4;
@@ -457,19 +460,37 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
                     tma_load_4d(dst, which ? &v_map : &k_map, full, hf * 64, slot0, g, page_id, l2_policy);
                     if (git == 0 && lane == 0) DA_TRACE_STAMP(blockIdx.x, 2);
                 }
-                if (has_next && !next_ready) {                            // this unit is under way: look ahead
+                if (queued) {
+                    // One link of the look at the queue per stage issued, so that a run of masked rows
+                    // does not hold the loads up - and only over the unit's last stages: a block that
+                    // draws its next unit early takes it away from a block that has nothing to do.
+                    constexpr int kQueueLead = 8;
+                    if (next_state == 0 && n_iters - it <= kQueueLead) queue_step();
+                } else if (has_next && !next_ready) {                     // this unit is under way: look ahead
                     nt1 = unit_end(nu);
                     nids_first = first_ids(nu, nt1);
                     next_ready = true;
                 }
             }
-            if (has_next && !next_ready) {
+            if (queued) {
+                while (next_state == 0 && alive) queue_step();
+                if (next_state == 0) publish(nu, false);                  // a wait was given up: the consumers leave too
+                have = next_state == 1;
+            } else if (has_next && !next_ready) {
                 nt1 = unit_end(nu);
                 nids_first = first_ids(nu, nt1);
             }
             u = nu;
             t1 = nt1;
             ids_first = nids_first;
+        }
+        if (queued && lane == 0) {
+            // this block has drawn its last: count it; whoever is last puts the counters back
+            const int participants = min(nb, n_ranked);
+            if (atomicAdd(p.queue + 1, 1) == participants - 1) {
+                atomicExch(p.queue, 0);
+                atomicExch(p.queue + 1, 0);
+            }
         }
         return;
     }
@@ -506,12 +527,42 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
             }
         }
     };
+    // queue (launches with a RUN mask): entry `need - 1` of the producer's ring has been published
+    auto wait_published = [&](int need) {
+        if (sm_pub[0] < need) {
+            const long long c0 = clock64();
+            while (sm_pub[0] < need)
+                if (sm_flags[0] != 0 || clock64() - c0 > p.wait_limit) return false;
+        }
+        __threadfence_block();
+        return true;
+    };
+    auto ring_unit = [&](int k) {
+        const int4 a = sm_ring[2 * (k % kRing)], b2 = sm_ring[2 * (k % kRing) + 1];
+        decode_attn_unit_t x;
+        x.seq = a.x; x.kv_head = a.y; x.tok_begin = a.z; x.tok_end = a.w;
+        x.slot = b2.x; x.seq_len = b2.y; x.split_index = b2.z; x.n_splits = b2.w;
+        return x;
+    };
+    if (queued) {
+        // the block's first unit is the first one of its draws whose row runs, if any does
+        const bool late = block_sync_or(1, kConsumerThreads, !wait_published(1));
+        if (late) {
+            if (tid == 0) {
+                record_status(p.status, DA_ERR_TIMEOUT);
+                sm_flags[0] = 1;
+            }
+            return;
+        }
+        u = ring_unit(0);
+        if (u.seq < 0) return;
+    }
     Pre cur;
     prefetch(u, cur);
-    for (int uid = ubeg; uid < uend; ++uid) {
-        const bool last_unit = uid + 1 >= uend;
+    for (int uid = ubeg; queued || uid < uend; ++uid) {
+        bool last_unit = !queued && uid + 1 >= uend;          // (queue: known once the next entry has been published)
         decode_attn_unit_t nu = u;
-        if (!last_unit) nu = load_unit(p.units, unit_at(uid + 1));        // lands while this unit is consumed
+        if (!queued && !last_unit) nu = load_unit(p.units, uid + 1);      // lands while this unit is consumed
         Pre nxt = cur;
         const int b = u.seq, g = u.kv_head & 0xffff;
         const int nseq = u.kv_head >> 16;                                  // > 0: a shared-prefix unit
@@ -857,6 +908,22 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
             if (lane == 0) mbar_arrive(bar_base + 8 * (NS + s));          // this warp is done with the stage
         }
         if (uid == ubeg && tid == 0) DA_TRACE_STAMP(blockIdx.x, 4);
+        if (queued) {
+            // the producer drew the next unit while this one streamed
+            const int need = uid - ubeg + 2;
+            if (!failed && !wait_published(need)) {
+                if (lane == 0) {
+                    record_status(p.status, DA_ERR_TIMEOUT);
+                    sm_flags[0] = 1;
+                }
+                failed = true;
+            }
+            last_unit = true;
+            if (!failed) {
+                nu = ring_unit(need - 1);
+                last_unit = nu.seq < 0;
+            }
+        }
         if (last_unit && MODE == kModeAttend) pdl_launch_dependents();    // the combine kernel may start getting scheduled
         if (!last_unit) prefetch(nu, nxt);                                // in flight during this unit's epilogue
 
@@ -880,6 +947,7 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
             // result is written straight away - no states to merge, no barrier, the scratch untouched.
             block_finish_empty<D>(p, u, G, tid, kConsumerThreads);
             if (uid == ubeg && tid == 0) DA_TRACE_STAMP(blockIdx.x, 6);
+            if (queued && last_unit) break;
             u = nu;
             cur = nxt;
             continue;
@@ -941,6 +1009,7 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
         }
         if (uid == ubeg && tid == 0) DA_TRACE_STAMP(blockIdx.x, 6);
         if (gave_up) return;
+        if (queued && last_unit) break;
         u = nu;
         cur = nxt;
     }
