@@ -15,7 +15,8 @@ from typing import Optional, Sequence
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libdecode_attn.so")
+# DECODE_ATTN_LIB: another build of the same library (a trace build, a variant under measurement)
+LIB_PATH = os.environ.get("DECODE_ATTN_LIB") or os.path.join(_HERE, "libdecode_attn.so")
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(

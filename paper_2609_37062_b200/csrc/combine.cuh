@@ -24,9 +24,13 @@ __global__ void __launch_bounds__(kCombineThreads) decode_attn_combine_kernel(co
     SeqInfo si;
     si.slot_base = -1;
     if (in_batch) si = p.seq_info[b];
+    // (trace builds: the combine blocks' stamps follow the partial kernel's rows)
+    if (threadIdx.x == 0) DA_TRACE_STAMP(p.n_work_blocks + blockIdx.x, 0);
     pdl_wait_primary();                                   // the records of the launch before this one are complete
+    if (threadIdx.x == 0) DA_TRACE_STAMP(p.n_work_blocks + blockIdx.x, 1);
     if (si.slot_base < 0) return;                         // a single split, written directly by the partial kernel
     combine_slice<D, BATCH>(p, b, g, slice, G, si.slot_base, si.n_splits, threadIdx.x, sm, 0);
+    if (threadIdx.x == 0) DA_TRACE_STAMP(p.n_work_blocks + blockIdx.x, 2);
 }
 
 // Plans whose sequences have at most MAXS (4 or 8) splits: one thread per output column, 128
@@ -42,9 +46,12 @@ __global__ void __launch_bounds__(kCombineThreads) decode_attn_combine_few_kerne
     SeqInfo si;
     si.slot_base = -1;
     if (in_batch) si = p.seq_info[b];
+    if (threadIdx.x == 0) DA_TRACE_STAMP(p.n_work_blocks + blockIdx.x, 0);
     pdl_wait_primary();
+    if (threadIdx.x == 0) DA_TRACE_STAMP(p.n_work_blocks + blockIdx.x, 1);
     if (si.slot_base < 0 || col >= G * (D / 4)) return;
     combine_column<D, MAXS>(p, b, g, col, G, si.slot_base, si.n_splits);
+    if (threadIdx.x == 0) DA_TRACE_STAMP(p.n_work_blocks + blockIdx.x, 2);
 }
 
 // Merge of KV-range shards: every shard holds a normalised output and its log-sum-exp (natural

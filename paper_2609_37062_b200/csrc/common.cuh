@@ -316,7 +316,9 @@ __device__ __forceinline__ void combine_slice(const KernelParams& p, int b, int 
     for (int t = 0; t < kCombineBatch; ++t) mloc = fmaxf(mloc, ml[t].x);
     for (int j = q + 4 * kCombineBatch; j < S; j += 4) mloc = fmaxf(mloc, __ldcg(mlp + j * (rec_stride / 2)).x);
     sm_m[q * 32 + lane] = mloc;
+    if (tid == 0) DA_TRACE_STAMP(p.n_work_blocks + blockIdx.x, 3);
     block_sync(bar_id, kCombineThreads);
+    if (tid == 0) DA_TRACE_STAMP(p.n_work_blocks + blockIdx.x, 4);
     const float M = fmaxf(fmaxf(sm_m[lane], sm_m[32 + lane]), fmaxf(sm_m[64 + lane], sm_m[96 + lane]));
 
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -348,6 +350,7 @@ __device__ __forceinline__ void combine_slice(const KernelParams& p, int b, int 
     }
     sm_acc[q * 32 + lane] = acc;
     sm_l[q * 32 + lane] = lch;
+    if (tid == 0) DA_TRACE_STAMP(p.n_work_blocks + blockIdx.x, 5);
     block_sync(bar_id, kCombineThreads);
     if (q == 0 && live) {
         const int d4 = col % D4;
