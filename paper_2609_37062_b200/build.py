@@ -60,5 +60,22 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return LIB
 
 
+TRACE_LIB = os.path.join(HERE, "libdecode_attn_trace.so")
+
+
+def build_trace() -> str:
+    """The same library compiled with -DDA_TRACE: its kernels stamp %globaltimer at a few points of
+    every block into a buffer set with decode_attn_trace_set_buffer (see timeline.py).  A diagnostic
+    build; the product library carries none of this."""
+    if os.path.exists(TRACE_LIB) and all(os.path.getmtime(f) <= os.path.getmtime(TRACE_LIB) for f in _deps()):
+        return TRACE_LIB
+    nvcc = os.environ.get("NVCC", "nvcc")
+    tmp = TRACE_LIB + f".{os.getpid()}.tmp"
+    subprocess.check_call([nvcc, *NVCC_FLAGS, "-DDA_TRACE", "-shared", "-I", os.path.join(ROOT, "include"), "-I", CSRC,
+                           *sources(), "-o", tmp, "-lcudart"])
+    os.replace(tmp, TRACE_LIB)
+    return TRACE_LIB
+
+
 if __name__ == "__main__":
     print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))

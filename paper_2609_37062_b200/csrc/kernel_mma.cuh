@@ -278,7 +278,7 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
     // kernel launched before this one may have produced (q, new K/V rows, lengths, page
     // mappings) is read only past this point; with a programmatic dependency the lines above
     // overlap that kernel's tail.
-    if (MODE == kModeAttend && warp == 0 && p.hint_first_pages != 0) {
+    if (MODE != kModeGather && warp == 0 && p.hint_first_pages != 0) {     // (the gather-only probe issues the same hints)
         // Hints, while the kernel before this one drains (from a consumer warp, which has nothing to do
         // until the first stage lands; the producer goes straight to its wait): the pages that will fill the ring first
         // are asked into L2.  The mask and the page ids read here may be about to change; they steer
@@ -297,10 +297,12 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
             const int first = (u.tok_begin >> 4) >> p.tile_shift;
             const int last = ((u.tok_begin >> 4) + min(unit_pages, 64) - 1) >> p.tile_shift;      // entries first .. last
             if (unit_pages > 0 && lane * 32 <= last - first) prefetch_l2(row + first + lane * 32);
-            const char* const qrows = reinterpret_cast<const char*>(
-                p.q + ((int64_t)u.seq * p.num_q_heads + (u.kv_head & 0xffff) * G) * D);
-            if (lane * 128 < G * D * 2) prefetch_l2(qrows + lane * 128);
-            if (lane == 31) prefetch_l2(p.seq_lens + u.seq);
+            if (MODE == kModeAttend) {
+                const char* const qrows = reinterpret_cast<const char*>(
+                    p.q + ((int64_t)u.seq * p.num_q_heads + (u.kv_head & 0xffff) * G) * D);
+                if (lane * 128 < G * D * 2) prefetch_l2(qrows + lane * 128);
+                if (lane == 31) prefetch_l2(p.seq_lens + u.seq);
+            }
         }
         if (lane < np && !masked) {
             const int tile = (u.tok_begin >> 4) + lane;
