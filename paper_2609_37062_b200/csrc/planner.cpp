@@ -129,16 +129,19 @@ struct SeqCut {
     bool even;       // spread the pages evenly instead of cutting at multiples of chunk
 };
 
+// (page counts are below 2^28: 32-bit divisions, which are several times cheaper than 64-bit ones)
 int64_t units_for_chunk(const std::vector<int64_t>& pages, int64_t c, int max_splits)
 {
     int64_t total = 0;
-    for (int64_t pg : pages) {
+    const uint32_t c32 = (uint32_t)std::min<int64_t>(c, INT32_MAX), ms = (uint32_t)max_splits;
+    for (int64_t pg64 : pages) {
+        const uint32_t pg = (uint32_t)pg64;
         if (pg == 0) {
             total += 1;
             continue;
         }
-        const int64_t cb = std::max(c, ceil_div(pg, max_splits));
-        total += ceil_div(pg, cb);
+        const uint32_t cb = std::max(c32, (pg + ms - 1) / ms);
+        total += (pg + cb - 1) / cb;
     }
     return total;
 }
@@ -205,18 +208,20 @@ int make_layout(const decode_attn_shape_t& s, const decode_attn_policy_t& p, con
 
     out.splits.assign(B, 1);
     out.slot_base.assign(B, -1);
-    out.units.clear();
     out.n_slots = 0;
     out.max_splits_used = B > 0 ? 1 : 0;
-    struct Keyed {
-        decode_attn_unit_t u;
-        int64_t cost;
-    };
-    std::vector<Keyed> keyed;
+    // Units in creation order (shared-prefix units first, then sequence by sequence, split by split,
+    // KV head by KV head) with their costs beside them; the launch order is found by sorting indices.
+    // This runs every decode step: no per-unit allocation, no moving of units but the final placement.
+    std::vector<decode_attn_unit_t>& made = out.scratch_units;
+    std::vector<int32_t>& cost = out.scratch_cost;
+    made.clear();
+    cost.clear();
     {
         size_t expect = 0;
         for (int b = 0; b < B; ++b) expect += (size_t)cuts[b].splits;
-        keyed.reserve((expect + (size_t)B) * (size_t)H + 64);
+        made.reserve((expect + (size_t)B) * (size_t)H + 64);
+        cost.reserve(made.capacity());
     }
 
     // Shared prefix: a unit is (block of sequences, KV head, chunk of the prefix); the query rows
@@ -226,6 +231,7 @@ int make_layout(const decode_attn_shape_t& s, const decode_attn_policy_t& p, con
     const bool umma = p.kernel == DA_KERNEL_UMMA_PREFIX && prefix_tokens > 0;
     const int seqs_per_block = prefix_tokens > 0 ? (umma ? kUmmaPrefixRows : kPrefixColumns) / G : 1;
     int32_t PC = 0;
+    size_t n_prefix_units = 0;
     if (prefix_tokens > 0 && B > 0) {
         const int64_t blocks = ceil_div(B, seqs_per_block);
         // the mma.sync kernel runs ctas_per_sm blocks on an SM, the tcgen05 kernel one
@@ -255,20 +261,21 @@ int make_layout(const decode_attn_shape_t& s, const decode_attn_policy_t& p, con
                     pe = pb + q + (i < r ? 1 : 0);
                 }
                 for (int g = 0; g < H; ++g) {
-                    Keyed k;
-                    k.u.seq = b0;
-                    k.u.kv_head = g | (nseq << 16);          // high half: sequences in the block
-                    k.u.tok_begin = (int32_t)(pb * P);
-                    k.u.tok_end = (int32_t)(pe * P);
-                    k.u.slot = -2;                            // records go to each sequence's own slots
-                    k.u.seq_len = seq_lens[b0];
-                    k.u.split_index = i;
-                    k.u.n_splits = 0;
-                    k.cost = (pe - pb) * 4 + (1LL << 40);     // heavier per page, and first in the launch order
-                    keyed.push_back(k);
+                    decode_attn_unit_t u;
+                    u.seq = b0;
+                    u.kv_head = g | (nseq << 16);          // high half: sequences in the block
+                    u.tok_begin = (int32_t)(pb * P);
+                    u.tok_end = (int32_t)(pe * P);
+                    u.slot = -2;                            // records go to each sequence's own slots
+                    u.seq_len = seq_lens[b0];
+                    u.split_index = i;
+                    u.n_splits = 0;
+                    made.push_back(u);
+                    cost.push_back((int32_t)((pe - pb) * 4));     // heavier per page: attended for a whole block of sequences
                 }
             }
         }
+        n_prefix_units = made.size();
     }
 
     for (int b = 0; b < B; ++b) {
@@ -285,89 +292,123 @@ int make_layout(const decode_attn_shape_t& s, const decode_attn_policy_t& p, con
             out.n_slots += S;
             if (out.n_slots > INT32_MAX) return DA_ERR_UNSUPPORTED;
         }
+        const int64_t even_q = S_own > 0 ? cut.pages / S_own : 0, even_r = S_own > 0 ? cut.pages % S_own : 0;
         for (int32_t i = 0; i < S_own; ++i) {
             int64_t pb, pe;
             if (cut.even) {
-                const int64_t q = cut.pages / S_own, r = cut.pages % S_own;
+                const int64_t q = even_q, r = even_r;
                 pb = i * q + std::min<int64_t>(i, r);
                 pe = pb + q + (i < r ? 1 : 0);
             } else {
                 pb = std::min(cut.pages, (int64_t)i * cut.chunk);
                 pe = std::min(cut.pages, (int64_t)(i + 1) * cut.chunk);
             }
+            decode_attn_unit_t u;
+            u.seq = b;
+            u.tok_begin = (int32_t)((prefix_pages + pb) * P);
+            u.tok_end = (int32_t)std::min<int64_t>((prefix_pages + pe) * P, seq_lens[b]);
+            if (u.tok_end < u.tok_begin) u.tok_end = u.tok_begin;
+            u.slot = base_slot >= 0 ? (int32_t)(base_slot + PC + i) : -1;
+            u.seq_len = seq_lens[b];
+            u.split_index = PC + i;
+            u.n_splits = S;
             for (int g = 0; g < H; ++g) {
-                Keyed k;
-                k.u.seq = b;
-                k.u.kv_head = g;
-                k.u.tok_begin = (int32_t)((prefix_pages + pb) * P);
-                k.u.tok_end = (int32_t)std::min<int64_t>((prefix_pages + pe) * P, seq_lens[b]);
-                if (k.u.tok_end < k.u.tok_begin) k.u.tok_end = k.u.tok_begin;
-                k.u.slot = base_slot >= 0 ? (int32_t)(base_slot + PC + i) : -1;
-                k.u.seq_len = seq_lens[b];
-                k.u.split_index = PC + i;
-                k.u.n_splits = S;
-                k.cost = pe - pb;
-                keyed.push_back(k);
+                u.kv_head = g;
+                made.push_back(u);
+                cost.push_back((int32_t)(pe - pb));
             }
         }
     }
     out.prefix_chunks = PC;
-    // Launch order: most expensive unit first, ties in creation order.  Sorting 4-byte indices is
-    // much cheaper than moving the units (this runs every decode step).
-    const size_t n = keyed.size();
-    std::vector<uint32_t> order(n);
+    // Launch order: shared-prefix units first, then most expensive unit first, ties in creation
+    // order.  Costs are small integers (16-token tiles of a unit), so a counting sort does it.
+    const size_t n = made.size();
+    std::vector<uint32_t>& order = out.scratch_order;
+    order.resize(n);
     for (size_t i = 0; i < n; ++i) order[i] = (uint32_t)i;
-    bool sorted = true;
-    for (size_t i = 1; i < n && sorted; ++i) sorted = keyed[i - 1].cost >= keyed[i].cost;
-    if (!sorted)
-        std::stable_sort(order.begin(), order.end(),
-                         [&keyed](uint32_t x, uint32_t y) { return keyed[x].cost > keyed[y].cost; });
-    out.units.clear();
+    auto sort_range = [&](size_t lo, size_t hi) {
+        bool sorted = true;
+        int32_t max_cost = 0;
+        for (size_t i = lo; i < hi; ++i) {
+            if (i > lo && cost[i - 1] < cost[i]) sorted = false;
+            max_cost = std::max(max_cost, cost[i]);
+        }
+        if (sorted) return;
+        if ((size_t)max_cost <= 4 * (hi - lo) + 1024) {
+            std::vector<uint32_t>& cnt = out.scratch_count;
+            cnt.assign((size_t)max_cost + 2, 0);
+            for (size_t i = lo; i < hi; ++i) ++cnt[(size_t)(max_cost - cost[i]) + 1];      // descending cost
+            for (size_t c = 1; c < cnt.size(); ++c) cnt[c] += cnt[c - 1];
+            for (size_t i = lo; i < hi; ++i) order[lo + cnt[(size_t)(max_cost - cost[i])]++] = (uint32_t)i;
+        } else {
+            std::stable_sort(order.begin() + lo, order.begin() + hi,
+                             [&cost](uint32_t x, uint32_t y) { return cost[x] > cost[y]; });
+        }
+    };
+    sort_range(0, n_prefix_units);
+    sort_range(n_prefix_units, n);
     out.units.resize(n);
     out.block_begin.clear();
     out.rank_pos.clear();
     out.n_front_units = 0;
     size_t first = 0;                       // units before this one stay out of the bins
     if (umma) {
-        while (first < n && keyed[order[first]].u.slot == -2) {
-            out.units[first] = keyed[order[first]].u;
-            ++first;
-        }
+        for (; first < n_prefix_units; ++first) out.units[first] = made[order[first]];
         out.n_front_units = (int32_t)first;
     }
     if (max_bins <= 0 || first == n) {
-        for (size_t i = first; i < n; ++i) out.units[i] = keyed[order[i]].u;
+        for (size_t i = first; i < n; ++i) out.units[i] = made[order[i]];
         return DA_OK;
     }
     // Longest unit first onto the lightest bin.  A unit costs its pages (a shared-prefix page
-    // counts four times: it is attended for a whole block of sequences) plus a fixed charge for
-    // the hand-over between units.
-    constexpr int64_t kHandOverPages = 24;
+    // counts four times) plus a fixed charge for the hand-over between units.  Loads are small
+    // integers that only grow, so the lightest bin is found with a bucket queue: one list of bins
+    // per load, the lightest non-empty list never moves down (ties: the bin that got there first).
+    constexpr int32_t kHandOverPages = 24;
     const int bins = (int)std::min<int64_t>((int64_t)(n - first), max_bins);
-    std::vector<int32_t> bin_of(n), count(bins + 1, 0);
-    const bool equal_costs = keyed[order[first]].cost == keyed[order[n - 1]].cost;     // (sorted: first is the largest)
+    std::vector<int32_t>& bin_of = out.scratch_bin_of;
+    std::vector<int32_t>& count = out.scratch_bin_count;
+    bin_of.resize(n);
+    count.assign((size_t)bins + 1, 0);
+    const bool equal_costs = cost[order[first]] == cost[order[n - 1]] && (first >= n_prefix_units || n_prefix_units == n);
     if ((size_t)bins == n - first) {
         for (size_t i = first; i < n; ++i) bin_of[i] = (int32_t)(i - first);      // a bin for every unit
     } else if (equal_costs) {
         for (size_t i = first; i < n; ++i) bin_of[i] = (int32_t)((i - first) % bins);   // what the rule below would do
     } else {
-        // binary min-heap of (load, bin) in an array; the top is replaced in place and sifted down
-        std::vector<std::pair<int64_t, int32_t>> heap(bins);
-        for (int i = 0; i < bins; ++i) heap[i] = {0, i};
+        int64_t total = 0;
+        int32_t biggest = 0;
         for (size_t i = first; i < n; ++i) {
-            bin_of[i] = heap[0].second;
-            std::pair<int64_t, int32_t> top = {heap[0].first + (keyed[order[i]].cost & ((1LL << 40) - 1)) + kHandOverPages,
-                                               heap[0].second};
-            int k = 0;
-            for (;;) {
-                int c = 2 * k + 1;
-                if (c >= bins) break;
-                if (c + 1 < bins && heap[c + 1] < heap[c]) ++c;
-                if (!(heap[c] < top)) break;
-                heap[k] = heap[c];
-                k = c;
-            }
-            heap[k] = top;
+            total += cost[order[i]] + kHandOverPages;
+            biggest = std::max(biggest, cost[order[i]] + kHandOverPages);
+        }
+        // no bin's load passes the mean by more than the biggest unit (the lightest bin is never above the mean)
+        const size_t levels = (size_t)(total / bins + 2 * (int64_t)biggest + 2);
+        std::vector<int32_t>& head = out.scratch_level_head;     // first bin of each load's list, -1: empty
+        std::vector<int32_t>& tail = out.scratch_level_tail;
+        std::vector<int32_t>& next = out.scratch_bin_next;       // next bin in the same list
+        std::vector<int32_t>& load = out.scratch_bin_load;
+        head.assign(levels, -1);
+        tail.assign(levels, -1);
+        next.assign((size_t)bins, -1);
+        load.assign((size_t)bins, 0);
+        for (int i = 0; i < bins; ++i) {                         // all bins start at load 0, in index order
+            next[i] = i + 1 < bins ? i + 1 : -1;
+        }
+        head[0] = 0;
+        tail[0] = bins - 1;
+        size_t lightest = 0;
+        for (size_t i = first; i < n; ++i) {
+            while (head[lightest] < 0) ++lightest;
+            const int32_t b = head[lightest];
+            head[lightest] = next[b];
+            if (head[lightest] < 0) tail[lightest] = -1;
+            bin_of[i] = b;
+            load[b] += cost[order[i]] + kHandOverPages;
+            const size_t l = (size_t)load[b];
+            next[b] = -1;
+            if (tail[l] < 0) head[l] = b; else next[tail[l]] = b;
+            tail[l] = b;
         }
     }
     // counting sort by bin, keeping the order within a bin
@@ -382,7 +423,7 @@ int make_layout(const decode_attn_shape_t& s, const decode_attn_policy_t& p, con
     out.rank_pos.resize(n - first);
     for (size_t i = first; i < n; ++i) {
         const int32_t pos = count[bin_of[i] + 1]++;
-        out.units[pos] = keyed[order[i]].u;
+        out.units[pos] = made[order[i]];
         out.rank_pos[i - first] = pos;
     }
     out.block_begin.push_back((int32_t)out.units.size());

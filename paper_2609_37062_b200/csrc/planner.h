@@ -32,6 +32,11 @@ struct Layout {
     std::vector<int32_t> block_begin;       // [bins + 1] when the units were packed into bins, else empty
     std::vector<int32_t> rank_pos;          // binned layouts: position in `units` of the binned unit with cost rank j
                                             // (j = 0: most expensive; ties in creation order)
+    // working storage of make_layout, kept so that a layout that is refilled every step allocates nothing
+    std::vector<decode_attn_unit_t> scratch_units;
+    std::vector<int32_t> scratch_cost, scratch_bin_of, scratch_bin_count, scratch_level_head, scratch_level_tail,
+        scratch_bin_next, scratch_bin_load;
+    std::vector<uint32_t> scratch_order, scratch_count;
 };
 
 // Validates the fields the planner and the kernels rely on.
