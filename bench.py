@@ -92,6 +92,8 @@ def parse_args(argv=None):
     ap.add_argument("--skip-e2e", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="leave out the list of other configurations")
     ap.add_argument("--extras", action="store_true", help="time the list of other configurations whatever the workload")
+    ap.add_argument("--sweep", action="store_true",
+                    help="instead of the list: every cell of the length x batch sweep (512..131072 x 1..256) in both split modes")
     ap.add_argument("--probe", action="store_true", help="also time the gather-only probe")
     ap.add_argument("--copies", type=int, default=0, help="pool copies to rotate over (0: enough for 1 GiB)")
     ap.add_argument("--alias-after", type=int, default=0,
@@ -382,11 +384,12 @@ def make_mask(torch, w, fraction, dev):
 
 
 def time_config(bench, name, steps, warmup, split="auto", prefix_aware=False, mask_fractions=None, probe=False,
-                replan=False):
+                replan=False, alias=None, pools_closed=None):
     """One entry (or, with mask fractions, several) of the `configs` list: the same timing method
-    as the headline on another workload.  Frees the workload before returning."""
+    as the headline on another workload.  Frees the workload before returning (unless the caller
+    passed the pools in)."""
     torch, da = bench.torch, bench.da
-    pools, closed = workload_copies(name, bench.dev, bench.rank, steps)
+    pools, closed = pools_closed or workload_copies(name, bench.dev, bench.rank, steps, alias=alias)
     w0 = pools[0]
     copies = len(pools)
     policy = da.make_policy(
@@ -421,6 +424,8 @@ def time_config(bench, name, steps, warmup, split="auto", prefix_aware=False, ma
              "GB/s": kv / us / 1e3, "pct_of_8tbs": kv / us / 1e3 / 80.0, "pct_of_measured_hbm": kv / us / 1e3 / peak * 100,
              "units": info.n_units, "chunk_tokens": info.chunk_tokens, "max_splits": info.max_splits_used,
              "copies": copies, "clocks": t["clocks"]}
+        if alias:
+            e["alias_after"] = alias
         if prefix_aware:
             e["shared_prefix_tokens"] = int(policy.shared_prefix_tokens)
             e["unique_GB/s"] = w0.unique_kv_bytes / us / 1e3
@@ -483,6 +488,22 @@ def time_replans(da, shape, policy, lens_host, n=200):
         res["plan_update_us_median"] = us[len(us) // 2]
         res["plan_update_us_p90"] = us[int(len(us) * 0.9)]
     return res
+
+
+def sweep_configs(bench, steps, warmup):
+    """Every cell of the length x batch sweep in both split modes.  The 128 GiB cell does not fit:
+    its sequences i >= 64 reuse the pages of sequence i mod 64 (it is partly served by L2)."""
+    out = []
+    for ctx in (512, 2048, 8192, 32768, 131072):
+        for batch in (1, 8, 64, 256):
+            name = f"sweep_{ctx}x{batch}"
+            alias = 64 if ctx * batch * 4096 > (100 << 30) else None
+            pc = workload_copies(name, bench.dev, bench.rank, steps, alias=alias, cap_bytes=70 << 30)
+            for split in ("auto", "deterministic"):
+                out += time_config(bench, name, steps, warmup, split=split, alias=alias, pools_closed=pc)
+            del pc
+            bench.torch.cuda.empty_cache()
+    return out
 
 
 def extra_configs(bench, steps, warmup):
@@ -832,13 +853,13 @@ def main(argv=None):
 
     # ---- the other configurations, same method (single-GPU default run)
     configs = None
-    want_extras = args.extras or (args.workload == "long_32k" and not args.no_extras and args.mask_fraction is None and
+    want_extras = args.extras or args.sweep or (args.workload == "long_32k" and not args.no_extras and args.mask_fraction is None and
                                   args.split == "auto" and not args.fuse and not args.partial_only)
     if want_extras and world == 1:
         plan.destroy()
         del pools, first
         torch.cuda.empty_cache()
-        configs = extra_configs(bench, min(args.steps, 64), min(max(args.warmup, 3), 8))
+        configs = (sweep_configs if args.sweep else extra_configs)(bench, min(args.steps, 64), min(max(args.warmup, 3), 8))
 
     # ---- the oracle on this machine's cores (rank 0, single-GPU runs only)
     cpu = None
