@@ -135,9 +135,11 @@ def maybe_spawn(args, argv) -> bool:
     if args.gpus <= 1 or "WORLD_SIZE" in os.environ or args.impl == "reference":
         return False
     env = dict(os.environ)
-    # the communicator's own lines (rank count, transport) stay visible in the output
+    # the communicator's own lines (rank count, transport) stay visible - on stderr, so that stdout
+    # carries the one JSON line and nothing else
     env.setdefault("NCCL_DEBUG", "INFO")
     env.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
+    env.setdefault("NCCL_DEBUG_FILE", "/dev/stderr")
     rc = subprocess.call(spawn_command(args.gpus, argv), env=env)
     if rc != 0:
         raise SystemExit(rc)
@@ -686,7 +688,8 @@ def run_kv_shard(args, bench):
                              "traffic_source": None, "kernel": "decode_attn_mma_kernel",
                              "how": "this rank's share of the K+V bytes / the whole step, exchange and merge included"},
                 "gpu_launches": steps * t_full["repeats"] * 3, "clocks": t_full["clocks"], "e2e": None, "cpu_baseline": None}
-        print(json.dumps(line))
+        return line
+    return None
 
 
 # ------------------------------------------------------------------------------------ main
@@ -724,9 +727,11 @@ def main(argv=None):
     bench = Bench(torch, da, dev, local_rank, world, rank)
     stream = bench.stream
     if args.shard == "kv":
-        run_kv_shard(args, bench)
+        line = run_kv_shard(args, bench)
         if world > 1:
             dist.destroy_process_group()
+        if line is not None:
+            print(json.dumps(line), flush=True)
         return
 
     # ---- inputs: R physical copies of the workload, this rank's own sequences
@@ -932,9 +937,10 @@ def main(argv=None):
                                             "arithmetic: the ceiling for this access pattern"}
         if configs is not None:
             line["configs"] = configs
-        print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(line), flush=True)          # the last thing on stdout
 
 
 if __name__ == "__main__":

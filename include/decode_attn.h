@@ -247,10 +247,18 @@ int decode_attn_plan_destroy(decode_attn_plan_t *plan);
  * block_table and run_mask - is read only after it has completed, so ordinary
  * stream order holds for every caller-visible buffer.  One thing happens
  * earlier in the tensor-core kernel: block_table and run_mask are also read
- * before that point to choose a few K/V lines to prefetch into L2.  Those
- * early values are used for nothing else and are read again
- * afterwards, so a kernel that is still writing them does no harm; the
- * buffers only have to be mapped device memory when the launch is enqueued.
+ * before that point to choose a few K/V lines to prefetch into L2, and the
+ * lines of q, seq_lens and block_table that the first unit of every block
+ * needs are asked into L2 as well.  The early values are used for nothing
+ * else and everything is read again afterwards (L2 is where the writes of
+ * the kernel before arrive, so a line brought in early is never stale), so a
+ * kernel that is still writing these buffers does no harm; they only have to
+ * be mapped device memory when the launch is enqueued.
+ *
+ * With a run_mask the units are handed to the thread blocks at run time (a
+ * queue in the plan's device buffer), so that the time a masked row saves
+ * follows the bytes it saves; the results do not depend on which block ran
+ * which unit.
  * ------------------------------------------------------------------------- */
 int decode_attn_run(const decode_attn_plan_t *plan, const void *q, const void *k_cache,
                     const void *v_cache, const int32_t *block_table, const int32_t *seq_lens, void *out,
