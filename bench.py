@@ -106,6 +106,8 @@ def parse_args(argv=None):
                     help="shared_prefix workload: tell the planner about the common prefix (attended once per block of sequences)")
     ap.add_argument("--mask-fraction", type=float, default=None,
                     help="RUN mask (Alg. 1 step 2): this fraction of the rows, picked by a seeded hash, reads no KV")
+    ap.add_argument("--append", default="none", choices=["none", "separate", "fused"],
+                    help="own-layer KV write in the step: a launch of its own before the attention launch, or fused into it")
     ap.add_argument("--dry-spawn", action="store_true",
                     help="start the ranks, join them in a gloo group on the CPU, print how many there are and exit")
     return ap.parse_args(argv)
@@ -766,10 +768,21 @@ def main(argv=None):
     if args.mask_fraction is not None:
         run_mask, masked_bytes = make_mask(torch, first, args.mask_fraction, dev)
 
+    new_k = new_v = None
+    if args.append != "none":
+        from paper_2609_37062_b200 import workloads as wl
+        n_new = first.batch * first.num_kv_heads * first.head_dim
+        new_k = wl.normal_bf16_bits(wl.stream_key(77, wl.TENSOR_NEW_K, 0), 0, n_new, dev).view(first.batch, first.num_kv_heads, -1)
+        new_v = wl.normal_bf16_bits(wl.stream_key(77, wl.TENSOR_NEW_V, 0), 0, n_new, dev).view(first.batch, first.num_kv_heads, -1)
+        launches_per_step += 1 if args.append == "separate" else 0
+
     def step(i, combine=True):
         w = pools[i % copies]
+        if args.append == "separate":
+            da.decode_attn_append_kv(shape, new_k, new_v, w.block_table, w.seq_lens, w.k_pool, w.v_pool)
         da.decode_attn_run(plan, w.q_bits, w.k_pool, w.v_pool, w.block_table, w.seq_lens, out, lse, ws,
-                           plan.workspace_bytes, run_mask=run_mask)
+                           plan.workspace_bytes, run_mask=run_mask,
+                           new_k=new_k if args.append == "fused" else None, new_v=new_v if args.append == "fused" else None)
         if combine and not policy.fuse_combine and not args.partial_only:
             da.decode_attn_combine(plan, ws, out, lse)
 
@@ -900,6 +913,7 @@ def main(argv=None):
                        "max_splits": info.max_splits_used, "kernel": kname, "ctas_per_sm": info.ctas_per_sm,
                        "fused_combine": bool(policy.fuse_combine), "cuda_graph": not args.no_graph,
                        "shared_prefix_tokens": int(policy.shared_prefix_tokens), "alias_after": args.alias_after,
+                       "kv_append": args.append,
                        "l2": f"rotating over {copies} physical pool copies ({copies * unique_bytes / 2**30:.2f} GiB)" +
                              ("" if closed else ", L2 flushed between regions"),
                        "timing": f"median of {timed['repeats']} back-to-back regions of {args.steps} graph-replayed steps, "

@@ -279,6 +279,16 @@ typedef struct {
     float *lse;
     void *workspace;
     size_t workspace_bytes;
+    /* Fused own-layer KV write (both NULL: none; struct_size may also stop before these two
+     * fields).  device, 16-bit (shape.kv_dtype) [batch, num_kv_heads, head_dim], 16-byte aligned:
+     * every row's new K and V rows.  The launch stores them at logical position seq_lens[b] - 1
+     * (as decode_attn_append_kv would: masked rows too, rows of length 0 not) and attends over
+     * them in the same pass, so k_cache and v_cache are modified although they are declared
+     * const here; the result is bit for bit that of decode_attn_append_kv followed by this call
+     * without the two pointers (Algorithm 1 step 2: the row's K/V is written, then the row
+     * attends).  Tensor-core kernel, plans without a shared prefix (DA_ERR_UNSUPPORTED else). */
+    const void *new_k;
+    const void *new_v;
 } decode_attn_run_args_t;
 
 int decode_attn_run_ex(const decode_attn_plan_t *plan, const decode_attn_run_args_t *args,

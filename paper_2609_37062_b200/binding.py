@@ -99,7 +99,8 @@ class RunArgs(ctypes.Structure):
                 ("q", ctypes.c_void_p), ("k_cache", ctypes.c_void_p), ("v_cache", ctypes.c_void_p),
                 ("block_table", ctypes.c_void_p), ("seq_lens", ctypes.c_void_p),
                 ("run_mask", ctypes.c_void_p), ("out", ctypes.c_void_p), ("lse", ctypes.c_void_p),
-                ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t)]
+                ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
+                ("new_k", ctypes.c_void_p), ("new_v", ctypes.c_void_p)]
 
 
 _vp = ctypes.c_void_p
@@ -300,10 +301,12 @@ def decode_attn_plan_destroy(plan: Plan) -> None:
 
 
 def decode_attn_run(plan: Plan, q, k_cache, v_cache, block_table, seq_lens, out, lse=None, workspace=None,
-                    workspace_bytes: Optional[int] = None, stream=None, run_mask=None, check: bool = True) -> int:
+                    workspace_bytes: Optional[int] = None, stream=None, run_mask=None, check: bool = True,
+                    new_k=None, new_v=None) -> int:
+    """new_k / new_v: the rows' new K and V, written at position seq_len - 1 and attended in the same launch."""
     if workspace_bytes is None:
         workspace_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
-    if run_mask is None:
+    if run_mask is None and new_k is None and new_v is None:
         rc = _lib.decode_attn_run(plan.handle, _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(block_table),
                                   _ptr(seq_lens), _ptr(out), _ptr(lse), _ptr(workspace), workspace_bytes,
                                   _stream(stream))
@@ -313,6 +316,7 @@ def decode_attn_run(plan: Plan, q, k_cache, v_cache, block_table, seq_lens, out,
         a.q, a.k_cache, a.v_cache = _ptr(q), _ptr(k_cache), _ptr(v_cache)
         a.block_table, a.seq_lens, a.run_mask = _ptr(block_table), _ptr(seq_lens), _ptr(run_mask)
         a.out, a.lse, a.workspace, a.workspace_bytes = _ptr(out), _ptr(lse), _ptr(workspace), workspace_bytes
+        a.new_k, a.new_v = _ptr(new_k), _ptr(new_v)
         rc = _lib.decode_attn_run_ex(plan.handle, ctypes.byref(a), _stream(stream))
     if check:
         _check(rc, "decode_attn_run")

@@ -5,6 +5,7 @@
 
 #include <algorithm>
 #include <cmath>
+#include <cstddef>
 #include <cstring>
 #include <mutex>
 #include <new>
@@ -348,6 +349,8 @@ KernelParams make_params(const decode_attn_plan_t* pl, const decode_attn_run_arg
     kp.block_table = a.block_table;
     kp.seq_lens = a.seq_lens;
     kp.run_mask = a.run_mask;
+    kp.new_k = static_cast<const __nv_bfloat16*>(a.new_k);
+    kp.new_v = static_cast<const __nv_bfloat16*>(a.new_v);
     kp.out = a.out;
     kp.lse = a.lse;
     kp.ws = static_cast<float*>(a.workspace);
@@ -648,7 +651,19 @@ int decode_attn_plan_destroy(decode_attn_plan_t* pl)
 static int run_impl(const decode_attn_plan_t* pl, const decode_attn_run_args_t* a, cudaStream_t stream, long long debug_limit)
 {
     if (!pl || !a) return DA_ERR_INVALID_ARG;
-    if (a->struct_size != sizeof(decode_attn_run_args_t) || a->flags != 0) return DA_ERR_INVALID_ARG;
+    // (callers built against the struct without its last two fields pass the shorter size)
+    constexpr uint32_t kLegacyArgs = (uint32_t)offsetof(decode_attn_run_args_t, new_k);
+    if ((a->struct_size != sizeof(decode_attn_run_args_t) && a->struct_size != kLegacyArgs) || a->flags != 0)
+        return DA_ERR_INVALID_ARG;
+    decode_attn_run_args_t full;
+    std::memset(&full, 0, sizeof full);
+    std::memcpy(&full, a, a->struct_size);
+    a = &full;
+    if ((a->new_k == nullptr) != (a->new_v == nullptr)) return DA_ERR_INVALID_ARG;
+    if (a->new_k != nullptr) {
+        if (!aligned(a->new_k, 16) || !aligned(a->new_v, 16)) return DA_ERR_INVALID_ARG;
+        if (pl->kernel != DA_KERNEL_MMA_TMA || pl->policy.shared_prefix_tokens > 0) return DA_ERR_UNSUPPORTED;
+    }
     if (pl->shape.batch == 0 && pl->policy.capacity_batch == 0) return DA_OK;
     if (!a->q || !a->k_cache || !a->v_cache || !a->block_table || !a->seq_lens || !a->out) return DA_ERR_INVALID_ARG;
     if (!aligned(a->q, 16) || !aligned(a->k_cache, 16) || !aligned(a->v_cache, 16) || !aligned(a->out, 16) ||

@@ -35,6 +35,10 @@ struct KernelParams {
     const int32_t* block_table;
     const int32_t* seq_lens;
     const uint8_t* run_mask;
+    // Own-layer KV write fused into the attention launch (NULL: none): new K and V rows [batch][Hkv][D] of the
+    // 16-bit input type, stored at position seq_len - 1 of every row and attended from there.
+    const __nv_bfloat16* new_k;
+    const __nv_bfloat16* new_v;
     void* out;
     float* lse;
     float* ws;     // [n_slots][Hkv] partial records, see rec_floats()
@@ -567,6 +571,36 @@ __device__ __forceinline__ void block_finish(const KernelParams& p, const decode
         __threadfence();
         atomicAdd(p.tickets + (int64_t)u.seq * p.num_kv_heads + u.kv_head, 1);
     }
+}
+
+// Own-layer KV write of one (sequence, KV head): the new K and V rows go to position seq_len - 1 of the paged
+// pools (Invariant 1: every valid row writes its K/V whether or not it then attends).  One warp; the unit must
+// be the one that holds the sequence's last token.  Page ids are range-checked like everywhere else.
+template <int D>
+__device__ __forceinline__ void append_new_row(const KernelParams& p, int seq, int g, int seq_len, int lane)
+{
+    if (p.new_k == nullptr || seq_len <= 0) return;
+    const int t = seq_len - 1;
+    const int page_shift = p.tile_shift + 4;
+    if ((t >> page_shift) >= p.max_pages_per_seq) {
+        if (lane == 0) record_status(p.status, DA_ERR_STALE_PLAN);
+        return;
+    }
+    const int page = __ldg(p.block_table + (int64_t)seq * p.max_pages_per_seq + (t >> page_shift));
+    if ((unsigned)page >= (unsigned)p.num_pages) {
+        if (lane == 0) record_status(p.status, DA_ERR_BAD_PAGE);
+        return;
+    }
+    const int slot = t & ((1 << page_shift) - 1);
+    constexpr int CH = D / 8;                               // 16-byte chunks of a row
+    const uint4* sk = reinterpret_cast<const uint4*>(p.new_k + ((int64_t)seq * p.num_kv_heads + g) * D);
+    const uint4* sv = reinterpret_cast<const uint4*>(p.new_v + ((int64_t)seq * p.num_kv_heads + g) * D);
+    uint4* dk = reinterpret_cast<uint4*>(const_cast<__nv_bfloat16*>(p.k) + (int64_t)page * p.k_stride_page +
+                                         (int64_t)slot * p.k_stride_token + (int64_t)g * p.k_stride_head);
+    uint4* dv = reinterpret_cast<uint4*>(const_cast<__nv_bfloat16*>(p.v) + (int64_t)page * p.v_stride_page +
+                                         (int64_t)slot * p.v_stride_token + (int64_t)g * p.v_stride_head);
+    if (lane < CH) dk[lane] = __ldg(sk + lane);
+    else if (lane < 2 * CH) dv[lane - CH] = __ldg(sv + lane - CH);
 }
 
 // The result of a unit that read nothing: zeros (and lse = -inf) for a sequence with a single split,

@@ -372,6 +372,8 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
                 ids = first_ids(x, end);
                 return 1;
             }
+            if (x.tok_end == x.seq_len && x.tok_end > x.tok_begin && (x.kv_head >> 16) == 0)
+                append_new_row<D>(p, x.seq, x.kv_head, x.seq_len, lane);     // a masked row still writes its K/V
             block_finish_empty<D>(p, x, G, lane, 32);
             return 0;
         };
@@ -384,6 +386,8 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
             t1 = unit_end(u);
             int r = 1;
             if (t1 <= u.tok_begin) {
+                if (u.tok_end == u.seq_len && u.tok_end > u.tok_begin && (u.kv_head >> 16) == 0)
+                    append_new_row<D>(p, u.seq, u.kv_head, u.seq_len, lane);
                 block_finish_empty<D>(p, u, G, lane, 32);
                 r = 0;
             }
@@ -431,6 +435,8 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
                         next_state = 1;
                         publish(nu, true);
                     } else {
+                        if (nu.tok_end == nu.seq_len && nu.tok_end > nu.tok_begin && (nu.kv_head >> 16) == 0)
+                            append_new_row<D>(p, nu.seq, nu.kv_head, nu.seq_len, lane);
                         block_finish_empty<D>(p, nu, G, lane, 32);
                         q_link = 0;
                     }
@@ -846,6 +852,25 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
                         *reinterpret_cast<uint4*>(ex.v_out + o) = vv;
                     }
                 } else {
+                    if (p.new_k != nullptr && nseq == 0 && tok0 + n_valid == u.seq_len) {
+                        // Fused own-layer KV write (Algorithm 1 step 2: the row's K/V is written, then the row
+                        // attends over it).  This page holds the sequence's last position, whose K and V rows
+                        // are the new ones: they replace what TMA brought from the pool in the staged tiles -
+                        // same bits as a write to the pool followed by the load - and go to the pool for the
+                        // steps to come.  The pool row belongs to this (sequence, KV head) unit alone.
+                        const int row = n_valid - 1;
+                        const uint4* nk = reinterpret_cast<const uint4*>(p.new_k + ((int64_t)b * p.num_kv_heads + g) * D);
+                        const uint4* nv = reinterpret_cast<const uint4*>(p.new_v + ((int64_t)b * p.num_kv_heads + g) * D);
+                        for (int i = lane; i < 2 * (D / 8); i += 32) {
+                            const int which = i / (D / 8), ch = i % (D / 8);
+                            const uint4 val = __ldg((which ? nv : nk) + ch);
+                            const uint32_t a = (which ? vpage : kpage) + (ch >> 3) * Cfg::kBoxBytes + swz(row, ch & 7);
+                            asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(val.x), "r"(val.y), "r"(val.z), "r"(val.w) : "memory");
+                        }
+                        append_new_row<D>(p, b, g, u.seq_len, lane);
+                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                        __syncwarp();
+                    }
                     if (n_valid < 16) {
                         // rows past the sequence end may hold anything (NaN patterns included) and a
                         // zero weight does not silence them in an mma: clear those V rows.  This is the
@@ -974,6 +999,8 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
         if (n_pages == 0) {
             // Nothing was read (a masked row, an empty split, a sequence of length 0): the empty
             // result is written straight away - no states to merge, no barrier, the scratch untouched.
+            if (MODE == kModeAttend && warp == 0 && nseq == 0 && u.tok_end == u.seq_len && u.tok_end > u.tok_begin)
+                append_new_row<D>(p, b, g, u.seq_len, lane);              // a masked row still writes its K/V
             block_finish_empty<D>(p, u, G, tid, kConsumerThreads);
             if (uid == ubeg && tid == 0) DA_TRACE_STAMP(blockIdx.x, 6);
             if (queued && last_unit) break;

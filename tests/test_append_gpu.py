@@ -79,3 +79,66 @@ def test_checked_append_reports_rows_it_could_not_write():
     assert da.decode_attn_last_device_status(plan) == da.DA_ERR_BAD_PAGE
     assert torch.equal(mid, w.k_pool)                        # the other rows rewrote the same bytes, row 2 wrote nothing
     assert da.decode_attn_last_device_status(plan) == da.DA_OK
+
+
+@pytest.mark.parametrize("page_size", [16, 64])
+@pytest.mark.parametrize("hq,hkv,d", [(8, 2, 64), (32, 8, 128), (64, 8, 128), (96, 8, 128)])
+@pytest.mark.parametrize("mode", ["auto", "deterministic", "fixed3"])
+def test_fused_write_and_attend_equals_write_then_attend(page_size, hq, hkv, d, mode):
+    """Algorithm 1 step 2 in one launch: the attention kernel stores every row's new K/V at
+    position seq_len - 1 (masked rows too) and attends over it in the same pass.  Pools and
+    outputs must equal, bit for bit, what decode_attn_append_kv followed by an ordinary launch
+    gives - and the oracle over the appended cache."""
+    lens = [1, 16, 17, 300, 0, 1024, 1025, 77, 4096, 31, 32, 33]
+    w = wl.make_workload("fused_append", lens, hq, hkv, d, seed=19, page_size=page_size, pool_pages=900 * 16 // page_size)
+    B = len(lens)
+    new_k = wl.normal_bf16_bits(wl.stream_key(19, wl.TENSOR_NEW_K, 0), 0, B * hkv * d).view(B, hkv, d).cuda()
+    new_v = wl.normal_bf16_bits(wl.stream_key(19, wl.TENSOR_NEW_V, 0), 0, B * hkv * d).view(B, hkv, d).cuda()
+    mask = torch.tensor([1, 0, 1, 0, 1, 1, 0, 1, 1, 1, 0, 1], dtype=torch.uint8, device="cuda")
+    pol = {"auto": da.make_policy(chunk_tokens=256),
+           "deterministic": da.make_policy(split_mode=da.DA_SPLIT_DETERMINISTIC),
+           "fixed3": da.make_policy(split_mode=da.DA_SPLIT_FIXED_COUNT, fixed_count=3)}[mode]
+    results = []
+    for fused in (False, True):
+        for run_mask in (None, mask):
+            wd = to_device(w)
+            shape = da.shape_of_workload(wd)
+            plan = da.decode_attn_plan(shape, pol, w.seq_lens)
+            out = torch.full((B, hq, d), float("nan"), dtype=torch.float32, device="cuda")
+            lse = torch.full((B, hq), float("nan"), dtype=torch.float32, device="cuda")
+            ws = torch.empty(max(plan.workspace_bytes, 256), dtype=torch.uint8, device="cuda")
+            if fused:
+                da.decode_attn_run(plan, wd.q_bits, wd.k_pool, wd.v_pool, wd.block_table, wd.seq_lens, out, lse, ws,
+                                   plan.workspace_bytes, run_mask=run_mask, new_k=new_k, new_v=new_v)
+            else:
+                da.decode_attn_append_kv(shape, new_k, new_v, wd.block_table, wd.seq_lens, wd.k_pool, wd.v_pool)
+                da.decode_attn_run(plan, wd.q_bits, wd.k_pool, wd.v_pool, wd.block_table, wd.seq_lens, out, lse, ws,
+                                   plan.workspace_bytes, run_mask=run_mask)
+            da.decode_attn_combine(plan, ws, out, lse)
+            assert da.decode_attn_last_device_status(plan) == da.DA_OK
+            results.append((out, lse, wd.k_pool.clone(), wd.v_pool.clone()))
+    for i in (0, 1):                                       # without / with the mask
+        a, b = results[i], results[2 + i]
+        assert torch.equal(a[2], b[2]) and torch.equal(a[3], b[3]), "pools differ"
+        assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1]), "outputs differ"
+    # against the oracle over the appended cache
+    inp = oracle.PagedInputs.from_workload(w)
+    k_ref, v_ref = oracle.append_kv(inp, new_k.cpu(), new_v.cpu())
+    assert np.array_equal(results[2][2].cpu().numpy().view(np.uint16).ravel(), k_ref.ravel())
+    w.k_pool = torch.from_numpy(k_ref.view(np.int16).reshape(tuple(w.k_pool.shape)))
+    w.v_pool = torch.from_numpy(v_ref.view(np.int16).reshape(tuple(w.v_pool.shape)))
+    ref_out, ref_lse = oracle.paged_decode_attention(oracle.PagedInputs.from_workload(w), run_mask=mask.cpu().numpy())
+    assert_parity(results[3][0], results[3][1], ref_out, ref_lse)
+
+
+def test_fused_write_is_refused_where_it_is_not_built():
+    w = to_device(wl.config_tiny())
+    nk = torch.zeros((4, 2, 64), dtype=torch.int16, device="cuda")
+    out = torch.zeros((4, 8, 64), dtype=torch.float32, device="cuda")
+    plan = da.decode_attn_plan(da.shape_of_workload(w), da.make_policy(kernel=da.DA_KERNEL_SIMT), w.seq_lens)
+    ws = torch.empty(max(plan.workspace_bytes, 256), dtype=torch.uint8, device="cuda")
+    args = (plan, w.q_bits, w.k_pool, w.v_pool, w.block_table, w.seq_lens, out, None, ws, plan.workspace_bytes)
+    assert da.decode_attn_run(*args, new_k=nk, new_v=nk, check=False) == da.DA_ERR_UNSUPPORTED
+    plan = da.decode_attn_plan(da.shape_of_workload(w), da.make_policy(), w.seq_lens)
+    args = (plan,) + args[1:]
+    assert da.decode_attn_run(*args, new_k=nk, new_v=None, check=False) == da.DA_ERR_INVALID_ARG
