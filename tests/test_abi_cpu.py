@@ -44,7 +44,7 @@ def test_struct_sizes_match_the_header():
     assert ctypes.sizeof(da.Unit) == 32
     assert ctypes.sizeof(da.Policy) == 64 and da.Policy.shared_prefix_tokens.offset == 40
     assert ctypes.sizeof(da.Shape) == 96
-    assert ctypes.sizeof(da.RunArgs) == 88
+    assert ctypes.sizeof(da.RunArgs) == 104 and da.RunArgs.new_k.offset == 88      # 88: the struct before new_k / new_v, still accepted
 
 
 def shape(B=4, Hq=32, Hkv=8, D=128, mpp=8192, pages=1 << 20):
