@@ -142,3 +142,26 @@ def test_fused_write_is_refused_where_it_is_not_built():
     plan = da.decode_attn_plan(da.shape_of_workload(w), da.make_policy(), w.seq_lens)
     args = (plan,) + args[1:]
     assert da.decode_attn_run(*args, new_k=nk, new_v=None, check=False) == da.DA_ERR_INVALID_ARG
+
+
+def test_run_args_without_the_new_fields_are_still_accepted():
+    """A caller built against decode_attn_run_args_t as it was before new_k / new_v passes the
+    shorter struct_size; whatever follows in memory must not be read."""
+    import ctypes
+    w = to_device(wl.config_tiny())
+    plan = da.decode_attn_plan(da.shape_of_workload(w), da.make_policy(), w.seq_lens)
+    out = torch.zeros((4, 8, 64), dtype=torch.float32, device="cuda")
+    ws = torch.empty(max(plan.workspace_bytes, 256), dtype=torch.uint8, device="cuda")
+    a = da.RunArgs()
+    a.struct_size = da.RunArgs.new_k.offset
+    a.q, a.k_cache, a.v_cache = w.q_bits.data_ptr(), w.k_pool.data_ptr(), w.v_pool.data_ptr()
+    a.block_table, a.seq_lens, a.out = w.block_table.data_ptr(), w.seq_lens.data_ptr(), out.data_ptr()
+    a.workspace, a.workspace_bytes = ws.data_ptr(), plan.workspace_bytes
+    a.new_k = a.new_v = 0xdead0                          # garbage behind the declared size
+    before = w.k_pool.clone()
+    assert da._lib.decode_attn_run_ex(plan.handle, ctypes.byref(a), torch.cuda.current_stream().cuda_stream) == da.DA_OK
+    da.decode_attn_combine(plan, ws, out)
+    assert da.decode_attn_last_device_status(plan) == da.DA_OK
+    assert torch.equal(before, w.k_pool) and out.abs().sum() > 0
+    a.struct_size = 80
+    assert da._lib.decode_attn_run_ex(plan.handle, ctypes.byref(a), torch.cuda.current_stream().cuda_stream) == da.DA_ERR_INVALID_ARG
