@@ -10,7 +10,7 @@
 namespace da {
 
 // BATCH: records a thread keeps in flight (see combine_slice).
-template <int D, int BATCH>
+template <int D, int BATCH, bool ONE_PASS>
 __global__ void __launch_bounds__(kCombineThreads) decode_attn_combine_kernel(const KernelParams p, int G, int n_slices)
 {
     __shared__ __align__(16) float sm[kCombineSmemFloats];
@@ -29,7 +29,7 @@ __global__ void __launch_bounds__(kCombineThreads) decode_attn_combine_kernel(co
     pdl_wait_primary();                                   // the records of the launch before this one are complete
     if (threadIdx.x == 0) DA_TRACE_STAMP(p.n_work_blocks + blockIdx.x, 1);
     if (si.slot_base < 0) return;                         // a single split, written directly by the partial kernel
-    combine_slice<D, BATCH>(p, b, g, slice, G, si.slot_base, si.n_splits, threadIdx.x, sm, 0);
+    combine_slice<D, BATCH, ONE_PASS>(p, b, g, slice, G, si.slot_base, si.n_splits, threadIdx.x, sm, 0);
     if (threadIdx.x == 0) DA_TRACE_STAMP(p.n_work_blocks + blockIdx.x, 2);
 }
 
@@ -109,9 +109,10 @@ inline int combine_launch_dim(int G, const KernelParams& kp, unsigned groups, cu
     const cudaError_t e =
         max_splits <= 4    ? cudaLaunchKernelEx(&cfg, decode_attn_combine_few_kernel<D, 4>, kp, G, blocks_per_group)
         : max_splits <= 8  ? cudaLaunchKernelEx(&cfg, decode_attn_combine_few_kernel<D, 8>, kp, G, blocks_per_group)
-        : max_splits <= 32 ? cudaLaunchKernelEx(&cfg, decode_attn_combine_kernel<D, 8>, kp, G, n_slices)
-        : max_splits <= 40 ? cudaLaunchKernelEx(&cfg, decode_attn_combine_kernel<D, 10>, kp, G, n_slices)
-                           : cudaLaunchKernelEx(&cfg, decode_attn_combine_kernel<D, kCombineBatch>, kp, G, n_slices);
+        : max_splits <= 32 ? cudaLaunchKernelEx(&cfg, decode_attn_combine_kernel<D, 8, true>, kp, G, n_slices)
+        : max_splits <= 40 ? cudaLaunchKernelEx(&cfg, decode_attn_combine_kernel<D, 10, true>, kp, G, n_slices)
+        : max_splits <= 48 ? cudaLaunchKernelEx(&cfg, decode_attn_combine_kernel<D, kCombineBatch, true>, kp, G, n_slices)
+                           : cudaLaunchKernelEx(&cfg, decode_attn_combine_kernel<D, kCombineBatch, false>, kp, G, n_slices);
     if (e != cudaSuccess) {
         (void)cudaGetLastError();
         return DA_ERR_CUDA;

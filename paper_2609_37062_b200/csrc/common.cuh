@@ -284,7 +284,8 @@ constexpr int kCombineThreads = 128;
 constexpr int kCombineBatch = 12;
 constexpr int kCombineSmemFloats = 4 * 32 * 6;
 
-template <int D, int BATCH = kCombineBatch>
+// ONE_PASS: the caller knows S <= 4 * BATCH, so the code for further rounds is left out.
+template <int D, int BATCH = kCombineBatch, bool ONE_PASS = false>
 __device__ __forceinline__ void combine_slice(const KernelParams& p, int b, int g, int slice, int G, int slot_base,
                                               int S, int tid, float* sm, int bar_id)
 {
@@ -318,7 +319,8 @@ __device__ __forceinline__ void combine_slice(const KernelParams& p, int b, int 
     float mloc = -INFINITY;
 #pragma unroll
     for (int t = 0; t < kCombineBatch; ++t) mloc = fmaxf(mloc, ml[t].x);
-    for (int j = q + 4 * kCombineBatch; j < S; j += 4) mloc = fmaxf(mloc, __ldcg(mlp + j * (rec_stride / 2)).x);
+    if (!ONE_PASS)
+        for (int j = q + 4 * kCombineBatch; j < S; j += 4) mloc = fmaxf(mloc, __ldcg(mlp + j * (rec_stride / 2)).x);
     sm_m[q * 32 + lane] = mloc;
     if (tid == 0) DA_TRACE_STAMP(p.n_work_blocks + blockIdx.x, 3);
     block_sync(bar_id, kCombineThreads);
@@ -327,8 +329,8 @@ __device__ __forceinline__ void combine_slice(const KernelParams& p, int b, int 
 
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     float lch = 0.f;
-    for (int t0 = 0; q + 4 * t0 < S; t0 += kCombineBatch) {
-        if (t0 > 0) {
+    for (int t0 = 0; q + 4 * t0 < S && (!ONE_PASS || t0 == 0); t0 += kCombineBatch) {
+        if (!ONE_PASS && t0 > 0) {
 #pragma unroll
             for (int t = 0; t < kCombineBatch; ++t) {
                 const int j = q + 4 * (t0 + t);
