@@ -527,11 +527,13 @@ __device__ __forceinline__ void block_finish(const KernelParams& p, const decode
     const int h0 = u.kv_head * G;
     const int RF = rec_floats(G, D);
     float* const rec = (u.slot >= 0) ? p.ws + ((int64_t)u.slot * p.num_kv_heads + u.kv_head) * RF : nullptr;
+    if (tid == 0) DA_TRACE_CLOCK(blockIdx.x + 4096, 0);
     for (int task = tid; task < head_count * D4; task += nthreads) {
         const int h = task / D4, d4 = task % D4;          // source column h is head head_first + h
         float M = -INFINITY;
 #pragma unroll kUnroll
         for (int r = 0; r < R; ++r) M = fmaxf(M, src_m[r * COLS + h]);
+        if (tid == 0) DA_TRACE_CLOCK(blockIdx.x + 4096, 1);
         float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
         float ls = 0.f;
         if (M != -INFINITY) {
@@ -550,6 +552,7 @@ __device__ __forceinline__ void block_finish(const KernelParams& p, const decode
                 ls = fmaf(w, src_l[r * COLS + h], ls);
             }
         }
+        if (tid == 0) DA_TRACE_CLOCK(blockIdx.x + 4096, 2);
         if (rec == nullptr) {
             if (ls > 0.f) {
                 const float inv = 1.0f / ls;
@@ -565,6 +568,7 @@ __device__ __forceinline__ void block_finish(const KernelParams& p, const decode
             if (d4 == 0) __stcg(reinterpret_cast<float2*>(rec + G * D) + head_first + h, make_float2(M, ls));
         }
     }
+    if (tid == 0) DA_TRACE_CLOCK(blockIdx.x + 4096, 3);
     if (rec == nullptr || !p.fused || !publish) return;
     // The barrier orders every thread's record stores before thread 0's fence, which publishes
     // them device-wide ahead of the arrival.

@@ -494,6 +494,9 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
                     const int slot0 = ((tile0 + it * kPagesPerStage + pg) & ((1 << ts) - 1)) << 4;   // of the tile within its page
                     tma_load_4d(dst, which ? &v_map : &k_map, full, hf * 64, slot0, g, page_id, l2_policy);
                     if (git == 0 && lane == 0) DA_TRACE_STAMP(blockIdx.x, 2);
+#ifdef DA_TRACE
+                    if (lane == 0 && uid - ubeg == 1 && it == 0) DA_TRACE_CLOCK(blockIdx.x, 30);   // second unit's first copy
+#endif
                 }
                 if (queued) {
                     // One link of the look at the queue per stage issued, so that a run of masked rows
@@ -599,6 +602,13 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
         decode_attn_unit_t nu = u;
         if (!queued && !last_unit) nu = load_unit(p.units, uid + 1);      // lands while this unit is consumed
         Pre nxt = cur;
+#ifdef DA_TRACE
+        // per-unit cycle stamps of a block's first four units: slots 10 + 4k .. 13 + 4k = the unit is taken up, its
+        // first stage has landed, its streaming loop is done, it is finished; slots 26 .. 29 split the second unit's
+        // finish (before / behind the vote barrier, states in the scratch, behind the second barrier)
+        const int trace_k = uid - ubeg;
+        if (tid == 0 && trace_k < 4) DA_TRACE_CLOCK(blockIdx.x, 10 + trace_k * 4);
+#endif
         const int b = u.seq, g = u.kv_head & 0xffff;
         const int nseq = u.kv_head >> 16;                                  // > 0: a shared-prefix unit
         const int t0 = u.tok_begin;
@@ -825,6 +835,9 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
                 break;
             }
             if (git == 0 && tid == 0) DA_TRACE_STAMP(blockIdx.x, 3);
+#ifdef DA_TRACE
+            if (it == 0 && tid == 0 && trace_k < 4) DA_TRACE_CLOCK(blockIdx.x, 11 + trace_k * 4);
+#endif
             const int page_idx = it * kPagesPerStage + warp;
             if (page_idx < n_pages) {
                 const int tok0 = t0 + page_idx * 16;
@@ -962,6 +975,9 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
             if (lane == 0) mbar_arrive(bar_base + 8 * (NS + s));          // this warp is done with the stage
         }
         if (uid == ubeg && tid == 0) DA_TRACE_STAMP(blockIdx.x, 4);
+#ifdef DA_TRACE
+        if (tid == 0 && trace_k < 4) DA_TRACE_CLOCK(blockIdx.x, 12 + trace_k * 4);
+#endif
         if (queued) {
             // the producer drew the next unit while this one streamed
             const int need = uid - ubeg + 2;
@@ -1019,7 +1035,13 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
         // Every warp is done reading the previous unit's results.  A warp may have given up on a
         // wait just before the others saw the flag: the barrier carries a vote, every warp gets
         // the same answer, the unit's result is voided and the block leaves together.
+#ifdef DA_TRACE
+        if (tid == 0 && trace_k == 1) DA_TRACE_CLOCK(blockIdx.x, 26);
+#endif
         const bool gave_up = block_sync_or(1, kConsumerThreads, failed || sm_flags[0] != 0);
+#ifdef DA_TRACE
+        if (tid == 0 && trace_k == 1) DA_TRACE_CLOCK(blockIdx.x, 27);
+#endif
         if (gave_up || stale) {
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
@@ -1059,11 +1081,20 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
                     wo[D + mt * 16 + r + 8] = oacc[mt][nt][3];
                 }
             }
+#ifdef DA_TRACE
+            if (tid == 0 && trace_k == 1 && q == 0) DA_TRACE_CLOCK(blockIdx.x, 28);
+#endif
             block_sync(1, kConsumerThreads);
+#ifdef DA_TRACE
+            if (tid == 0 && trace_k == 1 && q == 0) DA_TRACE_CLOCK(blockIdx.x, 29);
+#endif
             block_finish<D, kMmaConsumerWarps, COLS, false>(p, u, G, sm_wo, sm_wm, sm_wl, tid, kConsumerThreads, 1, 4 * q,
                                                             min(4, G - 4 * q), DUP || 4 * (q + 1) >= G);
         }
         if (uid == ubeg && tid == 0) DA_TRACE_STAMP(blockIdx.x, 6);
+#ifdef DA_TRACE
+        if (tid == 0 && trace_k < 4) DA_TRACE_CLOCK(blockIdx.x, 13 + trace_k * 4);
+#endif
         if (gave_up) return;
         if (queued && last_unit) break;
         u = nu;

@@ -29,6 +29,14 @@ def main(argv=None):
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--copies", type=int, default=10)
     ap.add_argument("--fuse", action="store_true")
+    ap.add_argument("--split", default="auto", choices=["auto", "deterministic"])
+    ap.add_argument("--workload", default="sweep", choices=["sweep", "short_chat", "few_shot_suffixes"],
+                    help="sweep: --batch sequences of --context tokens; short_chat: the 64-sequence chat mix; "
+                         "few_shot_suffixes: the 256 private suffixes (16..256 tokens) of the few-shot batch, by themselves")
+    ap.add_argument("--units", action="store_true",
+                    help="also print, in SM clock cycles turned into microseconds at --mhz, what a block's first four units "
+                         "spend waiting for their first stage, streaming and finishing, and how the second unit's finish divides")
+    ap.add_argument("--mhz", type=float, default=1965.0)
     args = ap.parse_args(argv)
 
     from . import build as da_build
@@ -41,9 +49,17 @@ def main(argv=None):
     lib = da._lib
     lib.decode_attn_trace_set_buffer.argtypes = [ctypes.c_void_p]
     K, copies = args.steps, args.copies
-    pools = [wl.config_sweep_cell(args.context, args.batch, device="cuda", table_seed=i) for i in range(copies)]
+    if args.workload == "short_chat":
+        pools = [wl.config_short_chat(device="cuda", table_seed=i) for i in range(copies)]
+    elif args.workload == "few_shot_suffixes":
+        lens = [x - 1536 for x in wl.lengths_shared_prefix(256, 3)]
+        pools = [wl.make_workload("few_shot_suffixes", lens, 32, 8, 128, seed=3, device="cuda", table_seed=i) for i in range(copies)]
+    else:
+        pools = [wl.config_sweep_cell(args.context, args.batch, device="cuda", table_seed=i) for i in range(copies)]
     w = pools[0]
-    plan = da.decode_attn_plan(da.shape_of_workload(w), da.make_policy(fuse_combine=int(args.fuse)), w.seq_lens)
+    policy = da.make_policy(fuse_combine=int(args.fuse),
+                            split_mode=da.DA_SPLIT_DETERMINISTIC if args.split == "deterministic" else da.DA_SPLIT_AUTO)
+    plan = da.decode_attn_plan(da.shape_of_workload(w), policy, w.seq_lens)
     info = plan.info()
     if info.kernel != da.DA_KERNEL_MMA_TMA:
         raise SystemExit("the timeline covers plans of the tensor-core kernel")
@@ -82,7 +98,8 @@ def main(argv=None):
         e1.record(s)
         s.synchronize()
     lib.decode_attn_trace_set_buffer(None)
-    print(f"{args.context} tokens x {args.batch}: {info.n_units} units on {n} blocks; "
+    what = f"{args.context} tokens x {args.batch}" if args.workload == "sweep" else args.workload
+    print(f"{what} ({args.split}): {info.n_units} units on {n} blocks; "
           f"region of {K} steps: {e0.elapsed_time(e1) * 1e3 / K:.2f} us per step (traced build)")
     t = trace.cpu().numpy().astype(np.float64)
     P, C = t[:, :n, :], t[:, n:, :]
@@ -114,6 +131,38 @@ def main(argv=None):
     period = [per_step[i + 1]["partial: dependency wait over"][0] - per_step[i]["partial: dependency wait over"][0]
               for i in range(2, K - 1)]
     print(f"step period (end of wait to end of wait): median {np.median(period) / 1e3:.2f} us")
+    if args.units:
+        c = P[2:]                                     # steps 2.., every block
+
+        def med(a, ok):
+            a = a[ok]
+            return float(np.median(a)) / args.mhz if a.size else float("nan")
+
+        print(f"per unit, SM cycles at {args.mhz:.0f} MHz, medians over blocks and steps (us):")
+        for k in range(4):
+            c0, c1, c2, c3 = (c[:, :, 10 + 4 * k + j] for j in range(4))
+            ok = (c0 > 0) & (c1 > 0) & (c2 > 0) & (c3 > 0)
+            if not ok.any():
+                continue
+            line = (f"  unit {k}: waits for its first stage {med(c1 - c0, ok):.2f}, streams {med(c2 - c1, ok):.2f}, "
+                    f"finishes {med(c3 - c2, ok):.2f}")
+            if k > 0:
+                prev = c[:, :, 13 + 4 * (k - 1)]
+                line += f" (taken up {med(c0 - prev, ok & (prev > 0)):.2f} after the unit before was finished)"
+            print(line)
+        c2, c3 = c[:, :, 16], c[:, :, 17]
+        a, b2, cc, d = (c[:, :, 26 + j] for j in range(4))
+        ok = (c2 > 0) & (a > 0) & (b2 > 0) & (cc > 0) & (d > 0) & (c3 > 0)
+        if ok.any():
+            print(f"  the second unit's finish: next unit's loads asked for, sums shuffled {med(a - c2, ok):.2f} | vote barrier "
+                  f"{med(b2 - a, ok):.2f} | low parts added, states into the scratch {med(cc - b2, ok):.2f} | barrier "
+                  f"{med(d - cc, ok):.2f} | merge of the four warps' states and the record {med(c3 - d, ok):.2f}")
+        f = t[2:, 4096:4096 + n, :]                   # stamps inside the merge of a block's last unit
+        f0, f1, f2, f3 = (f[:, :, j] for j in range(4))
+        ok = (f0 > 0) & (f1 > f0) & (f2 > f1) & (f3 > f2)
+        if ok.any():
+            print(f"  inside that merge (a block's last unit): maximum over the warps {med(f1 - f0, ok):.2f} | weights and sums "
+                  f"{med(f2 - f1, ok):.2f} | stores {med(f3 - f2, ok):.2f}")
 
 
 if __name__ == "__main__":
