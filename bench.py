@@ -510,11 +510,22 @@ def sweep_configs(bench, steps, warmup):
     return out
 
 
-def extra_configs(bench, steps, warmup):
+def oracle_beside(entry, name, skip):
+    """The oracle as it stands on this machine's cores, on the same workload (a reported baseline)."""
+    if skip:
+        return
+    sec, reps, cores = time_oracle(make_workload(name, "cpu"), budget_s=2.0)
+    entry["cpu_baseline"] = {"ms_per_step": sec * 1e3, "value": entry["logical_kv_bytes"] / sec / 1e9, "unit": UNIT,
+                             "cores": cores, "kind": "oracle", "sample": f"whole batch, {reps} runs"}
+
+
+def extra_configs(bench, steps, warmup, skip_cpu=False):
     """The other workload configurations, timed like the headline (median of repeated regions)."""
     out = []
     out += time_config(bench, "short_chat", steps, warmup, replan=True)
+    oracle_beside(out[-1], "short_chat", skip_cpu)
     out += time_config(bench, "shared_prefix", steps, warmup)
+    oracle_beside(out[-1], "shared_prefix", skip_cpu)
     out += time_config(bench, "shared_prefix", steps, warmup, prefix_aware=True)
     for cell, probe in (("sweep_512x256", False), ("sweep_2048x1", False), ("sweep_8192x64", True),
                         ("sweep_32768x8", False), ("sweep_131072x1", False)):
@@ -877,7 +888,8 @@ def main(argv=None):
         plan.destroy()
         del pools, first
         torch.cuda.empty_cache()
-        configs = (sweep_configs if args.sweep else extra_configs)(bench, min(args.steps, 64), min(max(args.warmup, 3), 8))
+        k_extra, w_extra = min(args.steps, 64), min(max(args.warmup, 3), 8)
+        configs = sweep_configs(bench, k_extra, w_extra) if args.sweep else extra_configs(bench, k_extra, w_extra, args.skip_cpu)
 
     # ---- the oracle on this machine's cores (rank 0, single-GPU runs only)
     cpu = None

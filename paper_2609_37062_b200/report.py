@@ -74,6 +74,9 @@ def configs(d):
             peak = c["GB/s"] / (c["pct_of_measured_hbm"] / 100.0)
             print(f"| {c['workload']} | {plan} | {c['us_per_step']:.2f} ({c['us_per_step_min']:.2f}) | {c['GB/s']:.0f} | "
                   f"{c['pct_of_8tbs']:.1f} | {uq:.0f} | {uq / peak * 100:.1f} | {c['units']} | {_clk(c['clocks'])} |")
+            if c.get("cpu_baseline"):
+                o = c["cpu_baseline"]
+                print(f"| | oracle on {o['cores']} host cores | {o['ms_per_step']:.1f} ms per step | {o['value']:.2f} | | | | | |")
             if c.get("replan"):
                 r = c["replan"]
                 print(f"| | re-plan us median / p90 | {r['plan_destroy_us_median']:.1f} / {r['plan_destroy_us_p90']:.1f}"
