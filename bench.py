@@ -32,7 +32,13 @@ every rank attends its range, one all-gather moves (out, lse) and the
 library's shard merge finishes the step (strong scaling).
 
 The default single-GPU run also times a fixed list of the other workload
-configurations with the same method and prints them under `configs`.
+configurations with the same method and prints them under `configs`
+(short_chat and the few-shot batch with the oracle's time beside them, five
+sweep cells in both split modes, the RUN-mask series, gather-only probes);
+--sweep times all 20 cells of the length x batch sweep instead.  --append
+puts the own-layer KV write into the step, as a launch of its own or fused
+into the attention launch.  `python -m paper_2609_37062_b200.report` turns
+the JSON line into tables.
 """
 from __future__ import annotations
 
