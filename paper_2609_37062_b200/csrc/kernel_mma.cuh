@@ -1100,6 +1100,7 @@ __global__ void __launch_bounds__(kMmaThreads, 2) decode_attn_mma_kernel(const K
         u = nu;
         cur = nxt;
     }
+    if (tid == 0) DA_TRACE_STAMP(blockIdx.x, 5);                  // (trace builds) the block's last unit is finished
 }
 
 // ---------------------------------------------------------------- host side

@@ -112,6 +112,7 @@ def main(argv=None):
              ("partial: producer past the wait", "P", 8), ("partial: first page ids in hand", "P", 9),
              ("partial: first copy issued", "P", 2), ("partial: first stage landed", "P", 3),
              ("partial: first unit's streaming loop done", "P", 4), ("partial: first unit finished", "P", 6),
+             ("partial: last unit finished", "P", 5),
              ("combine: block entry", "C", 0), ("combine: dependency wait over", "C", 1),
              ("combine: loads landed", "C", 3), ("combine: sums done", "C", 5), ("combine: done", "C", 2)]
     per_step = [{nm: rng((P if src == "P" else C)[i, :, slot]) for nm, src, slot in names} for i in range(K)]
