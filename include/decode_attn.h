@@ -205,7 +205,10 @@ int decode_attn_plan(const decode_attn_shape_t *shape, const decode_attn_policy_
  * and enqueues the upload of the refreshed work list on `stream`; the device
  * addresses, grid and kernel stay the same, so a CUDA graph captured around
  * run/combine keeps working.  Only for plans made with capacity_batch > 0.
- * seq_lens_host must stay valid until the call returns (it is copied). */
+ * The copy is ordered like any other work on `stream`: behind the launches
+ * already queued there, ahead of those that follow; launches on another
+ * stream are for the caller to order.  seq_lens_host must stay valid until
+ * the call returns (it is copied). */
 int decode_attn_plan_update(decode_attn_plan_t *plan, int32_t batch, const int32_t *seq_lens_host,
                             cudaStream_t stream);
 
