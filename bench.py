@@ -574,6 +574,14 @@ def oracle_sample(name):
     return w, "whole batch", 1.0
 
 
+def workload_keys(name, w):
+    """The keys of `config` that name the workload; the same in both arms."""
+    return {"workload": name, "batch": int(w.batch), "num_q_heads": int(w.num_q_heads),
+            "num_kv_heads": int(w.num_kv_heads), "head_dim": int(w.head_dim), "page_size": int(w.page_size),
+            "tokens": int(w.logical_kv_bytes) // (int(w.num_kv_heads) * int(w.head_dim) * 4),
+            "logical_kv_bytes": int(w.logical_kv_bytes), "unique_kv_bytes": int(w.unique_kv_bytes)}
+
+
 def run_reference(args):
     """The oracle as it stands on this machine's cores: W warm-up and exactly K timed steps, each step a
     bounded sample of the workload sized so that the whole run ends within a few minutes."""
@@ -585,6 +593,11 @@ def run_reference(args):
     # torch's launcher sets OMP_NUM_THREADS=1 for its ranks; the oracle takes the machine's cores all the same
     threads = (os.cpu_count() or 1) if os.environ.get("TORCHELASTIC_RUN_ID") else oracle.max_threads()
     w, sample, _ = oracle_sample(args.workload)
+    full_keys = workload_keys(args.workload, w)
+    if sample != "whole batch":                           # a sweep cell: the whole cell's size, without generating it
+        ctx, batch = (int(x) for x in args.workload[len("sweep_"):].split("x"))
+        nbytes = ctx * batch * int(w.num_kv_heads) * int(w.head_dim) * 4
+        full_keys.update(batch=batch, tokens=ctx * batch, logical_kv_bytes=nbytes, unique_kv_bytes=nbytes)
     inp = oracle.PagedInputs.from_workload(w)
     t0 = time.perf_counter()
     oracle.paged_decode_attention(inp, num_threads=threads)
@@ -613,7 +626,7 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": gbs, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
             "warmup": warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": args.workload, "sample": sample, "tokens": w.logical_tokens},
+            "config": dict(full_keys, sample=sample, sample_tokens=w.logical_tokens),
             "cpu_baseline": {"value": gbs, "unit": UNIT, "cores": threads, "kind": "oracle",
                              "sample": sample},
             "e2e": {"value": gbs, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
@@ -759,6 +772,7 @@ def main(argv=None):
     first, copies = pools[0], len(pools)
     kv_bytes = first.logical_kv_bytes
     unique_bytes = first.unique_kv_bytes
+    wl_keys = workload_keys(args.workload, first)
 
     kernel = {"auto": da.DA_KERNEL_AUTO, "simt": da.DA_KERNEL_SIMT, "mma": da.DA_KERNEL_MMA_TMA,
               "umma": da.DA_KERNEL_UMMA_PREFIX}[args.kernel]
@@ -915,18 +929,13 @@ def main(argv=None):
         kname = {da.DA_KERNEL_SIMT: "decode_attn_simt_kernel", da.DA_KERNEL_MMA_TMA: "decode_attn_mma_kernel",
                  da.DA_KERNEL_UMMA_PREFIX: "decode_attn_umma_prefix_kernel + decode_attn_mma_kernel"}[info.kernel]
         traffic, traffic_src = NCU_TRAFFIC_BYTES.get(args.workload, (None, None))
-        shape_batch = int(shape.batch)
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "repeats": timed["repeats"], "ms_per_step": sec_per_step * 1e3,
             "us_per_step": sec_per_step * 1e6, "us_per_step_min": ms_min * 1e3 / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": f"{IN_DTYPE} in, f32 accumulate",
             "data": "synthetic",
-            "config": {"workload": args.workload, "batch": shape_batch, "num_q_heads": int(shape.num_q_heads),
-                       "num_kv_heads": int(shape.num_kv_heads), "head_dim": int(shape.head_dim),
-                       "page_size": int(shape.page_size),
-                       "tokens": kv_bytes // (int(shape.num_kv_heads) * int(shape.head_dim) * 4),
-                       "logical_kv_bytes": kv_bytes, "unique_kv_bytes": unique_bytes,
+            "config": {**wl_keys,
                        "split": args.split, "chunk_tokens": info.chunk_tokens, "units": info.n_units,
                        "max_splits": info.max_splits_used, "kernel": kname, "ctas_per_sm": info.ctas_per_sm,
                        "fused_combine": bool(policy.fuse_combine), "cuda_graph": not args.no_graph,
