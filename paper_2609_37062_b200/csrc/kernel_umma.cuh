@@ -59,7 +59,7 @@
 namespace da {
 
 constexpr int kUmmaTraceBase = 2048;              // debug timelines: rows of this kernel's units
-constexpr int kUmmaSoftmaxWarps = 8;              // a multiple of 4: warps w, w + 4, ... share 32 lanes of tensor memory
+constexpr int kUmmaSoftmaxWarps = 8;              // 8 or 16 (measured: no faster): warps w, w + 4, ... share 32 lanes of tensor memory
 constexpr int kUmmaThreadsPerRow = kUmmaSoftmaxWarps / 4;
 constexpr int kUmmaGroupsPerThread = 4 / kUmmaThreadsPerRow;     // 32-token groups of a tile a thread owns
 constexpr int kUmmaOutColsPerThread = 128 / kUmmaThreadsPerRow;  // output columns a thread owns
@@ -387,8 +387,9 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
             for (int i = 0; i < OC; ++i) acc[i] = 0.f;
             float M = -INFINITY, L = 0.f;       // running maximum (log2 domain), this thread's share of the row sum
             float m_prev = 0.f, l_prev = 0.f;   // of the tile whose output is still to be folded in
-            static_assert(GP == 2 && OC == 64, "a thread owns 64 consecutive logit columns and 64 output columns");
-            uint32_t sg[64];                        // logits of the thread's columns; also the output tile on its way in
+            static_assert(32 * GP == OC && (OC == 64 || OC == 32), "a thread owns as many consecutive logit columns as output columns");
+            uint32_t sg[OC];                        // logits of the thread's columns; also the output tile on its way in
+            auto ld_cols = [&](uint32_t taddr) { umma::ld_cols(taddr, sg); };
             bool ok = true;
 
             // folds tile i's output into the running state
@@ -399,7 +400,7 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
                 if (tid == 0 && i < 8) DA_TRACE_CLOCK(kUmmaTraceBase + 1024 + unit_index, 16 + i);
                 umma::fence_after_thread_sync();
                 const uint32_t oc = lane_base + kUmmaOutCol + b * 128 + hh * OC;
-                umma::ld64(oc, sg);
+                ld_cols(oc);
                 umma::wait_ld();
                 umma::fence_before_thread_sync();
                 mbar_arrive(bar_ofree + 8 * b);                              // the buffer may be overwritten
@@ -432,7 +433,7 @@ __device__ __forceinline__ void umma_prefix_units(const KernelParams& p, const C
                     // pass 1: the maximum of this thread's logits; the row's other parts are exchanged
                     // through shared memory (their logits may not be read once they start writing weights)
                     float mx = -INFINITY;
-                    umma::ld64(sc + hh * 64, sg);                           // columns 64 hh .. 64 hh + 63
+                    ld_cols(sc + hh * OC);                                  // columns OC hh .. OC hh + OC - 1
                     umma::wait_ld();
 #pragma unroll
                     for (int q = 0; q < GP; ++q)

@@ -129,6 +129,9 @@ __device__ __forceinline__ void ld64(uint32_t taddr, uint32_t (&r)[64])
         : "memory");
 }
 
+// 32 or 64 columns, by the size of the destination
+__device__ __forceinline__ void ld_cols(uint32_t taddr, uint32_t (&r)[32]) { ld32(taddr, r); }
+__device__ __forceinline__ void ld_cols(uint32_t taddr, uint32_t (&r)[64]) { ld64(taddr, r); }
 __device__ __forceinline__ void wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // 16 consecutive columns of this thread's lane.
