@@ -383,13 +383,14 @@ KernelParams make_params(const decode_attn_plan_t* pl, const decode_attn_run_arg
     kp.n_units = (int32_t)pl->layout.units.size();
     kp.wait_limit = kWaitLimitCycles;
     // The tensor-core kernel asks the first pages of every block into L2 ahead of its dependency
-    // wait.  Two stages' worth when a block has a single unit (the opening burst is then a visible
-    // share of the step: 24.9 -> 23.0 us on one 32k sequence), one stage's worth otherwise
-    // (short_chat 20.0 -> 19.1 us); more than that costs more than it brings.
+    // wait.  Seven pages, just short of two stages' worth, when a block has a single unit (the opening
+    // burst is then a visible share of the step: 24.8 us without hints, 23.9 / 23.6 / 23.2 / 23.2 /
+    // 23.4 with 2 / 4 / 6 / 7 / 8 pages on one 32k sequence, more pages slower again), one stage's
+    // worth otherwise (short_chat 20.0 -> 19.1 us).
     if (pl->kernel != DA_KERNEL_SIMT) {
         const bool single = pl->policy.capacity_batch == 0 &&
                             (int64_t)pl->layout.units.size() - pl->layout.n_front_units <= pl->work_grid;
-        kp.hint_first_pages = single ? 8 : 4;
+        kp.hint_first_pages = single ? 7 : 4;
     }
 #ifdef DA_TRACE
     kp.trace = g_trace_buffer;
