@@ -118,6 +118,23 @@ def test_auto_uses_whole_waves_for_large_batches():
     assert set(splits) == {1} and n_slots == 0 and len(units) == 2048
 
 
+def test_auto_cuts_long_sequences_finer_when_whole_waves_do_not_divide():
+    # 64 sequences x 8 heads = 512 units on 296 resident blocks: two units for most blocks, one for the rest.
+    # Four splits of 32,768 tokens make 2,048 units, seven for most blocks: the heaviest block carries 12 % less.
+    units, splits, _, _, chunk = layout([131072] * 64, da.make_policy(), mpp=8192)
+    assert set(splits) == {4} and chunk == 32768 and len(units) == 2048
+    covered_exactly_once(units, [131072] * 64, 8)
+    # units that a cut would bring under 4,096 tokens stay whole
+    units, splits, _, _, chunk = layout([8192] * 64, da.make_policy())
+    assert set(splits) == {1} and chunk == 8192 and len(units) == 512
+    # waves that divide well enough are left alone (2,048 units on 296 blocks: 6.9 per block)
+    units, splits, _, _, _ = layout([32768] * 256, da.make_policy())
+    assert set(splits) == {1} and len(units) == 2048
+    # one long sequence still fills the machine exactly
+    units, splits, _, _, _ = layout([32768], da.make_policy())
+    assert len(units) == 296
+
+
 def test_auto_is_a_pure_function_of_its_inputs():
     lens = wl.lengths_short_chat(64, 2)
     a = layout(lens, da.make_policy())
