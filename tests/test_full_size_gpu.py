@@ -64,10 +64,16 @@ def test_shared_prefix_full_size():
     assert_parity(out, lse, ref_out, ref_lse, "shared_prefix")
 
 
-@pytest.mark.parametrize("context,batch", [(512, 256), (2048, 64), (8192, 64), (32768, 8), (131072, 2)])
+@pytest.mark.parametrize("context,batch", [(512, 256), (2048, 64), (8192, 64), (32768, 8), (131072, 2), (16384, 64)])
 def test_sweep_cells_on_sampled_sequences(context, batch):
-    """First, last and two seeded picks of the cell, one by one against the oracle."""
+    """First, last and two seeded picks of the cell, one by one against the oracle.  (16,384 x 64 is
+    a cell whose 512 whole-sequence units do not divide over the resident blocks: the planner cuts
+    every sequence in four.)"""
     w = wl.config_sweep_cell(context, batch, device="cuda")
+    if (context, batch) == (16384, 64):
+        plan = da.decode_attn_plan(da.shape_of_workload(w), bench_policy(), w.seq_lens)
+        assert plan.info().n_units == 2048 and plan.info().chunk_tokens == 4096
+        plan.destroy()
     out, lse = da.run_workload(w, bench_policy())
     g = torch.Generator().manual_seed(context + batch)
     picks = sorted({0, batch - 1, *torch.randint(0, batch, (2,), generator=g).tolist()})
