@@ -199,13 +199,14 @@ int make_layout(const decode_attn_shape_t& s, const decode_attn_policy_t& p, con
             c = lo;
             // Whole waves do not always divide: 64 long sequences x 8 heads are 512 units on 296 blocks,
             // so most blocks get two units and the rest one.  Where the units are long enough for a
-            // cut to cost nothing (chunks stay at 4,096 tokens or more), a chunk that is a fraction
-            // of c is taken when it brings the heaviest block's load down by more than 3 % - load in
-            // pages, three pages per unit for its hand-over, 24 for a combine launch the plan did not
-            // need before (131,072 x 64: 5.12 -> 4.9x ms, what the deterministic mode's finer cut got).
+            // cut to cost next to nothing (chunks stay at 2,048 tokens or more; 1,024 was measured and
+            // loses), a chunk that is a fraction of c is taken when it brings the heaviest block's
+            // load down by more than 3 % - load in pages, three pages per unit for its hand-over, 24
+            // for a combine launch the plan did not need before (131,072 x 64: 5.11 -> 4.85 ms,
+            // 32,768 x 64: 1.28 -> 1.23 ms, 8,192 x 64: 312 -> 308.5 us).
             const int64_t u0 = H * units_for_chunk(pages, c, max_splits);
             const int64_t waves0 = ceil_div(u0, slots);
-            constexpr int64_t kLongChunk = 256, kUnitPages = 3, kCombinePages = 24;
+            constexpr int64_t kLongChunk = 128, kUnitPages = 3, kCombinePages = 24;
             if (waves0 * slots * 100 > u0 * 106 && c >= 2 * kLongChunk) {
                 const bool split0 = u0 > floor_units;
                 int64_t best = c, best_cost = waves0 * (c + kUnitPages) + (split0 ? kCombinePages : 0);

@@ -124,9 +124,11 @@ def test_auto_cuts_long_sequences_finer_when_whole_waves_do_not_divide():
     units, splits, _, _, chunk = layout([131072] * 64, da.make_policy(), mpp=8192)
     assert set(splits) == {4} and chunk == 32768 and len(units) == 2048
     covered_exactly_once(units, [131072] * 64, 8)
-    # units that a cut would bring under 4,096 tokens stay whole
     units, splits, _, _, chunk = layout([8192] * 64, da.make_policy())
-    assert set(splits) == {1} and chunk == 8192 and len(units) == 512
+    assert set(splits) == {4} and chunk == 2048 and len(units) == 2048
+    # units that a cut would bring under 2,048 tokens stay whole
+    units, splits, _, _, chunk = layout([4096] * 64, da.make_policy())
+    assert set(splits) == {1} and chunk == 4096 and len(units) == 512
     # waves that divide well enough are left alone (2,048 units on 296 blocks: 6.9 per block)
     units, splits, _, _, _ = layout([32768] * 256, da.make_policy())
     assert set(splits) == {1} and len(units) == 2048
