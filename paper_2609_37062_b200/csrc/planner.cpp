@@ -181,6 +181,7 @@ int make_layout(const decode_attn_shape_t& s, const decode_attn_policy_t& p, con
         }
     } else {
         int64_t c = min_chunk_pages(s, p);
+        const int64_t c_min = c;                              // the policy's smallest chunk: nothing below goes
         if (p.split_mode == DA_SPLIT_AUTO && B > 0) {
             const int64_t slots = (int64_t)sm_count * ctas_per_sm;
             const int64_t floor_units = (int64_t)H * B;  // one unit per (sequence, KV head) at least
@@ -212,7 +213,7 @@ int make_layout(const decode_attn_shape_t& s, const decode_attn_policy_t& p, con
                 int64_t best = c, best_cost = waves0 * (c + kUnitPages) + (split0 ? kCombinePages : 0);
                 for (int k = 2; k <= 8; ++k) {
                     const int64_t ck = ceil_div(c, k);
-                    if (ck < kLongChunk) break;
+                    if (ck < std::max(kLongChunk, c_min)) break;
                     const int64_t wk = ceil_div(H * units_for_chunk(pages, ck, max_splits), slots);
                     const int64_t cost = wk * (ck + kUnitPages) + kCombinePages;
                     if (cost * 100 < best_cost * 97) {

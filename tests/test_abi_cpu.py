@@ -126,6 +126,9 @@ def test_auto_cuts_long_sequences_finer_when_whole_waves_do_not_divide():
     covered_exactly_once(units, [131072] * 64, 8)
     units, splits, _, _, chunk = layout([8192] * 64, da.make_policy())
     assert set(splits) == {4} and chunk == 2048 and len(units) == 2048
+    # never below the policy's own smallest chunk
+    units, splits, _, _, chunk = layout([8192] * 64, da.make_policy(chunk_tokens=4096))
+    assert set(splits) == {1} and chunk == 8192
     # units that a cut would bring under 2,048 tokens stay whole
     units, splits, _, _, chunk = layout([4096] * 64, da.make_policy())
     assert set(splits) == {1} and chunk == 4096 and len(units) == 512
