@@ -102,7 +102,7 @@ def main(argv=None):
     print(f"{what} ({args.split}): {info.n_units} units on {n} blocks; "
           f"region of {K} steps: {e0.elapsed_time(e1) * 1e3 / K:.2f} us per step (traced build)")
     t = trace.cpu().numpy().astype(np.float64)
-    P, C = t[:, :n, :], t[:, n:, :]
+    P, C = t[:, :n, :], t[:, n:4096, :]          # (rows from 4096 on hold the cycle stamps of the blocks' merges)
 
     def rng(a):
         a = a[a > 0]
